@@ -1,0 +1,475 @@
+"""Pins of the CPU oracle against what the paper and plain mathematics fix (no GPU needed).
+
+Each test names the passage of the paper it rests on. A mistake in the simulator (a dropped
+message, a wrong group or tree index, a value combined twice, a swapped operand) fails at least
+one of them.
+"""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import checker as K
+from oracle import oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+U64 = np.uint64
+
+
+def rand_u64(P, k, seed):
+    return np.random.Generator(np.random.PCG64(seed)).integers(0, 2**64, size=(P, k), dtype=np.uint64)
+
+
+def uc_messages(n, f):      # Theorem on the number of messages, up-correction phase
+    a = ((n - 1) % (f + 1)) + 1
+    return f * (f + 1) * ((n - 1) // (f + 1)) + a * (a - 1)
+
+
+# ---------------------------------------------------------------------------------------------
+# worked example (section "Reduce", prose around the second tree figure)
+# ---------------------------------------------------------------------------------------------
+def parse_golden():
+    d = {}
+    for line in open(os.path.join(GOLDEN, "worked_example_n7_f1.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        key, *rest = line.split()
+        d[key] = rest
+    return d
+
+
+def test_worked_example_every_printed_number():
+    g = parse_golden()
+    n, f = int(g["n"][0]), int(g["f"][0])
+    failed = [int(v) for v in g["failed"]]
+    x = np.arange(n, dtype=np.int64).reshape(n, 1)
+    d = O.run(x, f, "sum", failed, detail=True, track_sets=True)
+    assert d["code"] == 0 and int(d["result"][0]) == int(g["expected_result"][0]) == 20
+    for item in g["after_upcorrection"]:
+        p, v = map(int, item.split(":"))
+        assert int(d["uc_values"][p, 0]) == v, (p, v)
+    for item in g["tree_message"]:
+        p, v = map(int, item.split(":"))
+        assert d["tree_sent"][p] & 1 and int(d["tree_values"][p, 0]) == v
+    for p in map(int, g["no_message"]):
+        assert d["tree_sent"][p] == 0
+    for item in g["label"]:
+        p, ids = item.split(":")
+        assert K.bits(d["tree_sets"][int(p)], n) == [int(i) for i in ids.split(",")]
+    # the root's child that reports "no failures" is process 2 and its flag is clear
+    assert d["subtree"] == 1 and d["cand_flag"][1] == 0 and d["cand_flag"][0] == 2
+    assert K.bits(d["contrib"], n) == [0, 2, 3, 4, 5, 6]
+
+
+def test_worked_example_tree_shape_and_groups():
+    """The figure's tree and the exchanging pairs, observed through who receives whose value."""
+    g = parse_golden()
+    n, f = 7, 1
+    x = (U64(1) << np.arange(n, dtype=np.uint64)).reshape(n, 1)      # one-hot inputs: sums are set labels
+    d = O.run(x, f, "sum", [], detail=True, track_sets=True)
+    # up-correction: exactly the printed pairs hold each other's value, the root holds only its own
+    groups = [tuple(int(i) for i in grp.split(",")) for grp in g["groups"]]
+    for grp in groups:
+        want = sum(1 << i for i in grp)
+        for p in grp:
+            assert int(d["uc_values"][p, 0]) == want
+    assert int(d["uc_values"][0, 0]) == 1
+    # tree: a process' message carries its group plus everything its children sent
+    parent = dict(tuple(map(int, it.split(":"))) for it in g["parent"])
+    msg = {p: int(d["tree_values"][p, 0]) for p in range(1, n)}
+    for p in range(1, n):
+        kids = [c for c, par in parent.items() if par == p]
+        expect = int(d["uc_values"][p, 0])
+        for c in kids:
+            expect += msg[c]          # multiset sum: a label counted twice would show as a carry
+        assert msg[p] == expect
+
+
+# ---------------------------------------------------------------------------------------------
+# Theorem (number of messages) and "when processes fail, fewer messages are sent"
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("n,f", [(n, f) for f in range(0, 5) for n in range(f + 2, 20)] +
+                         [(8, 1), (64, 2), (1024, 3), (4096, 4)])
+def test_message_counts_failure_free(n, f):
+    x = np.ones((n, 1), dtype=np.int32)
+    d = O.run(x, f, "sum", [], detail=True)
+    assert int(d["msgs"][0]) == uc_messages(n, f)
+    assert int(d["msgs"][1]) == n - 1
+    assert int(d["result"][0]) == n
+
+
+def test_message_counts_config5_and_printed_values():
+    # values evaluated from the theorem for the five configurations
+    table = {(8, 1): (8, 7), (64, 2): (126, 63), (1024, 3): (3072, 1023), (4096, 4): (16380, 4095),
+             (65536, 8): (524274, 65535)}
+    for (n, f), (uc, tree) in table.items():
+        assert uc_messages(n, f) == uc and tree == n - 1
+    n, f = 65536, 8
+    d = O.run(np.ones((n, 1), dtype=np.int32), f, "sum", [], detail=True)
+    assert (int(d["msgs"][0]), int(d["msgs"][1])) == table[(n, f)]
+
+
+@pytest.mark.parametrize("n,f", [(7, 1), (11, 2), (14, 3), (9, 2)])
+def test_fewer_messages_with_failures_and_nobody_sends_more(n, f):
+    x = np.ones((n, 1), dtype=np.int32)
+    base = O.run(x, f, "sum", [], detail=True)
+    for size in range(1, f + 1):
+        for dead in itertools.combinations(range(n), size):
+            d = O.run(x, f, "sum", dead, detail=True)
+            assert np.all(d["sends"] <= base["sends"])
+            for p in dead:
+                assert d["sends"][p] == 0
+            live = [p for p in range(n) if p not in dead]
+            assert np.array_equal(d["sends"][live], base["sends"][live])     # no process sends more, or fewer
+            assert int(d["msgs"][0] + d["msgs"][1]) == int(base["sends"][live].sum())
+
+
+# ---------------------------------------------------------------------------------------------
+# Semantics of reduce with pre-operation failures: unique correct result = reduction over the
+# non-failed processes (sections "Semantics", "Failure information": "only one correct result")
+# ---------------------------------------------------------------------------------------------
+def _exhaustive_cases():
+    for f in (1, 2, 3):
+        for n in range(f + 2, 13):
+            yield n, f
+
+
+@pytest.mark.parametrize("n,f", list(_exhaustive_cases()))
+def test_reduce_equals_direct_reduction_over_survivors_exhaustive(n, f):
+    x = rand_u64(n, 2, 1000 * n + f)       # random 64-bit weights: a sum matches only if every survivor is in
+    roots = range(n) if n <= 9 else (0, 1, f + 1, n - 1)      # exactly once and no failed process is in at all
+    for size in range(0, f + 1):
+        for dead in itertools.combinations(range(n), size):
+            for root in roots:
+                d = O.run(x, f, "sum", dead, root=root, track_sets=True, detail=True)
+                live = [p for p in range(n) if p not in dead]
+                if root in dead:
+                    assert d["code"] == 1 and not d["result"].any()          # reduce to a failed root: no-op
+                    continue
+                assert d["code"] == 0, (n, f, dead, root)                     # a failure-free subtree exists
+                assert np.array_equal(d["result"], K.reduce_over(x, live, "sum"))
+                assert K.bits(d["contrib"], n) == live and d["count"] == len(live)
+                assert d["cand_flag"][d["subtree"]] == 0
+                assert all(d["cand_flag"][s] != 0 for s in range(d["subtree"]))
+
+
+@pytest.mark.parametrize("op,dtype", [("max", np.int32), ("xor", np.uint64), ("sum", np.int64), ("max", np.int64),
+                                      ("max", np.uint64), ("xor", np.int32)])
+def test_other_ops_and_dtypes_match_definition(op, dtype):
+    n, f = 11, 2
+    rng = np.random.Generator(np.random.PCG64(7))
+    info = np.iinfo(dtype)
+    x = rng.integers(info.min, info.max, size=(n, 3), dtype=dtype, endpoint=True)
+    for dead in itertools.chain([()], itertools.combinations(range(n), 1), itertools.combinations(range(n), 2)):
+        for root in (0, 4):
+            if root in dead:
+                continue
+            d = O.run(x, f, op, dead, root=root)
+            live = [p for p in range(n) if p not in dead]
+            assert np.array_equal(d["result"], K.reduce_over(x, live, op)), (op, dead, root)
+
+
+def test_integer_sum_wraps():
+    x = np.full((5, 1), 2**31 - 1, dtype=np.int32)
+    d = O.run(x, 1, "sum", [])
+    assert int(d["result"][0]) == ((5 * (2**31 - 1) + 2**31) % 2**32) - 2**31
+
+
+def test_more_than_f_failures_never_yield_a_wrong_value():
+    """Outside the theorems' hypothesis: the result is right or the root reports no failure-free subtree."""
+    n, f = 10, 2
+    x = rand_u64(n, 1, 5)
+    seen = set()
+    for dead in itertools.combinations(range(1, n), f + 1):
+        d = O.run(x, f, "sum", dead)
+        live = [p for p in range(n) if p not in dead]
+        seen.add(d["code"])
+        if d["code"] == 0:
+            assert np.array_equal(d["result"], K.reduce_over(x, live, "sum"))
+        else:
+            assert d["code"] == 2 and not d["result"].any()
+    assert seen == {0, 2}
+
+
+# ---------------------------------------------------------------------------------------------
+# copies of every value that reach the root in the failure-free case (section "Algorithm":
+# "include each value f+1 times", made exact): a process of a full group is in f+1 child
+# messages; a member of the last, short group (root included) in r child messages
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("n,f", [(7, 1), (8, 1), (12, 2), (13, 3), (16, 3), (30, 4)])
+def test_copies_of_each_value_at_the_root(n, f):
+    d = O.run(np.ones((n, 1), np.int32), f, "sum", [], detail=True, track_sets=True)
+    q, r = (n - 1) // (f + 1), (n - 1) % (f + 1)
+    copies = np.zeros(n, dtype=int)
+    for s in range(f + 1):
+        child = s + 1
+        for p in K.bits(d["tree_sets"][child], n):
+            copies[p] += 1
+    for p in range(1, n):
+        full = (p - 1) // (f + 1) < q
+        assert copies[p] == (f + 1 if full else r)
+    assert copies[0] == r
+    # sizes of the root's subtrees differ by at most one (definition of the I(f)-tree)
+    sizes = [int(d["tree_values"][s + 1, 0]) for s in range(f + 1)]    # inputs are 1: value = values included
+    assert d["cand_flag"].tolist() == [0] * (f + 1)
+    incl = [len(K.bits(d["tree_sets"][s + 1], n)) for s in range(f + 1)]
+    assert incl == sizes
+
+
+# ---------------------------------------------------------------------------------------------
+# in-operation failures (Theorem on the semantics, item 4): every (victim, round), value equals the
+# reduction over Live plus a subset of the victims, never a partial or doubled contribution
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("n,f", [(6, 1), (7, 1), (8, 2), (11, 2), (12, 3), (14, 3)])
+def test_inop_reduce_allowed_results_exhaustive(n, f):
+    x = rand_u64(n, 1, 77 * n + f)
+    rounds = O.schedule(n, f)["rounds_reduce"]
+    outcomes = set()
+    for victim in range(n):
+        for t in range(1, rounds + 2):
+            for pre in itertools.chain([()], itertools.combinations([p for p in range(1, n) if p != victim], 1)
+                                       if f >= 2 else []):
+                d = O.run(x, f, "sum", pre, inop=[(victim, t)], track_sets=True, detail=True)
+                if victim == 0:
+                    if t < rounds:
+                        assert d["code"] == 1            # the root failed: no-op
+                        continue
+                assert d["code"] == 0, (victim, t, pre)
+                C = K.bits(d["contrib"], n)
+                assert K.contribution_allowed(n, C, pre, [victim])
+                assert np.array_equal(d["result"], K.reduce_over(x, C, "sum"))
+                assert d["count"] == len(C) and d["inop_included"] == int(victim in C)
+                outcomes.add(victim in C)
+                if t >= rounds:
+                    assert victim in C                   # it completed every send of the reduce
+    # with f = 1 a victim's only up-correction send is round 0, so a round >= 1 always includes it
+    assert outcomes == ({True, False} if f >= 2 else {True})
+
+
+def test_inop_value_can_arrive_along_one_path_and_not_another():
+    """Section "Failure information": a process that completes up-correction but not its tree send
+    reaches the root through its partners only."""
+    n, f = 7, 1
+    x = (U64(1) << np.arange(n, dtype=np.uint64)).reshape(n, 1)
+    sch = O.schedule(n, f)
+    # process 3 (depth 2) sends to its partner 4 in round 0, its tree send is round f+H-2 = 1
+    d = O.run(x, f, "sum", [], inop=[(3, 1)], detail=True, track_sets=True)
+    assert d["cand_flag"].tolist() == [1, 0] and d["subtree"] == 1
+    assert K.bits(d["contrib"], n) == list(range(n))
+    d = O.run(x, f, "sum", [], inop=[(4, 1)], detail=True, track_sets=True)    # 4 is in subtree 1
+    assert d["cand_flag"].tolist() == [0, 1] and d["subtree"] == 0
+    assert K.bits(d["contrib"], n) == list(range(n))
+    assert sch["rounds_reduce"] == 3
+
+
+# ---------------------------------------------------------------------------------------------
+# allreduce (Algorithm "Allreduce", its semantics and the theorem on its number of messages)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("n,f", [(6, 1), (9, 2), (12, 3), (13, 2)])
+def test_allreduce_semantics_exhaustive_pre_op(n, f):
+    x = rand_u64(n, 2, 31 * n + f)
+    free = O.run(x, f, "sum", [], allreduce=True, detail=True)
+    per_attempt = int(free["msgs"][:4].sum())
+    assert int(free["msgs"][2]) == n - 1                       # the value travels down the same tree
+    assert int(free["msgs"][0]) == uc_messages(n, f) and int(free["msgs"][1]) == n - 1
+    for size in range(0, f + 1):
+        for dead in itertools.combinations(range(n), size):
+            for first in (0, 3):
+                d = O.run(x, f, "sum", dead, root=first, allreduce=True, detail=True, track_sets=True)
+                live = [p for p in range(n) if p not in dead]
+                lead = 0
+                while (first + lead) % n in dead:
+                    lead += 1
+                assert d["code"] == 0 and d["attempts"] == lead + 1       # one attempt per failed candidate
+                want = K.reduce_over(x, live, "sum")
+                assert np.array_equal(d["result"], want)
+                assert K.bits(d["holders"], n) == live and d["n_holders"] == len(live)
+                for p in range(n):                                       # every live process holds the same bits
+                    assert np.array_equal(d["expanded"][p], want if p in live else np.zeros_like(want))
+                assert int(d["msgs"][:4].sum()) <= (f + 1) * per_attempt   # at most (f+1)-fold
+                ev = d["events"]
+                assert all(ev[p] == 3 for p in live) and all(ev[p] == 0 for p in dead)
+
+
+def test_allreduce_no_live_candidate_and_inop_candidate():
+    n, f = 8, 1
+    x = rand_u64(n, 1, 3)
+    d = O.run(x, f, "sum", [0, 1], allreduce=True)
+    assert d["code"] == 3 and d["attempts"] == 2 and not d["result"].any()
+    d = O.run(x, f, "sum", [], inop=[(1, 2)], allreduce=True)
+    assert d["code"] == 4
+
+
+@pytest.mark.parametrize("n,f", [(7, 1), (10, 2), (13, 3)])
+def test_allreduce_inop_all_or_nothing_and_consistent(n, f):
+    """Allreduce semantics items 4 and 5 under one in-operation failure outside the candidates."""
+    x = rand_u64(n, 1, 900 + n)
+    R = O.schedule(n, f)["rounds_attempt"]
+    for victim in range(f + 1, n):
+        for t in range(1, R + 1):
+            d = O.run(x, f, "sum", [], inop=[(victim, t)], allreduce=True, detail=True, track_sets=True)
+            assert d["code"] == 0
+            C = K.bits(d["contrib"], n)
+            assert K.contribution_allowed(n, C, [], [victim])
+            want = K.reduce_over(x, C, "sum")
+            holders = K.bits(d["holders"], n)
+            alive_end = [p for p in range(n) if p != victim or t >= R]
+            assert holders == alive_end
+            for p in holders:
+                assert np.array_equal(d["expanded"][p], want)
+
+
+def test_allreduce_dead_first_candidate_then_inop_victim_counts_as_failed_before():
+    """A victim that dies during a fruitless first attempt is dead from the start of the second."""
+    n, f = 9, 2
+    x = rand_u64(n, 1, 11)
+    R = O.schedule(n, f)["rounds_attempt"]
+    d = O.run(x, f, "sum", [0], inop=[(5, 1)], allreduce=True, detail=True, track_sets=True)
+    assert d["attempts"] == 2 and K.bits(d["contrib"], n) == [1, 2, 3, 4, 6, 7, 8]
+    # second attempt, root 1: process 5 (group {4,5,6}, subtree of root child 2 -> unclean once 5 is gone) sends
+    # to 4 in local round 0 and to 6 in local round 1; subtree of child 1 has the dead process 0 at its top,
+    # so the root takes child 3, whose member of that group is 6
+    d = O.run(x, f, "sum", [0], inop=[(5, R + 1)], allreduce=True, detail=True, track_sets=True)
+    assert d["attempts"] == 2 and d["subtree"] == 2 and K.bits(d["contrib"], n) == [1, 2, 3, 4, 6, 7, 8]
+    d = O.run(x, f, "sum", [0], inop=[(5, R + 2)], allreduce=True, detail=True, track_sets=True)
+    assert d["attempts"] == 2 and d["subtree"] == 2 and K.bits(d["contrib"], n) == [1, 2, 3, 4, 5, 6, 7, 8]
+    assert K.bits(d["holders"], n) == [1, 2, 3, 4, 6, 7, 8]
+
+
+# ---------------------------------------------------------------------------------------------
+# protocol items 1, 2, 5 of the reduce semantics, seen through the event log
+# ---------------------------------------------------------------------------------------------
+def test_reduce_events_init_and_deliver_once():
+    n, f = 12, 2
+    x = rand_u64(n, 1, 2)
+    for dead in itertools.combinations(range(1, n), 2):
+        d = O.run(x, f, "sum", dead, detail=True)
+        for p in range(n):
+            assert d["events"][p] == (0 if p in dead else 3)        # init once, deliver exactly once
+
+
+# ---------------------------------------------------------------------------------------------
+# the scheduler is irrelevant: any interleaving of the processes gives the same messages
+# ---------------------------------------------------------------------------------------------
+def test_result_independent_of_scheduler_order():
+    n, f = 23, 3
+    x = np.random.Generator(np.random.PCG64(4)).standard_normal((n, 3)).astype(np.float32)
+    for allred in (False, True):
+        for dead, inop in (((), ()), ((2,), ((9, 2),)), ((5, 6), ((7, 1), (22, 4)))):
+            ref = O.run(x, f, "sum", dead, inop=list(inop), allreduce=allred, detail=True)
+            for sweep in (1, 2, 3, 99):
+                d = O.run(x, f, "sum", dead, inop=list(inop), allreduce=allred, sweep=sweep, detail=True)
+                for key in ("result", "status", "cand", "cand_flag", "msgs", "sends", "tree_values", "expanded"):
+                    assert np.array_equal(ref[key], d[key]), (key, sweep)
+
+
+# ---------------------------------------------------------------------------------------------
+# float32
+# ---------------------------------------------------------------------------------------------
+def test_f32_within_tolerance_of_float64_sum():
+    n, f = 1024, 3
+    rng = np.random.Generator(np.random.PCG64(9))
+    x = rng.standard_normal((n, 16)).astype(np.float32)
+    for dead in ((), (0,), (1, 2, 3), (17, 500, 1023)):
+        d = O.run(x, f, "sum", dead, allreduce=True)
+        live = [p for p in range(n) if p not in dead]
+        assert d["code"] == 0 and K.value_matches(x, live, "sum", d["result"])
+
+
+def test_f32_small_integers_are_exact():
+    n, f = 200, 3
+    x = np.random.Generator(np.random.PCG64(1)).integers(-1000, 1000, size=(n, 4)).astype(np.float32)
+    d = O.run(x, f, "sum", [3, 50])
+    live = [p for p in range(n) if p not in (3, 50)]
+    assert np.array_equal(d["result"].astype(np.int64), x[live].astype(np.int64).sum(axis=0))
+
+
+def test_f32_combine_order_of_the_documented_reading():
+    """n=5, f=1: groups {1,2},{3,4}; tree 0->{1,2}, 1->{3}, 2->{4}. The root takes child 1:
+    result = x0 + ((x1+x2) + (x3+x4)), each parenthesis one float32 rounding, accumulator left."""
+    x = np.array([[1.0], [1e8], [3.0], [-1e8], [5.0]], dtype=np.float32)
+    f32 = np.float32
+    want = f32(x[0, 0] + f32(f32(x[1, 0] + x[2, 0]) + f32(x[3, 0] + x[4, 0])))
+    d = O.run(x, 1, "sum", [])
+    assert d["result"][0] == want
+    # with process 1 failed the root takes child 2: x0 + ((x2) + (x4 + x3))
+    want2 = f32(x[0, 0] + f32(x[2, 0] + f32(x[4, 0] + x[3, 0])))
+    d = O.run(x, 1, "sum", [1])
+    assert d["result"][0] == want2 and d["subtree"] == 1
+
+
+def test_schedule_constants_of_the_five_configurations():
+    want = {(8, 1): (3, 4, 8), (64, 2): (5, 7, 14), (1024, 3): (9, 12, 24), (4096, 4): (10, 14, 28),
+            (65536, 8): (13, 21, 42)}
+    for (n, f), (H, rr, ra) in want.items():
+        s = O.schedule(n, f)
+        assert (s["H"], s["rounds_reduce"], s["rounds_attempt"]) == (H, rr, ra)
+        assert s["H"] == 1 + math.floor(math.log2(math.ceil((n - 1) / (f + 1))))
+
+
+# ---------------------------------------------------------------------------------------------
+# hand-evaluated cases of the documented readings (orders and the round clock), so that a change
+# of a reading cannot slip through unnoticed
+# ---------------------------------------------------------------------------------------------
+def test_reading_children_order_and_root_first_in_last_group_f32():
+    f32 = np.float32
+    # n=7, f=1: 1 -> {3,5}: message of 1 = ((x1+x2) + (x3+x4)) + (x5+x6); root adds its own on the left
+    x = np.array([[0.5], [1e8], [1.0], [-1e8], [3.0], [7.0], [-5.0]], dtype=np.float32)
+    v1 = f32(f32(f32(x[1, 0] + x[2, 0]) + f32(x[3, 0] + x[4, 0])) + f32(x[5, 0] + x[6, 0]))
+    d = O.run(x, 1, "sum", [], detail=True)
+    assert d["tree_values"][1, 0] == v1 and d["result"][0] == f32(x[0, 0] + v1)
+    swapped = f32(f32(f32(x[1, 0] + x[2, 0]) + f32(x[5, 0] + x[6, 0])) + f32(x[3, 0] + x[4, 0]))
+    assert swapped != v1            # the inputs do tell the two orders apart
+    # n=6, f=2: groups {1,2,3} and the short one {4,5,root}; the root takes child 1, whose subtree holds 4:
+    # message of 4 = (x4 + x0) + x5 (the root is the first partner), message of 1 = ((x1+x2)+x3) + that
+    y = np.array([[1e8], [2.0], [3.0], [4.0], [-1e8], [1.0]], dtype=np.float32)
+    m4 = f32(f32(y[4, 0] + y[0, 0]) + y[5, 0])
+    assert m4 != f32(f32(y[4, 0] + y[5, 0]) + y[0, 0])
+    d = O.run(y, 2, "sum", [], detail=True)
+    assert d["tree_values"][4, 0] == m4
+    assert d["result"][0] == f32(f32(f32(y[1, 0] + y[2, 0]) + y[3, 0]) + m4) and d["subtree"] == 0
+
+
+def test_reading_round_clock_of_tree_sends():
+    """n=7, f=1: H=2; leaves (depth 2) send to their parents in round f+H-2 = 1, root children in round 2."""
+    x = (U64(1) << np.arange(7, dtype=np.uint64)).reshape(7, 1)
+    flags = lambda vic, t: O.run(x, 1, "sum", [], inop=[(vic, t)], detail=True)["cand_flag"].tolist()
+    assert flags(3, 1) == [1, 0] and flags(3, 2) == [0, 0]
+    assert flags(1, 2) == [2, 0] and flags(1, 3) == [0, 0]
+    assert flags(2, 2) == [0, 2] and flags(2, 3) == [0, 0]
+
+
+def test_reading_partner_order_decides_whom_a_dying_process_reached():
+    """n=6, f=2, short last group {4, 5, root}: process 5 sends to the root in round 0 and to 4 in round 1.
+    Subtree of child 1 (holding 4) is chosen; it has 5's value only if the second send happened."""
+    x = (U64(1) << np.arange(6, dtype=np.uint64)).reshape(6, 1)
+    d = O.run(x, 2, "sum", [], inop=[(5, 1)], detail=True, track_sets=True)
+    assert d["subtree"] == 0 and K.bits(d["contrib"], 6) == [0, 1, 2, 3, 4]
+    d = O.run(x, 2, "sum", [], inop=[(5, 2)], detail=True, track_sets=True)
+    assert d["subtree"] == 0 and K.bits(d["contrib"], 6) == [0, 1, 2, 3, 4, 5]
+    # full group {1,2,3}: process 3 sends to 1 in round 0, to 2 in round 1, up the tree in round f+H-1 = 2
+    d = O.run(x, 2, "sum", [1], inop=[(3, 1)], detail=True, track_sets=True)
+    assert d["subtree"] == 1 and K.bits(d["contrib"], 6) == [0, 2, 4, 5]
+    d = O.run(x, 2, "sum", [1], inop=[(3, 2)], detail=True, track_sets=True)
+    assert d["subtree"] == 1 and K.bits(d["contrib"], 6) == [0, 2, 3, 4, 5]
+
+
+def test_reading_broadcast_correction_is_sent_by_tree_holders_only():
+    """n=10, f=2, allreduce from root 0 with 2 and 3 failed beforehand and 4 dying after its first
+    correction send (three failures: outside the theorems, played anyway). 4 is the only process of
+    {4,5,6} the tree reaches; it hands the value to 5 and dies; 5 does not pass it on to 6."""
+    x = rand_u64(10, 1, 8)
+    sch = O.schedule(10, 2)
+    assert (sch["H"], sch["rounds_reduce"], sch["rounds_attempt"]) == (2, 4, 8)
+    first_corr = sch["rounds_reduce"] + sch["H"]                # round of correction iteration 0
+    d = O.run(x, 2, "sum", [2, 3], inop=[(4, first_corr + 1)], allreduce=True, detail=True, track_sets=True)
+    assert d["code"] == 0 and d["subtree"] == 0
+    assert K.bits(d["holders"], 10) == [0, 1, 5, 7, 8, 9]
+    d = O.run(x, 2, "sum", [2, 3], inop=[(4, first_corr + 2)], allreduce=True, detail=True, track_sets=True)
+    # a failure round equal to the attempt's length: every send was made and the process is alive at the end
+    assert first_corr + 2 == sch["rounds_attempt"] and K.bits(d["holders"], 10) == [0, 1, 4, 5, 6, 7, 8, 9]
+    d = O.run(x, 2, "sum", [2, 3], inop=[(4, first_corr)], allreduce=True, detail=True, track_sets=True)
+    assert K.bits(d["holders"], 10) == [0, 1, 7, 8, 9]
