@@ -1,0 +1,196 @@
+/*
+ * ftc.h -- C ABI of the batched executor for the correction-based fault-tolerant
+ * reduce and allreduce (Kuettler & Haertig, "Fault-tolerant Reduce and Allreduce
+ * operations based on correction").
+ *
+ * The library plays the paper's message schedule for S independent scenarios at once
+ * on one NVIDIA B200 (sm_100a). A scenario is one input vector of k elements for each
+ * of P logical processes plus a failure pattern; the result is the value the root
+ * (reduce) or every surviving process (allreduce) ends up with, and a status record.
+ *
+ * Conventions for every entry point
+ *   - plain C linkage, no exceptions, no global state (except where an entry point
+ *     says otherwise); pointers named d_* are DEVICE pointers, h_* HOST pointers;
+ *   - the caller owns every buffer and the stream; inputs are read-only; the library
+ *     allocates nothing and never synchronises the host unless stated;
+ *   - work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = the
+ *     default stream) and is complete when that stream has drained;
+ *   - the return value reports call-level errors only (0 = FTC_OK, negative = error,
+ *     see ftc_strerror). What happens inside a scenario (failed root, no failure-free
+ *     subtree, ...) is not an error: it is written to that scenario's status record.
+ *
+ * Readings of the paper that fix the schedule (the paper leaves them open):
+ *   - the root swaps numbers with process 0 (section "Reduce"); all rules below apply
+ *     to the renumbered ranks v;
+ *   - up-correction group of v >= 1 is floor((v-1)/(f+1)); the root joins the last
+ *     group iff that group is short (section "Up-Correction"); partners are visited in
+ *     ascending rank, the root first;
+ *   - v >= 1 lies below root child s = (v-1) mod (f+1) (proof of the first theorem of
+ *     section "Properties"); within a subtree the nodes j = floor((v-1)/(f+1)) form a
+ *     binary heap: children 2j+1, 2j+2, received in that order, accumulator on the left;
+ *   - failure information is the single failed bit (third scheme of section "Failure
+ *     information"); the root takes the lowest-numbered child that delivered with the
+ *     bit clear (Algorithm "reduce_root");
+ *   - rounds: up-correction iteration i is round i (0..f-1); a node at depth d sends up
+ *     the tree in round f+H-d, H = 1+floor(log2(ceil((P-1)/(f+1)))); one reduce has
+ *     f+H rounds. The broadcast of the allreduce sends down the same tree (depth d in
+ *     round f+H+d) and then lets every process the tree reached send the value to its
+ *     up-correction partners (iteration i in round f+2H+i); one allreduce attempt has
+ *     2(f+H) rounds and attempt a starts at round a*2(f+H). A process with failure
+ *     round t performs exactly the sends scheduled in rounds < t;
+ *   - allreduce root candidates are first, first+1, ... (mod P), f+1 of them
+ *     (Algorithm "Allreduce"; "at least f+1 processes must eventually be tried").
+ */
+#ifndef FTC_H
+#define FTC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define FTC_API __attribute__((visibility("default")))
+#else
+#define FTC_API
+#endif
+
+#define FTC_VERSION 0x00010000u
+
+/* element types and reduction functions (section "Reduce": associative and commutative) */
+enum { FTC_I32 = 0, FTC_I64 = 1, FTC_U64 = 2, FTC_F32 = 3 };
+enum { FTC_SUM = 0, FTC_MAX = 1, FTC_XOR = 2 };   /* integer sums wrap; FTC_F32 supports FTC_SUM only */
+
+/* call-level return codes */
+enum {
+    FTC_OK = 0,
+    FTC_EINVAL = -1,        /* P < f+2, k = 0, root >= P, NULL or misaligned required pointer, f > 31, max_inop > 32 */
+    FTC_EUNSUPPORTED = -2,  /* unknown dtype/op, xor or max on f32 */
+    FTC_EWORKSPACE = -3,    /* workspace missing or smaller than ftc_workspace_bytes() */
+    FTC_ECUDA = -4          /* a CUDA call or launch failed */
+};
+
+/* per-scenario outcome, low byte of status word 0 */
+enum {
+    FTC_ST_OK = 0,
+    FTC_ST_ROOT_FAILED = 1,             /* reduce to a failed root is a no-op (section "Semantics") */
+    FTC_ST_NO_CLEAN_SUBTREE = 2,        /* Algorithm "reduce_root": "No failure-free subtree" (needs > f failures) */
+    FTC_ST_NO_LIVE_ROOT_CANDIDATE = 3,  /* allreduce: all f+1 candidates had failed before the operation */
+    FTC_ST_PRECONDITION_INOP_ROOT = 4,  /* allreduce: a root candidate is listed as failing in-operation */
+    FTC_ST_BAD_ROOT = 5                 /* d_roots[s] >= P */
+};
+
+/*
+ * Status record, FTC_STATUS_WORDS uint32 per scenario:
+ *   word 0: outcome | selected root child (0..f, 0xFF none) << 8 | attempts used << 16
+ *   word 1: number of processes whose input is included in the result
+ *   word 2: bit i set = the victim of in-operation slot i is included in the result
+ *   word 3: allreduce: processes that are alive at the end and hold the result; reduce: 0
+ * When the outcome is not FTC_ST_OK words 1..3 are 0 and the result is all zero bytes.
+ */
+#define FTC_STATUS_WORDS 4
+
+/* An in-operation failure: `victim` performs exactly the sends scheduled in rounds < `round`.
+ * victim = FTC_INOP_UNUSED marks an empty slot; a victim that is also pre-failed counts as pre-failed;
+ * round 0 is the same as a pre-operation failure. (Sections "Introduction", "Failures".) */
+typedef struct { uint32_t victim; uint32_t round; } ftc_inop_t;
+#define FTC_INOP_UNUSED 0xFFFFFFFFu
+#define FTC_MAX_INOP 32u
+#define FTC_MAX_F 31u
+
+/* flags */
+#define FTC_OUT_EXPANDED   0x1u   /* allreduce: d_out is [S][P][k], zeros for processes that do not hold the result */
+#define FTC_KERNEL_GENERIC 0x100u /* force the general level-by-level kernel (needs the workspace) */
+
+typedef struct {
+    uint32_t P;         /* processes, P >= f+2 (the root needs f+1 children: definition of the I(f)-tree) */
+    uint32_t f;         /* failures to tolerate, 0..31; up-correction groups have f+1 members */
+    uint32_t k;         /* elements per process */
+    uint32_t dtype;     /* FTC_I32 ... */
+    uint32_t op;        /* FTC_SUM ... */
+    int32_t  root;      /* >= 0: root (reduce) / first root candidate (allreduce) of every scenario; -1: d_roots[s] */
+    uint32_t max_inop;  /* in-operation slots per scenario in d_inop, 0..32 */
+    uint32_t flags;
+} ftc_desc_t;
+
+/* Schedule constants under the readings above and the failure-free message counts of the theorem on the
+ * number of messages (section "Properties"). */
+typedef struct {
+    uint32_t q, r;              /* full groups, size of the short last group without the root: P-1 = q(f+1)+r */
+    uint32_t H;                 /* depth of the deepest node */
+    uint32_t rounds_reduce;     /* f+H */
+    uint32_t rounds_attempt;    /* 2(f+H): reduce plus broadcast */
+    uint64_t msgs_upcorrection; /* f(f+1)q + a(a-1), a = r+1 */
+    uint64_t msgs_tree;         /* P-1 */
+} ftc_sched_t;
+
+/*
+ * Corrected reduce (Algorithms "Up-correction", "reduce_root", "reduce_non_root", "reduce") for S scenarios.
+ *   d_in      [S][P][k] elements of desc->dtype, process order as the caller numbers them; 16-byte aligned
+ *   d_prefail [S][ceil(P/32)] uint32, bit p of a scenario's words set = process p failed before the operation
+ *   d_inop    [S][max_inop] or NULL when max_inop = 0
+ *   d_roots   [S] or NULL; read only when desc->root < 0
+ *   d_out     [S][k]: the value delivered at the root (zeros unless the outcome is FTC_ST_OK); 16-byte aligned
+ *   d_status  [S][FTC_STATUS_WORDS]
+ *   d_workspace, workspace_bytes: scratch of at least ftc_workspace_bytes(desc, S, 0) bytes (may be NULL if that is 0);
+ *             contents are undefined afterwards; calls that share a workspace must not overlap on the device
+ * S = 0 is valid and does nothing. Returns FTC_OK or an error before anything is enqueued.
+ */
+FTC_API int ftc_reduce_batch(const ftc_desc_t* desc, uint64_t S, const void* d_in, const uint32_t* d_prefail,
+                     const ftc_inop_t* d_inop, const uint32_t* d_roots, void* d_out, uint32_t* d_status,
+                     void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Corrected allreduce (Algorithm "Allreduce": reduce to a root candidate, broadcast from it, next candidate if
+ * it had failed before the operation). Arguments as for ftc_reduce_batch; desc->root / d_roots give the first
+ * candidate. d_out is [S][k] (the value every holder has) or, with FTC_OUT_EXPANDED, [S][P][k].
+ */
+FTC_API int ftc_allreduce_batch(const ftc_desc_t* desc, uint64_t S, const void* d_in, const uint32_t* d_prefail,
+                        const ftc_inop_t* d_inop, const uint32_t* d_roots, void* d_out, uint32_t* d_status,
+                        void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Scratch bytes the two calls above need for this descriptor and batch size (0 when the shape runs on the
+ * shared-memory kernel). Returns 0 for an invalid descriptor as well; the batch calls report that. */
+FTC_API size_t ftc_workspace_bytes(const ftc_desc_t* desc, uint64_t S, int is_allreduce);
+
+/*
+ * Same operations with HOST buffers (h_* as the d_* above): copies the inputs to the device in chunks, runs the
+ * kernels, copies results and status back, all on `cuda_stream`, then synchronises that stream before returning.
+ * d_staging is device scratch of at least ftc_host_staging_bytes(desc, 1) bytes; larger staging means larger
+ * chunks. Pinned host memory makes the copies asynchronous but is not required.
+ */
+FTC_API int ftc_reduce_batch_host(const ftc_desc_t* desc, uint64_t S, const void* h_in, const uint32_t* h_prefail,
+                          const ftc_inop_t* h_inop, const uint32_t* h_roots, void* h_out, uint32_t* h_status,
+                          void* d_staging, size_t staging_bytes, void* cuda_stream);
+FTC_API int ftc_allreduce_batch_host(const ftc_desc_t* desc, uint64_t S, const void* h_in, const uint32_t* h_prefail,
+                             const ftc_inop_t* h_inop, const uint32_t* h_roots, void* h_out, uint32_t* h_status,
+                             void* d_staging, size_t staging_bytes, void* cuda_stream);
+/* Device staging bytes for chunks of `chunk_scenarios` scenarios (inputs, masks, outputs and workspace). */
+FTC_API size_t ftc_host_staging_bytes(const ftc_desc_t* desc, uint64_t chunk_scenarios);
+
+/* Schedule constants and failure-free message counts for (P, f) of the descriptor. FTC_EINVAL if P < f+2. */
+FTC_API int ftc_schedule_info(const ftc_desc_t* desc, ftc_sched_t* out);
+
+/*
+ * Synthetic scenario inputs on the device (not part of the paper's method): element (s, p, e) of scenario
+ * first_scenario+s is a function of (seed, scenario, p, e) only -- the splitmix64 output function applied to
+ * seed + 0x9E3779B97F4A7C15 * (counter+1) -- mapped to one of the value kinds
+ *   0 int32 in [-2^20, 2^20]   1 int64 in [-2^40, 2^40]   2 float32, sum of twelve 21-bit uniforms scaled to unit variance
+ *   3 int32 full range         4 uint64 full range
+ * d_out is [S][P][k] of the kind's type. Returns FTC_OK, FTC_EINVAL (unknown kind, NULL) or FTC_ECUDA.
+ */
+FTC_API int ftc_fill_inputs(uint32_t kind, uint64_t seed, uint64_t first_scenario, uint64_t S, uint32_t P, uint32_t k,
+                    void* d_out, void* cuda_stream);
+
+/* Name of the kernel family the batch calls would use for this descriptor: "tiled" or "generic". */
+FTC_API const char* ftc_kernel_name(const ftc_desc_t* desc, int is_allreduce);
+
+FTC_API const char* ftc_strerror(int code);
+FTC_API uint32_t ftc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FTC_H */

@@ -358,11 +358,11 @@ static int advance(sim_t* s, uint32_t v, int* overlap) {
             s->phase[v] = PH_BC_SEND; progress = 1;
         } break;
         case PH_BC_SEND: {
-            if (!s->tree_holder[v]) { s->bct_state[v] = SLOT_SKIPPED; }
+            uint32_t nc = children(s, v, cb);
+            if (!s->tree_holder[v] || nc == 0) { s->bct_state[v] = SLOT_SKIPPED; }   /* nothing to pass on, or nobody below */
             else {
                 int64_t round = s->base + s->Rred + depth_of(s, v);
                 if (!can_send(s, v, round)) { die(s, v); return 1; }
-                uint32_t nc = children(s, v, cb);
                 s->bct_state[v] = SLOT_SENT;
                 s->msgs_attempt[2] += nc; s->nsent[v] += nc;
             }

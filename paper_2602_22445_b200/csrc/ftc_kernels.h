@@ -1,0 +1,27 @@
+// Host-side declarations of the kernel launchers (internal to the library).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace ftc {
+
+struct Params;
+
+// (element type, reduction) pairs the kernels are instantiated for. Signed and unsigned sums and xors of the
+// same width are the same bit operation, so int64 sum runs as uint64 sum, and so on.
+enum TypeSel { TS_U32_SUM = 0, TS_I32_MAX, TS_U32_XOR, TS_U64_SUM, TS_I64_MAX, TS_U64_MAX, TS_U64_XOR, TS_F32_SUM, TS_COUNT };
+
+size_t generic_smem_bytes(const Params& p);
+uint32_t generic_grid(const Params& p, int sm_count);
+cudaError_t launch_generic(const Params& p, int tsel, int sm_count, cudaStream_t st);
+
+// Tiled kernel: does the shape fit (16-byte chunks, power-of-two chunk count <= 32, shared memory)? Fills the
+// tile geometry into p when it does.
+bool tiled_supported(Params& p, int smem_optin_bytes);
+cudaError_t launch_tiled(const Params& p, int tsel, int sm_count, cudaStream_t st);
+
+cudaError_t launch_fill(uint32_t kind, uint64_t seed, uint64_t first, uint64_t S, uint32_t P, uint32_t k, void* out,
+                        int sm_count, cudaStream_t st);
+
+}  // namespace ftc

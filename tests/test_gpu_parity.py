@@ -1,0 +1,257 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, element by element.
+
+Integer and bitwise results, status records and float32 results are all compared bit for bit (the
+schedule fixes the float32 combine order, so no tolerance is needed; the documented fallback tolerance
+1e-6*ceil(log2 P) relative to the sum of magnitudes is checked against a float64 sum as well).
+"""
+import itertools
+
+import numpy as np
+import pytest
+
+from oracle import checker as K
+from oracle import oracle as O
+from paper_2602_22445_b200 import binding as B
+from paper_2602_22445_b200 import scenarios as sc
+from tests.gpu_util import assert_same, run_gpu, run_oracle, to_dev, to_host
+
+pytestmark = pytest.mark.gpu
+
+KERNELS = [0, B.FTC_KERNEL_GENERIC]
+
+
+def check_workload(w, idx=None, flags=0, collective=None):
+    ids = np.arange(w.S) if idx is None else np.asarray(idx)
+    x = w.host_inputs(ids)
+    pf = w.prefail[ids]
+    inop = None if w.inop is None else w.inop[ids]
+    roots = None if w.roots is None else w.roots[ids]
+    allred = (collective or w.collective) == "allreduce"
+    got = run_gpu(x, w.f, w.op, pf, inop, roots, max(w.root, 0), allred, flags)
+    want = run_oracle(x, w.f, w.op, pf, inop, roots, max(w.root, 0), allred)
+    assert_same(got, want, f"{w.name} flags={flags:#x}")
+    return x, got
+
+
+@pytest.mark.parametrize("flags", KERNELS)
+def test_config1_all_scenarios(flags):
+    w = sc.config1()
+    x, (out, st, _) = check_workload(w, flags=flags)
+    assert (st[:, 0] & 0xFF).tolist() == [0, 1] + [0] * 7       # the set {0} kills the root: no-op
+
+
+@pytest.mark.parametrize("flags", KERNELS)
+def test_config2_all_scenarios(flags):
+    w = sc.config2()
+    assert w.S == 33296
+    x, (out, st, desc) = check_workload(w, flags=flags)
+    assert B.ftc_kernel_name(desc) == ("generic" if flags else "tiled")
+    live_ok = (st[:, 0] & 0xFF) == 0
+    assert live_ok.sum() == 16 * (2081 - 1 - 63)                 # every set without process 0 succeeds
+
+
+@pytest.mark.parametrize("flags", KERNELS)
+def test_config3_sample_float32_bit_exact(flags):
+    w = sc.config3(S=384)
+    x, (out, st, _) = check_workload(w, flags=flags)
+    for i in range(0, 384, 37):                                   # and within the documented tolerance of float64
+        live = [p for p in range(w.P) if not (w.prefail[i, p >> 5] >> (p & 31)) & 1]
+        assert K.value_matches(x[i], live, "sum", out[i])
+    assert set((st[:, 0] >> 16) & 0xFF) >= {1, 2}                 # some first candidates were dead
+
+
+@pytest.mark.parametrize("flags", KERNELS)
+def test_config4_sample_with_inop_failures(flags):
+    ratt = O.schedule(4096, 4)["rounds_attempt"]
+    w = sc.config4(ratt, S=96)
+    check_workload(w, flags=flags)
+
+
+@pytest.mark.parametrize("collective,op", [("reduce", "sum"), ("reduce", "xor"), ("allreduce", "sum"), ("allreduce", "xor")])
+def test_config5_sample(collective, op):
+    w = sc.config5(collective, op, S=12)
+    check_workload(w)
+
+
+def test_config5_sample_generic_kernel():
+    w = sc.config5("allreduce", "sum", S=4)
+    check_workload(w, flags=B.FTC_KERNEL_GENERIC)
+
+
+# ---------------------------------------------------------------------------------------------
+# exhaustive small cases and edge cases
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("flags", KERNELS)
+@pytest.mark.parametrize("allreduce", [False, True])
+def test_exhaustive_failure_sets_small_P(flags, allreduce):
+    rng = np.random.Generator(np.random.PCG64(5))
+    for f in (0, 1, 2, 3):
+        for P in (f + 2, f + 3, 7, 9, 13, 16):
+            if P < f + 2:
+                continue
+            sets = sc.all_failure_sets(P, min(f + 1, 3))          # one more failure than tolerated as well
+            roots = rng.integers(0, P, size=len(sets)).astype(np.uint32)
+            x = rng.integers(0, 2**64, size=(len(sets), P, 2), dtype=np.uint64)
+            pf = sc.sets_to_masks(sets, P)
+            got = run_gpu(x, f, "sum", pf, None, roots, 0, allreduce, flags)
+            want = run_oracle(x, f, "sum", pf, None, roots, 0, allreduce)
+            assert_same(got, want, f"P={P} f={f}")
+
+
+@pytest.mark.parametrize("flags", KERNELS)
+@pytest.mark.parametrize("allreduce", [False, True])
+def test_exhaustive_inop_victim_and_round(flags, allreduce):
+    """Every (victim, round) with zero or one pre-operation failure."""
+    for P, f in ((7, 1), (11, 2), (14, 3)):
+        R = O.schedule(P, f)["rounds_attempt" if allreduce else "rounds_reduce"]
+        cases = []
+        for victim in range(P):
+            for t in range(0, 2 * R + 2):
+                cases.append(((), victim, t))
+                cases.append((((victim + 3) % P,), victim, t))
+                cases.append(((0,), victim, t))
+        S = len(cases)
+        x = np.random.Generator(np.random.PCG64(P)).integers(0, 2**64, size=(S, P, 2), dtype=np.uint64)
+        pf = sc.sets_to_masks([c[0] for c in cases], P)
+        inop = np.zeros((S, 2, 2), dtype=np.uint32)
+        inop[:, 0, 0] = [c[1] for c in cases]
+        inop[:, 0, 1] = [c[2] for c in cases]
+        inop[:, 1, 0] = sc.UNUSED
+        got = run_gpu(x, f, "sum", pf, inop, None, 0, allreduce, flags)
+        want = run_oracle(x, f, "sum", pf, inop, None, 0, allreduce)
+        assert_same(got, want, f"P={P} f={f}")
+
+
+DT = {"i32": np.int32, "i64": np.int64, "u64": np.uint64, "f32": np.float32}
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_shapes_ops_and_failure_patterns(seed):
+    """Random (P, f, k, dtype, op), up to f+2 pre-operation failures, up to 3 in-operation failures (victims may
+    repeat, may be pre-failed, may be the reduce root), per-scenario roots, both collectives, both kernels."""
+    rng = np.random.Generator(np.random.PCG64(1000 + seed))
+    for _ in range(10):
+        f = int(rng.integers(0, 6))
+        P = int(rng.integers(f + 2, 400))
+        dname = ["i32", "i64", "u64", "f32"][int(rng.integers(0, 4))]
+        op = "sum" if dname == "f32" else ["sum", "max", "xor"][int(rng.integers(0, 3))]
+        k = int(rng.choice([1, 2, 3, 4, 8, 12, 16, 32, 64, 128] if DT[dname]().itemsize == 4 else [1, 2, 3, 4, 6, 8, 16, 64]))
+        S = 40
+        allred = bool(rng.integers(0, 2))
+        if dname == "f32":
+            x = rng.standard_normal((S, P, k)).astype(np.float32)
+        else:
+            info = np.iinfo(DT[dname])
+            x = rng.integers(info.min, info.max, size=(S, P, k), dtype=DT[dname], endpoint=True)
+        sizes = rng.integers(0, f + 3, size=S)
+        pf = sc.picks_to_masks(sc.random_subsets(rng, S, P, np.minimum(sizes, P - 1)), P)
+        R = O.schedule(P, f)["rounds_attempt"]
+        inop = np.zeros((S, 3, 2), dtype=np.uint32)
+        lo = f + 1 if allred and P > f + 2 else 0
+        inop[:, :, 0] = rng.integers(lo, P, size=(S, 3))
+        inop[:, :, 1] = rng.integers(0, 2 * R + 2, size=(S, 3))
+        inop[rng.random((S, 3)) < 0.4, 0] = sc.UNUSED
+        roots = rng.integers(0, P, size=S).astype(np.uint32)
+        if allred and lo:
+            roots = rng.integers(0, 1, size=S).astype(np.uint32)      # candidates 0..f stay clear of the victims
+        for flags in KERNELS:
+            got = run_gpu(x, f, op, pf, inop, roots, 0, allred, flags)
+            want = run_oracle(x, f, op, pf, inop, roots, 0, allred)
+            assert_same(got, want, f"P={P} f={f} k={k} {dname} {op} allreduce={allred} flags={flags:#x}")
+
+
+def test_chunk_counts_up_to_32_and_beyond():
+    """k*elem = 16 B .. 512 B run on the tiled kernel, larger or odd sizes on the general one."""
+    rng = np.random.Generator(np.random.PCG64(3))
+    P, f, S = 300, 2, 16
+    pf = sc.picks_to_masks(sc.random_subsets(rng, S, P, rng.integers(0, 3, size=S)), P)
+    for k, kernel in ((4, "tiled"), (8, "tiled"), (16, "tiled"), (32, "tiled"), (64, "tiled"), (128, "tiled"),
+                      (256, "generic"), (20, "generic"), (5, "generic")):
+        x = rng.integers(-2**31, 2**31 - 1, size=(S, P, k), dtype=np.int32)
+        got = run_gpu(x, f, "max", pf)
+        assert B.ftc_kernel_name(got[2]) == kernel
+        assert_same(got, run_oracle(x, f, "max", pf), f"k={k}")
+
+
+def test_wide_groups_f_up_to_31():
+    rng = np.random.Generator(np.random.PCG64(8))
+    for f in (9, 12, 31):
+        P, S, k = 40 * (f + 1) + 5, 12, 4
+        x = rng.integers(0, 2**64, size=(S, P, k), dtype=np.uint64)
+        pf = sc.picks_to_masks(sc.random_subsets(rng, S, P, rng.integers(0, f + 1, size=S)), P)
+        for allred in (False, True):
+            for flags in KERNELS:
+                assert_same(run_gpu(x, f, "sum", pf, allreduce=allred, flags=flags),
+                            run_oracle(x, f, "sum", pf, allreduce=allred), f"f={f}")
+
+
+def test_empty_batch_and_argument_errors():
+    import torch
+    d = B.make_desc(8, 1, 4, B.FTC_I32, "sum")
+    z = torch.zeros(16, dtype=torch.int32, device="cuda")
+    assert B.ftc_reduce_batch(d, 0, None, None, None, None, None, None) == B.FTC_OK
+    bad = [B.make_desc(2, 1, 4, B.FTC_I32, "sum"), B.make_desc(8, 1, 0, B.FTC_I32, "sum"),
+           B.make_desc(8, 1, 4, B.FTC_I32, "sum", root=8), B.make_desc(8, 32, 4, B.FTC_I32, "sum"),
+           B.make_desc(64, 1, 4, B.FTC_I32, "sum", max_inop=33)]
+    for desc in bad:
+        assert B.ftc_reduce_batch(desc, 1, z, z, z, z, z, z, check=False) == B.FTC_EINVAL
+    assert B.ftc_reduce_batch(B.make_desc(8, 1, 4, B.FTC_F32, "xor"), 1, z, z, z, z, z, z, check=False) == B.FTC_EUNSUPPORTED
+    assert B.ftc_reduce_batch(B.make_desc(8, 1, 4, 9, "sum"), 1, z, z, z, z, z, z, check=False) == B.FTC_EUNSUPPORTED
+    assert B.ftc_reduce_batch(d, 1, None, z, None, None, z, z, check=False) == B.FTC_EINVAL
+    assert B.ftc_reduce_batch(B.make_desc(8, 1, 4, B.FTC_I32, "sum", root=-1), 1, z, z, None, None, z, z, check=False) == B.FTC_EINVAL
+    assert B.ftc_reduce_batch(d, 1, z[1:], z, None, None, z, z, check=False) == B.FTC_EINVAL          # misaligned
+    g = B.make_desc(8, 1, 1, B.FTC_I32, "sum")                                                          # needs workspace
+    assert B.ftc_workspace_bytes(g, 4) > 0
+    assert B.ftc_reduce_batch(g, 4, z, z, None, None, z, z, None, check=False) == B.FTC_EWORKSPACE
+    with pytest.raises(B.FtcError):
+        B.ftc_reduce_batch(g, 4, z, z, None, None, z, z, None)
+    torch.cuda.synchronize()
+
+
+def test_bad_per_scenario_root_is_a_status_not_an_error():
+    rng = np.random.Generator(np.random.PCG64(2))
+    x = rng.integers(0, 100, size=(3, 10, 4), dtype=np.int32)
+    pf = np.zeros((3, 1), dtype=np.uint32)
+    out, st, _ = run_gpu(x, 1, "sum", pf, roots=np.array([2, 10, 9], dtype=np.uint32))
+    assert (st[:, 0] & 0xFF).tolist() == [0, B.FTC_ST_BAD_ROOT, 0] and not out[1].any()
+    assert np.array_equal(out[0], x[0].sum(axis=0)) and np.array_equal(out[2], x[2].sum(axis=0))
+
+
+def test_mask_bits_beyond_P_are_ignored():
+    P, f = 40, 2
+    x = np.random.Generator(np.random.PCG64(2)).integers(0, 2**64, size=(2, P, 2), dtype=np.uint64)
+    pf = np.zeros((2, 2), dtype=np.uint32)
+    pf[1, 1] = 0xFFFFFF00                    # bits 40..63
+    out, st, _ = run_gpu(x, f, "sum", pf)
+    want = run_oracle(x, f, "sum", np.zeros((2, 2), dtype=np.uint32))
+    assert_same((out, st), want)
+
+
+def test_device_input_generator_matches_host_generator():
+    import torch
+    for kind, tdt in ((sc.KIND_I32_PM20, torch.int32), (sc.KIND_I64_PM40, torch.int64), (sc.KIND_F32_NORMAL, torch.float32),
+                      (sc.KIND_I32_FULL, torch.int32), (sc.KIND_U64_FULL, torch.uint64)):
+        S, P, k, first = 5, 70, 6, 123456
+        d = torch.empty((S, P, k), dtype=tdt, device="cuda")
+        B.ftc_fill_inputs(kind, 0xABCDEF12345, first, S, P, k, d)
+        torch.cuda.synchronize()
+        host = sc.gen_inputs(kind, 0xABCDEF12345, np.arange(S) + first, P, k)
+        got = to_host(d, host.dtype)
+        assert np.array_equal(got.view(np.uint8), host.view(np.uint8)), kind
+
+
+def test_host_buffer_entry_points_match_device_ones():
+    import torch
+    ratt = O.schedule(4096, 4)["rounds_attempt"]
+    w = sc.config4(ratt, S=40)
+    x = w.host_inputs()
+    desc = B.make_desc(w.P, w.f, w.k, B.FTC_I32, "max", max_inop=2)
+    out = np.full((w.S, w.k), 7, dtype=np.int32)
+    st = np.full((w.S, 4), 7, dtype=np.uint32)
+    nbytes = B.ftc_host_staging_bytes(desc, 16)                 # forces three chunks
+    staging = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    B.ftc_allreduce_batch_host(desc, w.S, x, w.prefail, np.ascontiguousarray(w.inop), None, out, st, staging)
+    assert_same((out, st), run_oracle(x, w.f, "max", w.prefail, w.inop, None, 0, True), "host variant")
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    assert B.ftc_allreduce_batch_host(desc, w.S, x, w.prefail, np.ascontiguousarray(w.inop), None, out, st, small,
+                                      check=False) == B.FTC_EWORKSPACE

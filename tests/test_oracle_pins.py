@@ -473,3 +473,17 @@ def test_reading_broadcast_correction_is_sent_by_tree_holders_only():
     assert first_corr + 2 == sch["rounds_attempt"] and K.bits(d["holders"], 10) == [0, 1, 4, 5, 6, 7, 8, 9]
     d = O.run(x, 2, "sum", [2, 3], inop=[(4, first_corr)], allreduce=True, detail=True, track_sets=True)
     assert K.bits(d["holders"], 10) == [0, 1, 7, 8, 9]
+
+
+def test_leaf_has_no_tree_down_send_to_miss():
+    """f = 0: the deepest leaves would send down the tree in the round the attempt ends; they have no
+    children, so a failure round equal to the attempt's length leaves them alive and holding the value."""
+    n = 12
+    x = rand_u64(n, 1, 6)
+    sch = O.schedule(n, 0)
+    assert sch["rounds_attempt"] == 2 * sch["H"]
+    leaf = n - 1
+    d = O.run(x, 0, "sum", [], inop=[(leaf, sch["rounds_attempt"])], allreduce=True, detail=True)
+    assert d["n_holders"] == n and leaf in K.bits(d["holders"], n)
+    d = O.run(x, 0, "sum", [], inop=[(leaf, sch["rounds_attempt"] - 1)], allreduce=True, detail=True)
+    assert d["n_holders"] == n - 1 and leaf not in K.bits(d["holders"], n)
