@@ -85,10 +85,25 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(gpu_index)],
+                                          "-lms", "50", "-i", str(gpu_index)],
                                          stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
+
+    def lines(self) -> int:
+        try:
+            return sum(1 for _ in open(self.path))
+        except OSError:
+            return 0
+
+    def wait_ready(self, timeout: float = 5.0) -> None:
+        t0 = time.time()
+        while self.proc is not None and self.lines() == 0 and time.time() - t0 < timeout:
+            time.sleep(0.05)
+
+    def mark(self) -> None:
+        """Samples from here on count (the timed region starts)."""
+        self.first = self.lines()
 
     def stop(self) -> dict:
         if self.proc is None:
@@ -99,7 +114,9 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
-        for line in open(self.path):
+        for ln, line in enumerate(open(self.path)):
+            if ln < getattr(self, "first", 0):
+                continue
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 9:
                 continue
@@ -118,14 +135,19 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 # CPU oracle timing (cpu_baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------
-def time_oracle(w, n_scen: int, chunk: int):
-    """Runs the oracle, as it stands, over the first n_scen scenarios of w on all host cores (threads; the C call
-    releases the GIL). Inputs come from the host generator and are prepared before the clock starts."""
+def prepare_oracle(w, n_scen: int, chunk: int):
+    """Host inputs of the first n_scen scenarios of w, in chunks (prepared before any clock starts)."""
+    ids = [np.arange(s, min(s + chunk, n_scen)) for s in range(0, n_scen, chunk)]
+    return ids, [w.host_inputs(i) for i in ids]
+
+
+def time_oracle(w, prepared):
+    """Runs the oracle, as it stands, over the prepared scenarios on all host cores (threads; the C call releases
+    the GIL). Returns (scenarios/s, seconds, threads used)."""
     from oracle import oracle as orc
     orc.lib()
+    ids, xs = prepared
     cores = os.cpu_count() or 1
-    ids = [np.arange(s, min(s + chunk, n_scen)) for s in range(0, n_scen, chunk)]
-    xs = [w.host_inputs(i) for i in ids]
     allred = w.collective == "allreduce"
 
     def work(j):
@@ -137,10 +159,11 @@ def time_oracle(w, n_scen: int, chunk: int):
     with ThreadPoolExecutor(max_workers=cores) as ex:
         list(ex.map(work, range(len(ids))))
     dt = time.perf_counter() - t0
+    n_scen = sum(len(i) for i in ids)
     return n_scen / dt, dt, min(cores, len(ids))
 
 
-ORACLE_SAMPLE = {"c3": (16384, 256), "c4": (4096, 64), "c5": (128, 2), "c5r": (128, 2)}
+ORACLE_SAMPLE = {"c3": (32768, 256), "c4": (8192, 64), "c5": (192, 2), "c5r": (192, 2)}
 
 
 def run_reference(args):
@@ -149,13 +172,18 @@ def run_reference(args):
         return
     from oracle import oracle as orc
     sched = orc.schedule(*{"c3": (1024, 3), "c4": (4096, 4), "c5": (65536, 8), "c5r": (65536, 8)}[args.workload])
-    n, chunk = ORACLE_SAMPLE[args.workload]
-    n = max(chunk, n // 4)                      # one step = a quarter of the cpu_baseline sample
-    w = make_workload(args.workload, n, 0, sched["rounds_attempt"])
+    n_max, chunk = ORACLE_SAMPLE[args.workload]
+    w = make_workload(args.workload, n_max, 0, sched["rounds_attempt"])
+    cores = os.cpu_count() or 1
+    # size one step so that the whole run stays near two minutes: probe the rate on one chunk per core first
+    probe = prepare_oracle(w, min(n_max, chunk * cores), chunk)
+    rate, _, _ = time_oracle(w, probe)
+    n = int(rate * 120.0 / max(1, args.steps + args.warmup))
+    n = max(chunk, min(n_max, (n // chunk) * chunk))
+    prepared = prepare_oracle(w, n, chunk)
     times = []
-    cores = 1
     for it in range(args.warmup + args.steps):
-        rate, dt, cores = time_oracle(w, n, chunk)
+        rate, dt, cores = time_oracle(w, prepared)
         if it >= args.warmup:
             times.append(dt)
     ms = 1e3 * sum(times) / len(times)
@@ -226,12 +254,16 @@ def run_gpu(args):
     def step():
         fn(desc, S, d_x, d_pf, d_inop, d_roots, d_out, d_st, d_ws)
 
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.wait_ready()
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
     if dist:
         dist.barrier()
-    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.mark()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     torch.cuda.synchronize()
     ev[0].record()
@@ -251,36 +283,40 @@ def run_gpu(args):
     ms_per_step = total_ms / args.steps
     value = world * S / (ms_per_step / 1e3)
 
-    # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region) ----
-    Se = min(S, args.e2e_scenarios or max(64, (1 << 30) // (w.P * w.k * ESZ[np.dtype(w.dtype).name])))
-    we = make_workload(name, Se, rank * S, sched["rounds_attempt"])
-    h_x = torch.empty((Se, w.P, w.k), dtype=tdt).pin_memory()
-    h_x.copy_(d_x[:Se])                                                   # same synthetic inputs, now resident on the host
-    h_pf = torch.from_numpy(we.prefail.view(np.int32)).pin_memory()
-    h_inop = None if we.inop is None else torch.from_numpy(np.ascontiguousarray(we.inop).view(np.int32)).pin_memory()
-    h_roots = None if we.roots is None else torch.from_numpy(we.roots.view(np.int32)).pin_memory()
-    h_out = torch.empty((Se, w.k), dtype=tdt).pin_memory()
-    h_st = torch.empty((Se, 4), dtype=torch.int32).pin_memory()
-    staging = torch.empty(B.ftc_host_staging_bytes(desc, Se), dtype=torch.uint8, device="cuda")
-    fn_host = B.ftc_allreduce_batch_host if allred else B.ftc_reduce_batch_host
-    e2e_steps = max(2, min(args.steps, 5))
-    fn_host(desc, Se, h_x, h_pf, h_inop, h_roots, h_out, h_st, staging)
-    torch.cuda.synchronize()
-    if dist:
-        dist.barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        fn_host(desc, Se, h_x, h_pf, h_inop, h_roots, h_out, h_st, staging)     # synchronises its stream itself
-    e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if dist:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    h2d = Se * (bytes_per_scenario(w) - w.k * ESZ[np.dtype(w.dtype).name] - 16)
-    d2h = Se * (w.k * ESZ[np.dtype(w.dtype).name] + 16)
-    same = bool((h_st.numpy() == d_st[:Se].cpu().numpy()).all() and
-                (h_out.view(torch.uint8).numpy() == d_out[:Se].cpu().view(torch.uint8).numpy()).all())
+    e2e = None
+    if not args.kernel_only:
+        # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region) ----
+        Se = min(S, args.e2e_scenarios or max(64, (1 << 30) // (w.P * w.k * ESZ[np.dtype(w.dtype).name])))
+        we = w
+        h_x = torch.empty((Se, w.P, w.k), dtype=tdt).pin_memory()
+        h_x.copy_(d_x[:Se])                                                   # same synthetic inputs, now resident on the host
+        h_pf = torch.from_numpy(np.ascontiguousarray(we.prefail[:Se]).view(np.int32)).pin_memory()
+        h_inop = None if we.inop is None else torch.from_numpy(np.ascontiguousarray(we.inop[:Se]).view(np.int32)).pin_memory()
+        h_roots = None if we.roots is None else torch.from_numpy(np.ascontiguousarray(we.roots[:Se]).view(np.int32)).pin_memory()
+        h_out = torch.empty((Se, w.k), dtype=tdt).pin_memory()
+        h_st = torch.empty((Se, 4), dtype=torch.int32).pin_memory()
+        staging = torch.empty(B.ftc_host_staging_bytes(desc, Se), dtype=torch.uint8, device="cuda")
+        fn_host = B.ftc_allreduce_batch_host if allred else B.ftc_reduce_batch_host
+        e2e_steps = max(2, min(args.steps, 5))
+        fn_host(desc, Se, h_x, h_pf, h_inop, h_roots, h_out, h_st, staging)
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            fn_host(desc, Se, h_x, h_pf, h_inop, h_roots, h_out, h_st, staging)     # synchronises its stream itself
+        e2e_s = (time.perf_counter() - t0) / e2e_steps
+        if dist:
+            t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        h2d = Se * (bytes_per_scenario(w) - w.k * ESZ[np.dtype(w.dtype).name] - 16)
+        d2h = Se * (w.k * ESZ[np.dtype(w.dtype).name] + 16)
+        same = bool((h_st.numpy() == d_st[:Se].cpu().numpy()).all() and
+                    (h_out.view(torch.uint8).numpy() == d_out[:Se].cpu().view(torch.uint8).numpy()).all())
 
+        e2e = {"value": world * Se / e2e_s, "unit": "scenarios/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "scenarios_per_step": Se, "matches_device_run": same}
     if rank != 0:
         if dist:
             dist.destroy_process_group()
@@ -304,10 +340,10 @@ def run_gpu(args):
 
     # ---- the oracle beside it, on a bounded sample ----
     cpu = None
-    if not args.no_cpu_baseline:
+    if not (args.no_cpu_baseline or args.kernel_only):
         n, chunk = ORACLE_SAMPLE[name]
         wo = make_workload(name, n, 0, sched["rounds_attempt"])
-        rate, dt, cores = time_oracle(wo, n, chunk)
+        rate, dt, cores = time_oracle(wo, prepare_oracle(wo, n, chunk))
         cpu = {"value": rate, "unit": "scenarios/s", "cores": cores, "kind": "oracle",
                "sample": f"first {n} scenarios of the workload ({dt:.1f} s wall on {cores} threads)"}
 
@@ -328,8 +364,7 @@ def run_gpu(args):
                      "bytes_per_launch": bytes_launch, "avg_launch_ms": avg_launch_ms,
                      "min_launch_ms": min(per_launch_ms)},
         "cpu_baseline": cpu,
-        "e2e": {"value": world * Se / e2e_s, "unit": "scenarios/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "scenarios_per_step": Se, "matches_device_run": same},
+        "e2e": e2e,
         "gpu_launches": args.steps,
         "clocks": clocks,
     }
@@ -341,13 +376,14 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c4", choices=sorted(DESCRIPTION))
     ap.add_argument("--batch", type=int, default=0, help="scenarios per step per GPU")
     ap.add_argument("--e2e-scenarios", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU legs (for profiler runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
