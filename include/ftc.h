@@ -79,7 +79,8 @@ enum {
     FTC_ST_NO_CLEAN_SUBTREE = 2,        /* Algorithm "reduce_root": "No failure-free subtree" (needs > f failures) */
     FTC_ST_NO_LIVE_ROOT_CANDIDATE = 3,  /* allreduce: all f+1 candidates had failed before the operation */
     FTC_ST_PRECONDITION_INOP_ROOT = 4,  /* allreduce: a root candidate is listed as failing in-operation */
-    FTC_ST_BAD_ROOT = 5                 /* d_roots[s] >= P */
+    FTC_ST_BAD_ROOT = 5,                /* d_roots[s] >= P */
+    FTC_ST_INTERNAL_TIMEOUT = 6         /* a bounded wait inside the kernel ran out; the scenario's result is not valid */
 };
 
 /*
@@ -103,6 +104,7 @@ typedef struct { uint32_t victim; uint32_t round; } ftc_inop_t;
 /* flags */
 #define FTC_OUT_EXPANDED   0x1u   /* allreduce: d_out is [S][P][k], zeros for processes that do not hold the result */
 #define FTC_KERNEL_GENERIC 0x100u /* force the general level-by-level kernel (needs the workspace) */
+#define FTC_KERNEL_DIRECT  0x200u /* force the register-tiled kernel (direct global loads) where the shape allows it */
 
 typedef struct {
     uint32_t P;         /* processes, P >= f+2 (the root needs f+1 children: definition of the I(f)-tree) */
@@ -184,7 +186,7 @@ FTC_API int ftc_schedule_info(const ftc_desc_t* desc, ftc_sched_t* out);
 FTC_API int ftc_fill_inputs(uint32_t kind, uint64_t seed, uint64_t first_scenario, uint64_t S, uint32_t P, uint32_t k,
                     void* d_out, void* cuda_stream);
 
-/* Name of the kernel family the batch calls would use for this descriptor: "tiled" or "generic". */
+/* Name of the kernel family the batch calls would use for this descriptor: "staged", "tiled" or "generic". */
 FTC_API const char* ftc_kernel_name(const ftc_desc_t* desc, int is_allreduce);
 
 FTC_API const char* ftc_strerror(int code);

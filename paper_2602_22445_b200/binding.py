@@ -18,11 +18,12 @@ FTC_I32, FTC_I64, FTC_U64, FTC_F32 = 0, 1, 2, 3
 FTC_SUM, FTC_MAX, FTC_XOR = 0, 1, 2
 FTC_OK, FTC_EINVAL, FTC_EUNSUPPORTED, FTC_EWORKSPACE, FTC_ECUDA = 0, -1, -2, -3, -4
 FTC_ST_OK, FTC_ST_ROOT_FAILED, FTC_ST_NO_CLEAN_SUBTREE, FTC_ST_NO_LIVE_ROOT_CANDIDATE = 0, 1, 2, 3
-FTC_ST_PRECONDITION_INOP_ROOT, FTC_ST_BAD_ROOT = 4, 5
+FTC_ST_PRECONDITION_INOP_ROOT, FTC_ST_BAD_ROOT, FTC_ST_INTERNAL_TIMEOUT = 4, 5, 6
 FTC_STATUS_WORDS = 4
 FTC_INOP_UNUSED = 0xFFFFFFFF
 FTC_OUT_EXPANDED = 0x1
 FTC_KERNEL_GENERIC = 0x100
+FTC_KERNEL_DIRECT = 0x200
 OPS = {"sum": FTC_SUM, "max": FTC_MAX, "xor": FTC_XOR}
 
 EXPORTS = ["ftc_reduce_batch", "ftc_allreduce_batch", "ftc_workspace_bytes", "ftc_reduce_batch_host",

@@ -51,13 +51,15 @@ static int device_info(DeviceInfo& di) {
 // B200 figures, used where no device can be asked (sizing queries on a machine without a GPU).
 static const DeviceInfo kB200 = {148, 232448};
 
-static bool use_tiled(Params& p, const DeviceInfo& di) {
-    if (p.flags & FTC_KERNEL_GENERIC) return false;
-    return tiled_supported(p, di.smem_optin);
+enum KernelKind { K_GENERIC = 0, K_TILED = 1, K_STAGED = 2 };
+static KernelKind pick_kernel(Params& p, const DeviceInfo& di) {
+    if (p.flags & FTC_KERNEL_GENERIC) return K_GENERIC;
+    if (!(p.flags & FTC_KERNEL_DIRECT) && staged_supported(p, di.smem_optin)) return K_STAGED;
+    return tiled_supported(p, di.smem_optin) ? K_TILED : K_GENERIC;
 }
 
 static size_t workspace_for(Params& p, const DeviceInfo& di) {
-    if (use_tiled(p, di)) return 0;
+    if (pick_kernel(p, di) != K_GENERIC) return 0;
     return (size_t)generic_grid(p, di.sm_count) * p.Gmax * p.kbytes;
 }
 
@@ -81,7 +83,10 @@ static int run_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const
     const int tsel = type_select(desc->dtype, desc->op);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
-    if (use_tiled(p, di)) {
+    const KernelKind kind = pick_kernel(p, di);
+    if (kind == K_STAGED) {
+        e = launch_staged(p, tsel, di.sm_count, di.smem_optin, st);
+    } else if (kind == K_TILED) {
         e = launch_tiled(p, tsel, di.sm_count, st);
     } else {
         const size_t need = (size_t)generic_grid(p, di.sm_count) * p.Gmax * p.kbytes;
@@ -221,7 +226,8 @@ const char* ftc_kernel_name(const ftc_desc_t* desc, int is_allreduce) {
     if (fill_params(desc, 1, is_allreduce, p) != FTC_OK) return "invalid";
     DeviceInfo di;
     if (device_info(di) != FTC_OK) di = kB200;
-    return use_tiled(p, di) ? "tiled" : "generic";
+    const KernelKind kind = pick_kernel(p, di);
+    return kind == K_STAGED ? "staged" : kind == K_TILED ? "tiled" : "generic";
 }
 
 const char* ftc_strerror(int code) {

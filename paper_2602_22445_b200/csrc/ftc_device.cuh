@@ -44,7 +44,7 @@ struct Ctx {
     uint32_t holders;
     uint32_t ndead_end; // in-operation victims (not pre-failed) that are dead at the end of the attempt
     uint32_t unreached_lost;
-    uint32_t pad;
+    uint32_t pad;       // set when a bounded wait gave up
     uint32_t iv[FTC_MAX_INOP];   // victim (physical id) per slot, FTC_INOP_UNUSED if the slot does not count
     uint32_t ir[FTC_MAX_INOP];   // its failure round on the global clock (minimum over slots naming it)
     uint32_t ifirst;             // bit i: slot i is the first slot naming its victim
@@ -98,7 +98,7 @@ static __device__ void decode_scenario(const Params& p, uint64_t s, Ctx* cx, uin
     if (tid == 0) {
         cx->Fmask = 0; cx->npre = 0; cx->nexcl = 0; cx->inop_incl = 0; cx->holders = 0; cx->ndead_end = 0;
         cx->unreached_lost = 0; cx->code = FTC_ST_OK; cx->sstar = 0xFF; cx->attempts = 0; cx->base = 0; cx->root = 0;
-        cx->G = 0; cx->ifirst = 0;
+        cx->G = 0; cx->ifirst = 0; cx->pad = 0;
         pf[p.W] = 0; inc[p.W] = 0;
     }
     if (tid < FTC_MAX_INOP) {

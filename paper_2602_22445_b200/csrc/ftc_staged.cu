@@ -1,0 +1,323 @@
+// Staged kernel: the main fast path. Same decomposition as the register-tiled kernel (one block per scenario,
+// the selected subtree's heap of up-correction groups cut into warp tiles, levels above the tiles combined in
+// shared memory), but the input bytes of a tile travel global -> shared memory as a few large asynchronous bulk
+// copies (one per heap level of the tile: each level of a sub-heap is one contiguous run of rows), tracked by an
+// mbarrier per buffer. A warp keeps one tile in flight per buffer while it works on another, so the bytes in
+// flight do not depend on registers, and no lane spends instructions on global addresses.
+//
+// A tile has lw + XL levels (lw = log2 of the lane rows, 32 / chunks per vector): each lane row evaluates a
+// sub-heap of XL levels by itself (post-order, values in registers), the lw levels above are combined with warp
+// shuffles. Groups that are not "plain" (a missing member, a renumbered slot, the short last group) are folded
+// from global memory by the general routine; they are a handful per scenario.
+#include <cstdlib>
+#include "ftc_tile_common.cuh"
+#include "ftc_kernels.h"
+
+namespace ftc {
+
+// ---- mbarrier / bulk-copy primitives (shared::cta addresses as 32-bit) ----
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kWaitTries polls and reports it; the caller flags the scenario and carries on so
+// that block-wide barriers stay matched.
+constexpr uint32_t kWaitTries = 1u << 22;
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitTries; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+struct LdShared {
+    __device__ __forceinline__ uint4 operator()(const char* q) const { return *reinterpret_cast<const uint4*>(q); }
+};
+
+struct StagedGeom {
+    uint32_t nwarps, nbuf, tile_cap;       // warps per block, buffers per warp, bytes per buffer (multiple of 128)
+    uint32_t off_special, off_rootv, off_hv, off_bar, off_tiles, smem_bytes;
+};
+
+// The rare groups that are not plain: folded from global memory by the general routine. Kept out of line so that
+// the common path stays small in code and registers.
+template <typename T, int OP>
+__device__ __noinline__ uint4 fold_special(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
+                                           const char* in_lc, uint32_t row) {
+    return fold16_general<T, OP, 0>(p, root, sstar, inc, in_lc, row);
+}
+
+// Fold of one group, chunk lc: from the staged copy when the group is plain, else from global memory.
+template <typename T, int OP>
+__device__ __forceinline__ uint4 fold_staged(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
+                                             const char* in_lc, const char* srow_lc, uint32_t row) {
+    if (group_is_plain(p, root, inc, row)) {
+        uint4 acc;
+        if (Ordered<T>::value) {
+            acc = LdShared()(srow_lc + sstar * p.kbytes);
+#pragma unroll 4
+            for (uint32_t sp = 0; sp < p.m; ++sp)
+                if (sp != sstar) acc = comb16<T, OP>(acc, LdShared()(srow_lc + sp * p.kbytes));
+        } else {
+            acc = LdShared()(srow_lc);
+#pragma unroll 4
+            for (uint32_t sp = 1; sp < p.m; ++sp) acc = comb16<T, OP>(acc, LdShared()(srow_lc + sp * p.kbytes));
+        }
+        return acc;
+    }
+    return fold_special<T, OP>(p, root, sstar, inc, in_lc, row);
+}
+
+// Value of the node at level u (of XL) of a lane's sub-heap: its group's fold, then child 1, then child 2.
+// trow/grow: tile-heap index and global row of the node.
+template <typename T, int OP, int XL, int U>
+struct SubHeap {
+    static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
+                                                 const char* in_lc, const char* buf_lc, uint32_t rowbytes,
+                                                 uint32_t trow, uint32_t grow, uint32_t G) {
+        uint4 v = fold_staged<T, OP>(p, root, sstar, inc, in_lc, buf_lc + trow * rowbytes, grow);
+        if (U + 1 < XL) {
+            if (2 * grow + 1 < G)
+                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U)>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
+            if (2 * grow + 2 < G)
+                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U)>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
+        }
+        return v;
+    }
+};
+
+constexpr int kStagedMaxThreads = 512;
+
+template <typename T, int OP, int XL>
+__global__ void __launch_bounds__(kStagedMaxThreads) staged_kernel(Params p, StagedGeom g) {
+    extern __shared__ __align__(128) uint32_t smem[];
+    char* sbase = reinterpret_cast<char*>(smem);
+    Ctx* cx = reinterpret_cast<Ctx*>(smem);
+    uint32_t* pf = smem + sizeof(Ctx) / 4;
+    uint32_t* inc = pf + p.W + 1;
+    uint32_t* unr = inc + p.W + 1;
+    uint4* rootv = reinterpret_cast<uint4*>(sbase + g.off_rootv);
+    uint4* hv = reinterpret_cast<uint4*>(sbase + g.off_hv);
+
+    const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
+    const uint32_t cwl = p.cw_log2, lw = 5 - cwl, RW = 1u << lw, Cmask = p.C - 1;
+    const uint32_t lr = lane >> cwl, lc = lane & Cmask;
+    const uint32_t D = lw + XL;                                   // levels of a tile
+    const uint32_t Lt = p.Lt, ntiles = 1u << Lt, ntop = ntiles - 1, ngroups = (ntop + RW - 1) >> lw;
+    const uint32_t nitems = ntiles + ngroups + 1;
+    const uint32_t rowbytes = p.m * p.kbytes;
+    const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
+
+    const uint32_t bar0 = smem_addr(sbase + g.off_bar) + wid * g.nbuf * 8;
+    char* tiles = sbase + g.off_tiles + (size_t)wid * g.nbuf * g.tile_cap;
+    if (lane < g.nbuf) mbar_init(bar0 + lane * 8, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    uint32_t phase_bits = 0;                                      // bit b: parity to wait for on buffer b
+
+    for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {
+        decode_scenario(p, s, cx, pf, inc);
+        char* out_s = reinterpret_cast<char*>(p.out) + s * p.kbytes;
+        if (cx->code != FTC_ST_OK) {
+            if (tid < p.C) reinterpret_cast<uint4*>(out_s)[tid] = make_uint4(0, 0, 0, 0);
+            if (tid == 0) write_status_rec(p, s, cx);
+            __syncthreads();
+            continue;
+        }
+        if (p.is_allreduce) count_holders(p, cx, pf, unr);
+        const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
+        const char* in_s = reinterpret_cast<const char*>(p.in) + s * scen_bytes;
+        const char* in_lc = in_s + lc * 16;
+
+        // Issue the bulk copies of work item `it` into buffer b: lane t copies level t of the tile.
+        auto issue = [&](uint32_t it, uint32_t b) {
+            uint32_t first_row = 0, nrows = 0, dst_off = 0;
+            if (it < ntiles) {
+                const uint32_t j0 = ntop + it;
+                if (lane < D && j0 < G) { first_row = ((j0 + 1) << lane) - 1; nrows = 1u << lane; dst_off = ((1u << lane) - 1) * rowbytes; }
+            } else if (it < ntiles + ngroups) {
+                if (lane == 0) { first_row = (it - ntiles) << lw; nrows = min(RW, ntop - first_row); }
+            }
+            uint64_t b0 = ((uint64_t)first_row * p.m + 1) * p.kbytes, b1 = ((uint64_t)(first_row + nrows) * p.m + 1) * p.kbytes;
+            if (b1 > scen_bytes) b1 = scen_bytes;
+            const uint32_t bytes = (nrows && b1 > b0) ? (uint32_t)(b1 - b0) : 0u;
+            const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, bytes);
+            if (total) {
+                if (lane == 0) mbar_expect_tx(bar0 + b * 8, total);
+                __syncwarp();
+                if (bytes) bulk_g2s(smem_addr(tiles + (size_t)b * g.tile_cap + dst_off), in_s + b0, bytes, bar0 + b * 8);
+            }
+            return total != 0;
+        };
+
+        const uint32_t n_my = wid < nitems ? (nitems - wid + nw - 1) / nw : 0;
+        uint32_t pending = 0;                                     // bit b: buffer b has a copy in flight
+        for (uint32_t i = 0; i < g.nbuf && i < n_my; ++i)
+            if (issue(wid + i * nw, i)) pending |= 1u << i;
+
+        for (uint32_t i = 0; i < n_my; ++i) {
+            const uint32_t it = wid + i * nw, b = i % g.nbuf;
+            if ((pending >> b) & 1u) {
+                if (!mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u)) { if (lane == 0) atomicOr(&cx->pad, 1u); }
+                phase_bits ^= 1u << b; pending &= ~(1u << b);
+            }
+            const char* buf_lc = tiles + (size_t)b * g.tile_cap + lc * 16;
+            if (it < ntiles) {
+                const uint32_t j0 = ntop + it;
+                if (j0 < G) {
+                    // bottom part: this lane row's sub-heap, rooted at level lw of the tile
+                    const uint32_t tA = RW - 1 + lr, rowA = ((j0 + 1) << lw) - 1 + lr;
+                    uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
+                    if (rowA < G) valA = SubHeap<T, OP, XL, 0>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, tA, rowA, G);
+                    const uint32_t tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB);
+                    const uint32_t rowB = ((j0 + 1) << tB) - 1 + idxB;
+                    const bool hasB = lr < RW - 1 && rowB < G;
+                    if (hasB) valB = fold_staged<T, OP>(p, root, sstar, inc, in_lc, buf_lc + lr * rowbytes, rowB);
+                    valB = tile_tree_phase<T, OP>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
+                    if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
+                }
+            } else if (it < ntiles + ngroups) {
+                const uint32_t row = ((it - ntiles) << lw) + lr;
+                if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged<T, OP>(p, root, sstar, inc, in_lc, buf_lc + lr * rowbytes, row);
+            } else if (sstar >= p.r) {
+                if (lr == 0) rootv[lc] = fold_root16<T, OP>(p, root, inc, in_lc);
+            }
+            __syncwarp();                                         // every lane is done with buffer b
+            if (i + g.nbuf < n_my && issue(wid + (i + g.nbuf) * nw, b)) pending |= 1u << b;
+        }
+        __syncthreads();
+        // ---- levels above the tiles, leaves first (Algorithm "reduce_non_root") ----
+        for (int lvl = (int)Lt - 1; lvl >= 0; --lvl) {
+            const uint32_t lo = (1u << lvl) - 1u, n = min(lo + 1u, G > lo ? G - lo : 0u);
+            for (uint32_t u = tid; u < n * p.C; u += nt) {
+                const uint32_t row = lo + (u >> cwl), c = u & Cmask;
+                uint4 v = hv[(size_t)row * p.C + c];
+                if (2 * row + 1 < G) v = comb16<T, OP>(v, hv[(size_t)(2 * row + 1) * p.C + c]);
+                if (2 * row + 2 < G) v = comb16<T, OP>(v, hv[(size_t)(2 * row + 2) * p.C + c]);
+                hv[(size_t)row * p.C + c] = v;
+            }
+            __syncthreads();
+        }
+        // ---- the root (Algorithm "reduce_root") ----
+        if (tid < p.C) {
+            uint4 recv = hv[tid];
+            reinterpret_cast<uint4*>(out_s)[tid] = sstar < p.r ? recv : comb16<T, OP>(rootv[tid], recv);
+        }
+        if (tid == 0) {
+            if (cx->pad) cx->code = FTC_ST_INTERNAL_TIMEOUT;
+            write_status_rec(p, s, cx);
+        }
+        __syncthreads();
+    }
+}
+
+// ---- host side ----
+static uint32_t env_u32(const char* name, uint32_t dflt) {
+    const char* e = getenv(name);
+    if (!e) return dflt;
+    int v = atoi(e);
+    return v > 0 ? (uint32_t)v : dflt;
+}
+
+static bool staged_geometry(Params& p, int smem_optin, uint32_t XL, StagedGeom& g) {
+    if (p.kbytes % 16) return false;
+    const uint32_t C = p.kbytes / 16;
+    if (C == 0 || C > 32 || (C & (C - 1))) return false;
+    uint32_t cwl = 0; while ((1u << cwl) < C) ++cwl;
+    const uint32_t lw = 5 - cwl, D = lw + XL;
+    uint32_t Hmax = 1; while ((1u << Hmax) <= p.Gmax) ++Hmax;
+    p.C = C; p.cw_log2 = cwl; p.Lt = Hmax > D ? Hmax - D : 0;
+    if (p.Lt > 16) return false;
+    const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
+    const uint64_t cap = ((((uint64_t)1 << D) - 1) * rowbytes + 127) & ~(uint64_t)127;
+    if (cap > 64 * 1024) return false;
+    const uint32_t RW = 1u << lw, ntiles = 1u << p.Lt;
+    const uint32_t nitems = ntiles + ((ntiles - 1 + RW - 1) >> lw) + 1;
+    uint32_t warps = env_u32("FTC_STAGED_WARPS", 0);
+    if (!warps) { warps = 1; while (warps < 8 && warps * 2 * 16 <= nitems) warps *= 2; }   // >= 16 work items per warp
+    if (warps > kStagedMaxThreads / 32) warps = kStagedMaxThreads / 32;
+    uint32_t nbuf = env_u32("FTC_STAGED_NBUF", 1);
+    if (nbuf > 4) nbuf = 4;
+    size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
+    o = (o + 15) & ~(size_t)15; g.off_special = (uint32_t)o;
+    g.off_rootv = (uint32_t)o; o += (size_t)C * 16;
+    g.off_hv = (uint32_t)o; o += (((size_t)2 << p.Lt) - 1) * C * 16;
+    g.off_bar = (uint32_t)o; o += (size_t)warps * nbuf * 8;
+    o = (o + 127) & ~(size_t)127; g.off_tiles = (uint32_t)o;
+    while (nbuf > 1 && o + (size_t)warps * nbuf * cap > (size_t)smem_optin - 1024) --nbuf;
+    while (warps > 1 && o + (size_t)warps * nbuf * cap > (size_t)smem_optin - 1024) --warps;
+    o += (size_t)warps * nbuf * cap;
+    if (o > (size_t)smem_optin - 1024) return false;
+    g.nwarps = warps; g.nbuf = nbuf; g.tile_cap = (uint32_t)cap; g.smem_bytes = (uint32_t)o;
+    return true;
+}
+
+static uint32_t staged_xl(const Params& p) {
+    uint32_t xl = env_u32("FTC_STAGED_XL", 0);
+    if (xl >= 1 && xl <= 3) return xl;
+    // deepest lane-local sub-heap that keeps a tile (all its levels, every member) within 12 KB
+    if (p.kbytes % 16 || p.kbytes > 512) return 1;
+    uint32_t C = p.kbytes / 16, cwl = 0; while ((1u << cwl) < C) ++cwl;
+    const uint32_t lw = 5 - cwl;
+    for (xl = 3; xl > 1; --xl)
+        if ((((uint64_t)1 << (lw + xl)) - 1) * p.m * p.kbytes <= 12 * 1024) break;
+    return xl;
+}
+
+bool staged_supported(Params& p, int smem_optin_bytes) {
+    StagedGeom g;
+    return staged_geometry(p, smem_optin_bytes, staged_xl(p), g);
+}
+
+template <typename T, int OP, int XL>
+static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
+    StagedGeom g;
+    if (!staged_geometry(p, smem_optin, XL, g)) return cudaErrorInvalidConfiguration;
+    cudaError_t e = cudaFuncSetAttribute(staged_kernel<T, OP, XL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, staged_kernel<T, OP, XL>, (int)g.nwarps * 32, g.smem_bytes);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    const uint64_t cap = (uint64_t)sm_count * per_sm;
+    const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
+    staged_kernel<T, OP, XL><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
+    return cudaGetLastError();
+}
+
+template <typename T, int OP>
+static cudaError_t launch_staged_x(const Params& p, int sm_count, int smem_optin, cudaStream_t st) {
+    switch (staged_xl(p)) {
+    case 2: return launch_staged_t<T, OP, 2>(p, sm_count, smem_optin, st);
+    case 3: return launch_staged_t<T, OP, 3>(p, sm_count, smem_optin, st);
+    default: return launch_staged_t<T, OP, 1>(p, sm_count, smem_optin, st);
+    }
+}
+
+cudaError_t launch_staged(const Params& p, int tsel, int sm_count, int smem_optin, cudaStream_t st) {
+    switch (tsel) {
+    case TS_U32_SUM: return launch_staged_x<uint32_t, OP_SUM>(p, sm_count, smem_optin, st);
+    case TS_I32_MAX: return launch_staged_x<int32_t, OP_MAX>(p, sm_count, smem_optin, st);
+    case TS_U32_XOR: return launch_staged_x<uint32_t, OP_XOR>(p, sm_count, smem_optin, st);
+    case TS_U64_SUM: return launch_staged_x<unsigned long long, OP_SUM>(p, sm_count, smem_optin, st);
+    case TS_I64_MAX: return launch_staged_x<long long, OP_MAX>(p, sm_count, smem_optin, st);
+    case TS_U64_MAX: return launch_staged_x<unsigned long long, OP_MAX>(p, sm_count, smem_optin, st);
+    case TS_U64_XOR: return launch_staged_x<unsigned long long, OP_XOR>(p, sm_count, smem_optin, st);
+    case TS_F32_SUM: return launch_staged_x<float, OP_SUM>(p, sm_count, smem_optin, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace ftc

@@ -10,112 +10,16 @@
 //   * rows above level Lt are folded by the same lanes into shared memory and combined there level by level.
 // Every input byte is read from global memory exactly once; the combine order is the schedule's order, so
 // float32 sums come out bit-identical to a message-by-message execution.
-#include "ftc_device.cuh"
+#include <cstdlib>
+#include "ftc_tile_common.cuh"
 #include "ftc_kernels.h"
 
 namespace ftc {
 
-template <typename T> struct Vec16 { static constexpr int N = 16 / sizeof(T); };
-
-template <typename T, int OP>
-__device__ __forceinline__ uint4 comb16(uint4 a, uint4 b) {
-    union U { uint4 v; T t[Vec16<T>::N]; } A, B;
-    A.v = a; B.v = b;
-#pragma unroll
-    for (int i = 0; i < Vec16<T>::N; ++i) A.t[i] = Comb<T, OP>::f(A.t[i], B.t[i]);
-    return A.v;
-}
-
-__device__ __forceinline__ uint4 ld_stream(const char* ptr) {
-    return __ldg(reinterpret_cast<const uint4*>(ptr));
-}
-
-__device__ __forceinline__ uint4 shfl16(uint4 v, uint32_t src) {
-    uint4 r;
-    r.x = __shfl_sync(0xFFFFFFFFu, v.x, src); r.y = __shfl_sync(0xFFFFFFFFu, v.y, src);
-    r.z = __shfl_sync(0xFFFFFFFFu, v.z, src); r.w = __shfl_sync(0xFFFFFFFFu, v.w, src);
-    return r;
-}
-
-// Chunk lc of group `row` as the selected subtree's member holds it after up-correction: own input, then (short
-// last group only) the root's, then the partners whose message arrived, ascending. MCAP > 0: loads of up to MCAP
-// members are issued together; MCAP = 0: batches of eight.
-template <typename T, int OP, int MCAP>
-__device__ __forceinline__ uint4 fold16(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
-                                        const char* in_lc, uint32_t row) {
-    const uint32_t mj = row < p.q ? p.m : p.r, vbase = row * p.m + 1;
-    const uint32_t mask = extract_bits(inc, vbase, mj);
-    uint4 acc = make_uint4(0, 0, 0, 0);
-    if (MCAP > 0) {
-        uint4 v[MCAP > 0 ? MCAP : 1];
-#pragma unroll
-        for (int sp = 0; sp < MCAP; ++sp) {
-            v[sp] = make_uint4(0, 0, 0, 0);
-            if ((uint32_t)sp < mj && ((mask >> sp) & 1u)) {
-                const uint32_t vr = vbase + sp;
-                v[sp] = ld_stream(in_lc + (size_t)(vr == root ? 0u : vr) * p.kbytes);
-            }
-        }
-        uint4 vroot = make_uint4(0, 0, 0, 0);
-        if (row == p.q) vroot = ld_stream(in_lc + (size_t)root * p.kbytes);
-#pragma unroll
-        for (int sp = 0; sp < MCAP; ++sp) if ((uint32_t)sp == sstar) acc = v[sp];
-        if (row == p.q) acc = comb16<T, OP>(acc, vroot);
-#pragma unroll
-        for (int sp = 0; sp < MCAP; ++sp)
-            if ((uint32_t)sp < mj && (uint32_t)sp != sstar && ((mask >> sp) & 1u)) acc = comb16<T, OP>(acc, v[sp]);
-    } else {
-        const uint32_t vo = vbase + sstar;
-        acc = ld_stream(in_lc + (size_t)(vo == root ? 0u : vo) * p.kbytes);
-        if (row == p.q) acc = comb16<T, OP>(acc, ld_stream(in_lc + (size_t)root * p.kbytes));
-        for (uint32_t s0 = 0; s0 < mj; s0 += 8) {
-            uint4 v[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t sp = s0 + i, vr = vbase + sp;
-                v[i] = make_uint4(0, 0, 0, 0);
-                if (sp < mj && sp != sstar && ((mask >> sp) & 1u)) v[i] = ld_stream(in_lc + (size_t)(vr == root ? 0u : vr) * p.kbytes);
-            }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t sp = s0 + i;
-                if (sp < mj && sp != sstar && ((mask >> sp) & 1u)) acc = comb16<T, OP>(acc, v[i]);
-            }
-        }
-    }
-    return acc;
-}
-
-// The root's data after up-correction, for the case that no member of its (short, last) group lies in the
-// selected subtree: own input, then the members of that group whose message arrived.
-template <typename T, int OP>
-__device__ __forceinline__ uint4 fold_root16(const Params& p, uint32_t root, const uint32_t* inc, const char* in_lc) {
-    uint4 acc = ld_stream(in_lc + (size_t)root * p.kbytes);
-    if (p.r) {
-        const uint32_t vbase = p.q * p.m + 1, mask = extract_bits(inc, vbase, p.r);
-        for (uint32_t sp = 0; sp < p.r; ++sp) {
-            const uint32_t vr = vbase + sp;
-            if ((mask >> sp) & 1u) acc = comb16<T, OP>(acc, ld_stream(in_lc + (size_t)(vr == root ? 0u : vr) * p.kbytes));
-        }
-    }
-    return acc;
-}
-
-__device__ __forceinline__ void write_status_rec(const Params& p, uint64_t s, const Ctx* cx) {
-    uint32_t* st = p.status + s * FTC_STATUS_WORDS;
-    const bool ok = cx->code == FTC_ST_OK;
-    uint4 rec;
-    rec.x = cx->code | ((ok ? cx->sstar : 0xFFu) << 8) | (cx->attempts << 16);
-    rec.y = ok ? p.P - cx->npre - cx->nexcl : 0u;
-    rec.z = ok ? cx->inop_incl : 0u;
-    rec.w = (ok && p.is_allreduce) ? cx->holders : 0u;
-    *reinterpret_cast<uint4*>(st) = rec;
-}
-
 constexpr int kTiledMaxThreads = 512;
 
-template <typename T, int OP, int MCAP>
-__global__ void __launch_bounds__(kTiledMaxThreads) tiled_kernel(Params p) {
+template <typename T, int OP, int MCAP, int MINB>
+__global__ void __launch_bounds__(MINB == 1 ? 512 : 256, MINB) tiled_kernel(Params p) {
     extern __shared__ __align__(16) uint32_t smem[];
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
     uint32_t* pf = smem + sizeof(Ctx) / 4;
@@ -156,19 +60,7 @@ __global__ void __launch_bounds__(kTiledMaxThreads) tiled_kernel(Params p) {
                 const bool hasB = lr < RW - 1 && rowB < G;
                 if (rowA < G) valA = fold16<T, OP, MCAP>(p, root, sstar, inc, in_lc, rowA);
                 if (hasB) valB = fold16<T, OP, MCAP>(p, root, sstar, inc, in_lc, rowB);
-                for (int t = (int)lw - 1; t >= 0; --t) {
-                    // node idxB of level t takes its children from level t+1: data <- (data (op) child 1) (op) child 2
-                    const bool mine = hasB && tB == (uint32_t)t;
-                    const bool from_bottom = (uint32_t)(t + 1) == lw;
-                    const uint32_t src_row = from_bottom ? 2 * idxB : (2u << t) - 1 + 2 * idxB;
-                    const uint32_t src1 = mine ? ((src_row << cwl) | lc) : lane;
-                    const uint4 srcv = from_bottom ? valA : valB;
-                    const uint4 c1 = shfl16(srcv, src1), c2 = shfl16(srcv, mine ? src1 + p.C : lane);
-                    if (mine) {
-                        if (2 * rowB + 1 < G) valB = comb16<T, OP>(valB, c1);
-                        if (2 * rowB + 2 < G) valB = comb16<T, OP>(valB, c2);
-                    }
-                }
+                valB = tile_tree_phase<T, OP>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                 if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
             } else if (it < ntiles + ngroups) {
                 // ---- rows above the tiles: fold now, combine later ----
@@ -221,34 +113,45 @@ bool tiled_supported(Params& p, int smem_optin_bytes) {
 static uint32_t tiled_threads(const Params& p) {
     const uint32_t lw = 5 - p.cw_log2, ntiles = 1u << p.Lt;
     const uint32_t nitems = ntiles + ((ntiles - 1 + (1u << lw) - 1) >> lw) + 1;
-    uint32_t t = nitems * 32;
-    if (t < 128) t = 128;
-    if (t > (uint32_t)kTiledMaxThreads) t = kTiledMaxThreads;
-    return t;
+    if (const char* e = getenv("FTC_TILED_THREADS")) { int v = atoi(e); if (v >= 32 && v <= kTiledMaxThreads && v % 32 == 0) return (uint32_t)v; }
+    uint32_t warps = nitems / 32;                 // about 32 work items per warp and scenario
+    if (warps < 1) warps = 1;
+    if (warps > 8) warps = 8;
+    return warps * 32;
 }
 
-template <typename T, int OP, int MCAP>
+template <typename T, int OP, int MCAP, int MINB>
 static cudaError_t launch_tiled_t(const Params& p, int sm_count, cudaStream_t st) {
     const size_t smem = tiled_smem_bytes(p);
     const uint32_t threads = tiled_threads(p);
-    cudaError_t e = cudaFuncSetAttribute(tiled_kernel<T, OP, MCAP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(tiled_kernel<T, OP, MCAP, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tiled_kernel<T, OP, MCAP>, (int)threads, smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, tiled_kernel<T, OP, MCAP, MINB>, (int)threads, smem);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     uint64_t g = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < g ? p.S : g);
-    tiled_kernel<T, OP, MCAP><<<grid, threads, smem, st>>>(p);
+    tiled_kernel<T, OP, MCAP, MINB><<<grid, threads, smem, st>>>(p);
     return cudaGetLastError();
+}
+
+template <typename T, int OP, int MCAP>
+static cudaError_t launch_tiled_b(const Params& p, int sm_count, cudaStream_t st) {
+    int minb = MCAP == 4 ? 4 : MCAP == 6 ? 3 : 2;
+    if (const char* e = getenv("FTC_TILED_MINB")) minb = atoi(e);
+    if (tiled_threads(p) > 256 || minb == 1) return launch_tiled_t<T, OP, MCAP, 1>(p, sm_count, st);
+    if (minb >= 4) return launch_tiled_t<T, OP, MCAP, 4>(p, sm_count, st);
+    if (minb == 3) return launch_tiled_t<T, OP, MCAP, 3>(p, sm_count, st);
+    return launch_tiled_t<T, OP, MCAP, 2>(p, sm_count, st);
 }
 
 template <typename T, int OP>
 static cudaError_t launch_tiled_m(const Params& p, int sm_count, cudaStream_t st) {
-    if (p.m <= 4) return launch_tiled_t<T, OP, 4>(p, sm_count, st);
-    if (p.m <= 6) return launch_tiled_t<T, OP, 6>(p, sm_count, st);
-    if (p.m <= 9) return launch_tiled_t<T, OP, 9>(p, sm_count, st);
-    return launch_tiled_t<T, OP, 0>(p, sm_count, st);
+    if (p.m <= 4) return launch_tiled_b<T, OP, 4>(p, sm_count, st);
+    if (p.m <= 6) return launch_tiled_b<T, OP, 6>(p, sm_count, st);
+    if (p.m <= 9) return launch_tiled_b<T, OP, 9>(p, sm_count, st);
+    return launch_tiled_b<T, OP, 0>(p, sm_count, st);
 }
 
 cudaError_t launch_tiled(const Params& p, int tsel, int sm_count, cudaStream_t st) {

@@ -17,7 +17,7 @@ from tests.gpu_util import assert_same, run_gpu, run_oracle, to_dev, to_host
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = [0, B.FTC_KERNEL_GENERIC]
+KERNELS = [0, B.FTC_KERNEL_DIRECT, B.FTC_KERNEL_GENERIC]
 
 
 def check_workload(w, idx=None, flags=0, collective=None):
@@ -45,7 +45,7 @@ def test_config2_all_scenarios(flags):
     w = sc.config2()
     assert w.S == 33296
     x, (out, st, desc) = check_workload(w, flags=flags)
-    assert B.ftc_kernel_name(desc) == ("generic" if flags else "tiled")
+    assert B.ftc_kernel_name(desc) == {0: "staged", B.FTC_KERNEL_DIRECT: "tiled", B.FTC_KERNEL_GENERIC: "generic"}[flags]
     live_ok = (st[:, 0] & 0xFF) == 0
     assert live_ok.sum() == 16 * (2081 - 1 - 63)                 # every set without process 0 succeeds
 
@@ -73,9 +73,10 @@ def test_config5_sample(collective, op):
     check_workload(w)
 
 
-def test_config5_sample_generic_kernel():
+@pytest.mark.parametrize("flags", KERNELS[1:])
+def test_config5_sample_other_kernels(flags):
     w = sc.config5("allreduce", "sum", S=4)
-    check_workload(w, flags=B.FTC_KERNEL_GENERIC)
+    check_workload(w, flags=flags)
 
 
 # ---------------------------------------------------------------------------------------------
@@ -165,7 +166,7 @@ def test_chunk_counts_up_to_32_and_beyond():
     rng = np.random.Generator(np.random.PCG64(3))
     P, f, S = 300, 2, 16
     pf = sc.picks_to_masks(sc.random_subsets(rng, S, P, rng.integers(0, 3, size=S)), P)
-    for k, kernel in ((4, "tiled"), (8, "tiled"), (16, "tiled"), (32, "tiled"), (64, "tiled"), (128, "tiled"),
+    for k, kernel in ((4, "staged"), (8, "staged"), (16, "staged"), (32, "staged"), (64, "staged"), (128, "staged"),
                       (256, "generic"), (20, "generic"), (5, "generic")):
         x = rng.integers(-2**31, 2**31 - 1, size=(S, P, k), dtype=np.int32)
         got = run_gpu(x, f, "max", pf)
