@@ -16,10 +16,10 @@
 
 namespace ftc {
 
-constexpr int kTiledMaxThreads = 512;
+constexpr int kTiledMaxThreads = 256;
 
 template <typename T, int OP, int MCAP, int MINB>
-__global__ void __launch_bounds__(MINB == 1 ? 512 : 256, MINB) tiled_kernel(Params p) {
+__global__ void __launch_bounds__(kTiledMaxThreads, MINB) tiled_kernel(Params p) {
     extern __shared__ __align__(16) uint32_t smem[];
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
     uint32_t* pf = smem + sizeof(Ctx) / 4;
@@ -113,7 +113,6 @@ bool tiled_supported(Params& p, int smem_optin_bytes) {
 static uint32_t tiled_threads(const Params& p) {
     const uint32_t lw = 5 - p.cw_log2, ntiles = 1u << p.Lt;
     const uint32_t nitems = ntiles + ((ntiles - 1 + (1u << lw) - 1) >> lw) + 1;
-    if (const char* e = getenv("FTC_TILED_THREADS")) { int v = atoi(e); if (v >= 32 && v <= kTiledMaxThreads && v % 32 == 0) return (uint32_t)v; }
     uint32_t warps = nitems / 32;                 // about 32 work items per warp and scenario
     if (warps < 1) warps = 1;
     if (warps > 8) warps = 8;
@@ -136,14 +135,11 @@ static cudaError_t launch_tiled_t(const Params& p, int sm_count, cudaStream_t st
     return cudaGetLastError();
 }
 
+// Register budget per MCAP (blocks of up to 256 threads): 3 blocks per SM (80 registers) for groups of up to four
+// members, 2 (128 registers) for wider groups whose loads are all issued together.
 template <typename T, int OP, int MCAP>
 static cudaError_t launch_tiled_b(const Params& p, int sm_count, cudaStream_t st) {
-    int minb = MCAP == 4 ? 4 : MCAP == 6 ? 3 : 2;
-    if (const char* e = getenv("FTC_TILED_MINB")) minb = atoi(e);
-    if (tiled_threads(p) > 256 || minb == 1) return launch_tiled_t<T, OP, MCAP, 1>(p, sm_count, st);
-    if (minb >= 4) return launch_tiled_t<T, OP, MCAP, 4>(p, sm_count, st);
-    if (minb == 3) return launch_tiled_t<T, OP, MCAP, 3>(p, sm_count, st);
-    return launch_tiled_t<T, OP, MCAP, 2>(p, sm_count, st);
+    return launch_tiled_t<T, OP, MCAP, (MCAP == 4 ? 3 : 2)>(p, sm_count, st);
 }
 
 template <typename T, int OP>
