@@ -69,7 +69,8 @@ enum {
     FTC_EINVAL = -1,        /* P < f+2, k = 0, root >= P, NULL or misaligned required pointer, f > 31, max_inop > 32 */
     FTC_EUNSUPPORTED = -2,  /* unknown dtype/op, xor or max on f32 */
     FTC_EWORKSPACE = -3,    /* workspace missing or smaller than ftc_workspace_bytes() */
-    FTC_ECUDA = -4          /* a CUDA call or launch failed */
+    FTC_ECUDA = -4,         /* a CUDA call or launch failed */
+    FTC_ETOOLARGE = -5      /* ftc_reduce_batch_noalloc: the shape does not fit the built-in scratch */
 };
 
 /* per-scenario outcome, low byte of status word 0 */
@@ -152,6 +153,35 @@ FTC_API int ftc_reduce_batch(const ftc_desc_t* desc, uint64_t S, const void* d_i
 FTC_API int ftc_allreduce_batch(const ftc_desc_t* desc, uint64_t S, const void* d_in, const uint32_t* d_prefail,
                         const ftc_inop_t* d_inop, const uint32_t* d_roots, void* d_out, uint32_t* d_status,
                         void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Corrected reduce for callers that cannot give the library any scratch memory and cannot allocate it either.
+ * (The paper has no counterpart to this entry point: it exists for the sake of the host program, not the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a latency-critical loop, where an
+ * allocation's implicit device-wide synchronisation would stall unrelated streams; inside a plug-in or callback
+ * of another framework that owns the memory budget and hands out no allocator; or after start-up in a service
+ * whose device memory is fully accounted for. ftc_reduce_batch wants a caller-provided workspace for shapes that
+ * run on the general kernel; this variant needs none.
+ *
+ * How: the general kernel's per-block node values go to an array of FTC_NOALLOC_SCRATCH_BYTES bytes that is part
+ * of the library image. Every GPU that loads the library holds that array until the process exits. The call
+ * allocates nothing (no cudaMalloc, cudaFree or allocating library routine), results and status records are
+ * identical to ftc_reduce_batch's, and it is slower when fewer blocks than usual fit into the array.
+ *   - Limit: one block's slice, ceil((P-1)/(f+1)) * k * element size bytes, must fit the array; otherwise
+ *     FTC_ETOOLARGE is returned and nothing is enqueued.
+ *   - The first call on each device looks the array's device address up (one runtime query, with that device
+ *     current). Make that first call before starting any stream capture on that device.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left in it. Nothing in it
+ *     needs clearing: within a scenario every slot is written before it is read. But two calls whose kernels can
+ *     overlap on the same GPU (different streams, or different host threads) race on it: serialise them.
+ * Arguments and all other rules as for ftc_reduce_batch, without the workspace pair. The always-general kernel
+ * is used whatever the shape.
+ */
+#define FTC_NOALLOC_SCRATCH_BYTES (8u << 20)
+FTC_API int ftc_reduce_batch_noalloc(const ftc_desc_t* desc, uint64_t S, const void* d_in, const uint32_t* d_prefail,
+                                     const ftc_inop_t* d_inop, const uint32_t* d_roots, void* d_out,
+                                     uint32_t* d_status, void* cuda_stream);
 
 /* Scratch bytes the two calls above need for this descriptor and batch size (0 when the shape runs on the
  * shared-memory kernel). Returns 0 for an invalid descriptor as well; the batch calls report that. */

@@ -16,7 +16,8 @@ LIB_PATH = os.path.join(_HERE, "libftc.so")
 
 FTC_I32, FTC_I64, FTC_U64, FTC_F32 = 0, 1, 2, 3
 FTC_SUM, FTC_MAX, FTC_XOR = 0, 1, 2
-FTC_OK, FTC_EINVAL, FTC_EUNSUPPORTED, FTC_EWORKSPACE, FTC_ECUDA = 0, -1, -2, -3, -4
+FTC_OK, FTC_EINVAL, FTC_EUNSUPPORTED, FTC_EWORKSPACE, FTC_ECUDA, FTC_ETOOLARGE = 0, -1, -2, -3, -4, -5
+FTC_NOALLOC_SCRATCH_BYTES = 8 << 20
 FTC_ST_OK, FTC_ST_ROOT_FAILED, FTC_ST_NO_CLEAN_SUBTREE, FTC_ST_NO_LIVE_ROOT_CANDIDATE = 0, 1, 2, 3
 FTC_ST_PRECONDITION_INOP_ROOT, FTC_ST_BAD_ROOT, FTC_ST_INTERNAL_TIMEOUT = 4, 5, 6
 FTC_STATUS_WORDS = 4
@@ -26,7 +27,7 @@ FTC_KERNEL_GENERIC = 0x100
 FTC_KERNEL_DIRECT = 0x200
 OPS = {"sum": FTC_SUM, "max": FTC_MAX, "xor": FTC_XOR}
 
-EXPORTS = ["ftc_reduce_batch", "ftc_allreduce_batch", "ftc_workspace_bytes", "ftc_reduce_batch_host",
+EXPORTS = ["ftc_reduce_batch", "ftc_allreduce_batch", "ftc_reduce_batch_noalloc", "ftc_workspace_bytes", "ftc_reduce_batch_host",
            "ftc_allreduce_batch_host", "ftc_host_staging_bytes", "ftc_schedule_info", "ftc_fill_inputs",
            "ftc_kernel_name", "ftc_strerror", "ftc_version"]
 
@@ -65,6 +66,8 @@ def load():
     for name in ("ftc_reduce_batch", "ftc_allreduce_batch", "ftc_reduce_batch_host", "ftc_allreduce_batch_host"):
         getattr(lib, name).restype = C.c_int
         getattr(lib, name).argtypes = batch_args
+    lib.ftc_reduce_batch_noalloc.restype = C.c_int
+    lib.ftc_reduce_batch_noalloc.argtypes = [dp, u64, vp, vp, vp, vp, vp, vp, vp]
     lib.ftc_workspace_bytes.restype = sz
     lib.ftc_workspace_bytes.argtypes = [dp, u64, C.c_int]
     lib.ftc_host_staging_bytes.restype = sz
@@ -173,6 +176,17 @@ def ftc_allreduce_batch(desc, S, d_in, d_prefail, d_inop, d_roots, d_out, d_stat
                         check=True) -> int:
     return _batch("ftc_allreduce_batch", desc, S, d_in, d_prefail, d_inop, d_roots, d_out, d_status, d_workspace,
                   stream, check)
+
+
+def ftc_reduce_batch_noalloc(desc, S, d_in, d_prefail, d_inop, d_roots, d_out, d_status, stream=None,
+                             check=True) -> int:
+    """Reduce on the library's built-in scratch array: for callers that can neither pass a workspace nor
+    allocate one. Marshals the pointers only; no tensor is created here."""
+    rc = load().ftc_reduce_batch_noalloc(C.byref(desc), S, _dev_ptr(d_in), _dev_ptr(d_prefail), _dev_ptr(d_inop),
+                                         _dev_ptr(d_roots), _dev_ptr(d_out), _dev_ptr(d_status), _stream(stream))
+    if check and rc != FTC_OK:
+        raise FtcError(rc, "ftc_reduce_batch_noalloc")
+    return rc
 
 
 def _batch_host(fn_name, desc, S, h_in, h_prefail, h_inop, h_roots, h_out, h_status, d_staging, stream, check):

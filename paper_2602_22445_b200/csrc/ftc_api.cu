@@ -171,6 +171,29 @@ int ftc_allreduce_batch(const ftc_desc_t* desc, uint64_t S, const void* d_in, co
     return run_batch(desc, S, 1, d_in, d_prefail, d_inop, d_roots, d_out, d_status, d_workspace, workspace_bytes, cuda_stream);
 }
 
+int ftc_reduce_batch_noalloc(const ftc_desc_t* desc, uint64_t S, const void* d_in, const uint32_t* d_prefail,
+                             const ftc_inop_t* d_inop, const uint32_t* d_roots, void* d_out, uint32_t* d_status,
+                             void* cuda_stream) {
+    Params p;
+    int rc = fill_params(desc, S, 0, p);
+    if (rc != FTC_OK) return rc;
+    if (desc->flags & FTC_OUT_EXPANDED) return FTC_EUNSUPPORTED;
+    if (S == 0) return FTC_OK;
+    if (!d_in || !d_prefail || !d_out || !d_status) return FTC_EINVAL;
+    if (p.max_inop && !d_inop) return FTC_EINVAL;
+    if (p.root < 0 && !d_roots) return FTC_EINVAL;
+    if (!aligned16(d_in) || !aligned16(d_out) || !aligned16(d_status)) return FTC_EINVAL;
+    DeviceInfo di;
+    if ((rc = device_info(di)) != FTC_OK) return rc;
+    if (generic_smem_bytes(p) > (size_t)di.smem_optin) return FTC_EUNSUPPORTED;
+    p.in = d_in; p.prefail = d_prefail; p.inop = d_inop; p.roots = d_roots; p.out = d_out; p.status = d_status;
+    bool too_large = false;
+    cudaError_t e = launch_generic_static(p, type_select(desc->dtype, desc->op), di.sm_count,
+                                          static_cast<cudaStream_t>(cuda_stream), &too_large);
+    if (too_large) return FTC_ETOOLARGE;
+    return e == cudaSuccess ? FTC_OK : FTC_ECUDA;
+}
+
 size_t ftc_workspace_bytes(const ftc_desc_t* desc, uint64_t S, int is_allreduce) {
     Params p;
     if (fill_params(desc, S, is_allreduce, p) != FTC_OK || S == 0) return 0;
@@ -237,6 +260,7 @@ const char* ftc_strerror(int code) {
     case FTC_EUNSUPPORTED: return "unsupported dtype/op combination or flag";
     case FTC_EWORKSPACE: return "workspace missing, misaligned or smaller than ftc_workspace_bytes()";
     case FTC_ECUDA: return "a CUDA call or kernel launch failed";
+    case FTC_ETOOLARGE: return "shape too large for the built-in scratch: ceil((P-1)/(f+1)) * k * element size exceeds FTC_NOALLOC_SCRATCH_BYTES";
     }
     return "unknown error code";
 }

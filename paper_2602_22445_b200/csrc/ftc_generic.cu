@@ -1,5 +1,6 @@
 // General kernel: any P, f, k. One block per scenario (grid-stride), the selected subtree is evaluated level by
 // level from the leaves, node values pass through a per-block slice of the global workspace.
+#include <mutex>
 #include "ftc_device.cuh"
 #include "ftc_kernels.h"
 
@@ -116,6 +117,73 @@ cudaError_t launch_generic(const Params& p, int tsel, int sm_count, cudaStream_t
     case TS_U64_MAX: return launch_generic_t<unsigned long long, OP_MAX>(p, sm_count, st);
     case TS_U64_XOR: return launch_generic_t<unsigned long long, OP_XOR>(p, sm_count, st);
     case TS_F32_SUM: return launch_generic_t<float, OP_SUM>(p, sm_count, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Built-in scratch for callers that cannot hand the library a workspace.
+// The array lives in device memory of every GPU that loads the library, from load to process exit. Its name is
+// only meaningful to device code; host code must ask the runtime for its device address (below) and may never
+// pass the symbol itself to a kernel.
+// ---------------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[FTC_NOALLOC_SCRATCH_BYTES];
+
+static std::mutex g_static_mutex;
+static void* g_static_ptr[64];          // device address of g_static_scratch, per device ordinal
+static bool g_static_ready[64];
+
+// First call on a device: looks the array's device address up (with that device current). Later calls reuse it.
+static cudaError_t static_scratch_address(void** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ready[dev]) {
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        if (!ptr) return cudaErrorInvalidSymbol;
+        g_static_ptr[dev] = ptr; g_static_ready[dev] = true;
+    }
+    *out = g_static_ptr[dev];
+    return cudaSuccess;
+}
+
+template <typename T, int OP>
+static cudaError_t launch_static_t(const Params& p, uint32_t grid, cudaStream_t st) {
+    size_t smem = generic_smem_bytes(p);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(generic_kernel<T, OP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    generic_kernel<T, OP><<<grid, 256, smem, st>>>(p);
+    return cudaGetLastError();
+}
+
+// The general kernel with its node values in the built-in scratch: as many blocks as slices fit (at most the
+// usual grid). *too_large is set when not even one block's slice fits.
+cudaError_t launch_generic_static(Params p, int tsel, int sm_count, cudaStream_t st, bool* too_large) {
+    const size_t slice = (size_t)p.Gmax * p.kbytes;
+    *too_large = slice > (size_t)FTC_NOALLOC_SCRATCH_BYTES;
+    if (*too_large) return cudaSuccess;
+    void* ptr = nullptr;
+    cudaError_t e = static_scratch_address(&ptr);
+    if (e != cudaSuccess) return e;
+    uint32_t grid = generic_grid(p, sm_count);
+    const size_t fit = (size_t)FTC_NOALLOC_SCRATCH_BYTES / slice;
+    if (grid > fit) grid = (uint32_t)fit;
+    p.ws = ptr;
+    switch (tsel) {
+    case TS_U32_SUM: return launch_static_t<uint32_t, OP_SUM>(p, grid, st);
+    case TS_I32_MAX: return launch_static_t<int32_t, OP_MAX>(p, grid, st);
+    case TS_U32_XOR: return launch_static_t<uint32_t, OP_XOR>(p, grid, st);
+    case TS_U64_SUM: return launch_static_t<unsigned long long, OP_SUM>(p, grid, st);
+    case TS_I64_MAX: return launch_static_t<long long, OP_MAX>(p, grid, st);
+    case TS_U64_MAX: return launch_static_t<unsigned long long, OP_MAX>(p, grid, st);
+    case TS_U64_XOR: return launch_static_t<unsigned long long, OP_XOR>(p, grid, st);
+    case TS_F32_SUM: return launch_static_t<float, OP_SUM>(p, grid, st);
     }
     return cudaErrorInvalidValue;
 }

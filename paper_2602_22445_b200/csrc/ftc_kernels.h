@@ -16,6 +16,9 @@ size_t generic_smem_bytes(const Params& p);
 uint32_t generic_grid(const Params& p, int sm_count);
 cudaError_t launch_generic(const Params& p, int tsel, int sm_count, cudaStream_t st);
 
+// General kernel on the library's built-in scratch array (no workspace from the caller).
+cudaError_t launch_generic_static(Params p, int tsel, int sm_count, cudaStream_t st, bool* too_large);
+
 // Tiled kernel: does the shape fit (16-byte chunks, power-of-two chunk count <= 32, shared memory)? Fills the
 // tile geometry into p when it does.
 bool tiled_supported(Params& p, int smem_optin_bytes);
