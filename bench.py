@@ -238,8 +238,9 @@ def run_gpu(args):
     sched = B.ftc_schedule_info(desc0)
     w = make_workload(name, S, rank * S, sched["rounds_attempt"])          # each rank its own scenarios
     allred = w.collective == "allreduce"
+    kflags = {"auto": 0, "direct": B.FTC_KERNEL_DIRECT, "generic": B.FTC_KERNEL_GENERIC}[args.kernel]
     desc = B.make_desc(w.P, w.f, w.k, B.dtype_code(tdt), w.op, root=-1 if w.roots is not None else 0,
-                       max_inop=0 if w.inop is None else w.inop.shape[1])
+                       max_inop=0 if w.inop is None else w.inop.shape[1], flags=kflags)
     fn = B.ftc_allreduce_batch if allred else B.ftc_reduce_batch
 
     d_x = torch.empty((S, w.P, w.k), dtype=tdt, device="cuda")
@@ -382,6 +383,7 @@ def main():
     ap.add_argument("--workload", default="c4", choices=sorted(DESCRIPTION))
     ap.add_argument("--batch", type=int, default=0, help="scenarios per step per GPU")
     ap.add_argument("--e2e-scenarios", type=int, default=0)
+    ap.add_argument("--kernel", default="auto", choices=["auto", "direct", "generic"], help="force a kernel family")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU legs (for profiler runs)")
     args = ap.parse_args()

@@ -42,72 +42,82 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
     return false;
 }
 
-struct LdShared {
-    __device__ __forceinline__ uint4 operator()(const char* q) const { return *reinterpret_cast<const uint4*>(q); }
-};
-
 struct StagedGeom {
     uint32_t nwarps, nbuf, tile_cap;       // warps per block, buffers per warp, bytes per buffer (multiple of 128)
+    uint32_t whole;                        // 1: the whole scenario is staged in one block-wide buffer
     uint32_t off_special, off_rootv, off_hv, off_bar, off_tiles, smem_bytes;
 };
 
-// The rare groups that are not plain: folded from global memory by the general routine. Kept out of line so that
-// the common path stays small in code and registers.
-template <typename T, int OP>
-__device__ __noinline__ uint4 fold_special(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
-                                           const char* in_lc, uint32_t row) {
-    return fold16_general<T, OP, 0>(p, root, sstar, inc, in_lc, row);
+// Where a row's bytes sit: at tile-heap position trow of the warp's buffer, or (WHOLE) at their place in the
+// block-wide copy of the scenario (grow = global row).
+template <bool WHOLE>
+__device__ __forceinline__ uint32_t staged_row_offset(const Params& p, uint32_t rowbytes, uint32_t trow, uint32_t grow) {
+    return WHOLE ? (grow * p.m + 1) * p.kbytes : trow * rowbytes;
 }
 
-// Fold of one group, chunk lc: from the staged copy when the group is plain, else from global memory.
+// Fold of a plain group from its staged copy.
 template <typename T, int OP>
+__device__ __forceinline__ uint4 fold_plain_staged(const Params& p, uint32_t sstar, const char* srow_lc) {
+    return fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdShared());
+}
+
+// Fold of one group on the careful path: by the general routine from the scenario in process order (`in_lc`:
+// global memory, or the block-wide shared copy when WHOLE).
+template <typename T, int OP, bool WHOLE>
 __device__ __forceinline__ uint4 fold_staged(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
-                                             const char* in_lc, const char* srow_lc, uint32_t row) {
-    if (group_is_plain(p, root, inc, row)) {
-        uint4 acc;
-        if (Ordered<T>::value) {
-            acc = LdShared()(srow_lc + sstar * p.kbytes);
-#pragma unroll 4
-            for (uint32_t sp = 0; sp < p.m; ++sp)
-                if (sp != sstar) acc = comb16<T, OP>(acc, LdShared()(srow_lc + sp * p.kbytes));
-        } else {
-            acc = LdShared()(srow_lc);
-#pragma unroll 4
-            for (uint32_t sp = 1; sp < p.m; ++sp) acc = comb16<T, OP>(acc, LdShared()(srow_lc + sp * p.kbytes));
-        }
-        return acc;
-    }
-    return fold_special<T, OP>(p, root, sstar, inc, in_lc, row);
+                                             const char* in_lc, uint32_t row) {
+    if (WHOLE) return fold16_careful<T, OP, LdShared>(p, root, sstar, inc, in_lc, row);
+    return fold16_careful<T, OP, LdGlobal>(p, root, sstar, inc, in_lc, row);
 }
 
-// Value of the node at level u (of XL) of a lane's sub-heap: its group's fold, then child 1, then child 2.
-// trow/grow: tile-heap index and global row of the node.
-template <typename T, int OP, int XL, int U>
-struct SubHeap {
-    static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
-                                                 const char* in_lc, const char* buf_lc, uint32_t rowbytes,
+// A lane's sub-heap in a tile whose rows are all plain and that is complete down to its second-to-last level:
+// only the children at the tile's last level (U + 1 == XL - 1) may be missing.
+template <typename T, int OP, int XL, int U, bool WHOLE>
+struct SubHeapPlain {
+    static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t sstar, const char* buf_lc, uint32_t rowbytes,
                                                  uint32_t trow, uint32_t grow, uint32_t G) {
-        uint4 v = fold_staged<T, OP>(p, root, sstar, inc, in_lc, buf_lc + trow * rowbytes, grow);
+        uint4 v = fold_plain_staged<T, OP>(p, sstar, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, trow, grow));
         if (U + 1 < XL) {
-            if (2 * grow + 1 < G)
-                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U)>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
-            if (2 * grow + 2 < G)
-                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U)>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
+            constexpr int UN = (U + 1 < XL ? U + 1 : U);
+            if (U + 2 < XL || 2 * grow + 1 < G)
+                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE>::eval(p, sstar, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
+            if (U + 2 < XL || 2 * grow + 2 < G)
+                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE>::eval(p, sstar, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
         }
         return v;
     }
 };
 
-constexpr int kStagedMaxThreads = 512;
+// Value of the node at level u (of XL) of a lane's sub-heap: its group's fold, then child 1, then child 2.
+// trow/grow: tile-heap index and global row of the node. Its bytes sit at tile-heap position trow of the warp's
+// buffer, or (WHOLE) at their place in the block-wide copy of the scenario.
+template <typename T, int OP, int XL, int U, bool WHOLE>
+struct SubHeap {
+    static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
+                                                 const char* in_lc, const char* buf_lc, uint32_t rowbytes,
+                                                 uint32_t trow, uint32_t grow, uint32_t G) {
+        uint4 v = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, grow);
+        if (U + 1 < XL) {
+            if (2 * grow + 1 < G)
+                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
+            if (2 * grow + 2 < G)
+                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
+        }
+        return v;
+    }
+};
 
-template <typename T, int OP, int XL>
-__global__ void __launch_bounds__(kStagedMaxThreads) staged_kernel(Params p, StagedGeom g) {
+constexpr int kStagedMaxThreads = 256;
+
+template <typename T, int OP, int XL, bool WHOLE>
+__global__ void __launch_bounds__(kStagedMaxThreads, 2) staged_kernel(Params p, StagedGeom g) {
     extern __shared__ __align__(128) uint32_t smem[];
     char* sbase = reinterpret_cast<char*>(smem);
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
     uint32_t* pf = smem + sizeof(Ctx) / 4;
     uint32_t* inc = pf + p.W + 1;
     uint32_t* unr = inc + p.W + 1;
+    uint32_t* tspec = reinterpret_cast<uint32_t*>(sbase + g.off_special);
     uint4* rootv = reinterpret_cast<uint4*>(sbase + g.off_rootv);
     uint4* hv = reinterpret_cast<uint4*>(sbase + g.off_hv);
 
@@ -122,14 +132,31 @@ __global__ void __launch_bounds__(kStagedMaxThreads) staged_kernel(Params p, Sta
 
     const uint32_t bar0 = smem_addr(sbase + g.off_bar) + wid * g.nbuf * 8;
     char* tiles = sbase + g.off_tiles + (size_t)wid * g.nbuf * g.tile_cap;
+    const uint32_t cbar = smem_addr(sbase + g.off_bar) + g.nwarps * g.nbuf * 8;   // block-wide barrier (WHOLE)
+    char* wbuf = sbase + g.off_tiles;                                            // block-wide scenario copy (WHOLE)
     if (lane < g.nbuf) mbar_init(bar0 + lane * 8, 1);
+    if (WHOLE && tid == 0) mbar_init(cbar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
     uint32_t phase_bits = 0;                                      // bit b: parity to wait for on buffer b
+    uint32_t cphase = 0;
 
     for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {
+        const char* in_s = reinterpret_cast<const char*>(p.in) + s * scen_bytes;
+        if (WHOLE && wid == 0) {
+            // the whole scenario, in pieces of at most 32 KB, lands while the masks are decoded
+            if (lane == 0) mbar_expect_tx(cbar, (uint32_t)scen_bytes);
+            __syncwarp();
+            for (uint64_t o = (uint64_t)lane * 32768; o < scen_bytes; o += 32u * 32768)
+                bulk_g2s(smem_addr(wbuf + o), in_s + o, (uint32_t)min((uint64_t)32768, scen_bytes - o), cbar);
+        }
         decode_scenario(p, s, cx, pf, inc);
         char* out_s = reinterpret_cast<char*>(p.out) + s * p.kbytes;
+        if (WHOLE) {
+            // every thread sees the copy complete before it reads it or leaves the iteration
+            if (!mbar_wait_bounded(cbar, cphase)) atomicOr(&cx->pad, 1u);
+            cphase ^= 1u;
+        }
         if (cx->code != FTC_ST_OK) {
             if (tid < p.C) reinterpret_cast<uint4*>(out_s)[tid] = make_uint4(0, 0, 0, 0);
             if (tid == 0) write_status_rec(p, s, cx);
@@ -137,12 +164,13 @@ __global__ void __launch_bounds__(kStagedMaxThreads) staged_kernel(Params p, Sta
             continue;
         }
         if (p.is_allreduce) count_holders(p, cx, pf, unr);
+        mark_special_items(p, cx, pf, tspec, Lt, lw, D);
         const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
-        const char* in_s = reinterpret_cast<const char*>(p.in) + s * scen_bytes;
-        const char* in_lc = in_s + lc * 16;
+        const char* in_lc = (WHOLE ? wbuf : in_s) + lc * 16;      // the scenario in process order, for the general fold
 
         // Issue the bulk copies of work item `it` into buffer b: lane t copies level t of the tile.
         auto issue = [&](uint32_t it, uint32_t b) {
+            if (WHOLE) return false;
             uint32_t first_row = 0, nrows = 0, dst_off = 0;
             if (it < ntiles) {
                 const uint32_t j0 = ntop + it;
@@ -173,26 +201,36 @@ __global__ void __launch_bounds__(kStagedMaxThreads) staged_kernel(Params p, Sta
                 if (!mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u)) { if (lane == 0) atomicOr(&cx->pad, 1u); }
                 phase_bits ^= 1u << b; pending &= ~(1u << b);
             }
-            const char* buf_lc = tiles + (size_t)b * g.tile_cap + lc * 16;
+            const char* buf_lc = (WHOLE ? wbuf : tiles + (size_t)b * g.tile_cap) + lc * 16;
+            const bool careful = it < ntiles + ngroups && test_bit(tspec, it);      // warp-uniform
             if (it < ntiles) {
                 const uint32_t j0 = ntop + it;
-                if (j0 < G) {
-                    // bottom part: this lane row's sub-heap, rooted at level lw of the tile
-                    const uint32_t tA = RW - 1 + lr, rowA = ((j0 + 1) << lw) - 1 + lr;
+                const uint32_t tA = RW - 1 + lr, rowA = ((j0 + 1) << lw) - 1 + lr;     // root of this lane row's sub-heap
+                const uint32_t tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB);
+                const uint32_t rowB = ((j0 + 1) << tB) - 1 + idxB;                     // this lane row's node above
+                if (!careful) {
+                    // XL == 1: the bottom rows are the tile's last level and may be missing; XL > 1: they exist
                     uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
-                    if (rowA < G) valA = SubHeap<T, OP, XL, 0>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, tA, rowA, G);
-                    const uint32_t tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB);
-                    const uint32_t rowB = ((j0 + 1) << tB) - 1 + idxB;
+                    if (XL > 1 || rowA < G) valA = SubHeapPlain<T, OP, XL, 0, WHOLE>::eval(p, sstar, buf_lc, rowbytes, tA, rowA, G);
+                    const bool hasB = lr < RW - 1;
+                    if (hasB) valB = fold_plain_staged<T, OP>(p, sstar, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB));
+                    valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
+                    if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
+                } else if (j0 < G) {
+                    uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
+                    if (rowA < G) valA = SubHeap<T, OP, XL, 0, WHOLE>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, tA, rowA, G);
                     const bool hasB = lr < RW - 1 && rowB < G;
-                    if (hasB) valB = fold_staged<T, OP>(p, root, sstar, inc, in_lc, buf_lc + lr * rowbytes, rowB);
+                    if (hasB) valB = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, rowB);
                     valB = tile_tree_phase<T, OP>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                     if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                 }
             } else if (it < ntiles + ngroups) {
                 const uint32_t row = ((it - ntiles) << lw) + lr;
-                if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged<T, OP>(p, root, sstar, inc, in_lc, buf_lc + lr * rowbytes, row);
+                const char* srow = buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, row);
+                if (!careful) hv[(size_t)row * p.C + lc] = fold_plain_staged<T, OP>(p, sstar, srow);
+                else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, row);
             } else if (sstar >= p.r) {
-                if (lr == 0) rootv[lc] = fold_root16<T, OP>(p, root, inc, in_lc);
+                if (lr == 0) rootv[lc] = WHOLE ? fold_root16<T, OP, LdShared>(p, root, inc, in_lc) : fold_root16<T, OP, LdGlobal>(p, root, inc, in_lc);
             }
             __syncwarp();                                         // every lane is done with buffer b
             if (i + g.nbuf < n_my && issue(wid + (i + g.nbuf) * nw, b)) pending |= 1u << b;
@@ -250,15 +288,24 @@ static bool staged_geometry(Params& p, int smem_optin, uint32_t XL, StagedGeom& 
     if (warps > kStagedMaxThreads / 32) warps = kStagedMaxThreads / 32;
     uint32_t nbuf = env_u32("FTC_STAGED_NBUF", 1);
     if (nbuf > 4) nbuf = 4;
+    // small scenarios are staged whole (three blocks of them fit an SM), large ones tile by tile
+    const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
+    g.whole = scen_bytes <= env_u32("FTC_STAGED_WHOLE_MAX", 72 * 1024) ? 1u : 0u;
+    if (g.whole) { nbuf = 0; if (!env_u32("FTC_STAGED_WARPS", 0)) { warps = 1; while (warps < 8 && warps * 2 * 4 <= nitems) warps *= 2; } }
     size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
     o = (o + 15) & ~(size_t)15; g.off_special = (uint32_t)o;
+    o += ((((size_t)nitems + 31) / 32 + 1) * 4 + 15) & ~(size_t)15;
     g.off_rootv = (uint32_t)o; o += (size_t)C * 16;
     g.off_hv = (uint32_t)o; o += (((size_t)2 << p.Lt) - 1) * C * 16;
-    g.off_bar = (uint32_t)o; o += (size_t)warps * nbuf * 8;
+    g.off_bar = (uint32_t)o; o += (size_t)(kStagedMaxThreads / 32) * 4 * 8 + 8;      // room for any warps x nbuf, plus one
     o = (o + 127) & ~(size_t)127; g.off_tiles = (uint32_t)o;
-    while (nbuf > 1 && o + (size_t)warps * nbuf * cap > (size_t)smem_optin - 1024) --nbuf;
-    while (warps > 1 && o + (size_t)warps * nbuf * cap > (size_t)smem_optin - 1024) --warps;
-    o += (size_t)warps * nbuf * cap;
+    if (g.whole) {
+        o += (size_t)((scen_bytes + 127) & ~(uint64_t)127);
+    } else {
+        while (nbuf > 1 && o + (size_t)warps * nbuf * cap > (size_t)smem_optin - 1024) --nbuf;
+        while (warps > 1 && o + (size_t)warps * nbuf * cap > (size_t)smem_optin - 1024) --warps;
+        o += (size_t)warps * nbuf * cap;
+    }
     if (o > (size_t)smem_optin - 1024) return false;
     g.nwarps = warps; g.nbuf = nbuf; g.tile_cap = (uint32_t)cap; g.smem_bytes = (uint32_t)o;
     return true;
@@ -281,20 +328,25 @@ bool staged_supported(Params& p, int smem_optin_bytes) {
     return staged_geometry(p, smem_optin_bytes, staged_xl(p), g);
 }
 
-template <typename T, int OP, int XL>
-static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
-    StagedGeom g;
-    if (!staged_geometry(p, smem_optin, XL, g)) return cudaErrorInvalidConfiguration;
-    cudaError_t e = cudaFuncSetAttribute(staged_kernel<T, OP, XL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
+template <typename T, int OP, int XL, bool WHOLE>
+static cudaError_t launch_staged_w(const Params& p, const StagedGeom& g, int sm_count, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(staged_kernel<T, OP, XL, WHOLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, staged_kernel<T, OP, XL>, (int)g.nwarps * 32, g.smem_bytes);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, staged_kernel<T, OP, XL, WHOLE>, (int)g.nwarps * 32, g.smem_bytes);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
-    staged_kernel<T, OP, XL><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
+    staged_kernel<T, OP, XL, WHOLE><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
     return cudaGetLastError();
+}
+
+template <typename T, int OP, int XL>
+static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
+    StagedGeom g;
+    if (!staged_geometry(p, smem_optin, XL, g)) return cudaErrorInvalidConfiguration;
+    return g.whole ? launch_staged_w<T, OP, XL, true>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, false>(p, g, sm_count, st);
 }
 
 template <typename T, int OP>

@@ -32,13 +32,18 @@ __device__ __forceinline__ uint4 shfl16(uint4 v, uint32_t src) {
 template <typename T> struct Ordered { static constexpr bool value = false; };
 template <> struct Ordered<float> { static constexpr bool value = true; };
 
-// Chunk lc of group `row` as the selected subtree's member holds it after up-correction, read from global memory:
+struct LdGlobal { __device__ __forceinline__ uint4 operator()(const char* q) const { return ld_stream(q); } };
+struct LdShared { __device__ __forceinline__ uint4 operator()(const char* q) const { return *reinterpret_cast<const uint4*>(q); } };
+
+// Chunk lc of group `row` as the selected subtree's member holds it after up-correction, read from a copy of the
+// scenario in the caller's process order (global memory, or shared memory when LD = LdShared):
 // own input, then (short last group only) the root's, then the partners whose message arrived, ascending.
 // Handles every case (missing members, the renumbered slots, the short group). MCAP > 0: loads of up to MCAP
-// members are issued together; MCAP = 0: batches of eight.
-template <typename T, int OP, int MCAP>
+// members are issued together; MCAP = 0: batches of four.
+template <typename T, int OP, int MCAP, typename LD = LdGlobal>
 __device__ __forceinline__ uint4 fold16_general(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
                                                 const char* in_lc, uint32_t row) {
+    const LD ld{};
     const uint32_t mj = row < p.q ? p.m : p.r, vbase = row * p.m + 1;
     const uint32_t mask = extract_bits(inc, vbase, mj);
     uint4 acc = make_uint4(0, 0, 0, 0);
@@ -49,11 +54,11 @@ __device__ __forceinline__ uint4 fold16_general(const Params& p, uint32_t root, 
             v[sp] = make_uint4(0, 0, 0, 0);
             if ((uint32_t)sp < mj && ((mask >> sp) & 1u)) {
                 const uint32_t vr = vbase + sp;
-                v[sp] = ld_stream(in_lc + (size_t)(vr == root ? 0u : vr) * p.kbytes);
+                v[sp] = ld(in_lc + (size_t)(vr == root ? 0u : vr) * p.kbytes);
             }
         }
         uint4 vroot = make_uint4(0, 0, 0, 0);
-        if (row == p.q) vroot = ld_stream(in_lc + (size_t)root * p.kbytes);
+        if (row == p.q) vroot = ld(in_lc + (size_t)root * p.kbytes);
 #pragma unroll
         for (int sp = 0; sp < MCAP; ++sp) if ((uint32_t)sp == sstar) acc = v[sp];
         if (row == p.q) acc = comb16<T, OP>(acc, vroot);
@@ -62,18 +67,18 @@ __device__ __forceinline__ uint4 fold16_general(const Params& p, uint32_t root, 
             if ((uint32_t)sp < mj && (uint32_t)sp != sstar && ((mask >> sp) & 1u)) acc = comb16<T, OP>(acc, v[sp]);
     } else {
         const uint32_t vo = vbase + sstar;
-        acc = ld_stream(in_lc + (size_t)(vo == root ? 0u : vo) * p.kbytes);
-        if (row == p.q) acc = comb16<T, OP>(acc, ld_stream(in_lc + (size_t)root * p.kbytes));
-        for (uint32_t s0 = 0; s0 < mj; s0 += 8) {
-            uint4 v[8];
+        acc = ld(in_lc + (size_t)(vo == root ? 0u : vo) * p.kbytes);
+        if (row == p.q) acc = comb16<T, OP>(acc, ld(in_lc + (size_t)root * p.kbytes));
+        for (uint32_t s0 = 0; s0 < mj; s0 += 4) {
+            uint4 v[4];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < 4; ++i) {
                 const uint32_t sp = s0 + i, vr = vbase + sp;
                 v[i] = make_uint4(0, 0, 0, 0);
-                if (sp < mj && sp != sstar && ((mask >> sp) & 1u)) v[i] = ld_stream(in_lc + (size_t)(vr == root ? 0u : vr) * p.kbytes);
+                if (sp < mj && sp != sstar && ((mask >> sp) & 1u)) v[i] = ld(in_lc + (size_t)(vr == root ? 0u : vr) * p.kbytes);
             }
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < 4; ++i) {
                 const uint32_t sp = s0 + i;
                 if (sp < mj && sp != sstar && ((mask >> sp) & 1u)) acc = comb16<T, OP>(acc, v[i]);
             }
@@ -82,37 +87,34 @@ __device__ __forceinline__ uint4 fold16_general(const Params& p, uint32_t root, 
     return acc;
 }
 
+// Position in memory of the i-th operand of a full group's fold: for float the member of the selected subtree
+// comes first, then the others ascending; for the exactly associative operations simply ascending.
+template <typename T>
+__device__ __forceinline__ uint32_t fold_member(uint32_t i, uint32_t sstar) {
+    return Ordered<T>::value ? (i == 0 ? sstar : i - (i <= sstar ? 1u : 0u)) : i;
+}
+
 // Fold of a full group all of whose members' messages are present, from m vectors `stride` bytes apart starting
-// at `ptr` (global or shared memory, LD loads 16 bytes). Own input first when the order is observable.
+// at `ptr` (global or shared memory, LD loads 16 bytes). MCAP > 0: all loads issued together.
 template <typename T, int OP, int MCAP, typename LD>
 __device__ __forceinline__ uint4 fold16_full(const char* ptr, uint32_t stride, uint32_t m, uint32_t sstar, LD ld) {
     uint4 acc;
     if (MCAP > 0) {
         uint4 v[MCAP > 0 ? MCAP : 1];
 #pragma unroll
-        for (int sp = 0; sp < MCAP; ++sp)
-            if ((uint32_t)sp < m) v[sp] = ld(ptr + (uint32_t)sp * stride);
+        for (int i = 0; i < MCAP; ++i)
+            if ((uint32_t)i < m) v[i] = ld(ptr + fold_member<T>(i, sstar) * stride);
         acc = v[0];
-        if (Ordered<T>::value) {
 #pragma unroll
-            for (int sp = 1; sp < MCAP; ++sp) if ((uint32_t)sp == sstar) acc = v[sp];
-#pragma unroll
-            for (int sp = 0; sp < MCAP; ++sp)
-                if ((uint32_t)sp < m && (uint32_t)sp != sstar) acc = comb16<T, OP>(acc, v[sp]);
-        } else {
-#pragma unroll
-            for (int sp = 1; sp < MCAP; ++sp)
-                if ((uint32_t)sp < m) acc = comb16<T, OP>(acc, v[sp]);
-        }
+        for (int i = 1; i < MCAP; ++i)
+            if ((uint32_t)i < m) acc = comb16<T, OP>(acc, v[i]);
     } else {
-        acc = ld(ptr + (Ordered<T>::value ? sstar : 0u) * stride);
-        for (uint32_t sp = 0; sp < m; ++sp)
-            if (sp != (Ordered<T>::value ? sstar : 0u)) acc = comb16<T, OP>(acc, ld(ptr + sp * stride));
+        acc = ld(ptr + fold_member<T>(0, sstar) * stride);
+#pragma unroll 4
+        for (uint32_t i = 1; i < m; ++i) acc = comb16<T, OP>(acc, ld(ptr + fold_member<T>(i, sstar) * stride));
     }
     return acc;
 }
-
-struct LdGlobal { __device__ __forceinline__ uint4 operator()(const char* q) const { return ld_stream(q); } };
 
 // A group is "plain" when it is full, every member's message reached the selected subtree's member, and neither
 // renumbered slot lies in it; then its fold needs one base address and constant strides.
@@ -122,18 +124,20 @@ __device__ __forceinline__ bool group_is_plain(const Params& p, uint32_t root, c
     return row < p.q && root - vbase >= p.m && extract_bits(inc, vbase, p.m) == full;   // unsigned wrap: root outside the row
 }
 
-template <typename T, int OP, int MCAP>
-__device__ __forceinline__ uint4 fold16(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
-                                        const char* in_lc, uint32_t row) {
-    if (group_is_plain(p, root, inc, row))
-        return fold16_full<T, OP, MCAP>(in_lc + (size_t)(row * p.m + 1) * p.kbytes, p.kbytes, p.m, sstar, LdGlobal());
-    return fold16_general<T, OP, MCAP>(p, root, sstar, inc, in_lc, row);
+// Any group, by the general routine (the careful path of the tiled kernels; rare). LD says where `in_lc`, the
+// scenario in process order, lives.
+template <typename T, int OP, typename LD>
+__device__ __forceinline__ uint4 fold16_careful(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
+                                             const char* in_lc, uint32_t row) {
+    return fold16_general<T, OP, 0, LD>(p, root, sstar, inc, in_lc, row);
 }
 
 // Tree phase inside a warp tile (Algorithm "reduce_non_root": data <- (data (op) child 1) (op) child 2).
 // valA: this lane's row of the tile's bottom level (lane row lr); valB: its row of the levels above (tile heap
 // index lr, level tB, position idxB; rowB its global row, hasB whether it exists). Returns the updated valB.
-template <typename T, int OP>
+// FULL: every row of the tile's upper levels and of its bottom level exists (no existence checks at all);
+// FULL_ABOVE: only the bottom level may be ragged (checked), everything above exists.
+template <typename T, int OP, bool FULL = false, bool FULL_ABOVE = false>
 __device__ __forceinline__ uint4 tile_tree_phase(uint4 valA, uint4 valB, uint32_t lw, uint32_t cwl, uint32_t C,
                                                  uint32_t lane, uint32_t lc, uint32_t tB, uint32_t idxB, uint32_t rowB,
                                                  bool hasB, uint32_t G) {
@@ -142,8 +146,8 @@ __device__ __forceinline__ uint4 tile_tree_phase(uint4 valA, uint4 valB, uint32_
         const uint32_t src1 = mine ? (((2 * idxB) << cwl) | lc) : lane;
         const uint4 c1 = shfl16(valA, src1), c2 = shfl16(valA, mine ? src1 + C : lane);
         if (mine) {
-            if (2 * rowB + 1 < G) valB = comb16<T, OP>(valB, c1);
-            if (2 * rowB + 2 < G) valB = comb16<T, OP>(valB, c2);
+            if (FULL || 2 * rowB + 1 < G) valB = comb16<T, OP>(valB, c1);
+            if (FULL || 2 * rowB + 2 < G) valB = comb16<T, OP>(valB, c2);
         }
     }
     for (int t = (int)lw - 2; t >= 0; --t) {
@@ -151,23 +155,66 @@ __device__ __forceinline__ uint4 tile_tree_phase(uint4 valA, uint4 valB, uint32_
         const uint32_t src1 = mine ? ((((2u << t) - 1 + 2 * idxB) << cwl) | lc) : lane;
         const uint4 c1 = shfl16(valB, src1), c2 = shfl16(valB, mine ? src1 + C : lane);
         if (mine) {
-            if (2 * rowB + 1 < G) valB = comb16<T, OP>(valB, c1);
-            if (2 * rowB + 2 < G) valB = comb16<T, OP>(valB, c2);
+            if (FULL || FULL_ABOVE || 2 * rowB + 1 < G) valB = comb16<T, OP>(valB, c1);
+            if (FULL || FULL_ABOVE || 2 * rowB + 2 < G) valB = comb16<T, OP>(valB, c2);
         }
     }
     return valB;
 }
 
+// Work items (warp tiles, then groups of rows above the tiles) that need the careful path: those containing a
+// group that is not plain (a member failed or is an in-operation victim, a renumbered slot, the short last group)
+// and those that are incomplete above their last level. One bit per item in `tspec`; all threads call.
+// Item numbering: tile i (rooted at heap row 2^Lt - 1 + i, D levels) is item i; rows [g*RW, (g+1)*RW) above the
+// tiles are item 2^Lt + g.
+static __device__ void mark_special_items(const Params& p, const Ctx* cx, const uint32_t* pf, uint32_t* tspec,
+                                          uint32_t Lt, uint32_t lw, uint32_t D) {
+    const uint32_t tid = threadIdx.x, nt = blockDim.x;
+    const uint32_t ntiles = 1u << Lt, ntop = ntiles - 1, RW = 1u << lw, ngroups = (ntop + RW - 1) >> lw;
+    const uint32_t nitems = ntiles + ngroups, root = cx->root, G = cx->G;
+    for (uint32_t w = tid; w < (nitems + 31) / 32 + 1; w += nt) tspec[w] = 0;
+    __syncthreads();
+    auto mark_row = [&](uint32_t j) {
+        const uint32_t lvl = ilog2u(j + 1);
+        const uint32_t it = lvl >= Lt ? ((j + 1) >> (lvl - Lt)) - ntiles : ntiles + (j >> lw);
+        atomicOr(&tspec[it >> 5], 1u << (it & 31));
+    };
+    for (uint32_t w = tid; w < p.W; w += nt) {
+        uint32_t word = pf[w];
+        while (word) {
+            const uint32_t b = __ffs(word) - 1; word &= word - 1;
+            const uint32_t v = renumber((w << 5) + b, root);
+            if (v && (v - 1) / p.m < G) mark_row((v - 1) / p.m);
+        }
+    }
+    if (tid < p.max_inop && cx->iv[tid] != FTC_INOP_UNUSED) {
+        const uint32_t v = renumber(cx->iv[tid], root);
+        if (v && (v - 1) / p.m < G) mark_row((v - 1) / p.m);
+    }
+    if (tid == 0) {
+        if (root != 0 && (root - 1) / p.m < G) mark_row((root - 1) / p.m);   // the slot that holds process 0's input
+        if (G > p.q) mark_row(p.q);                                          // the short last group
+    }
+    // tiles not complete down to their second-to-last level (the last row of level t of the tile rooted at j0 is
+    // ((j0+2) << t) - 2); their last level may be ragged, the common path checks it. And the ragged last group.
+    for (uint32_t it = tid; it < ntiles; it += nt)
+        if (((ntop + it + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= G) atomicOr(&tspec[it >> 5], 1u << (it & 31));
+    for (uint32_t g = tid; g < ngroups; g += nt)
+        if (((g + 1) << lw) > ntop || ((g + 1) << lw) > G) atomicOr(&tspec[(ntiles + g) >> 5], 1u << ((ntiles + g) & 31));
+    __syncthreads();
+}
+
 // The root's data after up-correction, for the case that no member of its (short, last) group lies in the
 // selected subtree: own input, then the members of that group whose message arrived.
-template <typename T, int OP>
+template <typename T, int OP, typename LD = LdGlobal>
 __device__ __forceinline__ uint4 fold_root16(const Params& p, uint32_t root, const uint32_t* inc, const char* in_lc) {
-    uint4 acc = ld_stream(in_lc + (size_t)root * p.kbytes);
+    const LD ld{};
+    uint4 acc = ld(in_lc + (size_t)root * p.kbytes);
     if (p.r) {
         const uint32_t vbase = p.q * p.m + 1, mask = extract_bits(inc, vbase, p.r);
         for (uint32_t sp = 0; sp < p.r; ++sp) {
             const uint32_t vr = vbase + sp;
-            if ((mask >> sp) & 1u) acc = comb16<T, OP>(acc, ld_stream(in_lc + (size_t)(vr == root ? 0u : vr) * p.kbytes));
+            if ((mask >> sp) & 1u) acc = comb16<T, OP>(acc, ld(in_lc + (size_t)(vr == root ? 0u : vr) * p.kbytes));
         }
     }
     return acc;

@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(kTiledMaxThreads, MINB) tiled_kernel(Params p)
     const uint32_t mask_words = ((sizeof(Ctx) / 4 + 3 * (p.W + 1)) + 3u) & ~3u;
     uint4* rootv = reinterpret_cast<uint4*>(smem + mask_words);      // [C] the root's own data after up-correction
     uint4* hv = rootv + p.C;                                          // [2^(Lt+1)-1][C] node values, heap order
+    uint32_t* tspec = reinterpret_cast<uint32_t*>(hv + (((size_t)2 << p.Lt) - 1) * p.C);   // careful-path bit per work item
 
     const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
     const uint32_t cwl = p.cw_log2, lw = 5 - cwl, RW = 1u << lw, Cmask = p.C - 1;
@@ -45,27 +46,39 @@ __global__ void __launch_bounds__(kTiledMaxThreads, MINB) tiled_kernel(Params p)
             continue;
         }
         if (p.is_allreduce) count_holders(p, cx, pf, unr);
+        mark_special_items(p, cx, pf, tspec, Lt, lw, lw + 1);
         const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
         const char* in_lc = reinterpret_cast<const char*>(p.in) + s * (size_t)p.P * p.kbytes + lc * 16;
 
         for (uint32_t it = wid; it < nitems; it += nw) {
+            const bool careful = it < ntiles + ngroups && test_bit(tspec, it);      // warp-uniform
             if (it < ntiles) {
                 // ---- one tile: the sub-heap below heap row j0, lw+1 levels ----
                 const uint32_t j0 = ntop + it;
-                if (j0 >= G) continue;
                 const uint32_t rowA = ((j0 + 1) << lw) - 1 + lr;              // bottom level of the tile
                 uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
                 const uint32_t tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB);
                 const uint32_t rowB = ((j0 + 1) << tB) - 1 + idxB;            // this lane's row of the upper levels
+                if (!careful) {
+                    // all rows plain, the levels above the bottom complete: constant strides; only the bottom may be ragged
+                    if (rowA < G) valA = fold16_full<T, OP, MCAP>(in_lc + (size_t)(rowA * p.m + 1) * p.kbytes, p.kbytes, p.m, sstar, LdGlobal());
+                    const bool hasBp = lr < RW - 1;
+                    if (hasBp) valB = fold16_full<T, OP, MCAP>(in_lc + (size_t)(rowB * p.m + 1) * p.kbytes, p.kbytes, p.m, sstar, LdGlobal());
+                    valB = tile_tree_phase<T, OP, false, true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasBp, G);
+                    if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
+                    continue;
+                }
+                if (j0 >= G) continue;
                 const bool hasB = lr < RW - 1 && rowB < G;
-                if (rowA < G) valA = fold16<T, OP, MCAP>(p, root, sstar, inc, in_lc, rowA);
-                if (hasB) valB = fold16<T, OP, MCAP>(p, root, sstar, inc, in_lc, rowB);
+                if (rowA < G) valA = fold16_careful<T, OP, LdGlobal>(p, root, sstar, inc, in_lc, rowA);
+                if (hasB) valB = fold16_careful<T, OP, LdGlobal>(p, root, sstar, inc, in_lc, rowB);
                 valB = tile_tree_phase<T, OP>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                 if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
             } else if (it < ntiles + ngroups) {
                 // ---- rows above the tiles: fold now, combine later ----
                 const uint32_t row = ((it - ntiles) << lw) + lr;
-                if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold16<T, OP, MCAP>(p, root, sstar, inc, in_lc, row);
+                if (!careful) hv[(size_t)row * p.C + lc] = fold16_full<T, OP, MCAP>(in_lc + (size_t)(row * p.m + 1) * p.kbytes, p.kbytes, p.m, sstar, LdGlobal());
+                else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold16_careful<T, OP, LdGlobal>(p, root, sstar, inc, in_lc, row);
             } else if (sstar >= p.r) {
                 if (lr == 0) rootv[lc] = fold_root16<T, OP>(p, root, inc, in_lc);
             }
@@ -95,7 +108,9 @@ __global__ void __launch_bounds__(kTiledMaxThreads, MINB) tiled_kernel(Params p)
 
 static size_t tiled_smem_bytes(const Params& p) {
     size_t mask_words = ((sizeof(Ctx) / 4 + 3 * (size_t)(p.W + 1)) + 3u) & ~(size_t)3u;
-    return mask_words * 4 + (size_t)p.C * 16 + (((size_t)2 << p.Lt) - 1) * p.C * 16;
+    const uint32_t lw = 5 - p.cw_log2, ntiles = 1u << p.Lt;
+    const size_t nitems = ntiles + ((ntiles - 1 + (1u << lw) - 1) >> lw);
+    return mask_words * 4 + (size_t)p.C * 16 + (((size_t)2 << p.Lt) - 1) * p.C * 16 + ((nitems + 31) / 32 + 1) * 4;
 }
 
 bool tiled_supported(Params& p, int smem_optin_bytes) {
