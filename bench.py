@@ -206,6 +206,21 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------------
+def max_over_ranks(value: float, dist, device) -> float:
+    """Largest value over all ranks (step times are reported as the slowest rank's)."""
+    if dist is None:
+        return value
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, scenarios_per_rank: int, ms_per_step: float) -> float:
+    """Scenarios per second of the whole job: every rank processed its own scenarios in the slowest rank's time."""
+    return world * scenarios_per_rank / (ms_per_step / 1e3)
+
+
 def upload(w, torch):
     d_pf = torch.from_numpy(w.prefail.view(np.int32)).cuda()
     d_inop = None if w.inop is None else torch.from_numpy(np.ascontiguousarray(w.inop).view(np.int32)).cuda()
@@ -237,6 +252,12 @@ def run_gpu(args):
     desc0 = B.make_desc(probe.P, probe.f, probe.k, B.dtype_code(tdt), probe.op)
     sched = B.ftc_schedule_info(desc0)
     w = make_workload(name, S, rank * S, sched["rounds_attempt"])          # each rank its own scenarios
+    if args.collective:
+        w.collective = args.collective
+    if args.failure_free:
+        w.prefail[:] = 0
+        if w.inop is not None:
+            w.inop[:, :, 0] = sc.UNUSED
     allred = w.collective == "allreduce"
     kflags = {"auto": 0, "direct": B.FTC_KERNEL_DIRECT, "generic": B.FTC_KERNEL_GENERIC}[args.kernel]
     desc = B.make_desc(w.P, w.f, w.k, B.dtype_code(tdt), w.op, root=-1 if w.roots is not None else 0,
@@ -277,12 +298,9 @@ def run_gpu(args):
     clocks = sampler.stop() if sampler else None
     per_launch_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
     total_ms = ev[0].elapsed_time(ev[-1])
-    if dist:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, torch.device("cuda", local))
     ms_per_step = total_ms / args.steps
-    value = world * S / (ms_per_step / 1e3)
+    value = whole_job_value(world, S, ms_per_step)
 
     e2e = None
     if not args.kernel_only:
@@ -307,10 +325,7 @@ def run_gpu(args):
         for _ in range(e2e_steps):
             fn_host(desc, Se, h_x, h_pf, h_inop, h_roots, h_out, h_st, staging)     # synchronises its stream itself
         e2e_s = (time.perf_counter() - t0) / e2e_steps
-        if dist:
-            t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = max_over_ranks(e2e_s, dist, torch.device("cuda", local))
         h2d = Se * (bytes_per_scenario(w) - w.k * ESZ[np.dtype(w.dtype).name] - 16)
         d2h = Se * (w.k * ESZ[np.dtype(w.dtype).name] + 16)
         same = bool((h_st.numpy() == d_st[:Se].cpu().numpy()).all() and
@@ -356,7 +371,8 @@ def run_gpu(args):
         "vs_baseline": None, "dtype": {"int32": "i32", "int64": "i64", "uint64": "u64", "float32": "f32"}[np.dtype(w.dtype).name],
         "data": "synthetic",
         "process_rounds_per_sec": value * w.P * R,
-        "config": {"workload": f"{name}: {DESCRIPTION[name]}", "scenarios_per_step_per_gpu": S,
+        "config": {"workload": f"{name}: {DESCRIPTION[name]}" + (f" [collective={args.collective}]" if args.collective else "")
+                   + (" [failure-free]" if args.failure_free else ""), "scenarios_per_step_per_gpu": S,
                    "input_bytes_per_step_per_gpu": S * w.P * w.k * ESZ[np.dtype(w.dtype).name],
                    "cache": "inputs larger than L2, no flush", "kernel": B.ftc_kernel_name(desc, allred),
                    "rounds_per_scenario": R, "ok_scenarios": int(((status[:, 0] & 0xFF) == 0).sum())},
@@ -384,6 +400,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="scenarios per step per GPU")
     ap.add_argument("--e2e-scenarios", type=int, default=0)
     ap.add_argument("--kernel", default="auto", choices=["auto", "direct", "generic"], help="force a kernel family")
+    ap.add_argument("--collective", default="", choices=["", "reduce", "allreduce"], help="override the workload's collective")
+    ap.add_argument("--failure-free", action="store_true", help="clear every failure of the workload (diagnostic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU legs (for profiler runs)")
     args = ap.parse_args()

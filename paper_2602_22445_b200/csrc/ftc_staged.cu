@@ -9,7 +9,6 @@
 // sub-heap of XL levels by itself (post-order, values in registers), the lw levels above are combined with warp
 // shuffles. Groups that are not "plain" (a missing member, a renumbered slot, the short last group) are folded
 // from global memory by the general routine; they are a handful per scenario.
-#include <cstdlib>
 #include "ftc_tile_common.cuh"
 #include "ftc_kernels.h"
 
@@ -141,6 +140,50 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) staged_kernel(Params p, 
     uint32_t phase_bits = 0;                                      // bit b: parity to wait for on buffer b
     uint32_t cphase = 0;
 
+    // ---- the copy pipeline of this warp: it runs over the flat sequence (scenario, work item) of everything the
+    // warp will process, g.nbuf items ahead of the item being computed, across scenario boundaries. What is copied
+    // depends on the geometry only (rows that exist for the largest subtree), never on a scenario's decode.
+    const uint32_t n_my = wid < nitems ? (nitems - wid + nw - 1) / nw : 0;     // work items of this warp per scenario
+    uint64_t is_s = blockIdx.x;                                   // scenario and local item of the next copy to issue
+    uint32_t is_i = 0, iseq = 0, cseq = 0;                        // items issued / consumed so far
+    uint32_t pending = 0;                                         // bit b: buffer b has a copy in flight
+    auto issue_next = [&]() {
+        if (WHOLE || n_my == 0 || is_s >= p.S) return;
+        const uint32_t it = wid + is_i * nw, b = iseq % g.nbuf;
+        const char* src_s = reinterpret_cast<const char*>(p.in) + is_s * scen_bytes;
+        uint32_t first_row = 0, nrows = 0, dst_off = 0;
+        if (it < ntiles) {                                        // lane t copies level t of the tile
+            const uint32_t j0 = ntop + it;
+            if (lane < D && j0 < p.Gmax) { first_row = ((j0 + 1) << lane) - 1; nrows = 1u << lane; dst_off = ((1u << lane) - 1) * rowbytes; }
+        } else if (it < ntiles + ngroups) {
+            if (lane == 0) { first_row = (it - ntiles) << lw; nrows = min(RW, ntop - first_row); }
+        }
+        uint64_t b0 = ((uint64_t)first_row * p.m + 1) * p.kbytes, b1 = ((uint64_t)(first_row + nrows) * p.m + 1) * p.kbytes;
+        if (b1 > scen_bytes) b1 = scen_bytes;
+        const uint32_t bytes = (nrows && b1 > b0) ? (uint32_t)(b1 - b0) : 0u;
+        const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, bytes);
+        if (total) {
+            if (lane == 0) mbar_expect_tx(bar0 + b * 8, total);
+            __syncwarp();
+            if (bytes) bulk_g2s(smem_addr(tiles + (size_t)b * g.tile_cap + dst_off), src_s + b0, bytes, bar0 + b * 8);
+            pending |= 1u << b;
+        }
+        ++iseq;
+        if (++is_i == n_my) { is_i = 0; is_s += gridDim.x; }
+    };
+    // the buffer of the item about to be computed: wait for its copy if one was issued
+    auto acquire = [&]() {
+        const uint32_t b = WHOLE ? 0u : cseq % g.nbuf;
+        if (!WHOLE && ((pending >> b) & 1u)) {
+            if (!mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u)) { if (lane == 0) atomicOr(&cx->pad, 1u); }
+            phase_bits ^= 1u << b; pending &= ~(1u << b);
+        }
+        return b;
+    };
+    // every lane is done with the buffer: hand it to the next copy
+    auto release = [&]() { __syncwarp(); ++cseq; issue_next(); };
+    if (!WHOLE) for (uint32_t i = 0; i < g.nbuf; ++i) issue_next();
+
     for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {
         const char* in_s = reinterpret_cast<const char*>(p.in) + s * scen_bytes;
         if (WHOLE && wid == 0) {
@@ -159,6 +202,7 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) staged_kernel(Params p, 
         }
         if (cx->code != FTC_ST_OK) {
             if (tid < p.C) reinterpret_cast<uint4*>(out_s)[tid] = make_uint4(0, 0, 0, 0);
+            for (uint32_t i = 0; i < n_my; ++i) { acquire(); release(); }        // its copies were issued: consume them unused
             if (tid == 0) write_status_rec(p, s, cx);
             __syncthreads();
             continue;
@@ -168,39 +212,8 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) staged_kernel(Params p, 
         const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
         const char* in_lc = (WHOLE ? wbuf : in_s) + lc * 16;      // the scenario in process order, for the general fold
 
-        // Issue the bulk copies of work item `it` into buffer b: lane t copies level t of the tile.
-        auto issue = [&](uint32_t it, uint32_t b) {
-            if (WHOLE) return false;
-            uint32_t first_row = 0, nrows = 0, dst_off = 0;
-            if (it < ntiles) {
-                const uint32_t j0 = ntop + it;
-                if (lane < D && j0 < G) { first_row = ((j0 + 1) << lane) - 1; nrows = 1u << lane; dst_off = ((1u << lane) - 1) * rowbytes; }
-            } else if (it < ntiles + ngroups) {
-                if (lane == 0) { first_row = (it - ntiles) << lw; nrows = min(RW, ntop - first_row); }
-            }
-            uint64_t b0 = ((uint64_t)first_row * p.m + 1) * p.kbytes, b1 = ((uint64_t)(first_row + nrows) * p.m + 1) * p.kbytes;
-            if (b1 > scen_bytes) b1 = scen_bytes;
-            const uint32_t bytes = (nrows && b1 > b0) ? (uint32_t)(b1 - b0) : 0u;
-            const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, bytes);
-            if (total) {
-                if (lane == 0) mbar_expect_tx(bar0 + b * 8, total);
-                __syncwarp();
-                if (bytes) bulk_g2s(smem_addr(tiles + (size_t)b * g.tile_cap + dst_off), in_s + b0, bytes, bar0 + b * 8);
-            }
-            return total != 0;
-        };
-
-        const uint32_t n_my = wid < nitems ? (nitems - wid + nw - 1) / nw : 0;
-        uint32_t pending = 0;                                     // bit b: buffer b has a copy in flight
-        for (uint32_t i = 0; i < g.nbuf && i < n_my; ++i)
-            if (issue(wid + i * nw, i)) pending |= 1u << i;
-
         for (uint32_t i = 0; i < n_my; ++i) {
-            const uint32_t it = wid + i * nw, b = i % g.nbuf;
-            if ((pending >> b) & 1u) {
-                if (!mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u)) { if (lane == 0) atomicOr(&cx->pad, 1u); }
-                phase_bits ^= 1u << b; pending &= ~(1u << b);
-            }
+            const uint32_t it = wid + i * nw, b = acquire();
             const char* buf_lc = (WHOLE ? wbuf : tiles + (size_t)b * g.tile_cap) + lc * 16;
             const bool careful = it < ntiles + ngroups && test_bit(tspec, it);      // warp-uniform
             if (it < ntiles) {
@@ -232,8 +245,7 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) staged_kernel(Params p, 
             } else if (sstar >= p.r) {
                 if (lr == 0) rootv[lc] = WHOLE ? fold_root16<T, OP, LdShared>(p, root, inc, in_lc) : fold_root16<T, OP, LdGlobal>(p, root, inc, in_lc);
             }
-            __syncwarp();                                         // every lane is done with buffer b
-            if (i + g.nbuf < n_my && issue(wid + (i + g.nbuf) * nw, b)) pending |= 1u << b;
+            release();
         }
         __syncthreads();
         // ---- levels above the tiles, leaves first (Algorithm "reduce_non_root") ----
@@ -262,13 +274,6 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) staged_kernel(Params p, 
 }
 
 // ---- host side ----
-static uint32_t env_u32(const char* name, uint32_t dflt) {
-    const char* e = getenv(name);
-    if (!e) return dflt;
-    int v = atoi(e);
-    return v > 0 ? (uint32_t)v : dflt;
-}
-
 static bool staged_geometry(Params& p, int smem_optin, uint32_t XL, StagedGeom& g) {
     if (p.kbytes % 16) return false;
     const uint32_t C = p.kbytes / 16;
@@ -283,15 +288,16 @@ static bool staged_geometry(Params& p, int smem_optin, uint32_t XL, StagedGeom& 
     if (cap > 64 * 1024) return false;
     const uint32_t RW = 1u << lw, ntiles = 1u << p.Lt;
     const uint32_t nitems = ntiles + ((ntiles - 1 + RW - 1) >> lw) + 1;
-    uint32_t warps = env_u32("FTC_STAGED_WARPS", 0);
-    if (!warps) { warps = 1; while (warps < 8 && warps * 2 * 16 <= nitems) warps *= 2; }   // >= 16 work items per warp
-    if (warps > kStagedMaxThreads / 32) warps = kStagedMaxThreads / 32;
-    uint32_t nbuf = env_u32("FTC_STAGED_NBUF", 1);
-    if (nbuf > 4) nbuf = 4;
-    // small scenarios are staged whole (three blocks of them fit an SM), large ones tile by tile
+    // Launch shape, from sweeps on B200: what limits the kernel is the number of resident warps doing the combine
+    // work, and shared memory per warp decides that number. So: one buffer per warp, and blocks just large enough
+    // to give every warp at least 16 work items per scenario (at most 8 warps).
+    uint32_t warps = 1;
+    while (warps < 8 && warps * 2 * 16 <= nitems) warps *= 2;
+    uint32_t nbuf = 1;
+    // tiny scenarios (up to 16 KB) are staged whole with one copy, larger ones tile by tile
     const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
-    g.whole = scen_bytes <= env_u32("FTC_STAGED_WHOLE_MAX", 72 * 1024) ? 1u : 0u;
-    if (g.whole) { nbuf = 0; if (!env_u32("FTC_STAGED_WARPS", 0)) { warps = 1; while (warps < 8 && warps * 2 * 4 <= nitems) warps *= 2; } }
+    g.whole = scen_bytes <= 16 * 1024 ? 1u : 0u;
+    if (g.whole) nbuf = 0;
     size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
     o = (o + 15) & ~(size_t)15; g.off_special = (uint32_t)o;
     o += ((((size_t)nitems + 31) / 32 + 1) * 4 + 15) & ~(size_t)15;
@@ -312,8 +318,7 @@ static bool staged_geometry(Params& p, int smem_optin, uint32_t XL, StagedGeom& 
 }
 
 static uint32_t staged_xl(const Params& p) {
-    uint32_t xl = env_u32("FTC_STAGED_XL", 0);
-    if (xl >= 1 && xl <= 3) return xl;
+    uint32_t xl;
     // deepest lane-local sub-heap that keeps a tile (all its levels, every member) within 12 KB
     if (p.kbytes % 16 || p.kbytes > 512) return 1;
     uint32_t C = p.kbytes / 16, cwl = 0; while ((1u << cwl) < C) ++cwl;

@@ -10,7 +10,6 @@
 //   * rows above level Lt are folded by the same lanes into shared memory and combined there level by level.
 // Every input byte is read from global memory exactly once; the combine order is the schedule's order, so
 // float32 sums come out bit-identical to a message-by-message execution.
-#include <cstdlib>
 #include "ftc_tile_common.cuh"
 #include "ftc_kernels.h"
 
