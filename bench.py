@@ -206,6 +206,29 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------------
+def kernel_source_hash() -> str:
+    """Hash of the CUDA sources: ncu counters taken from an older kernel must not be quoted for a newer one."""
+    import glob
+    import hashlib
+    h = hashlib.sha256()
+    base = os.path.join(ROOT, "paper_2602_22445_b200", "csrc")
+    for f in sorted(glob.glob(os.path.join(base, "*.cu")) + glob.glob(os.path.join(base, "*.cuh")) + glob.glob(os.path.join(base, "*.h"))):
+        h.update(open(f, "rb").read())
+    return h.hexdigest()[:16]
+
+
+def kernel_traffic(name: str, S: int):
+    """DRAM read+write bytes of one launch over S scenarios, scaled from the committed ncu capture of a 2 GiB batch
+    (traffic is proportional to the scenarios of a launch); None when there is no capture or the sources changed."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    rec = json.load(open(path))
+    if rec.get("source_sha256_16") != kernel_source_hash() or name not in rec or not rec[name].get("valid"):
+        return None
+    return rec[name]["dram_bytes_per_scenario"] * S
+
+
 def max_over_ranks(value: float, dist, device) -> float:
     """Largest value over all ranks (step times are reported as the slowest rank's)."""
     if dist is None:
@@ -347,12 +370,7 @@ def run_gpu(args):
     bytes_launch = S * bytes_per_scenario(w)
     avg_launch_ms = sum(per_launch_ms) / len(per_launch_ms)
     achieved = bytes_launch / (avg_launch_ms / 1e3) / 1e9
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
-        tr = json.load(open(tpath)).get(name)
-        if tr and tr.get("valid"):
-            traffic = tr["dram_bytes_per_scenario"] * S
+    traffic = kernel_traffic(name, S)
 
     # ---- the oracle beside it, on a bounded sample ----
     cpu = None
