@@ -148,7 +148,10 @@ FTC_API int ftc_reduce_batch(const ftc_desc_t* desc, uint64_t S, const void* d_i
 /*
  * Corrected allreduce (Algorithm "Allreduce": reduce to a root candidate, broadcast from it, next candidate if
  * it had failed before the operation). Arguments as for ftc_reduce_batch; desc->root / d_roots give the first
- * candidate. d_out is [S][k] (the value every holder has) or, with FTC_OUT_EXPANDED, [S][P][k].
+ * candidate. d_out is [S][k] (the value every holder has) or, with FTC_OUT_EXPANDED, [S][P][k]: the value in the
+ * slot of every process that is alive at the end and holds it, zero bytes in all other slots. The expanded form
+ * needs ftc_workspace_bytes() of 256-byte aligned workspace (the compact results pass through it); the host-buffer
+ * variants and ftc_reduce_batch do not offer it (FTC_EUNSUPPORTED).
  */
 FTC_API int ftc_allreduce_batch(const ftc_desc_t* desc, uint64_t S, const void* d_in, const uint32_t* d_prefail,
                         const ftc_inop_t* d_inop, const uint32_t* d_roots, void* d_out, uint32_t* d_status,

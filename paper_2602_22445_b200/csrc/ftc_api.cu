@@ -58,9 +58,17 @@ static KernelKind pick_kernel(Params& p, const DeviceInfo& di) {
     return tiled_supported(p, di.smem_optin) ? K_TILED : K_GENERIC;
 }
 
+static size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+// Bytes at the front of the workspace that hold the compact results while the expanded output is produced.
+static size_t compact_area(const Params& p) {
+    return (p.flags & FTC_OUT_EXPANDED) ? up256((size_t)p.S * p.kbytes) : 0;
+}
+
 static size_t workspace_for(Params& p, const DeviceInfo& di) {
-    if (pick_kernel(p, di) != K_GENERIC) return 0;
-    return (size_t)generic_grid(p, di.sm_count) * p.Gmax * p.kbytes;
+    size_t need = compact_area(p);
+    if (pick_kernel(p, di) == K_GENERIC) need += (size_t)generic_grid(p, di.sm_count) * p.Gmax * p.kbytes;
+    return need;
 }
 
 static bool aligned16(const void* ptr) { return (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; }
@@ -71,7 +79,8 @@ static int run_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const
     Params p;
     int rc = fill_params(desc, S, is_allreduce, p);
     if (rc != FTC_OK) return rc;
-    if (desc->flags & FTC_OUT_EXPANDED) return FTC_EUNSUPPORTED;
+    const bool expanded = (desc->flags & FTC_OUT_EXPANDED) != 0;
+    if (expanded && !is_allreduce) return FTC_EUNSUPPORTED;     // a reduce delivers at the root only
     if (S == 0) return FTC_OK;
     if (!d_in || !d_prefail || !d_out || !d_status) return FTC_EINVAL;
     if (p.max_inop && !d_inop) return FTC_EINVAL;
@@ -79,7 +88,11 @@ static int run_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const
     if (!aligned16(d_in) || !aligned16(d_out) || !aligned16(d_status)) return FTC_EINVAL;
     DeviceInfo di;
     if ((rc = device_info(di)) != FTC_OK) return rc;
-    p.in = d_in; p.prefail = d_prefail; p.inop = d_inop; p.roots = d_roots; p.out = d_out; p.status = d_status;
+    const size_t front = compact_area(p);
+    if (expanded && (!d_ws || ws_bytes < front || (reinterpret_cast<uintptr_t>(d_ws) & 255u))) return FTC_EWORKSPACE;
+    p.in = d_in; p.prefail = d_prefail; p.inop = d_inop; p.roots = d_roots; p.status = d_status;
+    p.out = expanded ? d_ws : d_out;                            // compact results first, expanded afterwards
+    if (expanded) { d_ws = static_cast<char*>(d_ws) + front; ws_bytes -= front; }
     const int tsel = type_select(desc->dtype, desc->op);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
@@ -95,11 +108,11 @@ static int run_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const
         p.ws = d_ws;
         e = launch_generic(p, tsel, di.sm_count, st);
     }
+    if (e == cudaSuccess && expanded) e = launch_expand(p, p.out, d_out, di.sm_count, st);
     return e == cudaSuccess ? FTC_OK : FTC_ECUDA;
 }
 
 struct StagingLayout { size_t in, prefail, inop, roots, out, status, ws, total; };
-static size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
 static StagingLayout staging_layout(Params& p, uint64_t chunk, const DeviceInfo& di) {
     StagingLayout L; size_t o = 0;
     L.in = o; o += up256(chunk * (size_t)p.P * p.kbytes);

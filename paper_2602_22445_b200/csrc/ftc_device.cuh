@@ -214,11 +214,19 @@ static __device__ void decode_scenario(const Params& p, uint64_t s, Ctx* cx, uin
 
 // Broadcast of the allreduce: how many processes are alive at the end of the attempt and hold the value.
 // `unr` (W+1 words) receives bit v for every renumbered process the tree-down phase does not reach.
+// `hold` (optional, W+1 words) receives the holders as a bitmask over the caller's process ids.
 // All threads of the block call it after decode_scenario returned with code OK.
-static __device__ void count_holders(const Params& p, Ctx* cx, const uint32_t* pf, uint32_t* unr) {
+static __device__ void count_holders(const Params& p, Ctx* cx, const uint32_t* pf, uint32_t* unr, uint32_t* hold = nullptr) {
     const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
     const uint32_t root = cx->root, base = cx->base;
-    for (uint32_t w = tid; w <= p.W; w += nt) unr[w] = 0;
+    for (uint32_t w = tid; w <= p.W; w += nt) {
+        unr[w] = 0;
+        if (hold) {                                   // start from everybody who had not failed before the operation
+            uint32_t word = w < p.W ? ~pf[w] : 0u;
+            if (w == p.W - 1 && (p.P & 31)) word &= (1u << (p.P & 31)) - 1u;
+            hold[w] = word;
+        }
+    }
     __syncthreads();
     // every process that does not forward the value down the tree cuts off all its descendants
     const uint32_t nwords_round = (p.W + 31) & ~31u;
@@ -247,7 +255,10 @@ static __device__ void count_holders(const Params& p, Ctx* cx, const uint32_t* p
         for (uint32_t i = 0; i < p.max_inop; ++i) {
             if (cx->iv[i] == FTC_INOP_UNUSED || !((cx->ifirst >> i) & 1u)) continue;
             uint32_t v = renumber(cx->iv[i], root), t = local_round(cx->ir[i], base);
-            if (lane == 0 && t < p.Ratt) atomicAdd(&cx->ndead_end, 1u);
+            if (lane == 0 && t < p.Ratt) {
+                atomicAdd(&cx->ndead_end, 1u);
+                if (hold) atomicAnd(&hold[cx->iv[i] >> 5], ~(1u << (cx->iv[i] & 31)));
+            }
             if (!v) continue;
             uint32_t j = (v - 1) / p.m, sv = (v - 1) % p.m, Gs = p.q + (sv < p.r ? 1u : 0u), d = 1 + ilog2u(j + 1);
             if (t > p.Rred + d) continue;                  // it does forward: tree-down send of depth d is round f+H+d
@@ -278,7 +289,10 @@ static __device__ void count_holders(const Params& p, Ctx* cx, const uint32_t* p
                 uint32_t tu = local_round(fail_round(p, cx, pf, renumber(u, root)), base);
                 if (tu > p.Rred + p.H + partner_slot(p, j, su, sv)) rescued = true;
             }
-            if (!rescued) ++lost;
+            if (!rescued) {
+                ++lost;
+                if (hold) { const uint32_t ph = renumber(v, root); atomicAnd(&hold[ph >> 5], ~(1u << (ph & 31))); }
+            }
         }
     }
     lost = __reduce_add_sync(0xFFFFFFFFu, lost);

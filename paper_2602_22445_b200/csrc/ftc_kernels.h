@@ -28,6 +28,9 @@ cudaError_t launch_tiled(const Params& p, int tsel, int sm_count, cudaStream_t s
 bool staged_supported(Params& p, int smem_optin_bytes);
 cudaError_t launch_staged(const Params& p, int tsel, int sm_count, int smem_optin_bytes, cudaStream_t st);
 
+// Expanded allreduce output from the compact results (one value per scenario) left by the main kernel.
+cudaError_t launch_expand(const Params& p, const void* compact, void* out, int sm_count, cudaStream_t st);
+
 cudaError_t launch_fill(uint32_t kind, uint64_t seed, uint64_t first, uint64_t S, uint32_t P, uint32_t k, void* out,
                         int sm_count, cudaStream_t st);
 

@@ -256,3 +256,52 @@ def test_host_buffer_entry_points_match_device_ones():
     small = torch.empty(1024, dtype=torch.uint8, device="cuda")
     assert B.ftc_allreduce_batch_host(desc, w.S, x, w.prefail, np.ascontiguousarray(w.inop), None, out, st, small,
                                       check=False) == B.FTC_EWORKSPACE
+
+
+# ---------------------------------------------------------------------------------------------
+# expanded allreduce output: the value in the slot of every holder, zeros elsewhere
+# ---------------------------------------------------------------------------------------------
+def run_gpu_expanded(x, f, op, pf, inop, roots, flags):
+    import torch
+    d_x = to_dev(x)
+    S, P, k = d_x.shape
+    max_inop = 0 if inop is None else inop.shape[1]
+    desc = B.make_desc(P, f, k, B.dtype_code(d_x.dtype), op, root=-1, max_inop=max_inop, flags=flags | B.FTC_OUT_EXPANDED)
+    d_out = torch.empty((S, P, k), dtype=d_x.dtype, device="cuda")
+    d_out.view(torch.uint8).fill_(0x5A)
+    d_st = torch.full((S, 4), 0x7FFFFFFF, dtype=torch.int32, device="cuda")
+    wsb = B.ftc_workspace_bytes(desc, S, True)
+    assert wsb >= S * k * x.dtype.itemsize
+    d_ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+    B.ftc_allreduce_batch(desc, S, d_x, to_dev(pf), to_dev(inop) if max_inop else None, to_dev(roots), d_out, d_st, d_ws)
+    torch.cuda.synchronize()
+    return to_host(d_out, x.dtype), d_st.cpu().numpy().view(np.uint32)
+
+
+@pytest.mark.parametrize("flags", KERNELS)
+def test_expanded_output_matches_oracle_holders(flags):
+    rng = np.random.Generator(np.random.PCG64(77))
+    for P, f, k, dtype in ((10, 2, 4, np.uint64), (37, 1, 3, np.int32), (64, 3, 8, np.float32), (200, 0, 4, np.int32)):
+        S = 60
+        x = rng.standard_normal((S, P, k)).astype(np.float32) if dtype == np.float32 else \
+            rng.integers(0, 2**31 - 1, size=(S, P, k)).astype(dtype)
+        pf = sc.picks_to_masks(sc.random_subsets(rng, S, P, rng.integers(0, f + 3, size=S), lo=0), P)
+        R = O.schedule(P, f)["rounds_attempt"]
+        inop = np.zeros((S, 2, 2), dtype=np.uint32)
+        inop[:, :, 0] = rng.integers(f + 1, P, size=(S, 2))
+        inop[:, :, 1] = rng.integers(0, R + 3, size=(S, 2))
+        inop[rng.random((S, 2)) < 0.3, 0] = sc.UNUSED
+        roots = np.zeros(S, dtype=np.uint32)
+        got, st = run_gpu_expanded(x, f, "sum", pf, inop, roots, flags)
+        for i in range(S):
+            d = O.run(x[i], f, "sum", pf[i], inop=[tuple(e) for e in inop[i]], root=0, allreduce=True, detail=True)
+            assert np.array_equal(st[i], d["status"]), (P, i)
+            assert np.array_equal(got[i].view(np.uint8), d["expanded"].view(np.uint8)), (P, f, i, d["code"])
+
+
+def test_expanded_needs_allreduce_and_workspace():
+    import torch
+    z = torch.zeros(4096, dtype=torch.int32, device="cuda")
+    d = B.make_desc(8, 1, 4, B.FTC_I32, "sum", flags=B.FTC_OUT_EXPANDED)
+    assert B.ftc_reduce_batch(d, 1, z, z, None, None, z, z, z, check=False) == B.FTC_EUNSUPPORTED
+    assert B.ftc_allreduce_batch(d, 1, z, z, None, None, z, z, None, check=False) == B.FTC_EWORKSPACE
