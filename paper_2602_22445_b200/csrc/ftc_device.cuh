@@ -219,6 +219,26 @@ static __device__ void decode_scenario(const Params& p, uint64_t s, Ctx* cx, uin
 static __device__ void count_holders(const Params& p, Ctx* cx, const uint32_t* pf, uint32_t* unr, uint32_t* hold = nullptr) {
     const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
     const uint32_t root = cx->root, base = cx->base;
+    // With at most f failed processes one root subtree is free of failures: all its processes are reached by the
+    // tree and alive throughout, every group has a member in it (the short last group has the root instead), so
+    // the correction phase reaches every process that is alive at the end. No marking is needed then.
+    if (cx->npre + __popc(cx->ifirst) <= p.f) {            // uniform: shared values, read after a barrier
+        for (uint32_t w = tid; hold && w <= p.W; w += nt) {
+            uint32_t word = w < p.W ? ~pf[w] : 0u;
+            if (w == p.W - 1 && (p.P & 31)) word &= (1u << (p.P & 31)) - 1u;
+            hold[w] = word;
+        }
+        __syncthreads();
+        if (tid < p.max_inop && cx->iv[tid] != FTC_INOP_UNUSED && ((cx->ifirst >> tid) & 1u) &&
+            local_round(cx->ir[tid], base) < p.Ratt) {
+            atomicAdd(&cx->ndead_end, 1u);
+            if (hold) atomicAnd(&hold[cx->iv[tid] >> 5], ~(1u << (cx->iv[tid] & 31)));
+        }
+        __syncthreads();
+        if (tid == 0) cx->holders = p.P - cx->npre - cx->ndead_end;
+        __syncthreads();
+        return;
+    }
     for (uint32_t w = tid; w <= p.W; w += nt) {
         unr[w] = 0;
         if (hold) {                                   // start from everybody who had not failed before the operation

@@ -41,6 +41,12 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
     return false;
 }
 
+// words of one per-item bitmap
+__host__ __device__ inline uint32_t nitems_words(uint32_t Lt, uint32_t lw) {
+    const uint32_t ntiles = 1u << Lt, nitems = ntiles + ((ntiles - 1 + (1u << lw) - 1) >> lw);
+    return (nitems + 31) / 32 + 1;
+}
+
 struct StagedGeom {
     uint32_t nwarps, nbuf, tile_cap;       // warps per block, buffers per warp, bytes per buffer (multiple of 128)
     uint32_t whole;                        // 1: the whole scenario is staged in one block-wide buffer
@@ -60,28 +66,39 @@ __device__ __forceinline__ uint4 fold_plain_staged(const Params& p, uint32_t sst
     return fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdShared());
 }
 
-// Fold of one group on the careful path: by the general routine from the scenario in process order (`in_lc`:
-// global memory, or the block-wide shared copy when WHOLE).
+// Fold of one group on the careful path: a full group without a renumbered slot comes from its staged copy
+// (`srow_lc`, NULL when the row is not in the buffer) under its arrival mask; the others by the general routine from the scenario in process order (`in_lc`: global
+// memory, or the block-wide shared copy when WHOLE).
 template <typename T, int OP, bool WHOLE>
 __device__ __forceinline__ uint4 fold_staged(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
-                                             const char* in_lc, uint32_t row) {
+                                             const char* in_lc, const char* srow_lc, uint32_t row) {
+    const uint32_t vbase = row * p.m + 1;
+    if (srow_lc && row < p.q && root - vbase >= p.m)      // full group, no renumbered slot in it: its staged copy serves
+        return fold16_masked<T, OP>(srow_lc, p.kbytes, p.m, extract_bits(inc, vbase, p.m), sstar, LdShared());
     if (WHOLE) return fold16_careful<T, OP, LdShared>(p, root, sstar, inc, in_lc, row);
     return fold16_careful<T, OP, LdGlobal>(p, root, sstar, inc, in_lc, row);
 }
 
 // A lane's sub-heap in a tile whose rows are all plain and that is complete down to its second-to-last level:
 // only the children at the tile's last level (U + 1 == XL - 1) may be missing.
-template <typename T, int OP, int XL, int U, bool WHOLE>
+// MASKED: groups may miss members (fold under the arrival mask in `inc`), otherwise the same.
+template <typename T, int OP, bool MASKED>
+__device__ __forceinline__ uint4 fold_fast_staged(const Params& p, uint32_t sstar, const uint32_t* inc, const char* srow_lc, uint32_t grow) {
+    if (MASKED) return fold16_masked<T, OP>(srow_lc, p.kbytes, p.m, extract_bits(inc, grow * p.m + 1, p.m), sstar, LdShared());
+    return fold_plain_staged<T, OP>(p, sstar, srow_lc);
+}
+
+template <typename T, int OP, int XL, int U, bool WHOLE, bool MASKED>
 struct SubHeapPlain {
-    static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t sstar, const char* buf_lc, uint32_t rowbytes,
+    static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t sstar, const uint32_t* inc, const char* buf_lc, uint32_t rowbytes,
                                                  uint32_t trow, uint32_t grow, uint32_t G) {
-        uint4 v = fold_plain_staged<T, OP>(p, sstar, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, trow, grow));
+        uint4 v = fold_fast_staged<T, OP, MASKED>(p, sstar, inc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, trow, grow), grow);
         if (U + 1 < XL) {
             constexpr int UN = (U + 1 < XL ? U + 1 : U);
             if (U + 2 < XL || 2 * grow + 1 < G)
-                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE>::eval(p, sstar, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
+                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE, MASKED>::eval(p, sstar, inc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
             if (U + 2 < XL || 2 * grow + 2 < G)
-                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE>::eval(p, sstar, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
+                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE, MASKED>::eval(p, sstar, inc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
         }
         return v;
     }
@@ -95,7 +112,9 @@ struct SubHeap {
     static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
                                                  const char* in_lc, const char* buf_lc, uint32_t rowbytes,
                                                  uint32_t trow, uint32_t grow, uint32_t G) {
-        uint4 v = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, grow);
+        // the deepest level of this recursion lies below the tile: its rows are not in the warp's buffer
+        const char* srow = (WHOLE || U + 1 < XL) ? buf_lc + staged_row_offset<WHOLE>(p, rowbytes, trow, grow) : nullptr;
+        uint4 v = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, grow);
         if (U + 1 < XL) {
             if (2 * grow + 1 < G)
                 v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
@@ -108,15 +127,16 @@ struct SubHeap {
 
 constexpr int kStagedMaxThreads = 256;
 
-template <typename T, int OP, int XL, bool WHOLE>
-__global__ void __launch_bounds__(kStagedMaxThreads, 2) staged_kernel(Params p, StagedGeom g) {
+template <typename T, int OP, int XL, bool WHOLE, int MINB>
+__global__ void __launch_bounds__(kStagedMaxThreads, MINB) staged_kernel(Params p, StagedGeom g) {
     extern __shared__ __align__(128) uint32_t smem[];
     char* sbase = reinterpret_cast<char*>(smem);
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
     uint32_t* pf = smem + sizeof(Ctx) / 4;
     uint32_t* inc = pf + p.W + 1;
     uint32_t* unr = inc + p.W + 1;
-    uint32_t* tspec = reinterpret_cast<uint32_t*>(sbase + g.off_special);
+    uint32_t* tspec = reinterpret_cast<uint32_t*>(sbase + g.off_special);            // items that need every check
+    uint32_t* tmask = tspec + (nitems_words(p.Lt, 5 - p.cw_log2));                     // items with missing group members only
     uint4* rootv = reinterpret_cast<uint4*>(sbase + g.off_rootv);
     uint4* hv = reinterpret_cast<uint4*>(sbase + g.off_hv);
 
@@ -208,7 +228,7 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) staged_kernel(Params p, 
             continue;
         }
         if (p.is_allreduce) count_holders(p, cx, pf, unr);
-        mark_special_items(p, cx, pf, tspec, Lt, lw, D);
+        mark_special_items(p, cx, pf, tspec, tmask, Lt, lw, D);
         const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
         const char* in_lc = (WHOLE ? wbuf : in_s) + lc * 16;      // the scenario in process order, for the general fold
 
@@ -216,32 +236,42 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) staged_kernel(Params p, 
             const uint32_t it = wid + i * nw, b = acquire();
             const char* buf_lc = (WHOLE ? wbuf : tiles + (size_t)b * g.tile_cap) + lc * 16;
             const bool careful = it < ntiles + ngroups && test_bit(tspec, it);      // warp-uniform
+            const bool masked = it < ntiles + ngroups && test_bit(tmask, it);
             if (it < ntiles) {
                 const uint32_t j0 = ntop + it;
                 const uint32_t tA = RW - 1 + lr, rowA = ((j0 + 1) << lw) - 1 + lr;     // root of this lane row's sub-heap
                 const uint32_t tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB);
                 const uint32_t rowB = ((j0 + 1) << tB) - 1 + idxB;                     // this lane row's node above
-                if (!careful) {
+                if (!careful && !masked) {
                     // XL == 1: the bottom rows are the tile's last level and may be missing; XL > 1: they exist
                     uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
-                    if (XL > 1 || rowA < G) valA = SubHeapPlain<T, OP, XL, 0, WHOLE>::eval(p, sstar, buf_lc, rowbytes, tA, rowA, G);
+                    if (XL > 1 || rowA < G) valA = SubHeapPlain<T, OP, XL, 0, WHOLE, false>::eval(p, sstar, inc, buf_lc, rowbytes, tA, rowA, G);
                     const bool hasB = lr < RW - 1;
-                    if (hasB) valB = fold_plain_staged<T, OP>(p, sstar, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB));
+                    if (hasB) valB = fold_fast_staged<T, OP, false>(p, sstar, inc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB), rowB);
+                    valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
+                    if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
+                } else if (!careful) {
+                    // the same with some group members missing
+                    uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
+                    if (XL > 1 || rowA < G) valA = SubHeapPlain<T, OP, XL, 0, WHOLE, true>::eval(p, sstar, inc, buf_lc, rowbytes, tA, rowA, G);
+                    const bool hasB = lr < RW - 1;
+                    if (hasB) valB = fold_fast_staged<T, OP, true>(p, sstar, inc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB), rowB);
                     valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                     if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                 } else if (j0 < G) {
                     uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
-                    if (rowA < G) valA = SubHeap<T, OP, XL, 0, WHOLE>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, tA, rowA, G);
+                    if (rowA < G) valA = SubHeap<T, OP, XL + 1, 0, WHOLE>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, tA, rowA, G);   // one level deeper: rows below the tile
                     const bool hasB = lr < RW - 1 && rowB < G;
-                    if (hasB) valB = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, rowB);
+                    if (hasB) valB = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB), rowB);
                     valB = tile_tree_phase<T, OP>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                     if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                 }
             } else if (it < ntiles + ngroups) {
                 const uint32_t row = ((it - ntiles) << lw) + lr;
                 const char* srow = buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, row);
-                if (!careful) hv[(size_t)row * p.C + lc] = fold_plain_staged<T, OP>(p, sstar, srow);
-                else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, row);
+                if (!careful && !masked) hv[(size_t)row * p.C + lc] = fold_plain_staged<T, OP>(p, sstar, srow);
+                else if (!careful) hv[(size_t)row * p.C + lc] = fold_fast_staged<T, OP, true>(p, sstar, inc, srow, row);
+                else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, row);
             } else if (sstar >= p.r) {
                 if (lr == 0) rootv[lc] = WHOLE ? fold_root16<T, OP, LdShared>(p, root, inc, in_lc) : fold_root16<T, OP, LdGlobal>(p, root, inc, in_lc);
             }
@@ -280,8 +310,12 @@ static bool staged_geometry(Params& p, int smem_optin, uint32_t XL, StagedGeom& 
     if (C == 0 || C > 32 || (C & (C - 1))) return false;
     uint32_t cwl = 0; while ((1u << cwl) < C) ++cwl;
     const uint32_t lw = 5 - cwl, D = lw + XL;
-    uint32_t Hmax = 1; while ((1u << Hmax) <= p.Gmax) ++Hmax;
-    p.C = C; p.cw_log2 = cwl; p.Lt = Hmax > D ? Hmax - D : 0;
+    uint32_t Hmax = 1; while ((1u << Hmax) <= p.Gmax) ++Hmax;      // levels of the largest subtree heap
+    // a last level filled to less than an eighth stays out of the tiles (its few rows go the careful way), so that
+    // the tiles, and with them the copy buffers, are full
+    const uint32_t last_rows = p.Gmax - ((1u << (Hmax - 1)) - 1);
+    const uint32_t Heff = (Hmax >= 2 && last_rows * 8 < (1u << (Hmax - 1))) ? Hmax - 1 : Hmax;
+    p.C = C; p.cw_log2 = cwl; p.Lt = Heff > D ? Heff - D : 0;
     if (p.Lt > 16) return false;
     const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
     const uint64_t cap = ((((uint64_t)1 << D) - 1) * rowbytes + 127) & ~(uint64_t)127;
@@ -300,7 +334,7 @@ static bool staged_geometry(Params& p, int smem_optin, uint32_t XL, StagedGeom& 
     if (g.whole) nbuf = 0;
     size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
     o = (o + 15) & ~(size_t)15; g.off_special = (uint32_t)o;
-    o += ((((size_t)nitems + 31) / 32 + 1) * 4 + 15) & ~(size_t)15;
+    o += (2 * (size_t)nitems_words(p.Lt, lw) * 4 + 15) & ~(size_t)15;
     g.off_rootv = (uint32_t)o; o += (size_t)C * 16;
     g.off_hv = (uint32_t)o; o += (((size_t)2 << p.Lt) - 1) * C * 16;
     g.off_bar = (uint32_t)o; o += (size_t)(kStagedMaxThreads / 32) * 4 * 8 + 8;      // room for any warps x nbuf, plus one
@@ -333,17 +367,17 @@ bool staged_supported(Params& p, int smem_optin_bytes) {
     return staged_geometry(p, smem_optin_bytes, staged_xl(p), g);
 }
 
-template <typename T, int OP, int XL, bool WHOLE>
+template <typename T, int OP, int XL, bool WHOLE, int MINB>
 static cudaError_t launch_staged_w(const Params& p, const StagedGeom& g, int sm_count, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(staged_kernel<T, OP, XL, WHOLE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
+    cudaError_t e = cudaFuncSetAttribute(staged_kernel<T, OP, XL, WHOLE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, staged_kernel<T, OP, XL, WHOLE>, (int)g.nwarps * 32, g.smem_bytes);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, staged_kernel<T, OP, XL, WHOLE, MINB>, (int)g.nwarps * 32, g.smem_bytes);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
-    staged_kernel<T, OP, XL, WHOLE><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
+    staged_kernel<T, OP, XL, WHOLE, MINB><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
     return cudaGetLastError();
 }
 
@@ -351,7 +385,10 @@ template <typename T, int OP, int XL>
 static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
     StagedGeom g;
     if (!staged_geometry(p, smem_optin, XL, g)) return cudaErrorInvalidConfiguration;
-    return g.whole ? launch_staged_w<T, OP, XL, true>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, false>(p, g, sm_count, st);
+    // one- and two-warp blocks are register-limited before they are shared-memory-limited: 64 registers for them
+    const bool lean = g.nwarps <= 2;
+    if (g.whole) return lean ? launch_staged_w<T, OP, XL, true, 4>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, true, 2>(p, g, sm_count, st);
+    return lean ? launch_staged_w<T, OP, XL, false, 4>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
 }
 
 template <typename T, int OP>

@@ -116,6 +116,17 @@ __device__ __forceinline__ uint4 fold16_full(const char* ptr, uint32_t stride, u
     return acc;
 }
 
+// Fold of a full-size group some of whose members' messages may be missing (`mask`), from a copy in which the
+// members sit `stride` bytes apart in rank order: own input first, then the arrived ones ascending.
+template <typename T, int OP, typename LD>
+__device__ __forceinline__ uint4 fold16_masked(const char* ptr, uint32_t stride, uint32_t m, uint32_t mask, uint32_t sstar, LD ld) {
+    uint4 acc = ld(ptr + sstar * stride);
+#pragma unroll 2
+    for (uint32_t sp = 0; sp < m; ++sp)
+        if (sp != sstar && ((mask >> sp) & 1u)) acc = comb16<T, OP>(acc, ld(ptr + sp * stride));
+    return acc;
+}
+
 // A group is "plain" when it is full, every member's message reached the selected subtree's member, and neither
 // renumbered slot lies in it; then its fold needs one base address and constant strides.
 __device__ __forceinline__ bool group_is_plain(const Params& p, uint32_t root, const uint32_t* inc, uint32_t row) {
@@ -167,38 +178,43 @@ __device__ __forceinline__ uint4 tile_tree_phase(uint4 valA, uint4 valB, uint32_
 // and those that are incomplete above their last level. One bit per item in `tspec`; all threads call.
 // Item numbering: tile i (rooted at heap row 2^Lt - 1 + i, D levels) is item i; rows [g*RW, (g+1)*RW) above the
 // tiles are item 2^Lt + g.
+// `tmask` gets the items whose only peculiarity is a group with missing members (fold under the arrival mask, no
+// other checks needed); pass tmask = tspec to send those the careful way too.
 static __device__ void mark_special_items(const Params& p, const Ctx* cx, const uint32_t* pf, uint32_t* tspec,
-                                          uint32_t Lt, uint32_t lw, uint32_t D) {
+                                          uint32_t* tmask, uint32_t Lt, uint32_t lw, uint32_t D) {
     const uint32_t tid = threadIdx.x, nt = blockDim.x;
     const uint32_t ntiles = 1u << Lt, ntop = ntiles - 1, RW = 1u << lw, ngroups = (ntop + RW - 1) >> lw;
     const uint32_t nitems = ntiles + ngroups, root = cx->root, G = cx->G;
-    for (uint32_t w = tid; w < (nitems + 31) / 32 + 1; w += nt) tspec[w] = 0;
+    for (uint32_t w = tid; w < (nitems + 31) / 32 + 1; w += nt) { tspec[w] = 0; tmask[w] = 0; }
     __syncthreads();
-    auto mark_row = [&](uint32_t j) {
+    auto mark_row = [&](uint32_t j, uint32_t* bm) {
         const uint32_t lvl = ilog2u(j + 1);
         const uint32_t it = lvl >= Lt ? ((j + 1) >> (lvl - Lt)) - ntiles : ntiles + (j >> lw);
-        atomicOr(&tspec[it >> 5], 1u << (it & 31));
+        atomicOr(&bm[it >> 5], 1u << (it & 31));
     };
     for (uint32_t w = tid; w < p.W; w += nt) {
         uint32_t word = pf[w];
         while (word) {
             const uint32_t b = __ffs(word) - 1; word &= word - 1;
             const uint32_t v = renumber((w << 5) + b, root);
-            if (v && (v - 1) / p.m < G) mark_row((v - 1) / p.m);
+            if (v && (v - 1) / p.m < G) mark_row((v - 1) / p.m, tmask);
         }
     }
     if (tid < p.max_inop && cx->iv[tid] != FTC_INOP_UNUSED) {
         const uint32_t v = renumber(cx->iv[tid], root);
-        if (v && (v - 1) / p.m < G) mark_row((v - 1) / p.m);
+        if (v && (v - 1) / p.m < G) mark_row((v - 1) / p.m, tmask);
     }
     if (tid == 0) {
-        if (root != 0 && (root - 1) / p.m < G) mark_row((root - 1) / p.m);   // the slot that holds process 0's input
-        if (G > p.q) mark_row(p.q);                                          // the short last group
+        if (root != 0 && (root - 1) / p.m < G) mark_row((root - 1) / p.m, tspec);   // the slot that holds process 0's input
+        if (G > p.q) mark_row(p.q, tspec);                                          // the short last group
     }
     // tiles not complete down to their second-to-last level (the last row of level t of the tile rooted at j0 is
     // ((j0+2) << t) - 2); their last level may be ragged, the common path checks it. And the ragged last group.
+    // Also tiles with rows of the subtree below their last level (a sparsely filled last heap level is left out
+    // of the tiles: the first row below tile j0 is ((j0+1) << D) - 1).
     for (uint32_t it = tid; it < ntiles; it += nt)
-        if (((ntop + it + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= G) atomicOr(&tspec[it >> 5], 1u << (it & 31));
+        if (((ntop + it + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= G || ((ntop + it + 1) << D) - 1 < G)
+            atomicOr(&tspec[it >> 5], 1u << (it & 31));
     for (uint32_t g = tid; g < ngroups; g += nt)
         if (((g + 1) << lw) > ntop || ((g + 1) << lw) > G) atomicOr(&tspec[(ntiles + g) >> 5], 1u << ((ntiles + g) & 31));
     __syncthreads();

@@ -45,7 +45,7 @@ __global__ void __launch_bounds__(kTiledMaxThreads, MINB) tiled_kernel(Params p)
             continue;
         }
         if (p.is_allreduce) count_holders(p, cx, pf, unr);
-        mark_special_items(p, cx, pf, tspec, Lt, lw, lw + 1);
+        mark_special_items(p, cx, pf, tspec, tspec, Lt, lw, lw + 1);
         const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
         const char* in_lc = reinterpret_cast<const char*>(p.in) + s * (size_t)p.P * p.kbytes + lc * 16;
 
