@@ -1,0 +1,399 @@
+// Staged kernel: the main fast path. Same decomposition as the register-tiled kernel (one block per scenario,
+// the selected subtree's heap of up-correction groups cut into warp tiles, levels above the tiles combined in
+// shared memory), but the input bytes of a tile travel global -> shared memory as a few large asynchronous bulk
+// copies (one per heap level of the tile: each level of a sub-heap is one contiguous run of rows), tracked by an
+// mbarrier per buffer. A warp keeps one tile in flight per buffer while it works on another, so the bytes in
+// flight do not depend on registers, and no lane spends instructions on global addresses.
+//
+// A tile has lw + XL levels (lw = log2 of the lane rows, 32 / chunks per vector): each lane row evaluates a
+// sub-heap of XL levels by itself (post-order, values in registers), the lw levels above are combined with warp
+// shuffles. Groups that are not "plain" (a missing member, a renumbered slot, the short last group) are folded
+// from global memory by the general routine; they are a handful per scenario.
+#pragma once
+#include "ftc_tile_common.cuh"
+#include "ftc_kernels.h"
+
+namespace ftc {
+
+// ---- mbarrier / bulk-copy primitives (shared::cta addresses as 32-bit) ----
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kWaitTries polls and reports it; the caller flags the scenario and carries on so
+// that block-wide barriers stay matched.
+constexpr uint32_t kWaitTries = 1u << 22;
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kWaitTries; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+// words of one per-item bitmap
+__host__ __device__ inline uint32_t nitems_words(uint32_t Lt, uint32_t lw) {
+    const uint32_t ntiles = 1u << Lt, nitems = ntiles + ((ntiles - 1 + (1u << lw) - 1) >> lw);
+    return (nitems + 31) / 32 + 1;
+}
+
+struct StagedGeom {
+    uint32_t nwarps, nbuf, tile_cap;       // warps per block, buffers per warp, bytes per buffer (multiple of 128)
+    uint32_t whole;                        // 1: the whole scenario is staged in one block-wide buffer
+    uint32_t off_special, off_rootv, off_hv, off_bar, off_tiles, smem_bytes;
+};
+
+// Where a row's bytes sit: at tile-heap position trow of the warp's buffer, or (WHOLE) at their place in the
+// block-wide copy of the scenario (grow = global row).
+template <bool WHOLE>
+__device__ __forceinline__ uint32_t staged_row_offset(const Params& p, uint32_t rowbytes, uint32_t trow, uint32_t grow) {
+    return WHOLE ? (grow * p.m + 1) * p.kbytes : trow * rowbytes;
+}
+
+// Fold of a plain group from its staged copy.
+template <typename T, int OP>
+__device__ __forceinline__ uint4 fold_plain_staged(const Params& p, uint32_t sstar, const char* srow_lc) {
+    return fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdShared());
+}
+
+// Fold of one group on the careful path: a full group without a renumbered slot comes from its staged copy
+// (`srow_lc`, NULL when the row is not in the buffer) under its arrival mask; the others by the general routine from the scenario in process order (`in_lc`: global
+// memory, or the block-wide shared copy when WHOLE).
+template <typename T, int OP, bool WHOLE>
+__device__ __forceinline__ uint4 fold_staged(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
+                                             const char* in_lc, const char* srow_lc, uint32_t row) {
+    const uint32_t vbase = row * p.m + 1;
+    if (srow_lc && row < p.q && root - vbase >= p.m)      // full group, no renumbered slot in it: its staged copy serves
+        return fold16_masked<T, OP>(srow_lc, p.kbytes, p.m, extract_bits(inc, vbase, p.m), sstar, LdShared());
+    if (WHOLE) return fold16_careful<T, OP, LdShared>(p, root, sstar, inc, in_lc, row);
+    return fold16_careful<T, OP, LdGlobal>(p, root, sstar, inc, in_lc, row);
+}
+
+// A lane's sub-heap in a tile whose rows are all plain and that is complete down to its second-to-last level:
+// only the children at the tile's last level (U + 1 == XL - 1) may be missing.
+// MASKED: groups may miss members (fold under the arrival mask in `inc`), otherwise the same.
+template <typename T, int OP, bool MASKED>
+__device__ __forceinline__ uint4 fold_fast_staged(const Params& p, uint32_t sstar, const uint32_t* inc, const char* srow_lc, uint32_t grow) {
+    if (MASKED) return fold16_masked<T, OP>(srow_lc, p.kbytes, p.m, extract_bits(inc, grow * p.m + 1, p.m), sstar, LdShared());
+    return fold_plain_staged<T, OP>(p, sstar, srow_lc);
+}
+
+template <typename T, int OP, int XL, int U, bool WHOLE, bool MASKED>
+struct SubHeapPlain {
+    static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t sstar, const uint32_t* inc, const char* buf_lc, uint32_t rowbytes,
+                                                 uint32_t trow, uint32_t grow, uint32_t G) {
+        uint4 v = fold_fast_staged<T, OP, MASKED>(p, sstar, inc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, trow, grow), grow);
+        if (U + 1 < XL) {
+            constexpr int UN = (U + 1 < XL ? U + 1 : U);
+            if (U + 2 < XL || 2 * grow + 1 < G)
+                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE, MASKED>::eval(p, sstar, inc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
+            if (U + 2 < XL || 2 * grow + 2 < G)
+                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE, MASKED>::eval(p, sstar, inc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
+        }
+        return v;
+    }
+};
+
+// Value of the node at level u (of XL) of a lane's sub-heap: its group's fold, then child 1, then child 2.
+// trow/grow: tile-heap index and global row of the node. Its bytes sit at tile-heap position trow of the warp's
+// buffer, or (WHOLE) at their place in the block-wide copy of the scenario.
+template <typename T, int OP, int XL, int U, bool WHOLE>
+struct SubHeap {
+    static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
+                                                 const char* in_lc, const char* buf_lc, uint32_t rowbytes,
+                                                 uint32_t trow, uint32_t grow, uint32_t G) {
+        // the deepest level of this recursion lies below the tile: its rows are not in the warp's buffer
+        const char* srow = (WHOLE || U + 1 < XL) ? buf_lc + staged_row_offset<WHOLE>(p, rowbytes, trow, grow) : nullptr;
+        uint4 v = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, grow);
+        if (U + 1 < XL) {
+            if (2 * grow + 1 < G)
+                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
+            if (2 * grow + 2 < G)
+                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
+        }
+        return v;
+    }
+};
+
+constexpr int kStagedMaxThreads = 256;
+
+template <typename T, int OP, int XL, bool WHOLE, int MINB>
+__global__ void __launch_bounds__(kStagedMaxThreads, MINB) staged_kernel(Params p, StagedGeom g) {
+    extern __shared__ __align__(128) uint32_t smem[];
+    char* sbase = reinterpret_cast<char*>(smem);
+    Ctx* cx = reinterpret_cast<Ctx*>(smem);
+    uint32_t* pf = smem + sizeof(Ctx) / 4;
+    uint32_t* inc = pf + p.W + 1;
+    uint32_t* unr = inc + p.W + 1;
+    uint32_t* tspec = reinterpret_cast<uint32_t*>(sbase + g.off_special);            // items that need every check
+    uint32_t* tmask = tspec + (nitems_words(p.Lt, 5 - p.cw_log2));                     // items with missing group members only
+    uint4* rootv = reinterpret_cast<uint4*>(sbase + g.off_rootv);
+    uint4* hv = reinterpret_cast<uint4*>(sbase + g.off_hv);
+
+    const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
+    const uint32_t cwl = p.cw_log2, lw = 5 - cwl, RW = 1u << lw, Cmask = p.C - 1;
+    const uint32_t lr = lane >> cwl, lc = lane & Cmask;
+    const uint32_t D = lw + XL;                                   // levels of a tile
+    const uint32_t Lt = p.Lt, ntiles = 1u << Lt, ntop = ntiles - 1, ngroups = (ntop + RW - 1) >> lw;
+    const uint32_t nitems = ntiles + ngroups + 1;
+    const uint32_t rowbytes = p.m * p.kbytes;
+    const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
+
+    const uint32_t bar0 = smem_addr(sbase + g.off_bar) + wid * g.nbuf * 8;
+    char* tiles = sbase + g.off_tiles + (size_t)wid * g.nbuf * g.tile_cap;
+    const uint32_t cbar = smem_addr(sbase + g.off_bar) + g.nwarps * g.nbuf * 8;   // block-wide barrier (WHOLE)
+    char* wbuf = sbase + g.off_tiles;                                            // block-wide scenario copy (WHOLE)
+    if (lane < g.nbuf) mbar_init(bar0 + lane * 8, 1);
+    if (WHOLE && tid == 0) mbar_init(cbar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    uint32_t phase_bits = 0;                                      // bit b: parity to wait for on buffer b
+    uint32_t cphase = 0;
+
+    // ---- the copy pipeline of this warp: it runs over the flat sequence (scenario, work item) of everything the
+    // warp will process, g.nbuf items ahead of the item being computed, across scenario boundaries. What is copied
+    // depends on the geometry only (rows that exist for the largest subtree), never on a scenario's decode.
+    const uint32_t n_my = wid < nitems ? (nitems - wid + nw - 1) / nw : 0;     // work items of this warp per scenario
+    uint64_t is_s = blockIdx.x;                                   // scenario and local item of the next copy to issue
+    uint32_t is_i = 0, iseq = 0, cseq = 0;                        // items issued / consumed so far
+    uint32_t pending = 0;                                         // bit b: buffer b has a copy in flight
+    auto issue_next = [&]() {
+        if (WHOLE || n_my == 0 || is_s >= p.S) return;
+        const uint32_t it = wid + is_i * nw, b = iseq % g.nbuf;
+        const char* src_s = reinterpret_cast<const char*>(p.in) + is_s * scen_bytes;
+        uint32_t first_row = 0, nrows = 0, dst_off = 0;
+        if (it < ntiles) {                                        // lane t copies level t of the tile
+            const uint32_t j0 = ntop + it;
+            if (lane < D && j0 < p.Gmax) { first_row = ((j0 + 1) << lane) - 1; nrows = 1u << lane; dst_off = ((1u << lane) - 1) * rowbytes; }
+        } else if (it < ntiles + ngroups) {
+            if (lane == 0) { first_row = (it - ntiles) << lw; nrows = min(RW, ntop - first_row); }
+        }
+        uint64_t b0 = ((uint64_t)first_row * p.m + 1) * p.kbytes, b1 = ((uint64_t)(first_row + nrows) * p.m + 1) * p.kbytes;
+        if (b1 > scen_bytes) b1 = scen_bytes;
+        const uint32_t bytes = (nrows && b1 > b0) ? (uint32_t)(b1 - b0) : 0u;
+        const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, bytes);
+        if (total) {
+            if (lane == 0) mbar_expect_tx(bar0 + b * 8, total);
+            __syncwarp();
+            if (bytes) bulk_g2s(smem_addr(tiles + (size_t)b * g.tile_cap + dst_off), src_s + b0, bytes, bar0 + b * 8);
+            pending |= 1u << b;
+        }
+        ++iseq;
+        if (++is_i == n_my) { is_i = 0; is_s += gridDim.x; }
+    };
+    // the buffer of the item about to be computed: wait for its copy if one was issued
+    auto acquire = [&]() {
+        const uint32_t b = WHOLE ? 0u : cseq % g.nbuf;
+        if (!WHOLE && ((pending >> b) & 1u)) {
+            if (!mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u)) { if (lane == 0) atomicOr(&cx->pad, 1u); }
+            phase_bits ^= 1u << b; pending &= ~(1u << b);
+        }
+        return b;
+    };
+    // every lane is done with the buffer: hand it to the next copy
+    auto release = [&]() { __syncwarp(); ++cseq; issue_next(); };
+    if (!WHOLE) for (uint32_t i = 0; i < g.nbuf; ++i) issue_next();
+
+    for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {
+        const char* in_s = reinterpret_cast<const char*>(p.in) + s * scen_bytes;
+        if (WHOLE && wid == 0) {
+            // the whole scenario, in pieces of at most 32 KB, lands while the masks are decoded
+            if (lane == 0) mbar_expect_tx(cbar, (uint32_t)scen_bytes);
+            __syncwarp();
+            for (uint64_t o = (uint64_t)lane * 32768; o < scen_bytes; o += 32u * 32768)
+                bulk_g2s(smem_addr(wbuf + o), in_s + o, (uint32_t)min((uint64_t)32768, scen_bytes - o), cbar);
+        }
+        decode_scenario(p, s, cx, pf, inc);
+        char* out_s = reinterpret_cast<char*>(p.out) + s * p.kbytes;
+        if (WHOLE) {
+            // every thread sees the copy complete before it reads it or leaves the iteration
+            if (!mbar_wait_bounded(cbar, cphase)) atomicOr(&cx->pad, 1u);
+            cphase ^= 1u;
+        }
+        if (cx->code != FTC_ST_OK) {
+            if (tid < p.C) reinterpret_cast<uint4*>(out_s)[tid] = make_uint4(0, 0, 0, 0);
+            for (uint32_t i = 0; i < n_my; ++i) { acquire(); release(); }        // its copies were issued: consume them unused
+            if (tid == 0) write_status_rec(p, s, cx);
+            __syncthreads();
+            continue;
+        }
+        if (p.is_allreduce) count_holders(p, cx, pf, unr);
+        mark_special_items(p, cx, pf, tspec, tmask, Lt, lw, D);
+        const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
+        const char* in_lc = (WHOLE ? wbuf : in_s) + lc * 16;      // the scenario in process order, for the general fold
+
+        for (uint32_t i = 0; i < n_my; ++i) {
+            const uint32_t it = wid + i * nw, b = acquire();
+            const char* buf_lc = (WHOLE ? wbuf : tiles + (size_t)b * g.tile_cap) + lc * 16;
+            const bool careful = it < ntiles + ngroups && test_bit(tspec, it);      // warp-uniform
+            const bool masked = it < ntiles + ngroups && test_bit(tmask, it);
+            if (it < ntiles) {
+                const uint32_t j0 = ntop + it;
+                const uint32_t tA = RW - 1 + lr, rowA = ((j0 + 1) << lw) - 1 + lr;     // root of this lane row's sub-heap
+                const uint32_t tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB);
+                const uint32_t rowB = ((j0 + 1) << tB) - 1 + idxB;                     // this lane row's node above
+                if (!careful && !masked) {
+                    // XL == 1: the bottom rows are the tile's last level and may be missing; XL > 1: they exist
+                    uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
+                    if (XL > 1 || rowA < G) valA = SubHeapPlain<T, OP, XL, 0, WHOLE, false>::eval(p, sstar, inc, buf_lc, rowbytes, tA, rowA, G);
+                    const bool hasB = lr < RW - 1;
+                    if (hasB) valB = fold_fast_staged<T, OP, false>(p, sstar, inc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB), rowB);
+                    valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
+                    if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
+                } else if (!careful) {
+                    // the same with some group members missing
+                    uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
+                    if (XL > 1 || rowA < G) valA = SubHeapPlain<T, OP, XL, 0, WHOLE, true>::eval(p, sstar, inc, buf_lc, rowbytes, tA, rowA, G);
+                    const bool hasB = lr < RW - 1;
+                    if (hasB) valB = fold_fast_staged<T, OP, true>(p, sstar, inc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB), rowB);
+                    valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
+                    if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
+                } else if (j0 < G) {
+                    uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
+                    if (rowA < G) valA = SubHeap<T, OP, XL + 1, 0, WHOLE>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, tA, rowA, G);   // one level deeper: rows below the tile
+                    const bool hasB = lr < RW - 1 && rowB < G;
+                    if (hasB) valB = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB), rowB);
+                    valB = tile_tree_phase<T, OP>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
+                    if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
+                }
+            } else if (it < ntiles + ngroups) {
+                const uint32_t row = ((it - ntiles) << lw) + lr;
+                const char* srow = buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, row);
+                if (!careful && !masked) hv[(size_t)row * p.C + lc] = fold_plain_staged<T, OP>(p, sstar, srow);
+                else if (!careful) hv[(size_t)row * p.C + lc] = fold_fast_staged<T, OP, true>(p, sstar, inc, srow, row);
+                else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, row);
+            } else if (sstar >= p.r) {
+                if (lr == 0) rootv[lc] = WHOLE ? fold_root16<T, OP, LdShared>(p, root, inc, in_lc) : fold_root16<T, OP, LdGlobal>(p, root, inc, in_lc);
+            }
+            release();
+        }
+        __syncthreads();
+        // ---- levels above the tiles, leaves first (Algorithm "reduce_non_root") ----
+        for (int lvl = (int)Lt - 1; lvl >= 0; --lvl) {
+            const uint32_t lo = (1u << lvl) - 1u, n = min(lo + 1u, G > lo ? G - lo : 0u);
+            for (uint32_t u = tid; u < n * p.C; u += nt) {
+                const uint32_t row = lo + (u >> cwl), c = u & Cmask;
+                uint4 v = hv[(size_t)row * p.C + c];
+                if (2 * row + 1 < G) v = comb16<T, OP>(v, hv[(size_t)(2 * row + 1) * p.C + c]);
+                if (2 * row + 2 < G) v = comb16<T, OP>(v, hv[(size_t)(2 * row + 2) * p.C + c]);
+                hv[(size_t)row * p.C + c] = v;
+            }
+            __syncthreads();
+        }
+        // ---- the root (Algorithm "reduce_root") ----
+        if (tid < p.C) {
+            uint4 recv = hv[tid];
+            reinterpret_cast<uint4*>(out_s)[tid] = sstar < p.r ? recv : comb16<T, OP>(rootv[tid], recv);
+        }
+        if (tid == 0) {
+            if (cx->pad) cx->code = FTC_ST_INTERNAL_TIMEOUT;
+            write_status_rec(p, s, cx);
+        }
+        __syncthreads();
+    }
+}
+
+// ---- host side ----
+static bool staged_geometry(Params& p, int smem_optin, uint32_t XL, StagedGeom& g) {
+    if (p.kbytes % 16) return false;
+    const uint32_t C = p.kbytes / 16;
+    if (C == 0 || C > 32 || (C & (C - 1))) return false;
+    uint32_t cwl = 0; while ((1u << cwl) < C) ++cwl;
+    const uint32_t lw = 5 - cwl, D = lw + XL;
+    uint32_t Hmax = 1; while ((1u << Hmax) <= p.Gmax) ++Hmax;      // levels of the largest subtree heap
+    // a last level filled to less than an eighth stays out of the tiles (its few rows go the careful way), so that
+    // the tiles, and with them the copy buffers, are full
+    const uint32_t last_rows = p.Gmax - ((1u << (Hmax - 1)) - 1);
+    const uint32_t Heff = (Hmax >= 2 && last_rows * 8 < (1u << (Hmax - 1))) ? Hmax - 1 : Hmax;
+    p.C = C; p.cw_log2 = cwl; p.Lt = Heff > D ? Heff - D : 0;
+    if (p.Lt > 16) return false;
+    const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
+    const uint64_t cap = ((((uint64_t)1 << D) - 1) * rowbytes + 127) & ~(uint64_t)127;
+    if (cap > 64 * 1024) return false;
+    const uint32_t RW = 1u << lw, ntiles = 1u << p.Lt;
+    const uint32_t nitems = ntiles + ((ntiles - 1 + RW - 1) >> lw) + 1;
+    // Launch shape, from sweeps on B200: what limits the kernel is the number of resident warps doing the combine
+    // work, and shared memory per warp decides that number. So: one buffer per warp, and blocks just large enough
+    // to give every warp at least 16 work items per scenario (at most 8 warps).
+    uint32_t warps = 1;
+    while (warps < 8 && warps * 2 * 16 <= nitems) warps *= 2;
+    uint32_t nbuf = 1;
+    // tiny scenarios (up to 16 KB) are staged whole with one copy, larger ones tile by tile
+    const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
+    g.whole = scen_bytes <= 16 * 1024 ? 1u : 0u;
+    if (g.whole) nbuf = 0;
+    size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
+    o = (o + 15) & ~(size_t)15; g.off_special = (uint32_t)o;
+    o += (2 * (size_t)nitems_words(p.Lt, lw) * 4 + 15) & ~(size_t)15;
+    g.off_rootv = (uint32_t)o; o += (size_t)C * 16;
+    g.off_hv = (uint32_t)o; o += (((size_t)2 << p.Lt) - 1) * C * 16;
+    g.off_bar = (uint32_t)o; o += (size_t)(kStagedMaxThreads / 32) * 4 * 8 + 8;      // room for any warps x nbuf, plus one
+    o = (o + 127) & ~(size_t)127; g.off_tiles = (uint32_t)o;
+    if (g.whole) {
+        o += (size_t)((scen_bytes + 127) & ~(uint64_t)127);
+    } else {
+        while (nbuf > 1 && o + (size_t)warps * nbuf * cap > (size_t)smem_optin - 1024) --nbuf;
+        while (warps > 1 && o + (size_t)warps * nbuf * cap > (size_t)smem_optin - 1024) --warps;
+        o += (size_t)warps * nbuf * cap;
+    }
+    if (o > (size_t)smem_optin - 1024) return false;
+    g.nwarps = warps; g.nbuf = nbuf; g.tile_cap = (uint32_t)cap; g.smem_bytes = (uint32_t)o;
+    return true;
+}
+
+static uint32_t staged_xl(const Params& p) {
+    uint32_t xl;
+    // deepest lane-local sub-heap that keeps a tile (all its levels, every member) within 12 KB
+    if (p.kbytes % 16 || p.kbytes > 512) return 1;
+    uint32_t C = p.kbytes / 16, cwl = 0; while ((1u << cwl) < C) ++cwl;
+    const uint32_t lw = 5 - cwl;
+    for (xl = 3; xl > 1; --xl)
+        if ((((uint64_t)1 << (lw + xl)) - 1) * p.m * p.kbytes <= 12 * 1024) break;
+    return xl;
+}
+
+template <typename T, int OP, int XL, bool WHOLE, int MINB>
+static cudaError_t launch_staged_w(const Params& p, const StagedGeom& g, int sm_count, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(staged_kernel<T, OP, XL, WHOLE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, staged_kernel<T, OP, XL, WHOLE, MINB>, (int)g.nwarps * 32, g.smem_bytes);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    const uint64_t cap = (uint64_t)sm_count * per_sm;
+    const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
+    staged_kernel<T, OP, XL, WHOLE, MINB><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
+    return cudaGetLastError();
+}
+
+template <typename T, int OP, int XL>
+static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
+    StagedGeom g;
+    if (!staged_geometry(p, smem_optin, XL, g)) return cudaErrorInvalidConfiguration;
+    // one- and two-warp blocks are register-limited before they are shared-memory-limited: 64 registers for them
+    const bool lean = g.nwarps <= 2;
+    if (g.whole) return lean ? launch_staged_w<T, OP, XL, true, 4>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, true, 2>(p, g, sm_count, st);
+    return lean ? launch_staged_w<T, OP, XL, false, 4>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
+}
+
+template <typename T, int OP>
+static cudaError_t launch_staged_x(const Params& p, int sm_count, int smem_optin, cudaStream_t st) {
+    switch (staged_xl(p)) {
+    case 2: return launch_staged_t<T, OP, 2>(p, sm_count, smem_optin, st);
+    case 3: return launch_staged_t<T, OP, 3>(p, sm_count, smem_optin, st);
+    default: return launch_staged_t<T, OP, 1>(p, sm_count, smem_optin, st);
+    }
+}
+
+}  // namespace ftc
