@@ -95,6 +95,9 @@ typedef struct {
     void*     tree_values;/* [P][k] payload of each physical process' tree message (zeros if unsent) */
     uint32_t* tree_sent;  /* [P] 1 if the tree message was sent, with bit1 = its failed bit */
     uint32_t* tree_sets;  /* [P][ceil(P/32)] contribution set of each tree message (needs track_sets) */
+    uint32_t* cand_nfail; /* [f+1] size of the failed-process list each root child delivered (0 if nothing) */
+    uint32_t* nfail;      /* [1] size of the root's final list of failed processes */
+    uint32_t* failed;     /* [ceil(P/32)] that list, physical ids (needs track_sets) */
 } orc_out_t;
 
 typedef struct {
@@ -115,6 +118,8 @@ typedef struct {
     uint8_t *phase, *sub;
     uint32_t *idx;
     uint32_t *cnt, *tcnt, *imask, *timask, *imask0;
+    uint32_t *nf, *tnf;     /* size of the list of known failed processes (second failure-information scheme) */
+    uint32_t *fl, *tfl;     /* the list itself as a P-bit set per process / per tree message, when tracking (first scheme) */
     uint32_t *set, *tset;  /* [P][W] when tracking */
     int64_t* fail_round;   /* per virtual rank, global clock */
     uint8_t *inited, *delivered;
@@ -184,6 +189,17 @@ static void merge_single(sim_t* s, uint32_t v, uint32_t u, int* overlap) {
         if (*w & (1u << (u & 31))) *overlap = 1;
         *w |= 1u << (u & 31);
     }
+}
+
+/* process v could not receive a value from u: append u to v's list of failed processes */
+static void note_failed(sim_t* s, uint32_t v, uint32_t u) {
+    s->nf[v] += 1;
+    if (s->fl) s->fl[(size_t)v * s->W + (u >> 5)] |= 1u << (u & 31);
+}
+/* v takes over the list that came with a message */
+static void take_list(sim_t* s, uint32_t v, uint32_t n, const uint32_t* list) {
+    s->nf[v] += n;
+    if (s->fl) for (uint32_t w = 0; w < s->W; ++w) s->fl[(size_t)v * s->W + w] |= list[w];
 }
 
 /* ---- topology in renumbered ranks ---- */
@@ -274,7 +290,7 @@ static int advance(sim_t* s, uint32_t v, int* overlap) {
             if (st == SLOT_SENT) {
                 combine(s, s->data + v * kb, s->x + u * kb);   /* payload is p's unmodified input */
                 merge_single(s, v, u, overlap);
-            } /* SLOT_SKIPPED: p has failed; the failed bit is not touched in this phase */
+            } else note_failed(s, v, u);   /* p has failed: noted in the list; the failed bit is not touched in this phase */
             s->idx[v]++; s->sub[v] = 0; progress = 1;
         } break;
         case PH_TREE_RECV: {
@@ -288,8 +304,10 @@ static int advance(sim_t* s, uint32_t v, int* overlap) {
                 s->failbit[v] |= s->tfail[c];
                 merge_contrib(s, &s->cnt[v], &s->imask[v], s->set ? s->set + (size_t)v * s->W : NULL,
                               s->tcnt[c], s->timask[c], s->tset ? s->tset + (size_t)c * s->W : NULL, overlap);
+                take_list(s, v, s->tnf[c], s->tfl ? s->tfl + (size_t)c * s->W : NULL);
             } else {
                 s->failbit[v] = 1;          /* no value from this child: set the failed bit */
+                note_failed(s, v, c);
             }
             s->idx[v]++; progress = 1;
         } break;
@@ -297,7 +315,8 @@ static int advance(sim_t* s, uint32_t v, int* overlap) {
             int64_t round = s->base + s->f + s->H - depth_of(s, v);
             if (!can_send(s, v, round)) { die(s, v); return 1; }
             memcpy(s->tdata + v * kb, s->data + v * kb, kb);
-            s->tfail[v] = s->failbit[v]; s->tcnt[v] = s->cnt[v]; s->timask[v] = s->imask[v];
+            s->tfail[v] = s->failbit[v]; s->tcnt[v] = s->cnt[v]; s->timask[v] = s->imask[v]; s->tnf[v] = s->nf[v];
+            if (s->tfl) memcpy(s->tfl + (size_t)v * s->W, s->fl + (size_t)v * s->W, (size_t)s->W * 4);
             if (s->tset) memcpy(s->tset + (size_t)v * s->W, s->set + (size_t)v * s->W, (size_t)s->W * 4);
             s->tree_state[v] = SLOT_SENT;
             s->msgs_attempt[1]++; s->nsent[v]++;
@@ -333,10 +352,13 @@ static int advance(sim_t* s, uint32_t v, int* overlap) {
                 memcpy(s->data + v * kb, s->tdata + c * kb, kb);
                 s->cnt[v] = s->tcnt[c]; s->imask[v] = s->timask[c];
                 if (s->set) memcpy(s->set + (size_t)v * s->W, s->tset + (size_t)c * s->W, (size_t)s->W * 4);
+                s->nf[v] = s->tnf[c];       /* and its list of failed processes is the complete one */
+                if (s->fl) memcpy(s->fl + (size_t)v * s->W, s->tfl + (size_t)c * s->W, (size_t)s->W * 4);
             } else {
                 combine(s, s->data + v * kb, s->tdata + c * kb);   /* root's data on the left */
                 merge_contrib(s, &s->cnt[v], &s->imask[v], s->set ? s->set + (size_t)v * s->W : NULL,
                               s->tcnt[c], s->timask[c], s->tset ? s->tset + (size_t)c * s->W : NULL, overlap);
+                take_list(s, v, s->tnf[c], s->tfl ? s->tfl + (size_t)c * s->W : NULL);
             }
             s->st_code = ST_OK; s->st_subtree = (uint32_t)chosen;
             if (!s->is_allreduce) { deliver(s, v); s->phase[v] = PH_DONE; }
@@ -419,7 +441,8 @@ static int play_attempt(sim_t* s, const void* in, const int64_t* fail_round_phys
         s->hold[v] = 0; s->tree_holder[v] = 0;
         for (uint32_t i = 0; i < f; ++i) { s->uc_state[(size_t)v * f + i] = SLOT_NOT_YET; s->corr_state[(size_t)v * f + i] = SLOT_NOT_YET; }
         s->phase[v] = PH_UC; s->idx[v] = 0; s->sub[v] = 0;
-        s->cnt[v] = 1; s->tcnt[v] = 0; s->timask[v] = 0;
+        s->cnt[v] = 1; s->tcnt[v] = 0; s->timask[v] = 0; s->nf[v] = 0; s->tnf[v] = 0;
+        if (s->fl) { memset(s->fl + (size_t)v * s->W, 0, (size_t)s->W * 4); memset(s->tfl + (size_t)v * s->W, 0, (size_t)s->W * 4); }
         s->imask[v] = imask_phys[p]; s->imask0[v] = imask_phys[p];
         if (s->set) { memset(s->set + (size_t)v * s->W, 0, (size_t)s->W * 4); s->set[(size_t)v * s->W + (v >> 5)] = 1u << (v & 31);
                       memset(s->tset + (size_t)v * s->W, 0, (size_t)s->W * 4); }
@@ -466,15 +489,18 @@ int ftc_oracle_run(const orc_cfg_t* cfg, int is_allreduce, const void* in, const
     s->uc_state = malloc(P * fz); s->corr_state = malloc(P * fz);
     s->phase = malloc(P); s->sub = malloc(P); s->idx = malloc(P * 4);
     s->cnt = malloc(P * 4); s->tcnt = malloc(P * 4); s->imask = malloc(P * 4); s->imask0 = malloc(P * 4); s->timask = malloc(P * 4);
+    s->nf = malloc(P * 4); s->tnf = malloc(P * 4);
     s->fail_round = malloc(P * 8); s->inited = malloc(P); s->delivered = malloc(P); s->nsent = malloc(P * 4);
     int64_t* frp = malloc(P * 8); uint32_t* imp = calloc(P, 4); uint32_t* order = malloc(P * 4);
     uint32_t* sends_tot = calloc(P, 4); uint8_t* ev = calloc(P, 1);
-    if (cfg->track_sets) { s->set = malloc((size_t)P * s->W * 4); s->tset = malloc((size_t)P * s->W * 4); }
+    if (cfg->track_sets) { s->set = malloc((size_t)P * s->W * 4); s->tset = malloc((size_t)P * s->W * 4);
+                           s->fl = malloc((size_t)P * s->W * 4); s->tfl = malloc((size_t)P * s->W * 4); }
     int rc = 0;
     if (!s->x || !s->data || !s->tdata || !s->hval || !s->failbit || !s->tfail || !s->tree_state || !s->bct_state ||
         !s->hold || !s->tree_holder || !s->uc_state || !s->corr_state || !s->phase || !s->sub || !s->idx || !s->cnt ||
         !s->tcnt || !s->imask || !s->imask0 || !s->ucval || !s->timask || !s->fail_round || !s->inited || !s->delivered || !s->nsent || !frp ||
-        !imp || !order || !sends_tot || !ev || (cfg->track_sets && (!s->set || !s->tset))) { rc = -2; goto done; }
+        !imp || !order || !sends_tot || !ev || !s->nf || !s->tnf ||
+        (cfg->track_sets && (!s->set || !s->tset || !s->fl || !s->tfl))) { rc = -2; goto done; }
 
     /* failure rounds on the global clock: 0 = failed before the operation */
     for (uint32_t p = 0; p < P; ++p) frp[p] = ((prefail[p >> 5] >> (p & 31)) & 1) ? 0 : ORC_NEVER;
@@ -554,6 +580,12 @@ int ftc_oracle_run(const orc_cfg_t* cfg, int is_allreduce, const void* in, const
     if (out->msgs) { for (int i = 0; i < 4; ++i) { out->msgs[i] = msgs_all[i]; out->msgs[4 + i] = attempts ? s->msgs_attempt[i] : 0; } }
     if (out->sends) memcpy(out->sends, sends_tot, P * 4);
     if (out->events) for (uint32_t p = 0; p < P; ++p) out->events[p] = ev[p];
+    if (out->nfail) out->nfail[0] = have_result ? s->nf[0] : 0;
+    if (out->failed) {
+        memset(out->failed, 0, (size_t)W * 4);
+        if (have_result && s->fl) for (uint32_t v = 0; v < P; ++v)
+            if ((s->fl[v >> 5] >> (v & 31)) & 1) { uint32_t p = v2p(s, v); out->failed[p >> 5] |= 1u << (p & 31); }
+    }
     if (out->contrib) {
         memset(out->contrib, 0, (size_t)W * 4);
         if (have_result && s->set) for (uint32_t v = 0; v < P; ++v)
@@ -565,6 +597,7 @@ int ftc_oracle_run(const orc_cfg_t* cfg, int is_allreduce, const void* in, const
             uint32_t c = cb[i];
             if (out->cand) memcpy((unsigned char*)out->cand + i * kb, s->tdata + c * kb, kb);
             if (out->cand_flag) out->cand_flag[i] = s->tree_state[c] != SLOT_SENT ? 2 : (s->tfail[c] ? 1 : 0);
+            if (out->cand_nfail) out->cand_nfail[i] = s->tree_state[c] == SLOT_SENT ? s->tnf[c] : 0;
         }
         for (uint32_t v = 0; v < P; ++v) {
             uint32_t p = v2p(s, v);
@@ -583,7 +616,7 @@ done:
     free(s->bct_state); free(s->hold); free(s->tree_holder); free(s->uc_state); free(s->corr_state); free(s->phase);
     free(s->sub); free(s->idx); free(s->cnt); free(s->tcnt); free(s->imask); free(s->imask0); free(s->ucval); free(s->timask); free(s->fail_round);
     free(s->inited); free(s->delivered); free(s->nsent); free(frp); free(imp); free(order); free(sends_tot); free(ev);
-    free(s->set); free(s->tset);
+    free(s->set); free(s->tset); free(s->nf); free(s->tnf); free(s->fl); free(s->tfl);
     return rc;
 }
 

@@ -29,7 +29,7 @@ class Cfg(C.Structure):
 class Out(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("result", "status", "cand", "cand_flag", "holders", "expanded", "msgs",
                                           "contrib", "sends", "events", "uc_values", "tree_values", "tree_sent",
-                                          "tree_sets")]
+                                          "tree_sets", "cand_nfail", "nfail", "failed")]
 
 
 def build(force: bool = False) -> str:
@@ -106,10 +106,11 @@ def run(x: np.ndarray, f: int, op: str, prefail, inop=None, root: int = 0, allre
                      holders=np.zeros(W, np.uint32), expanded=np.zeros((P, k), x.dtype),
                      msgs=np.zeros(8, np.uint64), sends=np.zeros(P, np.uint32), events=np.zeros(P, np.uint32),
                      uc_values=np.zeros((P, k), x.dtype), tree_values=np.zeros((P, k), x.dtype),
-                     tree_sent=np.zeros(P, np.uint32))
+                     tree_sent=np.zeros(P, np.uint32), cand_nfail=np.zeros(f + 1, np.uint32), nfail=np.zeros(1, np.uint32))
         if track_sets:
             extra["contrib"] = np.zeros(W, np.uint32)
             extra["tree_sets"] = np.zeros((P, W), np.uint32)
+            extra["failed"] = np.zeros(W, np.uint32)
         for name, arr in extra.items():
             setattr(out, name, _ptr(arr))
     rc = lib().ftc_oracle_run(C.byref(cfg), 1 if allreduce else 0, _ptr(x), _ptr(prefail), _ptr(inop_a), root,

@@ -487,3 +487,37 @@ def test_leaf_has_no_tree_down_send_to_miss():
     assert d["n_holders"] == n and leaf in K.bits(d["holders"], n)
     d = O.run(x, 0, "sum", [], inop=[(leaf, sch["rounds_attempt"] - 1)], allreduce=True, detail=True)
     assert d["n_holders"] == n - 1 and leaf not in K.bits(d["holders"], n)
+
+
+# ---------------------------------------------------------------------------------------------
+# failure information, first and second scheme (section "Failure information"): a child without a failure
+# in its subtree hands the root the complete list of failed processes; concatenated lists are disjoint, so
+# the list's size can be tracked instead of the list
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("n,f", [(7, 1), (9, 2), (12, 2), (13, 3)])
+def test_failed_process_list_is_complete_and_duplicate_free(n, f):
+    x = rand_u64(n, 1, 5 * n + f)
+    for size in range(0, f + 1):
+        for dead in itertools.combinations(range(n), size):
+            for root in (0, 2):
+                if root in dead:
+                    continue
+                d = O.run(x, f, "sum", dead, root=root, track_sets=True, detail=True)
+                assert K.bits(d["failed"], n) == list(dead)                 # complete list from the clean child
+                assert int(d["nfail"][0]) == len(dead)                      # its size: no id listed twice
+                assert d["cand_flag"][d["subtree"]] == 0
+
+
+def test_failed_list_under_inop_failure_is_the_complement_of_the_contributions():
+    n, f = 11, 2
+    x = rand_u64(n, 1, 3)
+    R = O.schedule(n, f)["rounds_reduce"]
+    for victim in range(1, n):
+        for t in range(1, R + 1):
+            for pre in ((), ((victim % (n - 1)) + 1,)):
+                if victim in pre:
+                    continue
+                d = O.run(x, f, "sum", pre, inop=[(victim, t)], track_sets=True, detail=True)
+                C = K.bits(d["contrib"], n)
+                assert K.bits(d["failed"], n) == [p for p in range(n) if p not in C]
+                assert int(d["nfail"][0]) == n - len(C)
