@@ -186,6 +186,24 @@ FTC_API int ftc_reduce_batch_noalloc(const ftc_desc_t* desc, uint64_t S, const v
                                      const ftc_inop_t* d_inop, const uint32_t* d_roots, void* d_out,
                                      uint32_t* d_status, void* cuda_stream);
 
+/*
+ * What the root receives from each of its f+1 children (Algorithm "reduce_root": "receive from any child (data,
+ * failure information)"; section "Failure information", second and third scheme), for S scenarios. The batch calls
+ * above evaluate only the child the root selects; this call plays all f+1 subtrees, nodes that deliver nothing
+ * included. is_allreduce != 0: the reduce of the allreduce attempt that counts (the last one if no candidate is alive).
+ *   d_cand      [S][f+1][k]: the value child s delivers (zeros if it delivers nothing); 16-byte aligned
+ *   d_cand_info [S][f+1][2] uint32: [0] 0 = delivered with the failed bit clear, 1 = delivered with the failed bit set,
+ *               2 = nothing delivered; [1] size of the list of failed processes that came with the value
+ *   workspace of at least ftc_candidates_workspace_bytes(desc, S) bytes, 16-byte aligned
+ * Other arguments as for ftc_reduce_batch. Scenarios whose root is invalid or violates the allreduce precondition
+ * play no attempt: zeros and "nothing delivered". Always runs on the general kernel (any k).
+ */
+FTC_API int ftc_candidates_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const void* d_in,
+                                 const uint32_t* d_prefail, const ftc_inop_t* d_inop, const uint32_t* d_roots,
+                                 void* d_cand, uint32_t* d_cand_info, void* d_workspace, size_t workspace_bytes,
+                                 void* cuda_stream);
+FTC_API size_t ftc_candidates_workspace_bytes(const ftc_desc_t* desc, uint64_t S);
+
 /* Scratch bytes the two calls above need for this descriptor and batch size (0 when the shape runs on the
  * shared-memory kernel). Returns 0 for an invalid descriptor as well; the batch calls report that. */
 FTC_API size_t ftc_workspace_bytes(const ftc_desc_t* desc, uint64_t S, int is_allreduce);

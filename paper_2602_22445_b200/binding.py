@@ -27,7 +27,8 @@ FTC_KERNEL_GENERIC = 0x100
 FTC_KERNEL_DIRECT = 0x200
 OPS = {"sum": FTC_SUM, "max": FTC_MAX, "xor": FTC_XOR}
 
-EXPORTS = ["ftc_reduce_batch", "ftc_allreduce_batch", "ftc_reduce_batch_noalloc", "ftc_workspace_bytes", "ftc_reduce_batch_host",
+EXPORTS = ["ftc_reduce_batch", "ftc_allreduce_batch", "ftc_reduce_batch_noalloc", "ftc_candidates_batch",
+           "ftc_candidates_workspace_bytes", "ftc_workspace_bytes", "ftc_reduce_batch_host",
            "ftc_allreduce_batch_host", "ftc_host_staging_bytes", "ftc_schedule_info", "ftc_fill_inputs",
            "ftc_kernel_name", "ftc_strerror", "ftc_version"]
 
@@ -68,6 +69,10 @@ def load():
         getattr(lib, name).argtypes = batch_args
     lib.ftc_reduce_batch_noalloc.restype = C.c_int
     lib.ftc_reduce_batch_noalloc.argtypes = [dp, u64, vp, vp, vp, vp, vp, vp, vp]
+    lib.ftc_candidates_batch.restype = C.c_int
+    lib.ftc_candidates_batch.argtypes = [dp, u64, C.c_int, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.ftc_candidates_workspace_bytes.restype = sz
+    lib.ftc_candidates_workspace_bytes.argtypes = [dp, u64]
     lib.ftc_workspace_bytes.restype = sz
     lib.ftc_workspace_bytes.argtypes = [dp, u64, C.c_int]
     lib.ftc_host_staging_bytes.restype = sz
@@ -186,6 +191,21 @@ def ftc_reduce_batch_noalloc(desc, S, d_in, d_prefail, d_inop, d_roots, d_out, d
                                          _dev_ptr(d_roots), _dev_ptr(d_out), _dev_ptr(d_status), _stream(stream))
     if check and rc != FTC_OK:
         raise FtcError(rc, "ftc_reduce_batch_noalloc")
+    return rc
+
+
+def ftc_candidates_workspace_bytes(desc, S) -> int:
+    return load().ftc_candidates_workspace_bytes(C.byref(desc), S)
+
+
+def ftc_candidates_batch(desc, S, is_allreduce, d_in, d_prefail, d_inop, d_roots, d_cand, d_cand_info, d_workspace,
+                         stream=None, check=True) -> int:
+    ws_bytes = 0 if d_workspace is None else d_workspace.numel() * d_workspace.element_size()
+    rc = load().ftc_candidates_batch(C.byref(desc), S, int(is_allreduce), _dev_ptr(d_in), _dev_ptr(d_prefail),
+                                     _dev_ptr(d_inop), _dev_ptr(d_roots), _dev_ptr(d_cand), _dev_ptr(d_cand_info),
+                                     _dev_ptr(d_workspace), ws_bytes, _stream(stream))
+    if check and rc != FTC_OK:
+        raise FtcError(rc, "ftc_candidates_batch")
     return rc
 
 

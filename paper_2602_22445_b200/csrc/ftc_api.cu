@@ -207,6 +207,36 @@ int ftc_reduce_batch_noalloc(const ftc_desc_t* desc, uint64_t S, const void* d_i
     return e == cudaSuccess ? FTC_OK : FTC_ECUDA;
 }
 
+int ftc_candidates_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const void* d_in, const uint32_t* d_prefail,
+                         const ftc_inop_t* d_inop, const uint32_t* d_roots, void* d_cand, uint32_t* d_cand_info,
+                         void* d_workspace, size_t workspace_bytes, void* cuda_stream) {
+    Params p;
+    int rc = fill_params(desc, S, is_allreduce ? 1 : 0, p);
+    if (rc != FTC_OK) return rc;
+    if (S == 0) return FTC_OK;
+    if (!d_in || !d_prefail || !d_cand || !d_cand_info) return FTC_EINVAL;
+    if (p.max_inop && !d_inop) return FTC_EINVAL;
+    if (p.root < 0 && !d_roots) return FTC_EINVAL;
+    if (!aligned16(d_in) || !aligned16(d_cand) || !aligned16(d_cand_info)) return FTC_EINVAL;
+    DeviceInfo di;
+    if ((rc = device_info(di)) != FTC_OK) return rc;
+    const size_t need = (size_t)generic_grid(p, di.sm_count) * candidates_slice_bytes(p);
+    if (!d_workspace || workspace_bytes < need || !aligned16(d_workspace)) return FTC_EWORKSPACE;
+    if (generic_smem_bytes(p) > (size_t)di.smem_optin) return FTC_EUNSUPPORTED;
+    p.in = d_in; p.prefail = d_prefail; p.inop = d_inop; p.roots = d_roots; p.ws = d_workspace;
+    cudaError_t e = launch_candidates(p, type_select(desc->dtype, desc->op), d_cand, d_cand_info, di.sm_count,
+                                      static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? FTC_OK : FTC_ECUDA;
+}
+
+size_t ftc_candidates_workspace_bytes(const ftc_desc_t* desc, uint64_t S) {
+    Params p;
+    if (fill_params(desc, S, 0, p) != FTC_OK || S == 0) return 0;
+    DeviceInfo di;
+    if (device_info(di) != FTC_OK) di = kB200;
+    return (size_t)generic_grid(p, di.sm_count) * candidates_slice_bytes(p);
+}
+
 size_t ftc_workspace_bytes(const ftc_desc_t* desc, uint64_t S, int is_allreduce) {
     Params p;
     if (fill_params(desc, S, is_allreduce, p) != FTC_OK || S == 0) return 0;

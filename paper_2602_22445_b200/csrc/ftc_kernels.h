@@ -28,6 +28,10 @@ cudaError_t launch_tiled(const Params& p, int tsel, int sm_count, cudaStream_t s
 bool staged_supported(Params& p, int smem_optin_bytes);
 cudaError_t launch_staged(const Params& p, int tsel, int sm_count, int smem_optin_bytes, cudaStream_t st);
 
+// Every root child's delivery (value, flag, failed-list size): general kernel, workspace slices of candidates_slice_bytes().
+size_t candidates_slice_bytes(const Params& p);
+cudaError_t launch_candidates(const Params& p, int tsel, void* cand, uint32_t* info, int sm_count, cudaStream_t st);
+
 // Expanded allreduce output from the compact results (one value per scenario) left by the main kernel.
 cudaError_t launch_expand(const Params& p, const void* compact, void* out, int sm_count, cudaStream_t st);
 

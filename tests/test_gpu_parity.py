@@ -305,3 +305,40 @@ def test_expanded_needs_allreduce_and_workspace():
     d = B.make_desc(8, 1, 4, B.FTC_I32, "sum", flags=B.FTC_OUT_EXPANDED)
     assert B.ftc_reduce_batch(d, 1, z, z, None, None, z, z, z, check=False) == B.FTC_EUNSUPPORTED
     assert B.ftc_allreduce_batch(d, 1, z, z, None, None, z, z, None, check=False) == B.FTC_EWORKSPACE
+
+
+# ---------------------------------------------------------------------------------------------
+# what every root child delivers: value, delivered / failed bit, size of the failed-process list
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("allreduce", [False, True])
+def test_candidates_of_every_root_child_match_oracle(allreduce):
+    import torch
+    rng = np.random.Generator(np.random.PCG64(91))
+    for P, f, k, dtype in ((7, 1, 1, np.int64), (14, 2, 4, np.uint64), (41, 3, 3, np.float32), (130, 4, 2, np.int32), (9, 0, 2, np.int32)):
+        S = 80
+        x = rng.standard_normal((S, P, k)).astype(np.float32) if dtype == np.float32 else \
+            rng.integers(0, 2**31 - 1, size=(S, P, k)).astype(dtype)
+        pf = sc.picks_to_masks(sc.random_subsets(rng, S, P, rng.integers(0, f + 3, size=S)), P)
+        R = O.schedule(P, f)["rounds_attempt"]
+        inop = np.zeros((S, 2, 2), dtype=np.uint32)
+        inop[:, :, 0] = rng.integers((f + 1) if allreduce else 0, P, size=(S, 2))
+        inop[:, :, 1] = rng.integers(0, R + 3, size=(S, 2))
+        inop[rng.random((S, 2)) < 0.3, 0] = sc.UNUSED
+        roots = (np.zeros(S) if allreduce else rng.integers(0, P, size=S)).astype(np.uint32)
+        d_x = to_dev(x)
+        desc = B.make_desc(P, f, k, B.dtype_code(d_x.dtype), "sum", root=-1, max_inop=2)
+        d_cand = torch.empty((S, f + 1, k), dtype=d_x.dtype, device="cuda")
+        d_cand.view(torch.uint8).fill_(0x5A)
+        d_info = torch.full((S, f + 1, 2), 0x7FFFFFFF, dtype=torch.int32, device="cuda")
+        d_ws = torch.empty(B.ftc_candidates_workspace_bytes(desc, S), dtype=torch.uint8, device="cuda")
+        B.ftc_candidates_batch(desc, S, allreduce, d_x, to_dev(pf), to_dev(inop), to_dev(roots), d_cand, d_info, d_ws)
+        torch.cuda.synchronize()
+        cand, info = to_host(d_cand, x.dtype), d_info.cpu().numpy()
+        for i in range(S):
+            d = O.run(x[i], f, "sum", pf[i], inop=[tuple(e) for e in inop[i]], root=int(roots[i]), allreduce=allreduce, detail=True)
+            if d["attempts"] == 0:
+                assert (info[i, :, 0] == 2).all() and not cand[i].any()
+                continue
+            assert np.array_equal(info[i, :, 0], d["cand_flag"]), (P, f, i, d["code"])
+            assert np.array_equal(info[i, :, 1], d["cand_nfail"]), (P, f, i)
+            assert np.array_equal(cand[i].view(np.uint8), d["cand"].view(np.uint8)), (P, f, i)
