@@ -246,3 +246,22 @@ def config5(collective: str = "allreduce", op: str = "sum", S: int = 1 << 14, fi
     roots = rng.integers(0, P, size=S).astype(np.uint32)
     return Workload("C5", collective, P, f, 4, KIND_U64_FULL, op, BASE_SEED + 5, S, masks, None, roots,
                     root=-1, first_scenario=first)
+
+
+def inop_sweep(P: int, f: int, k: int, kind: int, op: str, pre_sets, rounds, collective: str = "reduce",
+               victims=None, seed: int = BASE_SEED + 6) -> Workload:
+    """Exhaustive in-operation sweep: every pre-operation failure set of `pre_sets` x every victim x every failure
+    round of `rounds` (victims that are in the pre-failed set are skipped). One in-operation slot per scenario."""
+    victims = range(P) if victims is None else victims
+    masks, inop = [], []
+    for st in pre_sets:
+        for v in victims:
+            if v in st:
+                continue
+            for t in rounds:
+                masks.append(st)
+                inop.append((v, t))
+    S = len(masks)
+    io = np.asarray(inop, dtype=np.uint32).reshape(S, 1, 2)
+    return Workload("inop-sweep", collective, P, f, k, kind, op, seed, S, sets_to_masks(masks, P), io, None,
+                    extra={"sets": masks})
