@@ -204,7 +204,30 @@ FTC_API int ftc_candidates_batch(const ftc_desc_t* desc, uint64_t S, int is_allr
                                  void* cuda_stream);
 FTC_API size_t ftc_candidates_workspace_bytes(const ftc_desc_t* desc, uint64_t S);
 
-/* Scratch bytes the two calls above need for this descriptor and batch size (0 when the shape runs on the
+/*
+ * Messages sent in each scenario (theorem on the number of messages of the reduce and theorem on the messages of
+ * the allreduce, section "Properties": failure-free f(f+1)q + a(a-1) up-correction and P-1 tree messages; no
+ * process sends more when processes fail; an allreduce whose first candidates had failed repeats the reduce).
+ * A message counts when its sender performs the send, whether or not the receiver is alive (section "Failures":
+ * a send to a failed process completes). Only the failure pattern is read; desc->k, dtype and op must be valid
+ * but do not matter.
+ *   d_msgs [S][FTC_MSG_WORDS] uint64, 8-byte aligned:
+ *     [0..3] over all attempts that are played: up-correction, tree, tree-down (broadcast), correction (broadcast)
+ *     [4..7] the same four for the last attempt alone
+ *   A reduce plays one attempt and has no broadcast ([2], [3], [6], [7] are 0), also when its root has failed
+ *   (the others still send). An allreduce plays one attempt per root candidate up to the first one that had not
+ *   failed before the operation; only that candidate broadcasts, and only if it found a failure-free subtree.
+ *   Scenarios with outcome FTC_ST_BAD_ROOT or FTC_ST_PRECONDITION_INOP_ROOT play nothing: all zero.
+ *   The broadcast numbers rest on this library's reading of the broadcast (see the top of this file), which the
+ *   paper does not define.
+ * Other arguments as for ftc_reduce_batch. No workspace.
+ */
+#define FTC_MSG_WORDS 8
+FTC_API int ftc_message_counts_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const uint32_t* d_prefail,
+                                     const ftc_inop_t* d_inop, const uint32_t* d_roots, uint64_t* d_msgs,
+                                     void* cuda_stream);
+
+/* Scratch bytes ftc_reduce_batch / ftc_allreduce_batch need for this descriptor and batch size (0 when the shape runs on the
  * shared-memory kernel). Returns 0 for an invalid descriptor as well; the batch calls report that. */
 FTC_API size_t ftc_workspace_bytes(const ftc_desc_t* desc, uint64_t S, int is_allreduce);
 

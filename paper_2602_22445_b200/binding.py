@@ -21,6 +21,7 @@ FTC_NOALLOC_SCRATCH_BYTES = 8 << 20
 FTC_ST_OK, FTC_ST_ROOT_FAILED, FTC_ST_NO_CLEAN_SUBTREE, FTC_ST_NO_LIVE_ROOT_CANDIDATE = 0, 1, 2, 3
 FTC_ST_PRECONDITION_INOP_ROOT, FTC_ST_BAD_ROOT, FTC_ST_INTERNAL_TIMEOUT = 4, 5, 6
 FTC_STATUS_WORDS = 4
+FTC_MSG_WORDS = 8
 FTC_INOP_UNUSED = 0xFFFFFFFF
 FTC_OUT_EXPANDED = 0x1
 FTC_KERNEL_GENERIC = 0x100
@@ -28,7 +29,7 @@ FTC_KERNEL_DIRECT = 0x200
 OPS = {"sum": FTC_SUM, "max": FTC_MAX, "xor": FTC_XOR}
 
 EXPORTS = ["ftc_reduce_batch", "ftc_allreduce_batch", "ftc_reduce_batch_noalloc", "ftc_candidates_batch",
-           "ftc_candidates_workspace_bytes", "ftc_workspace_bytes", "ftc_reduce_batch_host",
+           "ftc_candidates_workspace_bytes", "ftc_message_counts_batch", "ftc_workspace_bytes", "ftc_reduce_batch_host",
            "ftc_allreduce_batch_host", "ftc_host_staging_bytes", "ftc_schedule_info", "ftc_fill_inputs",
            "ftc_kernel_name", "ftc_strerror", "ftc_version"]
 
@@ -73,6 +74,8 @@ def load():
     lib.ftc_candidates_batch.argtypes = [dp, u64, C.c_int, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.ftc_candidates_workspace_bytes.restype = sz
     lib.ftc_candidates_workspace_bytes.argtypes = [dp, u64]
+    lib.ftc_message_counts_batch.restype = C.c_int
+    lib.ftc_message_counts_batch.argtypes = [dp, u64, C.c_int, vp, vp, vp, vp, vp]
     lib.ftc_workspace_bytes.restype = sz
     lib.ftc_workspace_bytes.argtypes = [dp, u64, C.c_int]
     lib.ftc_host_staging_bytes.restype = sz
@@ -206,6 +209,14 @@ def ftc_candidates_batch(desc, S, is_allreduce, d_in, d_prefail, d_inop, d_roots
                                      _dev_ptr(d_workspace), ws_bytes, _stream(stream))
     if check and rc != FTC_OK:
         raise FtcError(rc, "ftc_candidates_batch")
+    return rc
+
+
+def ftc_message_counts_batch(desc, S, is_allreduce, d_prefail, d_inop, d_roots, d_msgs, stream=None, check=True) -> int:
+    rc = load().ftc_message_counts_batch(C.byref(desc), S, int(is_allreduce), _dev_ptr(d_prefail), _dev_ptr(d_inop),
+                                         _dev_ptr(d_roots), _dev_ptr(d_msgs), _stream(stream))
+    if check and rc != FTC_OK:
+        raise FtcError(rc, "ftc_message_counts_batch")
     return rc
 
 

@@ -32,6 +32,10 @@ cudaError_t launch_staged(const Params& p, int tsel, int sm_count, int smem_opti
 size_t candidates_slice_bytes(const Params& p);
 cudaError_t launch_candidates(const Params& p, int tsel, void* cand, uint32_t* info, int sm_count, cudaStream_t st);
 
+// Message counts per scenario (FTC_MSG_WORDS 64-bit words each); reads the failure pattern only.
+size_t messages_smem_bytes(const Params& p);
+cudaError_t launch_messages(const Params& p, unsigned long long* out, int sm_count, cudaStream_t st);
+
 // Expanded allreduce output from the compact results (one value per scenario) left by the main kernel.
 cudaError_t launch_expand(const Params& p, const void* compact, void* out, int sm_count, cudaStream_t st);
 
