@@ -29,6 +29,7 @@ struct Params {
     uint32_t C;        // 16-byte chunks per process vector
     uint32_t cw_log2;  // log2 of lanes along the chunk dimension (= log2 C)
     uint32_t Lt;       // heap level at which the warp tiles are rooted; levels above go through shared memory
+    uint32_t below;    // 1: the heap's sparsely filled last level lies below the tiles (its rows are folded one by one)
 };
 
 // Per-scenario facts, in shared memory.

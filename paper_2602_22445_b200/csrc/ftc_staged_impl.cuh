@@ -105,31 +105,147 @@ struct SubHeapPlain {
     }
 };
 
+// ---- the lean variant (blocks of one or two warps) ----
+// Small scenarios run as one- or two-warp blocks, many per SM, and each warp alternates between waiting for its
+// copy and computing: what counts there is the length of the dependent instruction chain per tile and the
+// registers per warp. So the lean variant folds all rows of a lane together (independent chains), and the folds
+// that few rows need are real function calls, which keeps the code every row runs through small.
+
+// Fold of one group by every rule: a full group without a renumbered slot comes from its staged copy (`srow_lc`,
+// NULL when the row is not in the buffer) under its arrival mask; the others by the general routine from the
+// scenario in process order (`in_lc`: global memory, or the block-wide shared copy when WHOLE).
+template <typename T, int OP, bool WHOLE>
+__device__ __noinline__ uint4 fold_staged_call(FoldShape fs, uint32_t root, uint32_t sstar, const uint32_t* inc,
+                                               const char* in_lc, const char* srow_lc, uint32_t row) {
+    const uint32_t vbase = row * fs.m + 1;
+    if (srow_lc && row < fs.q && root - vbase >= fs.m)      // full group, no renumbered slot in it: its staged copy serves
+        return fold16_masked<T, OP>(srow_lc, fs.kbytes, fs.m, extract_bits(inc, vbase, fs.m), sstar, LdShared());
+    if (WHOLE) return fold16_general<T, OP, 0, LdShared, FoldShape>(fs, root, sstar, inc, in_lc, row);
+    return fold16_general<T, OP, 0, LdGlobal, FoldShape>(fs, root, sstar, inc, in_lc, row);
+}
+
+// A full group some of whose members' messages are missing, from its staged copy.
+template <typename T, int OP>
+__device__ __noinline__ uint4 fold_masked_call(const char* srow_lc, uint32_t kbytes, uint32_t m, uint32_t mask, uint32_t sstar) {
+    return fold16_masked<T, OP>(srow_lc, kbytes, m, mask, sstar, LdShared());
+}
+
+// One row from its staged copy; `masked`: the work item holds a group with a missing member, so look at the mask.
+template <typename T, int OP>
+__device__ __forceinline__ uint4 fold_row_lean(const Params& p, uint32_t sstar, const uint32_t* inc, const char* srow_lc,
+                                               uint32_t grow, bool masked) {
+    if (masked) {
+        const uint32_t mask = extract_bits(inc, grow * p.m + 1, p.m), full = p.m >= 32 ? 0xFFFFFFFFu : (1u << p.m) - 1u;
+        if (mask != full) return fold_masked_call<T, OP>(srow_lc, p.kbytes, p.m, mask, sstar);
+    }
+    return fold_plain_staged<T, OP>(p, sstar, srow_lc);
+}
+
+__host__ __device__ constexpr int clog2(int v) { return v <= 1 ? 0 : 1 + clog2(v >> 1); }
+
+// Tree phase inside a lane's sub-heap from the folded rows, breadth-first index B (slot 1 + B of `acc`): the
+// node's own fold, then child 1, then child 2. Children on the tile's last level may be missing; children on the
+// heap's sparse last level, which is left out of the tiles, are leaves folded by the general routine.
+template <typename T, int OP, int XL, int B, bool WHOLE>
+struct SubComb {
+    static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc, const char* in_lc,
+                                                 const uint4* acc, const uint32_t* grow, uint32_t G) {
+        constexpr int U = clog2(B + 1);
+        uint4 v = acc[1 + B];
+        if (U + 1 < XL) {
+            constexpr int C1 = (U + 1 < XL) ? 2 * B + 1 : B, C2 = (U + 1 < XL) ? 2 * B + 2 : B;
+            if (U + 2 < XL || grow[1 + C1] < G) v = comb16<T, OP>(v, SubComb<T, OP, XL, C1, WHOLE>::eval(p, root, sstar, inc, in_lc, acc, grow, G));
+            if (U + 2 < XL || grow[1 + C2] < G) v = comb16<T, OP>(v, SubComb<T, OP, XL, C2, WHOLE>::eval(p, root, sstar, inc, in_lc, acc, grow, G));
+        } else if (p.below) {
+            const uint32_t c1 = 2 * grow[1 + B] + 1;
+            if (c1 < G) v = comb16<T, OP>(v, fold_staged_call<T, OP, WHOLE>(fold_shape(p), root, sstar, inc, in_lc, nullptr, c1));
+            if (c1 + 1 < G) v = comb16<T, OP>(v, fold_staged_call<T, OP, WHOLE>(fold_shape(p), root, sstar, inc, in_lc, nullptr, c1 + 1));
+        }
+        return v;
+    }
+};
+
+// Fast path of one tile for one lane: the rows it owns -- slot 0 its node of the tile's upper levels (tile heap
+// index lr, global row rowB, present iff hasB), slots 1.. the XL-level sub-heap rooted at tile heap index tA
+// (global row rowA), breadth first -- are folded together, one group member at a time across all rows (own input
+// of the selected subtree's member first, then the partners ascending: Algorithm "Up-correction"), so that the
+// loads and adds of different rows overlap; then the sub-heap is combined. The tile has no renumbered slot, no
+// short group and is complete down to its second-to-last level. `masked`: some group of the tile misses a member.
+template <typename T, int OP, int XL, bool WHOLE>
+__device__ __forceinline__ void fold_tile_fast(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc, const char* in_lc,
+                                               const char* buf_lc, uint32_t rowbytes, uint32_t j0, uint32_t lr, uint32_t rowB, bool hasB,
+                                               uint32_t tA, uint32_t rowA, uint32_t G, bool masked, uint4& valA, uint4& valB) {
+    constexpr int NS = 1 << XL;
+    const LdShared lds{};
+    uint32_t off[NS], grow[NS];
+    const uint32_t off0 = staged_row_offset<WHOLE>(p, rowbytes, 0, j0);        // the tile's root: always there
+    grow[0] = hasB ? rowB : j0;
+    off[0] = hasB ? staged_row_offset<WHOLE>(p, rowbytes, lr, rowB) : off0;
+#pragma unroll
+    for (int b = 0; b < NS - 1; ++b) {
+        const int u = clog2(b + 1), pos = b + 1 - (1 << u);
+        const uint32_t t = ((tA + 1) << u) - 1 + pos, g = ((rowA + 1) << u) - 1 + pos;
+        grow[1 + b] = g;
+        off[1 + b] = g < G ? staged_row_offset<WHOLE>(p, rowbytes, t, g) : off0;   // a missing row reads the root's bytes, unused
+    }
+    uint4 acc[NS];
+    const char* own = buf_lc + sstar * p.kbytes;
+#pragma unroll
+    for (int s = 0; s < NS; ++s) acc[s] = lds(own + off[s]);
+    if (!masked) {
+#pragma unroll 1
+        for (uint32_t i = 1; i < p.m; ++i) {
+            const char* mem = buf_lc + (i - (i <= sstar ? 1u : 0u)) * p.kbytes;      // partners ascending, own skipped
+#pragma unroll
+            for (int s = 0; s < NS; ++s) acc[s] = comb16<T, OP>(acc[s], lds(mem + off[s]));
+        }
+    } else {
+        uint32_t mask[NS];
+#pragma unroll
+        for (int s = 0; s < NS; ++s) mask[s] = grow[s] < G ? extract_bits(inc, grow[s] * p.m + 1, p.m) : 0u;
+#pragma unroll 1
+        for (uint32_t i = 1; i < p.m; ++i) {
+            const uint32_t sp = i - (i <= sstar ? 1u : 0u);
+            const char* mem = buf_lc + sp * p.kbytes;
+#pragma unroll
+            for (int s = 0; s < NS; ++s)
+                if ((mask[s] >> sp) & 1u) acc[s] = comb16<T, OP>(acc[s], lds(mem + off[s]));
+        }
+    }
+    valB = acc[0];
+    valA = SubComb<T, OP, XL, 0, WHOLE>::eval(p, root, sstar, inc, in_lc, acc, grow, G);
+}
+
 // Value of the node at level u (of XL) of a lane's sub-heap: its group's fold, then child 1, then child 2.
 // trow/grow: tile-heap index and global row of the node. Its bytes sit at tile-heap position trow of the warp's
 // buffer, or (WHOLE) at their place in the block-wide copy of the scenario.
-template <typename T, int OP, int XL, int U, bool WHOLE>
+// CALL: the fold is a function call (lean variant) instead of inline code.
+template <typename T, int OP, int XL, int U, bool WHOLE, bool CALL = false>
 struct SubHeap {
     static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
                                                  const char* in_lc, const char* buf_lc, uint32_t rowbytes,
                                                  uint32_t trow, uint32_t grow, uint32_t G) {
         // the deepest level of this recursion lies below the tile: its rows are not in the warp's buffer
         const char* srow = (WHOLE || U + 1 < XL) ? buf_lc + staged_row_offset<WHOLE>(p, rowbytes, trow, grow) : nullptr;
-        uint4 v = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, grow);
+        uint4 v = CALL ? fold_staged_call<T, OP, WHOLE>(fold_shape(p), root, sstar, inc, in_lc, srow, grow)
+                       : fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, grow);
         if (U + 1 < XL) {
             if (2 * grow + 1 < G)
-                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
+                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE, CALL>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
             if (2 * grow + 2 < G)
-                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
+                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE, CALL>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
         }
         return v;
     }
 };
 
 constexpr int kStagedMaxThreads = 256;
+constexpr int kStagedLeanThreads = 64;      // lean variant: at most two warps, about 96 registers a thread
+constexpr int kStagedLeanMinBlocks = 10;
 
 template <typename T, int OP, int XL, bool WHOLE, int MINB>
-__global__ void __launch_bounds__(kStagedMaxThreads, MINB) staged_kernel(Params p, StagedGeom g) {
+__global__ void __launch_bounds__(MINB > 2 ? kStagedLeanThreads : kStagedMaxThreads, MINB) staged_kernel(Params p, StagedGeom g) {
+    constexpr bool LEAN = MINB > 2;
     extern __shared__ __align__(128) uint32_t smem[];
     char* sbase = reinterpret_cast<char*>(smem);
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
@@ -229,7 +345,7 @@ __global__ void __launch_bounds__(kStagedMaxThreads, MINB) staged_kernel(Params 
             continue;
         }
         if (p.is_allreduce) count_holders(p, cx, pf, unr);
-        mark_special_items(p, cx, pf, tspec, tmask, Lt, lw, D);
+        mark_special_items(p, cx, pf, tspec, tmask, Lt, lw, D, LEAN && p.below != 0);
         const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
         const char* in_lc = (WHOLE ? wbuf : in_s) + lc * 16;      // the scenario in process order, for the general fold
 
@@ -243,7 +359,22 @@ __global__ void __launch_bounds__(kStagedMaxThreads, MINB) staged_kernel(Params 
                 const uint32_t tA = RW - 1 + lr, rowA = ((j0 + 1) << lw) - 1 + lr;     // root of this lane row's sub-heap
                 const uint32_t tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB);
                 const uint32_t rowB = ((j0 + 1) << tB) - 1 + idxB;                     // this lane row's node above
-                if (!careful && !masked) {
+                if (LEAN) {
+                    if (!careful) {
+                        uint4 valA, valB;
+                        const bool hasB = lr < RW - 1;
+                        fold_tile_fast<T, OP, XL, WHOLE>(p, root, sstar, inc, in_lc, buf_lc, rowbytes, j0, lr, rowB, hasB, tA, rowA, G, masked, valA, valB);
+                        valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
+                        if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
+                    } else if (j0 < G) {
+                        uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
+                        if (rowA < G) valA = SubHeap<T, OP, XL + 1, 0, WHOLE, true>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, tA, rowA, G);
+                        const bool hasB = lr < RW - 1 && rowB < G;
+                        if (hasB) valB = fold_staged_call<T, OP, WHOLE>(fold_shape(p), root, sstar, inc, in_lc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB), rowB);
+                        valB = tile_tree_phase<T, OP>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
+                        if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
+                    }
+                } else if (!careful && !masked) {
                     // XL == 1: the bottom rows are the tile's last level and may be missing; XL > 1: they exist
                     uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
                     if (XL > 1 || rowA < G) valA = SubHeapPlain<T, OP, XL, 0, WHOLE, false>::eval(p, sstar, inc, buf_lc, rowbytes, tA, rowA, G);
@@ -270,7 +401,10 @@ __global__ void __launch_bounds__(kStagedMaxThreads, MINB) staged_kernel(Params 
             } else if (it < ntiles + ngroups) {
                 const uint32_t row = ((it - ntiles) << lw) + lr;
                 const char* srow = buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, row);
-                if (!careful && !masked) hv[(size_t)row * p.C + lc] = fold_plain_staged<T, OP>(p, sstar, srow);
+                if (LEAN) {
+                    if (!careful) hv[(size_t)row * p.C + lc] = fold_row_lean<T, OP>(p, sstar, inc, srow, row, masked);
+                    else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged_call<T, OP, WHOLE>(fold_shape(p), root, sstar, inc, in_lc, srow, row);
+                } else if (!careful && !masked) hv[(size_t)row * p.C + lc] = fold_plain_staged<T, OP>(p, sstar, srow);
                 else if (!careful) hv[(size_t)row * p.C + lc] = fold_fast_staged<T, OP, true>(p, sstar, inc, srow, row);
                 else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, row);
             } else if (sstar >= p.r) {
@@ -317,6 +451,7 @@ static bool staged_geometry(Params& p, int smem_optin, uint32_t XL, StagedGeom& 
     const uint32_t last_rows = p.Gmax - ((1u << (Hmax - 1)) - 1);
     const uint32_t Heff = (Hmax >= 2 && last_rows * 8 < (1u << (Hmax - 1))) ? Hmax - 1 : Hmax;
     p.C = C; p.cw_log2 = cwl; p.Lt = Heff > D ? Heff - D : 0;
+    p.below = (Heff < Hmax && Heff >= D) ? 1u : 0u;
     if (p.Lt > 16) return false;
     const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
     const uint64_t cap = ((((uint64_t)1 << D) - 1) * rowbytes + 127) & ~(uint64_t)127;
@@ -381,10 +516,10 @@ template <typename T, int OP, int XL>
 static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
     StagedGeom g;
     if (!staged_geometry(p, smem_optin, XL, g)) return cudaErrorInvalidConfiguration;
-    // one- and two-warp blocks are register-limited before they are shared-memory-limited: 64 registers for them
+    // one- and two-warp blocks get the lean variant; its register cap (about 96) matches the blocks that fit by shared memory
     const bool lean = g.nwarps <= 2;
-    if (g.whole) return lean ? launch_staged_w<T, OP, XL, true, 4>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, true, 2>(p, g, sm_count, st);
-    return lean ? launch_staged_w<T, OP, XL, false, 4>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
+    if (g.whole) return lean ? launch_staged_w<T, OP, XL, true, kStagedLeanMinBlocks>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, true, 2>(p, g, sm_count, st);
+    return lean ? launch_staged_w<T, OP, XL, false, kStagedLeanMinBlocks>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
 }
 
 template <typename T, int OP>

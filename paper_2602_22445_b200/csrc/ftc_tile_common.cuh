@@ -40,8 +40,8 @@ struct LdShared { __device__ __forceinline__ uint4 operator()(const char* q) con
 // own input, then (short last group only) the root's, then the partners whose message arrived, ascending.
 // Handles every case (missing members, the renumbered slots, the short group). MCAP > 0: loads of up to MCAP
 // members are issued together; MCAP = 0: batches of four.
-template <typename T, int OP, int MCAP, typename LD = LdGlobal>
-__device__ __forceinline__ uint4 fold16_general(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
+template <typename T, int OP, int MCAP, typename LD = LdGlobal, typename SHAPE = Params>
+__device__ __forceinline__ uint4 fold16_general(const SHAPE& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
                                                 const char* in_lc, uint32_t row) {
     const LD ld{};
     const uint32_t mj = row < p.q ? p.m : p.r, vbase = row * p.m + 1;
@@ -135,6 +135,10 @@ __device__ __forceinline__ bool group_is_plain(const Params& p, uint32_t root, c
     return row < p.q && root - vbase >= p.m && extract_bits(inc, vbase, p.m) == full;   // unsigned wrap: root outside the row
 }
 
+// The four numbers the general fold needs, for passing by value.
+struct FoldShape { uint32_t m, q, r, kbytes; };
+__device__ __forceinline__ FoldShape fold_shape(const Params& p) { return FoldShape{p.m, p.q, p.r, p.kbytes}; }
+
 // Any group, by the general routine (the careful path of the tiled kernels; rare). LD says where `in_lc`, the
 // scenario in process order, lives.
 template <typename T, int OP, typename LD>
@@ -180,8 +184,10 @@ __device__ __forceinline__ uint4 tile_tree_phase(uint4 valA, uint4 valB, uint32_
 // tiles are item 2^Lt + g.
 // `tmask` gets the items whose only peculiarity is a group with missing members (fold under the arrival mask, no
 // other checks needed); pass tmask = tspec to send those the careful way too.
+// `below`: rows under the tiles' last level (a sparsely filled last heap level) are folded one by one by the general
+// routine wherever a tile meets them, so they mark nothing.
 static __device__ void mark_special_items(const Params& p, const Ctx* cx, const uint32_t* pf, uint32_t* tspec,
-                                          uint32_t* tmask, uint32_t Lt, uint32_t lw, uint32_t D) {
+                                          uint32_t* tmask, uint32_t Lt, uint32_t lw, uint32_t D, bool below = false) {
     const uint32_t tid = threadIdx.x, nt = blockDim.x;
     const uint32_t ntiles = 1u << Lt, ntop = ntiles - 1, RW = 1u << lw, ngroups = (ntop + RW - 1) >> lw;
     const uint32_t nitems = ntiles + ngroups, root = cx->root, G = cx->G;
@@ -189,6 +195,7 @@ static __device__ void mark_special_items(const Params& p, const Ctx* cx, const 
     __syncthreads();
     auto mark_row = [&](uint32_t j, uint32_t* bm) {
         const uint32_t lvl = ilog2u(j + 1);
+        if (below && lvl >= Lt + D) return;
         const uint32_t it = lvl >= Lt ? ((j + 1) >> (lvl - Lt)) - ntiles : ntiles + (j >> lw);
         atomicOr(&bm[it >> 5], 1u << (it & 31));
     };
@@ -213,7 +220,7 @@ static __device__ void mark_special_items(const Params& p, const Ctx* cx, const 
     // Also tiles with rows of the subtree below their last level (a sparsely filled last heap level is left out
     // of the tiles: the first row below tile j0 is ((j0+1) << D) - 1).
     for (uint32_t it = tid; it < ntiles; it += nt)
-        if (((ntop + it + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= G || ((ntop + it + 1) << D) - 1 < G)
+        if (((ntop + it + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= G || (!below && ((ntop + it + 1) << D) - 1 < G))
             atomicOr(&tspec[it >> 5], 1u << (it & 31));
     for (uint32_t g = tid; g < ngroups; g += nt)
         if (((g + 1) << lw) > ntop || ((g + 1) << lw) > G) atomicOr(&tspec[(ntiles + g) >> 5], 1u << ((ntiles + g) & 31));
