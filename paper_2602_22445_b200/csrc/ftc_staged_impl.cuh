@@ -282,35 +282,38 @@ __global__ void __launch_bounds__(MINB > 2 ? kStagedLeanThreads : kStagedMaxThre
     // depends on the geometry only (rows that exist for the largest subtree), never on a scenario's decode.
     const uint32_t n_my = wid < nitems ? (nitems - wid + nw - 1) / nw : 0;     // work items of this warp per scenario
     uint64_t is_s = blockIdx.x;                                   // scenario and local item of the next copy to issue
-    uint32_t is_i = 0, iseq = 0, cseq = 0;                        // items issued / consumed so far
+    const char* is_src = reinterpret_cast<const char*>(p.in) + is_s * scen_bytes;
+    uint32_t is_i = 0, ibuf = 0, cbuf = 0;                        // buffer of the next copy to issue / item to consume
     uint32_t pending = 0;                                         // bit b: buffer b has a copy in flight
+    // lane t copies level t of a tile: 2^t rows, placed after the 2^t - 1 rows of the levels above
+    const uint32_t lvl_rows = lane < D ? 1u << lane : 0u, lvl_dst = (lvl_rows ? lvl_rows - 1 : 0u) * rowbytes;
     auto issue_next = [&]() {
         if (WHOLE || n_my == 0 || is_s >= p.S) return;
-        const uint32_t it = wid + is_i * nw, b = iseq % g.nbuf;
-        const char* src_s = reinterpret_cast<const char*>(p.in) + is_s * scen_bytes;
+        const uint32_t it = wid + is_i * nw, b = ibuf;
         uint32_t first_row = 0, nrows = 0, dst_off = 0;
-        if (it < ntiles) {                                        // lane t copies level t of the tile
+        if (it < ntiles) {
             const uint32_t j0 = ntop + it;
-            if (lane < D && j0 < p.Gmax) { first_row = ((j0 + 1) << lane) - 1; nrows = 1u << lane; dst_off = ((1u << lane) - 1) * rowbytes; }
+            if (j0 < p.Gmax) { first_row = ((j0 + 1) << lane) - 1; nrows = lvl_rows; dst_off = lvl_dst; }
         } else if (it < ntiles + ngroups) {
             if (lane == 0) { first_row = (it - ntiles) << lw; nrows = min(RW, ntop - first_row); }
         }
-        uint64_t b0 = ((uint64_t)first_row * p.m + 1) * p.kbytes, b1 = ((uint64_t)(first_row + nrows) * p.m + 1) * p.kbytes;
-        if (b1 > scen_bytes) b1 = scen_bytes;
-        const uint32_t bytes = (nrows && b1 > b0) ? (uint32_t)(b1 - b0) : 0u;
+        // rows first_row .. first_row+nrows-1 are bytes [first_row*rowbytes + kbytes, ...) of the scenario, cut at its end
+        const uint64_t b0 = (uint64_t)first_row * rowbytes + p.kbytes;
+        uint32_t bytes = 0;
+        if (nrows && b0 < scen_bytes) bytes = (uint32_t)min((uint64_t)nrows * rowbytes, scen_bytes - b0);
         const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, bytes);
         if (total) {
             if (lane == 0) mbar_expect_tx(bar0 + b * 8, total);
             __syncwarp();
-            if (bytes) bulk_g2s(smem_addr(tiles + (size_t)b * g.tile_cap + dst_off), src_s + b0, bytes, bar0 + b * 8);
+            if (bytes) bulk_g2s(smem_addr(tiles + (size_t)b * g.tile_cap + dst_off), is_src + b0, bytes, bar0 + b * 8);
             pending |= 1u << b;
         }
-        ++iseq;
-        if (++is_i == n_my) { is_i = 0; is_s += gridDim.x; }
+        if (++ibuf == g.nbuf) ibuf = 0;
+        if (++is_i == n_my) { is_i = 0; is_s += gridDim.x; is_src += (uint64_t)gridDim.x * scen_bytes; }
     };
     // the buffer of the item about to be computed: wait for its copy if one was issued
     auto acquire = [&]() {
-        const uint32_t b = WHOLE ? 0u : cseq % g.nbuf;
+        const uint32_t b = WHOLE ? 0u : cbuf;
         if (!WHOLE && ((pending >> b) & 1u)) {
             if (!mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u)) { if (lane == 0) atomicOr(&cx->pad, 1u); }
             phase_bits ^= 1u << b; pending &= ~(1u << b);
@@ -318,7 +321,7 @@ __global__ void __launch_bounds__(MINB > 2 ? kStagedLeanThreads : kStagedMaxThre
         return b;
     };
     // every lane is done with the buffer: hand it to the next copy
-    auto release = [&]() { __syncwarp(); ++cseq; issue_next(); };
+    auto release = [&]() { __syncwarp(); if (!WHOLE && ++cbuf == g.nbuf) cbuf = 0; issue_next(); };
     if (!WHOLE) for (uint32_t i = 0; i < g.nbuf; ++i) issue_next();
 
     for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {
