@@ -29,14 +29,17 @@
  *
  * Readings where the paper is silent (the same ones the documentation lists):
  *   - group partners are visited in ascending (renumbered) rank, skipping self;
- *   - below each root child the subtree is a binary heap on the local index
- *     j = floor((v-1)/(f+1)): children 2j+1 and 2j+2, received in that order;
+ *   - below each root child the subtree is a heap on the local index
+ *     j = floor((v-1)/(f+1)): binary by default (children 2j+1 and 2j+2), or
+ *     a-ary on request (children a*j+1 .. a*j+a), received in ascending order;
+ *     the paper asks only for f+1 root children whose subtree sizes differ by
+ *     at most one, which the interleaved numbering gives for any such shape;
  *   - the root examines its children in ascending order and takes the first
  *     message that arrived with the failed bit clear;
  *   - a "failure round" t of a process means: it performs exactly those of
  *     its sends that are scheduled in rounds < t.  Up-correction iteration i
  *     is round i (rounds 0..f-1), the tree send of a node at depth d is round
- *     f+H-d, H = 1+floor(log2(ceil((n-1)/(f+1)))).  A broadcast adds H rounds
+ *     f+H-d, H = depth of the deepest node (binary: 1+floor(log2(ceil((n-1)/(f+1))))).  A broadcast adds H rounds
  *     of tree-down sends (a node at depth d sends to all its children in
  *     round d of the broadcast) and f rounds of correction.  An allreduce
  *     attempt therefore has 2(f+H) rounds and attempt a starts at a*2(f+H);
@@ -75,6 +78,7 @@ typedef struct {
     uint32_t max_inop;   /* in-operation failure slots per scenario */
     uint32_t sweep;      /* scheduler order: 0 descending rank, 1 ascending, >=2 seeded shuffle */
     uint32_t track_sets; /* carry a P-bit contribution set with every value (instrumentation) */
+    uint32_t arity;      /* children per node below the root's children: 0 or 2 = binary heap, a >= 2 = a-ary heap */
 } orc_cfg_t;
 
 typedef struct { uint32_t victim, round; } orc_inop_t;
@@ -103,6 +107,7 @@ typedef struct {
 typedef struct {
     const orc_cfg_t* cfg;
     uint32_t P, f, k, m, esz, W;
+    uint32_t arity;     /* children per node below the root's children */
     uint32_t q, r, H, Rred, Ratt;
     int is_allreduce;
     uint32_t root;      /* physical id of the current root */
@@ -129,7 +134,6 @@ typedef struct {
     uint32_t st_code, st_subtree;
 } sim_t;
 
-static uint32_t ilog2(uint32_t v) { uint32_t l = 0; while (v >>= 1) ++l; return l; }
 
 /* ---- renumbering: the root swaps numbers with process 0 ---- */
 static uint32_t v2p(const sim_t* s, uint32_t v) { return v == 0 ? s->root : (v == s->root ? 0 : v); }
@@ -206,7 +210,13 @@ static void take_list(sim_t* s, uint32_t v, uint32_t n, const uint32_t* list) {
 static uint32_t row_of(const sim_t* s, uint32_t v) { return (v - 1) / s->m; }      /* group number */
 static uint32_t sub_of(const sim_t* s, uint32_t v) { return (v - 1) % s->m; }      /* root child index */
 static uint32_t rank_of(const sim_t* s, uint32_t j, uint32_t sidx) { return j * s->m + sidx + 1; }
-static uint32_t depth_of(const sim_t* s, uint32_t v) { return v == 0 ? 0 : 1 + ilog2(row_of(s, v) + 1); }
+/* level of local index j in an a-ary heap: level l holds the a^l indices after those of the levels above */
+static uint32_t heap_level(uint32_t arity, uint32_t j) {
+    uint32_t l = 0; uint64_t start = 0, width = 1;
+    while (j >= start + width) { start += width; width *= arity; ++l; }
+    return l;
+}
+static uint32_t depth_of(const sim_t* s, uint32_t v) { return v == 0 ? 0 : 1 + heap_level(s->arity, row_of(s, v)); }
 
 /* members of the up-correction group of v in ascending rank, v excluded; returns their number */
 static uint32_t partners(const sim_t* s, uint32_t v, uint32_t* out) {
@@ -233,14 +243,15 @@ static uint32_t children(const sim_t* s, uint32_t v, uint32_t* out) {
     uint32_t n = 0;
     if (v == 0) { for (uint32_t c = 1; c <= s->m && c < s->P; ++c) out[n++] = c; return n; }
     uint32_t j = row_of(s, v), sidx = sub_of(s, v);
-    uint32_t c1 = rank_of(s, 2 * j + 1, sidx), c2 = rank_of(s, 2 * j + 2, sidx);
-    if (c1 < s->P) out[n++] = c1;
-    if (c2 < s->P) out[n++] = c2;
+    for (uint32_t c = 1; c <= s->arity; ++c) {
+        uint64_t jc = (uint64_t)s->arity * j + c;                 /* heap children of j: a*j+1 .. a*j+a */
+        if (jc * s->m + sidx + 1 < s->P) out[n++] = rank_of(s, (uint32_t)jc, sidx);
+    }
     return n;
 }
 static uint32_t parent_of(const sim_t* s, uint32_t v) {
     uint32_t j = row_of(s, v);
-    return j == 0 ? 0 : rank_of(s, (j - 1) / 2, sub_of(s, v));
+    return j == 0 ? 0 : rank_of(s, (j - 1) / s->arity, sub_of(s, v));
 }
 
 /* A send scheduled in round `round` happens iff the sender's failure round is later. */
@@ -471,6 +482,7 @@ int ftc_oracle_run(const orc_cfg_t* cfg, int is_allreduce, const void* in, const
     if (!cfg || !in || !prefail || !out) return -1;
     uint32_t P = cfg->P, f = cfg->f, k = cfg->k;
     if (k == 0 || P < f + 2 || f + 1 > 60 || root >= P || cfg->max_inop > 32) return -1;
+    if (cfg->arity == 1 || cfg->arity > 32) return -1;
     if (cfg->dtype > DT_F32 || cfg->op > OP_XOR) return -1;
     if (cfg->dtype == DT_F32 && cfg->op != OP_SUM) return -1;
     sim_t S; memset(&S, 0, sizeof S);
@@ -479,7 +491,8 @@ int ftc_oracle_run(const orc_cfg_t* cfg, int is_allreduce, const void* in, const
     s->esz = (cfg->dtype == DT_I32 || cfg->dtype == DT_F32) ? 4 : 8;
     s->W = (P + 31) / 32;
     s->q = (P - 1) / s->m; s->r = (P - 1) % s->m;
-    s->H = 1 + ilog2(s->q + (s->r ? 1 : 0));
+    s->arity = cfg->arity ? cfg->arity : 2;
+    s->H = 1 + heap_level(s->arity, s->q + (s->r ? 1 : 0) - 1);     /* depth of the deepest node of the largest subtree */
     s->Rred = f + s->H; s->Ratt = 2 * s->Rred;
     s->is_allreduce = is_allreduce;
     size_t kb = (size_t)k * s->esz, fz = f ? f : 1;
@@ -641,9 +654,9 @@ int ftc_oracle_batch(const orc_cfg_t* cfg, int is_allreduce, uint64_t S, const v
 }
 
 /* Schedule constants under the readings above: q, r, H, rounds of a reduce, rounds of an allreduce attempt. */
-int ftc_oracle_schedule(uint32_t P, uint32_t f, uint32_t* out5) {
-    if (P < f + 2) return -1;
-    uint32_t m = f + 1, q = (P - 1) / m, r = (P - 1) % m, H = 1 + ilog2(q + (r ? 1 : 0));
+int ftc_oracle_schedule(uint32_t P, uint32_t f, uint32_t arity, uint32_t* out5) {
+    if (P < f + 2 || arity == 1) return -1;
+    uint32_t m = f + 1, q = (P - 1) / m, r = (P - 1) % m, H = 1 + heap_level(arity ? arity : 2, q + (r ? 1 : 0) - 1);
     out5[0] = q; out5[1] = r; out5[2] = H; out5[3] = f + H; out5[4] = 2 * (f + H);
     return 0;
 }

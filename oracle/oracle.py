@@ -23,7 +23,7 @@ UNUSED = 0xFFFFFFFF
 
 
 class Cfg(C.Structure):
-    _fields_ = [(n, C.c_uint32) for n in ("P", "f", "k", "dtype", "op", "max_inop", "sweep", "track_sets")]
+    _fields_ = [(n, C.c_uint32) for n in ("P", "f", "k", "dtype", "op", "max_inop", "sweep", "track_sets", "arity")]
 
 
 class Out(C.Structure):
@@ -54,14 +54,14 @@ def lib():
         _lib.ftc_oracle_batch.argtypes = [C.POINTER(Cfg), C.c_int, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p,
                                           C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p]
         _lib.ftc_oracle_schedule.restype = C.c_int
-        _lib.ftc_oracle_schedule.argtypes = [C.c_uint32, C.c_uint32, C.POINTER(C.c_uint32)]
+        _lib.ftc_oracle_schedule.argtypes = [C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(C.c_uint32)]
     return _lib
 
 
-def schedule(P: int, f: int) -> dict:
-    """q, r, H and the round counts of one reduce / one allreduce attempt."""
+def schedule(P: int, f: int, arity: int = 2) -> dict:
+    """q, r, H and the round counts of one reduce / one allreduce attempt (subtrees: `arity`-ary heaps)."""
     buf = (C.c_uint32 * 5)()
-    if lib().ftc_oracle_schedule(P, f, buf) != 0:
+    if lib().ftc_oracle_schedule(P, f, arity, buf) != 0:
         raise ValueError("P must be at least f+2")
     return dict(q=buf[0], r=buf[1], H=buf[2], rounds_reduce=buf[3], rounds_attempt=buf[4])
 
@@ -78,7 +78,7 @@ def _prep_inop(inop, max_inop):
 
 
 def run(x: np.ndarray, f: int, op: str, prefail, inop=None, root: int = 0, allreduce: bool = False,
-        sweep: int = 0, track_sets: bool = False, detail: bool = False) -> dict:
+        sweep: int = 0, track_sets: bool = False, detail: bool = False, arity: int = 2) -> dict:
     """Simulate one scenario. x: [P][k]; prefail: uint32 words or an iterable of failed ids;
     inop: [(victim, round), ...]. Returns result, status fields and (detail=True) instrumentation."""
     x = np.ascontiguousarray(x)
@@ -95,7 +95,7 @@ def run(x: np.ndarray, f: int, op: str, prefail, inop=None, root: int = 0, allre
     if inop is not None and len(inop):
         inop_a = np.ascontiguousarray(np.asarray(inop, dtype=np.uint32).reshape(-1, 2))
         max_inop = inop_a.shape[0]
-    cfg = Cfg(P, f, k, DTYPES[x.dtype], OPS[op], max_inop, sweep, 1 if track_sets else 0)
+    cfg = Cfg(P, f, k, DTYPES[x.dtype], OPS[op], max_inop, sweep, 1 if track_sets else 0, arity)
     res = np.zeros(k, dtype=x.dtype)
     status = np.zeros(4, dtype=np.uint32)
     out = Out()
@@ -125,7 +125,7 @@ def run(x: np.ndarray, f: int, op: str, prefail, inop=None, root: int = 0, allre
 
 
 def batch(x: np.ndarray, f: int, op: str, prefail: np.ndarray, inop=None, roots=None, root: int = 0,
-          allreduce: bool = False):
+          allreduce: bool = False, arity: int = 2):
     """Simulate S scenarios one after the other. x: [S][P][k]; prefail: [S][W] uint32;
     inop: [S][max_inop][2] uint32 or None; roots: [S] uint32 or None. Returns (result [S][k], status [S][4])."""
     x = np.ascontiguousarray(x)
@@ -137,7 +137,7 @@ def batch(x: np.ndarray, f: int, op: str, prefail: np.ndarray, inop=None, roots=
         max_inop = inop.shape[1]
     if roots is not None:
         roots = np.ascontiguousarray(roots, dtype=np.uint32)
-    cfg = Cfg(P, f, k, DTYPES[x.dtype], OPS[op], max_inop, 0, 0)
+    cfg = Cfg(P, f, k, DTYPES[x.dtype], OPS[op], max_inop, 0, 0, arity)
     res = np.zeros((S, k), dtype=x.dtype)
     status = np.zeros((S, 4), dtype=np.uint32)
     rc = lib().ftc_oracle_batch(C.byref(cfg), 1 if allreduce else 0, S, _ptr(x), _ptr(prefail), _ptr(inop),

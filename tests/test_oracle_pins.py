@@ -521,3 +521,97 @@ def test_failed_list_under_inop_failure_is_the_complement_of_the_contributions()
                 C = K.bits(d["contrib"], n)
                 assert K.bits(d["failed"], n) == [p for p in range(n) if p not in C]
                 assert int(d["nfail"][0]) == n - len(C)
+
+
+# ---------------------------------------------------------------------------------------------
+# Other subtree shapes: below each root child an a-ary heap instead of the binary one. The paper fixes only
+# the I(f)-tree property (f+1 root children, subtree sizes within one of each other: definition before the
+# first theorem of section "Properties"), so every statement pinned above must hold for these shapes too.
+# ---------------------------------------------------------------------------------------------
+ARITIES = [3, 4, 5]
+
+
+def test_arity_tree_structure_by_hand():
+    """n = 14, f = 1, ternary: subtree 0 holds ranks 1,3,..,13 (local index j = (v-1)/2); node j has children
+    3j+1..3j+3, so rank 1 receives from 3, 5, 7 and rank 3 from 9, 11, 13. A tree message carries the groups of
+    the sender's whole subtree (each group {2j+1, 2j+2}; the short last group {13} also holds the root)."""
+    n, f = 14, 1
+    x = (U64(1) << np.arange(n, dtype=np.uint64)).reshape(n, 1)
+    d = O.run(x, f, "sum", [], detail=True, track_sets=True, arity=3)
+    sets = {v: K.bits(d["tree_sets"][v], n) for v in range(1, n)}
+    assert sets[3] == sorted([3, 4, 9, 10, 11, 12, 13, 0])
+    assert sets[5] == [5, 6] and sets[7] == [7, 8] and sets[9] == [9, 10] and sets[13] == [0, 13]
+    assert sets[1] == list(range(n))                       # root child 1 collects every group once
+    assert sets[2] == sorted([2, 1] + sets[4] + sets[6] + sets[8])
+    assert sets[4] == sorted([4, 3, 10, 9, 12, 11])          # j = 1 of subtree 1: children j = 4, 5 (rank 14 does not exist)
+    assert int(d["result"][0]) == (1 << n) - 1
+    # depth of the deepest node: rows 0..6 fill ternary levels 1 + 3 + 3, binary levels 1 + 2 + 4: H = 3 either way;
+    # n = 20 (rows 0..9): binary 1+2+4+3 -> H = 4, ternary 1+3+6 -> H = 3
+    assert O.schedule(14, 1, 3)["H"] == 3 and O.schedule(14, 1, 2)["H"] == 3
+    assert O.schedule(20, 1, 2)["H"] == 4 and O.schedule(20, 1, 3)["H"] == 3 and O.schedule(20, 1, 4)["H"] == 3
+
+
+def test_arity_f32_children_combined_in_ascending_order():
+    """Algorithm "reduce_non_root" with three children: data <- ((data + c1) + c2) + c3 in float32."""
+    n, f = 5, 0                      # one subtree: ranks 1..4, rank 1 has children 2, 3, 4; no up-correction
+    vals = np.array([0.0, 1.0, 2.0**24, 1.0, -(2.0**24)], dtype=np.float32).reshape(n, 1)
+    d = O.run(vals, f, "sum", [], arity=3)
+    acc = np.float32(1.0)
+    for c in (2, 3, 4):
+        acc = np.float32(acc + vals[c, 0])
+    assert d["result"][0] == np.float32(np.float32(0.0) + acc) and d["result"][0] == np.float32(0.0)
+    d2 = O.run(vals, f, "sum", [], arity=2)               # binary: 1 <- (1 + (2 + 4)) + 3: another rounding
+    assert d2["result"][0] == np.float32(2.0)
+
+
+@pytest.mark.parametrize("arity", ARITIES)
+def test_arity_message_counts_do_not_depend_on_the_shape(arity):
+    for f in range(0, 4):
+        for n in list(range(f + 2, 24)) + [64, 257]:
+            d = O.run(np.ones((n, 1), dtype=np.int32), f, "sum", [], detail=True, arity=arity)
+            assert (int(d["msgs"][0]), int(d["msgs"][1])) == (uc_messages(n, f), n - 1)
+            assert int(d["result"][0]) == n
+            da = O.run(np.ones((n, 1), dtype=np.int32), f, "sum", [], allreduce=True, detail=True, arity=arity)
+            assert [int(v) for v in da["msgs"][:4]] == [uc_messages(n, f), n - 1, n - 1, uc_messages(n, f)]
+
+
+@pytest.mark.parametrize("arity", ARITIES)
+@pytest.mark.parametrize("n,f", [(9, 1), (14, 1), (13, 2), (16, 2), (17, 3)])
+def test_arity_reduce_equals_direct_reduction_exhaustive(n, f, arity):
+    x = rand_u64(n, 2, 500 * n + f + arity)
+    for size in range(0, f + 1):
+        for dead in itertools.combinations(range(n), size):
+            for root in (0, 2, n - 1):
+                d = O.run(x, f, "sum", dead, root=root, track_sets=True, detail=True, arity=arity)
+                live = [p for p in range(n) if p not in dead]
+                if root in dead:
+                    assert d["code"] == 1 and not d["result"].any()
+                    continue
+                assert d["code"] == 0
+                assert np.array_equal(d["result"], K.reduce_over(x, live, "sum"))
+                assert K.bits(d["contrib"], n) == live and d["count"] == len(live)
+
+
+@pytest.mark.parametrize("arity", ARITIES)
+@pytest.mark.parametrize("n,f", [(10, 1), (14, 2), (17, 3)])
+def test_arity_inop_allowed_results_and_allreduce_consistency(n, f, arity):
+    x = rand_u64(n, 1, 91 * n + f + arity)
+    sch = O.schedule(n, f, arity)
+    for victim in range(f + 1, n):
+        for t in range(1, sch["rounds_attempt"] + 2):
+            for allred in (False, True):
+                if not allred and t > sch["rounds_reduce"] + 1:
+                    continue
+                d = O.run(x, f, "sum", [1] if f >= 2 and victim != 1 else [], inop=[(victim, t)], allreduce=allred,
+                          track_sets=True, detail=True, arity=arity)
+                pre = [1] if f >= 2 and victim != 1 else []
+                assert d["code"] == 0
+                C = K.bits(d["contrib"], n)
+                assert K.contribution_allowed(n, C, pre, [victim])
+                assert np.array_equal(d["result"], K.reduce_over(x, C, "sum"))
+                if allred:
+                    holders = K.bits(d["holders"], n)
+                    alive_end = [p for p in range(n) if p not in pre and not (p == victim and t < sch["rounds_attempt"])]
+                    assert holders == alive_end                  # at most f failures: every survivor holds the value
+                    for p in holders:
+                        assert np.array_equal(d["expanded"][p], d["result"])
