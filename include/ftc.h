@@ -27,7 +27,9 @@
  *     ascending rank, the root first;
  *   - v >= 1 lies below root child s = (v-1) mod (f+1) (proof of the first theorem of
  *     section "Properties"); within a subtree the nodes j = floor((v-1)/(f+1)) form a
- *     binary heap: children 2j+1, 2j+2, received in that order, accumulator on the left;
+ *     heap, binary unless FTC_TREE_ARITY(a) in the flags asks for a children per node: children a*j+1 .. a*j+a,
+ *     received in that order, accumulator on the left (the paper's I(f)-tree fixes only the root's f+1 children
+ *     and their subtree sizes; shapes other than binary run on the general kernel and need its workspace);
  *   - failure information is the single failed bit (third scheme of section "Failure
  *     information"); the root takes the lowest-numbered child that delivered with the
  *     bit clear (Algorithm "reduce_root");
@@ -66,7 +68,7 @@ enum { FTC_SUM = 0, FTC_MAX = 1, FTC_XOR = 2 };   /* integer sums wrap; FTC_F32 
 /* call-level return codes */
 enum {
     FTC_OK = 0,
-    FTC_EINVAL = -1,        /* P < f+2, k = 0, root >= P, NULL or misaligned required pointer, f > 31, max_inop > 32 */
+    FTC_EINVAL = -1,        /* P < f+2, k = 0, root >= P, NULL or misaligned required pointer, f > 31, max_inop > 32, tree arity 1 or > 32 */
     FTC_EUNSUPPORTED = -2,  /* unknown dtype/op, xor or max on f32 */
     FTC_EWORKSPACE = -3,    /* workspace missing or smaller than ftc_workspace_bytes() */
     FTC_ECUDA = -4,         /* a CUDA call or launch failed */
@@ -104,6 +106,8 @@ typedef struct { uint32_t victim; uint32_t round; } ftc_inop_t;
 
 /* flags */
 #define FTC_OUT_EXPANDED   0x1u   /* allreduce: d_out is [S][P][k], zeros for processes that do not hold the result */
+#define FTC_TREE_ARITY(a)  (((uint32_t)(a) & 0xFFu) << 16)  /* subtrees below the root's children are a-ary heaps, 2 <= a <= FTC_MAX_ARITY (not given: binary) */
+#define FTC_MAX_ARITY 32u
 #define FTC_KERNEL_GENERIC 0x100u /* force the general level-by-level kernel (needs the workspace) */
 #define FTC_KERNEL_DIRECT  0x200u /* force the register-tiled kernel (direct global loads) where the shape allows it */
 

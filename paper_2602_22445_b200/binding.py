@@ -25,6 +25,13 @@ FTC_MSG_WORDS = 8
 FTC_INOP_UNUSED = 0xFFFFFFFF
 FTC_OUT_EXPANDED = 0x1
 FTC_KERNEL_GENERIC = 0x100
+FTC_MAX_ARITY = 32
+
+
+def FTC_TREE_ARITY(a: int) -> int:
+    """Flag bits asking for a-ary heaps below the root's children."""
+    return (a & 0xFF) << 16
+
 FTC_KERNEL_DIRECT = 0x200
 OPS = {"sum": FTC_SUM, "max": FTC_MAX, "xor": FTC_XOR}
 

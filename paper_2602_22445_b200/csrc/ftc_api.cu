@@ -5,7 +5,19 @@
 
 namespace ftc {
 
-static uint32_t ilog2h(uint32_t v) { uint32_t l = 0; while (v >>= 1) ++l; return l; }
+
+// level of index j in an a-ary heap (level l holds a^l indices)
+static uint32_t heap_level_h(uint32_t arity, uint32_t j) {
+    uint32_t l = 0; uint64_t start = 0, width = 1;
+    while (j >= start + width) { start += width; width *= arity; ++l; }
+    return l;
+}
+// children per node from the descriptor's flags: 0 = not given = binary; 1 and values above FTC_MAX_ARITY are invalid
+static bool tree_arity(uint32_t flags, uint32_t& arity) {
+    const uint32_t a = (flags >> 16) & 0xFFu;
+    arity = a ? a : 2u;
+    return a != 1 && a <= FTC_MAX_ARITY;
+}
 
 static uint32_t elem_size(uint32_t dtype) { return (dtype == FTC_I32 || dtype == FTC_F32) ? 4u : 8u; }
 
@@ -27,11 +39,14 @@ static int fill_params(const ftc_desc_t* d, uint64_t S, int is_allreduce, Params
     if (d->k == 0 || d->f > FTC_MAX_F || d->P < d->f + 2 || d->max_inop > FTC_MAX_INOP) return FTC_EINVAL;
     if (d->root >= 0 && (uint32_t)d->root >= d->P) return FTC_EINVAL;
     if ((uint64_t)d->k * elem_size(d->dtype) > 0x7FFFFFFFull || (uint64_t)d->P * d->k > (1ull << 40)) return FTC_EINVAL;
+    uint32_t arity;
+    if (!tree_arity(d->flags, arity)) return FTC_EINVAL;
     std::memset(&p, 0, sizeof p);
+    p.arity = arity;
     p.P = d->P; p.f = d->f; p.m = d->f + 1; p.k = d->k; p.W = (d->P + 31) / 32;
     p.q = (d->P - 1) / p.m; p.r = (d->P - 1) % p.m;
     p.Gmax = p.q + (p.r ? 1u : 0u);
-    p.H = 1 + ilog2h(p.Gmax);
+    p.H = 1 + heap_level_h(p.arity, p.Gmax - 1);
     p.Rred = p.f + p.H; p.Ratt = 2 * p.Rred;
     p.max_inop = d->max_inop; p.flags = d->flags; p.root = d->root; p.is_allreduce = is_allreduce;
     p.kbytes = d->k * elem_size(d->dtype);
@@ -53,7 +68,7 @@ static const DeviceInfo kB200 = {148, 232448};
 
 enum KernelKind { K_GENERIC = 0, K_TILED = 1, K_STAGED = 2 };
 static KernelKind pick_kernel(Params& p, const DeviceInfo& di) {
-    if (p.flags & FTC_KERNEL_GENERIC) return K_GENERIC;
+    if ((p.flags & FTC_KERNEL_GENERIC) || p.arity != 2) return K_GENERIC;      // the tiled kernels are built on the binary heap
     if (!(p.flags & FTC_KERNEL_DIRECT) && staged_supported(p, di.smem_optin)) return K_STAGED;
     return tiled_supported(p, di.smem_optin) ? K_TILED : K_GENERIC;
 }
@@ -285,10 +300,11 @@ size_t ftc_host_staging_bytes(const ftc_desc_t* desc, uint64_t chunk_scenarios) 
 }
 
 int ftc_schedule_info(const ftc_desc_t* desc, ftc_sched_t* out) {
-    if (!desc || !out || desc->f > FTC_MAX_F || desc->P < desc->f + 2) return FTC_EINVAL;
+    uint32_t arity;
+    if (!desc || !out || desc->f > FTC_MAX_F || desc->P < desc->f + 2 || !tree_arity(desc->flags, arity)) return FTC_EINVAL;
     const uint32_t m = desc->f + 1, q = (desc->P - 1) / m, r = (desc->P - 1) % m;
     out->q = q; out->r = r;
-    out->H = 1 + ilog2h(q + (r ? 1u : 0u));
+    out->H = 1 + heap_level_h(arity, q + (r ? 1u : 0u) - 1);
     out->rounds_reduce = desc->f + out->H;
     out->rounds_attempt = 2 * out->rounds_reduce;
     out->msgs_upcorrection = (uint64_t)desc->f * m * q + (uint64_t)(r + 1) * r;

@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(256) candidates_kernel(Params p, T* cand, uint
         if (tid < p.max_inop && cx->iv[tid] != FTC_INOP_UNUSED) {
             const uint32_t v = renumber(cx->iv[tid], root);
             if (v) {
-                const uint32_t d = 1 + ilog2u((v - 1) / p.m + 1), t = local_round(cx->ir[tid], base);
+                const uint32_t d = 1 + heap_level(p.arity, (v - 1) / p.m), t = local_round(cx->ir[tid], base);
                 if (!(p.f + p.H - d < t)) atomicAnd(&snd[v >> 5], ~(1u << (v & 31)));
             }
         }
@@ -90,8 +90,9 @@ __global__ void __launch_bounds__(256) candidates_kernel(Params p, T* cand, uint
             }
             __syncthreads();
             const uint32_t G = p.q + (sc < p.r ? 1u : 0u);
-            for (int lvl = (int)ilog2u(G); lvl >= 0; --lvl) {
-                const uint32_t lo = (1u << lvl) - 1u, hi = min(2u * lo + 1u, G);
+            for (int lvl = (int)heap_level(p.arity, G - 1); lvl >= 0; --lvl) {
+                const uint32_t lo = (uint32_t)heap_level_start(p.arity, lvl);
+                const uint32_t hi = (uint32_t)min(heap_level_start(p.arity, lvl + 1), (uint64_t)G);
                 for (uint32_t u = tid; u < (hi - lo) * p.k; u += nt) {
                     const uint32_t j = lo + u / p.k, e = u % p.k;
                     const uint32_t v = j * p.m + sc + 1;
@@ -104,7 +105,7 @@ __global__ void __launch_bounds__(256) candidates_kernel(Params p, T* cand, uint
                     for (uint32_t sp = 0; sp < mj; ++sp)
                         if (sp != sc && ((mask >> sp) & 1u)) acc = Comb<T, OP>::f(acc, in_s[(size_t)renumber(vbase + sp, root) * p.k + e]);
                     uint32_t fb = 0, nf = mj - __popc(mask) + ((j == p.q && !from_root) ? 1u : 0u);   // partners whose message did not arrive
-                    for (uint32_t c = 2 * j + 1; c <= 2 * j + 2 && c < G; ++c) {
+                    for (uint64_t c = (uint64_t)p.arity * j + 1; c <= (uint64_t)p.arity * j + p.arity && c < G; ++c) {
                         if (pres[c]) { acc = Comb<T, OP>::f(acc, val[(size_t)c * p.k + e]); fb |= fbit[c]; nf += nfl[c]; }
                         else { fb = 1; nf += 1; }
                     }

@@ -13,6 +13,7 @@ struct Params {
     uint32_t P, f, m, k, W;          // m = f+1 (group size = root children); W = mask words per scenario
     uint32_t q, r, H, Rred, Ratt;    // P-1 = q*m + r; deepest node; rounds of a reduce / of an allreduce attempt
     uint32_t Gmax;                   // nodes of the largest root subtree: q + (r > 0)
+    uint32_t arity;                  // children per node below the root's children (2: binary heap)
     uint32_t max_inop, flags;
     int32_t  root;
     int32_t  is_allreduce;
@@ -53,6 +54,32 @@ struct Ctx {
 
 __device__ __forceinline__ uint32_t ilog2u(uint32_t v) { return 31u - __clz(v); }
 __device__ __forceinline__ bool test_bit(const uint32_t* bm, uint32_t i) { return (bm[i >> 5] >> (i & 31)) & 1u; }
+
+// ---- subtree shape: below each root child a heap on the local index j with p.arity children per node ----
+// Level l holds the arity^l indices that follow those of the levels above; node j has children a*j+1 .. a*j+a.
+__device__ __forceinline__ uint32_t heap_level(uint32_t arity, uint32_t j) {
+    if (arity == 2) return ilog2u(j + 1);
+    uint32_t l = 0; uint64_t start = 0, width = 1;
+    while (j >= start + width) { start += width; width *= arity; ++l; }
+    return l;
+}
+// First index of level l (the levels above hold (a^l - 1)/(a - 1) indices); saturates far beyond any index.
+__device__ __forceinline__ uint64_t heap_level_start(uint32_t arity, uint32_t l) {
+    if (arity == 2) return ((uint64_t)1 << l) - 1;
+    uint64_t start = 0, width = 1;
+    for (uint32_t i = 0; i < l && start < ((uint64_t)1 << 40); ++i) { start += width; width *= arity; }
+    return start;
+}
+// Sets in `bm` (bits = renumbered ranks) every process below local index j of root subtree sv, which has Gs nodes.
+// All lanes of a warp call it with the same arguments.
+__device__ __forceinline__ void mark_descendants(uint32_t arity, uint32_t m, uint32_t* bm, uint32_t j, uint32_t sv,
+                                                 uint32_t Gs, uint32_t lane) {
+    for (uint64_t lo = (uint64_t)arity * j + 1, n = arity; lo < Gs; lo = arity * lo + 1, n *= arity)
+        for (uint64_t i = lane; i < n && lo + i < Gs; i += 32) {
+            const uint32_t u = (uint32_t)(lo + i) * m + sv + 1;
+            atomicOr(&bm[u >> 5], 1u << (u & 31));
+        }
+}
 
 // n <= 32 bits of a bitmask starting at bit `pos`; the mask has one zero word of padding at its end.
 __device__ __forceinline__ uint32_t extract_bits(const uint32_t* bm, uint32_t pos, uint32_t n) {
@@ -163,7 +190,7 @@ static __device__ void decode_scenario(const Params& p, uint64_t s, Ctx* cx, uin
     if (tid < p.max_inop && cx->iv[tid] != FTC_INOP_UNUSED) {
         uint32_t v = renumber(cx->iv[tid], root);
         if (v) {
-            uint32_t j = (v - 1) / p.m, d = 1 + ilog2u(j + 1);
+            uint32_t j = (v - 1) / p.m, d = 1 + heap_level(p.arity, j);
             uint32_t t = local_round(cx->ir[tid], base);
             if (!(p.f + p.H - d < t)) F |= 1u << ((v - 1) % p.m);     // tree send of depth d is round f+H-d
         }
@@ -264,11 +291,7 @@ static __device__ void count_holders(const Params& p, Ctx* cx, const uint32_t* p
                 uint32_t v = renumber(wbase + b, root);
                 if (!v) continue;
                 uint32_t j = (v - 1) / p.m, sv = (v - 1) % p.m, Gs = p.q + (sv < p.r ? 1u : 0u);
-                for (uint32_t lo = 2 * j + 1, n = 2; lo < Gs; lo = 2 * lo + 1, n *= 2)
-                    for (uint32_t i = lane; i < n && lo + i < Gs; i += 32) {
-                        uint32_t u = (lo + i) * p.m + sv + 1;
-                        atomicOr(&unr[u >> 5], 1u << (u & 31));
-                    }
+                mark_descendants(p.arity, p.m, unr, j, sv, Gs, lane);
             }
         }
     }
@@ -281,13 +304,9 @@ static __device__ void count_holders(const Params& p, Ctx* cx, const uint32_t* p
                 if (hold) atomicAnd(&hold[cx->iv[i] >> 5], ~(1u << (cx->iv[i] & 31)));
             }
             if (!v) continue;
-            uint32_t j = (v - 1) / p.m, sv = (v - 1) % p.m, Gs = p.q + (sv < p.r ? 1u : 0u), d = 1 + ilog2u(j + 1);
+            uint32_t j = (v - 1) / p.m, sv = (v - 1) % p.m, Gs = p.q + (sv < p.r ? 1u : 0u), d = 1 + heap_level(p.arity, j);
             if (t > p.Rred + d) continue;                  // it does forward: tree-down send of depth d is round f+H+d
-            for (uint32_t lo = 2 * j + 1, n = 2; lo < Gs; lo = 2 * lo + 1, n *= 2)
-                for (uint32_t k2 = lane; k2 < n && lo + k2 < Gs; k2 += 32) {
-                    uint32_t u = (lo + k2) * p.m + sv + 1;
-                    atomicOr(&unr[u >> 5], 1u << (u & 31));
-                }
+            mark_descendants(p.arity, p.m, unr, j, sv, Gs, lane);
         }
     }
     __syncthreads();

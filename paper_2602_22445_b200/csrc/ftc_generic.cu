@@ -66,14 +66,15 @@ __global__ void __launch_bounds__(256) generic_kernel(Params p) {
         if (p.is_allreduce) count_holders(p, cx, pf, unr);
         const T* in_s = reinterpret_cast<const T*>(p.in) + s * (size_t)p.P * p.k;
         const uint32_t G = cx->G;
-        // tree phase (Algorithm "reduce_non_root"): data <- data (op) child 1 (op) child 2, leaves first
-        for (int lvl = (int)ilog2u(G); lvl >= 0; --lvl) {
-            const uint32_t lo = (1u << lvl) - 1u, hi = min(2u * lo + 1u, G);
+        // tree phase (Algorithm "reduce_non_root"): data <- data (op) child 1 (op) child 2 ..., leaves first
+        for (int lvl = (int)heap_level(p.arity, G - 1); lvl >= 0; --lvl) {
+            const uint32_t lo = (uint32_t)heap_level_start(p.arity, lvl);
+            const uint32_t hi = (uint32_t)min(heap_level_start(p.arity, lvl + 1), (uint64_t)G);
             for (uint32_t u = tid; u < (hi - lo) * p.k; u += nt) {
                 const uint32_t j = lo + u / p.k, e = u % p.k;
                 T v = fold_group_scalar<T, OP>(p, cx, inc, in_s, j, e);
-                if (2 * j + 1 < G) v = Comb<T, OP>::f(v, ws[(size_t)(2 * j + 1) * p.k + e]);
-                if (2 * j + 2 < G) v = Comb<T, OP>::f(v, ws[(size_t)(2 * j + 2) * p.k + e]);
+                for (uint64_t c = (uint64_t)p.arity * j + 1; c <= (uint64_t)p.arity * j + p.arity && c < G; ++c)
+                    v = Comb<T, OP>::f(v, ws[(size_t)c * p.k + e]);
                 ws[(size_t)j * p.k + e] = v;
             }
             __syncthreads();

@@ -18,7 +18,7 @@ __device__ __forceinline__ uint32_t n_partners(const Params& p, uint32_t v) {
     if (v == 0) return p.r;
     return (v - 1) / p.m < p.q ? p.f : p.r;
 }
-__device__ __forceinline__ uint32_t depth_of(const Params& p, uint32_t v) { return v ? 1u + ilog2u((v - 1) / p.m + 1) : 0u; }
+__device__ __forceinline__ uint32_t depth_of(const Params& p, uint32_t v) { return v ? 1u + heap_level(p.arity, (v - 1) / p.m) : 0u; }
 
 // What a process with failure round t (on the attempt's clock, t != kNever) does not send in the reduce of an
 // attempt: up-correction sends i >= t, and its tree send when that lies in a round >= t.
@@ -89,12 +89,8 @@ __global__ void __launch_bounds__(kMsgThreads) messages_kernel(Params p, unsigne
             // a process that does not pass the value on cuts off everything below it: bit v of unr = the tree-down
             // phase sends no message to renumbered process v
             auto mark_below = [&](uint32_t v) {
-                const uint32_t j = (v - 1) / p.m, sv = (v - 1) % p.m, Gs = p.q + (sv < p.r ? 1u : 0u);
-                for (uint32_t lo = 2 * j + 1, n = 2; lo < Gs; lo = 2 * lo + 1, n *= 2)
-                    for (uint32_t i = lane; i < n && lo + i < Gs; i += 32) {
-                        const uint32_t u = (lo + i) * p.m + sv + 1;
-                        atomicOr(&unr[u >> 5], 1u << (u & 31));
-                    }
+                const uint32_t sv = (v - 1) % p.m;
+                mark_descendants(p.arity, p.m, unr, (v - 1) / p.m, sv, p.q + (sv < p.r ? 1u : 0u), lane);
             };
             const uint32_t nwords_round = (p.W + 31) & ~31u;
             for (uint32_t w0 = wid * 32; w0 < nwords_round; w0 += nw * 32) {

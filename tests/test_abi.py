@@ -35,6 +35,11 @@ def test_host_only_calls():
     assert B.ftc_workspace_bytes(B.make_desc(8, 1, 1, B.FTC_I32, "sum"), 9) == 9 * 4 * 4
     assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_KERNEL_DIRECT)) == "tiled"
     assert B.ftc_kernel_name(B.make_desc(2, 1, 1, B.FTC_I32, "sum")) == "invalid"
+    # other subtree shapes: depth of the deepest node of an a-ary heap; they run on the general kernel
+    t = B.ftc_schedule_info(B.make_desc(1024, 3, 16, B.FTC_F32, "sum", flags=B.FTC_TREE_ARITY(4)))
+    assert (t["H"], t["rounds_reduce"], t["rounds_attempt"]) == (5, 8, 16)       # 256 rows: levels of 1, 4, 16, 64, 171
+    assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(3))) == "generic"
+    assert B.ftc_kernel_name(B.make_desc(8, 1, 1, B.FTC_I32, "sum", flags=B.FTC_TREE_ARITY(1))) == "invalid"
     for code in (0, -1, -2, -3, -4, -5):
         assert B.ftc_strerror(code) and "unknown" not in B.ftc_strerror(code)
     assert "unknown" in B.ftc_strerror(-99)
