@@ -189,27 +189,43 @@ __device__ __forceinline__ void fold_tile_fast(const Params& p, uint32_t root, u
         off[1 + b] = g < G ? staged_row_offset<WHOLE>(p, rowbytes, t, g) : off0;   // a missing row reads the root's bytes, unused
     }
     uint4 acc[NS];
-    const char* own = buf_lc + sstar * p.kbytes;
+    if (!Ordered<T>::value && !masked) {
+        // Any member order gives the same bits. When a group's bytes are a multiple of 128, the rows of different
+        // lane rows start in the same shared-memory bank: each lane row then starts at another member.
+        uint32_t mem = (rowbytes & 127u) ? 0u : lr % p.m;
+        const char* src = buf_lc + mem * p.kbytes;
 #pragma unroll
-    for (int s = 0; s < NS; ++s) acc[s] = lds(own + off[s]);
-    if (!masked) {
+        for (int s = 0; s < NS; ++s) acc[s] = lds(src + off[s]);
 #pragma unroll 1
         for (uint32_t i = 1; i < p.m; ++i) {
-            const char* mem = buf_lc + (i - (i <= sstar ? 1u : 0u)) * p.kbytes;      // partners ascending, own skipped
+            if (++mem == p.m) mem = 0;
+            src = buf_lc + mem * p.kbytes;
 #pragma unroll
-            for (int s = 0; s < NS; ++s) acc[s] = comb16<T, OP>(acc[s], lds(mem + off[s]));
+            for (int s = 0; s < NS; ++s) acc[s] = comb16<T, OP>(acc[s], lds(src + off[s]));
         }
     } else {
-        uint32_t mask[NS];
+        const char* own = buf_lc + sstar * p.kbytes;
 #pragma unroll
-        for (int s = 0; s < NS; ++s) mask[s] = grow[s] < G ? extract_bits(inc, grow[s] * p.m + 1, p.m) : 0u;
+        for (int s = 0; s < NS; ++s) acc[s] = lds(own + off[s]);
+        if (!masked) {
 #pragma unroll 1
-        for (uint32_t i = 1; i < p.m; ++i) {
-            const uint32_t sp = i - (i <= sstar ? 1u : 0u);
-            const char* mem = buf_lc + sp * p.kbytes;
+            for (uint32_t i = 1; i < p.m; ++i) {
+                const char* mem = buf_lc + (i - (i <= sstar ? 1u : 0u)) * p.kbytes;      // partners ascending, own skipped
 #pragma unroll
-            for (int s = 0; s < NS; ++s)
-                if ((mask[s] >> sp) & 1u) acc[s] = comb16<T, OP>(acc[s], lds(mem + off[s]));
+                for (int s = 0; s < NS; ++s) acc[s] = comb16<T, OP>(acc[s], lds(mem + off[s]));
+            }
+        } else {
+            uint32_t mask[NS];
+#pragma unroll
+            for (int s = 0; s < NS; ++s) mask[s] = grow[s] < G ? extract_bits(inc, grow[s] * p.m + 1, p.m) : 0u;
+#pragma unroll 1
+            for (uint32_t i = 1; i < p.m; ++i) {
+                const uint32_t sp = i - (i <= sstar ? 1u : 0u);
+                const char* mem = buf_lc + sp * p.kbytes;
+#pragma unroll
+                for (int s = 0; s < NS; ++s)
+                    if ((mask[s] >> sp) & 1u) acc[s] = comb16<T, OP>(acc[s], lds(mem + off[s]));
+            }
         }
     }
     valB = acc[0];
@@ -244,8 +260,8 @@ constexpr int kStagedLeanThreads = 64;      // lean variant: at most two warps, 
 constexpr int kStagedLeanMinBlocks = 10;
 
 template <typename T, int OP, int XL, bool WHOLE, int MINB>
-__global__ void __launch_bounds__(MINB > 2 ? kStagedLeanThreads : kStagedMaxThreads, MINB) staged_kernel(Params p, StagedGeom g) {
-    constexpr bool LEAN = MINB > 2;
+__global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThreads : kStagedMaxThreads, MINB) staged_kernel(Params p, StagedGeom g) {
+    constexpr bool LEAN = MINB == kStagedLeanMinBlocks;
     extern __shared__ __align__(128) uint32_t smem[];
     char* sbase = reinterpret_cast<char*>(smem);
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
@@ -519,9 +535,11 @@ template <typename T, int OP, int XL>
 static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
     StagedGeom g;
     if (!staged_geometry(p, smem_optin, XL, g)) return cudaErrorInvalidConfiguration;
-    // one- and two-warp blocks get the lean variant; its register cap (about 96) matches the blocks that fit by shared memory
+    // one- and two-warp blocks get the lean variant; its register cap (about 96) matches the blocks that fit by shared
+    // memory. Scenarios staged whole are so small that many more blocks fit: for them 64 registers, so that the
+    // SM's block limit and not the register file decides
     const bool lean = g.nwarps <= 2;
-    if (g.whole) return lean ? launch_staged_w<T, OP, XL, true, kStagedLeanMinBlocks>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, true, 2>(p, g, sm_count, st);
+    if (g.whole) return lean ? launch_staged_w<T, OP, XL, true, 4>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, true, 2>(p, g, sm_count, st);
     return lean ? launch_staged_w<T, OP, XL, false, kStagedLeanMinBlocks>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
 }
 
