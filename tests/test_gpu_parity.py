@@ -342,3 +342,45 @@ def test_candidates_of_every_root_child_match_oracle(allreduce):
             assert np.array_equal(info[i, :, 0], d["cand_flag"]), (P, f, i, d["code"])
             assert np.array_equal(info[i, :, 1], d["cand_nfail"]), (P, f, i)
             assert np.array_equal(cand[i].view(np.uint8), d["cand"].view(np.uint8)), (P, f, i)
+
+
+# ---------------------------------------------------------------------------------------------
+# a sparsely filled last heap level: its rows stay out of the warp tiles and are folded one by one
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("P,f,k,dname", [(1024, 3, 16, "f32"),     # 256 rows: one row (the short group) on the last level
+                                         (533, 1, 4, "i32"),       # 266 rows, 10 on the last level; staged whole
+                                         (1598, 2, 8, "i64"),      # 533 rows, 21 on the last level, short group among them
+                                         (2056, 7, 4, "f32")])     # 257 rows: one row on the last level, wide groups
+@pytest.mark.parametrize("allreduce", [False, True])
+def test_sparse_last_level_failures_roots_and_victims_there(P, f, k, dname, allreduce):
+    rng = np.random.Generator(np.random.PCG64(P + f))
+    S, m = 96, f + 1
+    Gmax = (P - 1 + m - 1) // m
+    first_last = (1 << (Gmax.bit_length() - 1)) - 1                 # first row of the last heap level
+    tail = list(range(first_last * m + 1, P))                        # processes of the last level's rows
+    assert 0 < len(tail) <= (m * (first_last + 1)) // 8 + m
+    x = rng.standard_normal((S, P, k)).astype(np.float32) if dname == "f32" else \
+        rng.integers(np.iinfo(DT[dname]).min, np.iinfo(DT[dname]).max, size=(S, P, k), dtype=DT[dname])
+    R = O.schedule(P, f)
+    sets, inop, roots = [], np.full((S, 2, 2), sc.UNUSED, dtype=np.uint32), np.zeros(S, dtype=np.uint32)
+    for i in range(S):
+        n_tail = int(rng.integers(0, min(f, len(tail)) + 1))
+        dead = set(int(v) for v in rng.choice(tail, size=n_tail, replace=False))
+        dead |= set(int(v) for v in rng.integers(0, P, size=int(rng.integers(0, f + 1 - n_tail + 1))))
+        roots[i] = int(rng.choice(tail)) if rng.random() < 0.5 else int(rng.integers(0, P))
+        if allreduce and rng.random() < 0.5:
+            roots[i] = P - 1 - int(rng.integers(0, 2))               # candidates wrap around to process 0
+        for j in range(2):
+            if rng.random() < 0.6:
+                v = int(rng.choice(tail)) if rng.random() < 0.7 else int(rng.integers(0, P))
+                if allreduce and (v - int(roots[i])) % P <= f:
+                    continue
+                inop[i, j] = (v, int(rng.integers(0, R["rounds_attempt"] + 2)))
+        sets.append(sorted(dead))
+    pf = sc.sets_to_masks(sets, P)
+    op = "sum" if dname == "f32" else "max"
+    for flags in KERNELS:
+        got = run_gpu(x, f, op, pf, inop, roots, 0, allreduce, flags)
+        want = run_oracle(x, f, op, pf, inop, roots, 0, allreduce)
+        assert_same(got, want, f"P={P} f={f} k={k} {dname} allreduce={allreduce} flags={flags:#x}")
+        assert ((want[1][:, 0] & 0xFF) == 0).sum() > S // 3
