@@ -207,12 +207,14 @@ def run_reference(args):
 # GPU arm
 # ------------------------------------------------------------------------------------------------
 def kernel_source_hash() -> str:
-    """Hash of the CUDA sources: ncu counters taken from an older kernel must not be quoted for a newer one."""
+    """Hash of the sources of the staged kernel (the one the traffic figures belong to): ncu counters taken from
+    an older kernel must not be quoted for a newer one."""
     import glob
     import hashlib
     h = hashlib.sha256()
     base = os.path.join(ROOT, "paper_2602_22445_b200", "csrc")
-    for f in sorted(glob.glob(os.path.join(base, "*.cu")) + glob.glob(os.path.join(base, "*.cuh")) + glob.glob(os.path.join(base, "*.h"))):
+    files = glob.glob(os.path.join(base, "ftc_staged*")) + [os.path.join(base, n) for n in ("ftc_tile_common.cuh", "ftc_device.cuh")]
+    for f in sorted(files):
         h.update(open(f, "rb").read())
     return h.hexdigest()[:16]
 
