@@ -1,36 +1,52 @@
 // General kernel: any P, f, k. One block per scenario (grid-stride), the selected subtree is evaluated level by
 // level from the leaves, node values pass through a per-block slice of the global workspace.
 #include <mutex>
-#include "ftc_device.cuh"
+#include "ftc_tile_common.cuh"
 #include "ftc_kernels.h"
 
 namespace ftc {
 
+// The unit a thread works on: one element, or (VEC) one 16-byte chunk of a process vector when vectors are a
+// whole number of chunks.
+template <typename T, int OP, bool VEC> struct Unit;
+template <typename T, int OP> struct Unit<T, OP, false> {
+    using V = T;
+    static __device__ __forceinline__ V comb(V a, V b) { return Comb<T, OP>::f(a, b); }
+    static __device__ __forceinline__ V zero() { return T(0); }
+    static __device__ __forceinline__ V ld(const V* q) { return __ldg(q); }
+};
+template <typename T, int OP> struct Unit<T, OP, true> {
+    using V = uint4;
+    static __device__ __forceinline__ V comb(V a, V b) { return comb16<T, OP>(a, b); }
+    static __device__ __forceinline__ V zero() { return make_uint4(0, 0, 0, 0); }
+    static __device__ __forceinline__ V ld(const V* q) { return __ldg(q); }
+};
+
 // Value of group `row` as the selected subtree's member sees it after up-correction (Algorithm "Up-correction"):
 // own input first, then the partners whose message arrived, in ascending rank (the root first in the short group).
-template <typename T, int OP>
-__device__ __forceinline__ T fold_group_scalar(const Params& p, const Ctx* cx, const uint32_t* inc, const T* in_s,
-                                               uint32_t row, uint32_t e) {
-    const uint32_t root = cx->root, sstar = cx->sstar;
+// `in_s`: the scenario as units, `nu` units per process, `u` the unit.
+template <typename U>
+__device__ __forceinline__ typename U::V fold_group_unit(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
+                                                          const typename U::V* in_s, uint32_t nu, uint32_t row, uint32_t u) {
     const uint32_t mj = row < p.q ? p.m : p.r, vbase = row * p.m + 1;
     const uint32_t mask = extract_bits(inc, vbase, mj);
-    T acc = in_s[(size_t)renumber(vbase + sstar, root) * p.k + e];
-    if (row == p.q) acc = Comb<T, OP>::f(acc, in_s[(size_t)root * p.k + e]);
+    typename U::V acc = U::ld(in_s + (size_t)renumber(vbase + sstar, root) * nu + u);
+    if (row == p.q) acc = U::comb(acc, U::ld(in_s + (size_t)root * nu + u));
     for (uint32_t sp = 0; sp < mj; ++sp)
-        if (sp != sstar && ((mask >> sp) & 1u)) acc = Comb<T, OP>::f(acc, in_s[(size_t)renumber(vbase + sp, root) * p.k + e]);
+        if (sp != sstar && ((mask >> sp) & 1u)) acc = U::comb(acc, U::ld(in_s + (size_t)renumber(vbase + sp, root) * nu + u));
     return acc;
 }
 
 // The root's own data after up-correction when it is a member of the short last group whose other members all
 // lie outside the selected subtree.
-template <typename T, int OP>
-__device__ __forceinline__ T fold_root_scalar(const Params& p, const Ctx* cx, const uint32_t* inc, const T* in_s, uint32_t e) {
-    const uint32_t root = cx->root;
-    T acc = in_s[(size_t)root * p.k + e];
+template <typename U>
+__device__ __forceinline__ typename U::V fold_root_unit(const Params& p, uint32_t root, const uint32_t* inc,
+                                                         const typename U::V* in_s, uint32_t nu, uint32_t u) {
+    typename U::V acc = U::ld(in_s + (size_t)root * nu + u);
     if (p.r) {
         const uint32_t vbase = p.q * p.m + 1, mask = extract_bits(inc, vbase, p.r);
         for (uint32_t sp = 0; sp < p.r; ++sp)
-            if ((mask >> sp) & 1u) acc = Comb<T, OP>::f(acc, in_s[(size_t)renumber(vbase + sp, root) * p.k + e]);
+            if ((mask >> sp) & 1u) acc = U::comb(acc, U::ld(in_s + (size_t)renumber(vbase + sp, root) * nu + u));
     }
     return acc;
 }
@@ -44,46 +60,64 @@ static __device__ void write_status(const Params& p, uint64_t s, const Ctx* cx) 
     st[3] = (ok && p.is_allreduce) ? cx->holders : 0u;
 }
 
-template <typename T, int OP>
-__global__ void __launch_bounds__(256) generic_kernel(Params p) {
+template <typename T, int OP, bool VEC>
+__global__ void __launch_bounds__(256, VEC ? 0 : 8) generic_kernel(Params p) {
+    using U = Unit<T, OP, VEC>;
+    using V = typename U::V;
     extern __shared__ uint32_t smem[];
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
     uint32_t* pf = smem + sizeof(Ctx) / 4;
     uint32_t* inc = pf + p.W + 1;
     uint32_t* unr = inc + p.W + 1;
     const uint32_t tid = threadIdx.x, nt = blockDim.x;
-    T* ws = reinterpret_cast<T*>(p.ws) + (size_t)blockIdx.x * p.Gmax * p.k;
+    const uint32_t nu = VEC ? p.kbytes / 16 : p.k;                 // units per process vector
+    // a power-of-two group of `upw` lanes walks the units of one row; 32/upw rows per warp, no divisions
+    uint32_t upw_log2 = 0; while ((1u << upw_log2) < nu && upw_log2 < 5) ++upw_log2;
+    const uint32_t upw = 1u << upw_log2, rows_per_pass = nt >> upw_log2, r0 = tid >> upw_log2, u0 = tid & (upw - 1);
+    V* ws = reinterpret_cast<V*>(p.ws) + (size_t)blockIdx.x * p.Gmax * nu;
 
     for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {
         decode_scenario(p, s, cx, pf, inc);
-        T* out_s = reinterpret_cast<T*>(p.out) + s * p.k;
+        V* out_s = reinterpret_cast<V*>(p.out) + s * nu;
         if (cx->code != FTC_ST_OK) {
-            for (uint32_t e = tid; e < p.k; e += nt) out_s[e] = T(0);
+            for (uint32_t u = tid; u < nu; u += nt) out_s[u] = U::zero();
             if (tid == 0) write_status(p, s, cx);
             __syncthreads();
             continue;
         }
         if (p.is_allreduce) count_holders(p, cx, pf, unr);
-        const T* in_s = reinterpret_cast<const T*>(p.in) + s * (size_t)p.P * p.k;
-        const uint32_t G = cx->G;
+        const V* in_s = reinterpret_cast<const V*>(p.in) + s * (size_t)p.P * nu;
+        const uint32_t G = cx->G, root = cx->root, sstar = cx->sstar;
         // tree phase (Algorithm "reduce_non_root"): data <- data (op) child 1 (op) child 2 ..., leaves first
         for (int lvl = (int)heap_level(p.arity, G - 1); lvl >= 0; --lvl) {
             const uint32_t lo = (uint32_t)heap_level_start(p.arity, lvl);
             const uint32_t hi = (uint32_t)min(heap_level_start(p.arity, lvl + 1), (uint64_t)G);
-            for (uint32_t u = tid; u < (hi - lo) * p.k; u += nt) {
-                const uint32_t j = lo + u / p.k, e = u % p.k;
-                T v = fold_group_scalar<T, OP>(p, cx, inc, in_s, j, e);
-                for (uint64_t c = (uint64_t)p.arity * j + 1; c <= (uint64_t)p.arity * j + p.arity && c < G; ++c)
-                    v = Comb<T, OP>::f(v, ws[(size_t)c * p.k + e]);
-                ws[(size_t)j * p.k + e] = v;
+            if (VEC) {
+                for (uint32_t j = lo + r0; j < hi; j += rows_per_pass) {
+                    const uint64_t c0 = (uint64_t)p.arity * j + 1, c1 = min(c0 + p.arity, (uint64_t)G);
+                    for (uint32_t u = u0; u < nu; u += upw) {
+                        V v = fold_group_unit<U>(p, root, sstar, inc, in_s, nu, j, u);
+                        for (uint64_t c = c0; c < c1; ++c) v = U::comb(v, ws[(size_t)c * nu + u]);
+                        ws[(size_t)j * nu + u] = v;
+                    }
+                }
+            } else {
+                // single elements: every thread takes the next (row, element) pair of the level, whatever k is
+                for (uint32_t x = tid; x < (hi - lo) * nu; x += nt) {
+                    const uint32_t j = lo + x / nu, u = x % nu;
+                    const uint64_t c0 = (uint64_t)p.arity * j + 1, c1 = min(c0 + p.arity, (uint64_t)G);
+                    V v = fold_group_unit<U>(p, root, sstar, inc, in_s, nu, j, u);
+                    for (uint64_t c = c0; c < c1; ++c) v = U::comb(v, ws[(size_t)c * nu + u]);
+                    ws[(size_t)j * nu + u] = v;
+                }
             }
             __syncthreads();
         }
         // root (Algorithm "reduce_root"): the selected child's value, combined with the root's own data unless the
         // child's subtree already holds it (it does iff it contains a member of the root's group)
-        for (uint32_t e = tid; e < p.k; e += nt) {
-            T recv = ws[e];
-            out_s[e] = cx->sstar < p.r ? recv : Comb<T, OP>::f(fold_root_scalar<T, OP>(p, cx, inc, in_s, e), recv);
+        for (uint32_t u = tid; u < nu; u += nt) {
+            V recv = ws[u];
+            out_s[u] = sstar < p.r ? recv : U::comb(fold_root_unit<U>(p, root, inc, in_s, nu, u), recv);
         }
         if (tid == 0) write_status(p, s, cx);
         __syncthreads();
@@ -97,15 +131,22 @@ uint32_t generic_grid(const Params& p, int sm_count) {
     return (uint32_t)(p.S < g ? p.S : g);
 }
 
-template <typename T, int OP>
-static cudaError_t launch_generic_t(const Params& p, int sm_count, cudaStream_t st) {
+template <typename T, int OP, bool VEC>
+static cudaError_t launch_generic_v(const Params& p, uint32_t grid, cudaStream_t st) {
     size_t smem = generic_smem_bytes(p);
     if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(generic_kernel<T, OP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(generic_kernel<T, OP, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    generic_kernel<T, OP><<<generic_grid(p, sm_count), 256, smem, st>>>(p);
+    generic_kernel<T, OP, VEC><<<grid, 256, smem, st>>>(p);
     return cudaGetLastError();
+}
+
+// 16-byte units when the process vectors are a whole number of them (inputs, results and workspace are 16-byte aligned)
+template <typename T, int OP>
+static cudaError_t launch_generic_t(const Params& p, int sm_count, cudaStream_t st) {
+    return p.kbytes % 16 == 0 ? launch_generic_v<T, OP, true>(p, generic_grid(p, sm_count), st)
+                              : launch_generic_v<T, OP, false>(p, generic_grid(p, sm_count), st);
 }
 
 cudaError_t launch_generic(const Params& p, int tsel, int sm_count, cudaStream_t st) {
@@ -154,13 +195,7 @@ static cudaError_t static_scratch_address(void** out) {
 
 template <typename T, int OP>
 static cudaError_t launch_static_t(const Params& p, uint32_t grid, cudaStream_t st) {
-    size_t smem = generic_smem_bytes(p);
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(generic_kernel<T, OP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
-    generic_kernel<T, OP><<<grid, 256, smem, st>>>(p);
-    return cudaGetLastError();
+    return p.kbytes % 16 == 0 ? launch_generic_v<T, OP, true>(p, grid, st) : launch_generic_v<T, OP, false>(p, grid, st);
 }
 
 // The general kernel with its node values in the built-in scratch: as many blocks as slices fit (at most the
