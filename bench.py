@@ -213,7 +213,8 @@ def kernel_source_hash() -> str:
     import hashlib
     h = hashlib.sha256()
     base = os.path.join(ROOT, "paper_2602_22445_b200", "csrc")
-    files = glob.glob(os.path.join(base, "ftc_staged*")) + [os.path.join(base, n) for n in ("ftc_tile_common.cuh", "ftc_device.cuh")]
+    files = glob.glob(os.path.join(base, "ftc_staged*.cu")) + glob.glob(os.path.join(base, "ftc_staged*.cuh")) + \
+        [os.path.join(base, n) for n in ("ftc_tile_common.cuh", "ftc_device.cuh")]
     for f in sorted(files):
         h.update(open(f, "rb").read())
     return h.hexdigest()[:16]
