@@ -141,8 +141,10 @@ typedef struct {
  *   d_roots   [S] or NULL; read only when desc->root < 0
  *   d_out     [S][k]: the value delivered at the root (zeros unless the outcome is FTC_ST_OK); 16-byte aligned
  *   d_status  [S][FTC_STATUS_WORDS]
- *   d_workspace, workspace_bytes: scratch of at least ftc_workspace_bytes(desc, S, 0) bytes (may be NULL if that is 0);
- *             contents are undefined afterwards; calls that share a workspace must not overlap on the device
+ *   d_workspace, workspace_bytes: scratch of at least ftc_workspace_bytes(desc, S, 0) bytes (may be NULL if that is 0),
+ *             16-byte aligned; contents are undefined afterwards; calls that share a workspace must not overlap on
+ *             the device. Shapes that run on the shared-memory kernels also run with less or none (large process
+ *             counts with wide vectors then more slowly); shapes that need the general kernel get FTC_EWORKSPACE
  * S = 0 is valid and does nothing. Returns FTC_OK or an error before anything is enqueued.
  */
 FTC_API int ftc_reduce_batch(const ftc_desc_t* desc, uint64_t S, const void* d_in, const uint32_t* d_prefail,
@@ -231,8 +233,9 @@ FTC_API int ftc_message_counts_batch(const ftc_desc_t* desc, uint64_t S, int is_
                                      const ftc_inop_t* d_inop, const uint32_t* d_roots, uint64_t* d_msgs,
                                      void* cuda_stream);
 
-/* Scratch bytes ftc_reduce_batch / ftc_allreduce_batch need for this descriptor and batch size (0 when the shape runs on the
- * shared-memory kernel). Returns 0 for an invalid descriptor as well; the batch calls report that. */
+/* Scratch bytes ftc_reduce_batch / ftc_allreduce_batch want for this descriptor and batch size: the general kernel's
+ * node values, the compact results of the expanded output, and for many processes with wide vectors the shared-memory
+ * kernel's array of tile results (0 otherwise). Returns 0 for an invalid descriptor as well; the batch calls report that. */
 FTC_API size_t ftc_workspace_bytes(const ftc_desc_t* desc, uint64_t S, int is_allreduce);
 
 /*

@@ -69,7 +69,7 @@ static const DeviceInfo kB200 = {148, 232448};
 enum KernelKind { K_GENERIC = 0, K_TILED = 1, K_STAGED = 2 };
 static KernelKind pick_kernel(Params& p, const DeviceInfo& di) {
     if ((p.flags & FTC_KERNEL_GENERIC) || p.arity != 2) return K_GENERIC;      // the tiled kernels are built on the binary heap
-    if (!(p.flags & FTC_KERNEL_DIRECT) && staged_supported(p, di.smem_optin)) return K_STAGED;
+    if (!(p.flags & FTC_KERNEL_DIRECT) && staged_supported(p, di.smem_optin, di.sm_count)) return K_STAGED;
     return tiled_supported(p, di.smem_optin) ? K_TILED : K_GENERIC;
 }
 
@@ -80,9 +80,14 @@ static size_t compact_area(const Params& p) {
     return (p.flags & FTC_OUT_EXPANDED) ? up256((size_t)p.S * p.kbytes) : 0;
 }
 
+// Workspace that lets the batch calls run at their best: the general kernel needs its slices; the staged kernel
+// uses one for large heap arrays (without it the shape runs more slowly, or on another kernel).
 static size_t workspace_for(Params& p, const DeviceInfo& di) {
     size_t need = compact_area(p);
-    if (pick_kernel(p, di) == K_GENERIC) need += (size_t)generic_grid(p, di.sm_count) * p.Gmax * p.kbytes;
+    p.ws_bytes = ~0ull;
+    const KernelKind kind = pick_kernel(p, di);
+    if (kind == K_GENERIC) need += (size_t)generic_grid(p, di.sm_count) * p.Gmax * p.kbytes;
+    else if (kind == K_STAGED) need += staged_workspace_bytes(p, di.smem_optin, di.sm_count);
     return need;
 }
 
@@ -111,6 +116,7 @@ static int run_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const
     const int tsel = type_select(desc->dtype, desc->op);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e;
+    p.ws = d_ws; p.ws_bytes = (d_ws && aligned16(d_ws)) ? ws_bytes : 0;
     const KernelKind kind = pick_kernel(p, di);
     if (kind == K_STAGED) {
         e = launch_staged(p, tsel, di.sm_count, di.smem_optin, st);
@@ -327,6 +333,7 @@ const char* ftc_kernel_name(const ftc_desc_t* desc, int is_allreduce) {
     if (fill_params(desc, 1, is_allreduce, p) != FTC_OK) return "invalid";
     DeviceInfo di;
     if (device_info(di) != FTC_OK) di = kB200;
+    p.ws_bytes = ~0ull;                                   // given the workspace ftc_workspace_bytes() asks for
     const KernelKind kind = pick_kernel(p, di);
     return kind == K_STAGED ? "staged" : kind == K_TILED ? "tiled" : "generic";
 }

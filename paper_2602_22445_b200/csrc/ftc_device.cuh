@@ -26,6 +26,7 @@ struct Params {
     void* out;
     uint32_t* status;
     void* ws;
+    uint64_t ws_bytes;               // bytes the caller's workspace offers at ws (0: none)
     // tiled kernel geometry
     uint32_t C;        // 16-byte chunks per process vector
     uint32_t cw_log2;  // log2 of lanes along the chunk dimension (= log2 C)

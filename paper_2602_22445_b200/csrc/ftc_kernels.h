@@ -25,7 +25,10 @@ bool tiled_supported(Params& p, int smem_optin_bytes);
 cudaError_t launch_tiled(const Params& p, int tsel, int sm_count, cudaStream_t st);
 
 // Staged kernel (bulk copies into shared memory): same shape limits plus room for the tile buffers.
-bool staged_supported(Params& p, int smem_optin_bytes);
+// With a workspace (p.ws_bytes) large heap arrays move there, which frees shared memory: more shapes fit and more
+// blocks are resident. staged_workspace_bytes: what that takes for this shape (0: nothing to gain).
+bool staged_supported(Params& p, int smem_optin_bytes, int sm_count);
+size_t staged_workspace_bytes(Params p, int smem_optin_bytes, int sm_count);
 cudaError_t launch_staged(const Params& p, int tsel, int sm_count, int smem_optin_bytes, cudaStream_t st);
 
 // Every root child's delivery (value, flag, failed-list size): general kernel, workspace slices of candidates_slice_bytes().

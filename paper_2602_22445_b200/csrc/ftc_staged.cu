@@ -13,9 +13,16 @@ cudaError_t launch_staged_u64_max(const Params& p, int sm_count, int smem_optin,
 cudaError_t launch_staged_u64_xor(const Params& p, int sm_count, int smem_optin, cudaStream_t st);
 cudaError_t launch_staged_f32_sum(const Params& p, int sm_count, int smem_optin, cudaStream_t st);
 
-bool staged_supported(Params& p, int smem_optin_bytes) {
+bool staged_supported(Params& p, int smem_optin_bytes, int sm_count) {
     StagedGeom g;
-    return staged_geometry(p, smem_optin_bytes, staged_xl(p), g);
+    return staged_geometry(p, smem_optin_bytes, sm_count, staged_xl(p), g);
+}
+
+size_t staged_workspace_bytes(Params p, int smem_optin_bytes, int sm_count) {
+    StagedGeom g;
+    p.ws_bytes = ~0ull;                       // what would be used if the workspace were there
+    if (!staged_geometry(p, smem_optin_bytes, sm_count, staged_xl(p), g) || !g.hv_global) return 0;
+    return (size_t)sm_count * kHvGlobalBlocksPerSm * (size_t)g.hv_bytes;
 }
 
 cudaError_t launch_staged(const Params& p, int tsel, int sm_count, int smem_optin, cudaStream_t st) {

@@ -52,6 +52,8 @@ struct StagedGeom {
     uint32_t nwarps, nbuf, tile_cap;       // warps per block, buffers per warp, bytes per buffer (multiple of 128)
     uint32_t whole;                        // 1: the whole scenario is staged in one block-wide buffer
     uint32_t off_special, off_rootv, off_hv, off_bar, off_tiles, smem_bytes;
+    uint32_t hv_global;                    // 1: the heap array of tile roots and upper rows lives in the workspace
+    uint64_t hv_bytes;                     // its size per block
 };
 
 // Where a row's bytes sit: at tile-heap position trow of the warp's buffer, or (WHOLE) at their place in the
@@ -271,7 +273,10 @@ __global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThre
     uint32_t* tspec = reinterpret_cast<uint32_t*>(sbase + g.off_special);            // items that need every check
     uint32_t* tmask = tspec + (nitems_words(p.Lt, 5 - p.cw_log2));                     // items with missing group members only
     uint4* rootv = reinterpret_cast<uint4*>(sbase + g.off_rootv);
-    uint4* hv = reinterpret_cast<uint4*>(sbase + g.off_hv);
+    // node values of the tile roots and of the rows above them, heap order: in shared memory, or, when that would
+    // crowd out resident blocks, in this block's slice of the workspace (it stays in L2: written and read once)
+    uint4* hv = g.hv_global ? reinterpret_cast<uint4*>(static_cast<char*>(p.ws) + (size_t)blockIdx.x * g.hv_bytes)
+                            : reinterpret_cast<uint4*>(sbase + g.off_hv);
 
     const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
     const uint32_t cwl = p.cw_log2, lw = 5 - cwl, RW = 1u << lw, Cmask = p.C - 1;
@@ -458,7 +463,12 @@ __global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThre
 }
 
 // ---- host side ----
-static bool staged_geometry(Params& p, int smem_optin, uint32_t XL, StagedGeom& g) {
+// The heap array moves to the workspace when it is at least this large and the workspace has a slice for every block
+// (at most kHvGlobalBlocksPerSm blocks per SM are launched then).
+constexpr size_t kHvGlobalMinBytes = 24 * 1024;
+constexpr int kHvGlobalBlocksPerSm = 4;
+
+static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL, StagedGeom& g) {
     if (p.kbytes % 16) return false;
     const uint32_t C = p.kbytes / 16;
     if (C == 0 || C > 32 || (C & (C - 1))) return false;
@@ -491,7 +501,10 @@ static bool staged_geometry(Params& p, int smem_optin, uint32_t XL, StagedGeom& 
     o = (o + 15) & ~(size_t)15; g.off_special = (uint32_t)o;
     o += (2 * (size_t)nitems_words(p.Lt, lw) * 4 + 15) & ~(size_t)15;
     g.off_rootv = (uint32_t)o; o += (size_t)C * 16;
-    g.off_hv = (uint32_t)o; o += (((size_t)2 << p.Lt) - 1) * C * 16;
+    g.hv_bytes = (((uint64_t)2 << p.Lt) - 1) * C * 16;
+    g.hv_global = (!g.whole && g.hv_bytes >= kHvGlobalMinBytes &&
+                   p.ws_bytes / ((uint64_t)sm_count * kHvGlobalBlocksPerSm) >= g.hv_bytes) ? 1u : 0u;
+    g.off_hv = (uint32_t)o; if (!g.hv_global) o += (size_t)g.hv_bytes;
     g.off_bar = (uint32_t)o; o += (size_t)(kStagedMaxThreads / 32) * 4 * 8 + 8;      // room for any warps x nbuf, plus one
     o = (o + 127) & ~(size_t)127; g.off_tiles = (uint32_t)o;
     if (g.whole) {
@@ -525,6 +538,7 @@ static cudaError_t launch_staged_w(const Params& p, const StagedGeom& g, int sm_
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, staged_kernel<T, OP, XL, WHOLE, MINB>, (int)g.nwarps * 32, g.smem_bytes);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
+    if (g.hv_global && per_sm > kHvGlobalBlocksPerSm) per_sm = kHvGlobalBlocksPerSm;      // one workspace slice per block
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
     staged_kernel<T, OP, XL, WHOLE, MINB><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
@@ -534,7 +548,7 @@ static cudaError_t launch_staged_w(const Params& p, const StagedGeom& g, int sm_
 template <typename T, int OP, int XL>
 static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
     StagedGeom g;
-    if (!staged_geometry(p, smem_optin, XL, g)) return cudaErrorInvalidConfiguration;
+    if (!staged_geometry(p, smem_optin, sm_count, XL, g)) return cudaErrorInvalidConfiguration;
     // one- and two-warp blocks get the lean variant; its register cap (about 96) matches the blocks that fit by shared
     // memory. Scenarios staged whole are so small that many more blocks fit: for them 64 registers, so that the
     // SM's block limit and not the register file decides

@@ -384,3 +384,33 @@ def test_sparse_last_level_failures_roots_and_victims_there(P, f, k, dname, allr
         want = run_oracle(x, f, op, pf, inop, roots, 0, allreduce)
         assert_same(got, want, f"P={P} f={f} k={k} {dname} allreduce={allreduce} flags={flags:#x}")
         assert ((want[1][:, 0] & 0xFF) == 0).sum() > S // 3
+
+
+# ---------------------------------------------------------------------------------------------
+# many processes with wide vectors: the staged kernel's array of tile results moves into the workspace
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("P,f,k,dname,S", [(16384, 5, 16, "u64", 6), (65536, 4, 32, "i32", 2), (1024, 3, 128, "f32", 24),
+                                           (65536, 8, 16, "f32", 2)])
+def test_large_heap_array_in_the_workspace_and_without(P, f, k, dname, S):
+    import torch
+    rng = np.random.Generator(np.random.PCG64(P + k))
+    x = rng.standard_normal((S, P, k)).astype(np.float32) if dname == "f32" else \
+        rng.integers(np.iinfo(DT[dname]).min, np.iinfo(DT[dname]).max, size=(S, P, k), dtype=DT[dname])
+    pf = sc.picks_to_masks(sc.random_subsets(rng, S, P, rng.integers(0, f + 1, size=S)), P)
+    roots = rng.integers(0, P, size=S).astype(np.uint32)
+    op = "sum" if dname in ("f32", "u64") else "max"
+    want = run_oracle(x, f, op, pf, None, roots, 0, True)
+    desc = B.make_desc(P, f, k, B.dtype_code(np.dtype(DT[dname])), op, root=-1)
+    assert B.ftc_kernel_name(desc, True) == "staged" and B.ftc_workspace_bytes(desc, S, True) > 0
+    got = run_gpu(x, f, op, pf, None, roots, 0, True)                   # with the workspace the library asks for
+    assert_same(got, want, f"P={P} k={k} {dname} with workspace")
+    # without a workspace the shape still runs (array in shared memory, or another kernel) unless only the general
+    # kernel is left, which reports the missing workspace
+    d_x, d_out = to_dev(x), torch.zeros((S, k), dtype=to_dev(x).dtype, device="cuda")
+    d_st = torch.zeros((S, 4), dtype=torch.int32, device="cuda")
+    rc = B.ftc_allreduce_batch(desc, S, d_x, to_dev(pf), None, to_dev(roots), d_out, d_st.view(torch.uint32), None, check=False)
+    torch.cuda.synchronize()
+    if rc == B.FTC_OK:
+        assert_same((to_host(d_out, x.dtype), d_st.cpu().numpy().view(np.uint32)), want, f"P={P} k={k} {dname} without workspace")
+    else:
+        assert rc == B.FTC_EWORKSPACE
