@@ -490,8 +490,11 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
     // Launch shape, from sweeps on B200: what limits the kernel is the number of resident warps doing the combine
     // work, and shared memory per warp decides that number. So: one buffer per warp, and blocks just large enough
     // to give every warp at least 16 work items per scenario (at most 8 warps).
+    // Vectors of 256 and 512 bytes leave one or two lane rows, so their tiles are small sub-heaps and their work items
+    // many and short: there 8 items per warp and at most 4 warps did better in the sweeps.
+    const uint32_t per_warp = C >= 16 ? 8u : 16u, max_warps = C >= 16 ? 4u : 8u;
     uint32_t warps = 1;
-    while (warps < 8 && warps * 2 * 16 <= nitems) warps *= 2;
+    while (warps < max_warps && warps * 2 * per_warp <= nitems) warps *= 2;
     uint32_t nbuf = 1;
     // tiny scenarios (up to 16 KB) are staged whole with one copy, larger ones tile by tile
     const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
@@ -521,12 +524,13 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
 
 static uint32_t staged_xl(const Params& p) {
     uint32_t xl;
-    // deepest lane-local sub-heap that keeps a tile (all its levels, every member) within 12 KB
+    // deepest lane-local sub-heap that keeps a tile (all its levels, every member) within 12 KB; 20 KB for vectors of
+    // 256 and 512 bytes, whose tiles would otherwise be three rows
     if (p.kbytes % 16 || p.kbytes > 512) return 1;
     uint32_t C = p.kbytes / 16, cwl = 0; while ((1u << cwl) < C) ++cwl;
-    const uint32_t lw = 5 - cwl;
+    const uint32_t lw = 5 - cwl, budget = (C >= 16 ? 20u : 12u) * 1024u;
     for (xl = 3; xl > 1; --xl)
-        if ((((uint64_t)1 << (lw + xl)) - 1) * p.m * p.kbytes <= 12 * 1024) break;
+        if ((((uint64_t)1 << (lw + xl)) - 1) * p.m * p.kbytes <= budget) break;
     return xl;
 }
 
