@@ -175,7 +175,7 @@ struct SubComb {
 // short group and is complete down to its second-to-last level. `masked`: some group of the tile misses a member.
 template <typename T, int OP, int XL, bool WHOLE>
 __device__ __forceinline__ void fold_tile_fast(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc, const char* in_lc,
-                                               const char* buf_lc, uint32_t rowbytes, uint32_t j0, uint32_t lr, uint32_t rowB, bool hasB,
+                                               const char* buf_lc, uint32_t rowbytes, uint32_t j0, uint32_t lr, uint32_t rot, uint32_t rowB, bool hasB,
                                                uint32_t tA, uint32_t rowA, uint32_t G, bool masked, uint4& valA, uint4& valB) {
     constexpr int NS = 1 << XL;
     const LdShared lds{};
@@ -192,9 +192,9 @@ __device__ __forceinline__ void fold_tile_fast(const Params& p, uint32_t root, u
     }
     uint4 acc[NS];
     if (!Ordered<T>::value && !masked) {
-        // Any member order gives the same bits. When a group's bytes are a multiple of 128, the rows of different
-        // lane rows start in the same shared-memory bank: each lane row then starts at another member.
-        uint32_t mem = (rowbytes & 127u) ? 0u : lr % p.m;
+        // Any member order gives the same bits: each lane row starts at member `rot`, chosen so that the lane rows
+        // that load together (a quarter warp) read from different shared-memory banks.
+        uint32_t mem = rot;
         const char* src = buf_lc + mem * p.kbytes;
 #pragma unroll
         for (int s = 0; s < NS; ++s) acc[s] = lds(src + off[s]);
@@ -282,6 +282,11 @@ __global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThre
     const uint32_t cwl = p.cw_log2, lw = 5 - cwl, RW = 1u << lw, Cmask = p.C - 1;
     const uint32_t lr = lane >> cwl, lc = lane & Cmask;
     const uint32_t D = lw + XL;                                   // levels of a tile
+    // Starting member of this lane row's folds for the exactly associative operations. A quarter warp holds
+    // nq = 8/C lane rows whose rows start m*C chunks apart; with g = gcd(m, nq), rows nq/g apart share their banks,
+    // and g different starting members (all < m) separate them.
+    const uint32_t nq = p.C < 8 ? 8u / p.C : 1u, gq = min(nq, p.m & (0u - p.m));
+    const uint32_t rot = (lr >> ilog2u(nq / gq)) & (gq - 1);
     const uint32_t Lt = p.Lt, ntiles = 1u << Lt, ntop = ntiles - 1, ngroups = (ntop + RW - 1) >> lw;
     const uint32_t nitems = ntiles + ngroups + 1;
     const uint32_t rowbytes = p.m * p.kbytes;
@@ -387,7 +392,7 @@ __global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThre
                     if (!careful) {
                         uint4 valA, valB;
                         const bool hasB = lr < RW - 1;
-                        fold_tile_fast<T, OP, XL, WHOLE>(p, root, sstar, inc, in_lc, buf_lc, rowbytes, j0, lr, rowB, hasB, tA, rowA, G, masked, valA, valB);
+                        fold_tile_fast<T, OP, XL, WHOLE>(p, root, sstar, inc, in_lc, buf_lc, rowbytes, j0, lr, rot, rowB, hasB, tA, rowA, G, masked, valA, valB);
                         valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                         if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                     } else if (j0 < G) {
