@@ -471,6 +471,7 @@ __global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThre
 // The heap array moves to the workspace when it is at least this large and the workspace has a slice for every block
 // (at most kHvGlobalBlocksPerSm blocks per SM are launched then).
 constexpr size_t kHvGlobalMinBytes = 24 * 1024;
+constexpr size_t kHvGlobalMaxBytes = 512 * 1024;   // beyond this the slices of all blocks no longer stay in L2
 constexpr int kHvGlobalBlocksPerSm = 4;
 
 static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL, StagedGeom& g) {
@@ -510,7 +511,7 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
     o += (2 * (size_t)nitems_words(p.Lt, lw) * 4 + 15) & ~(size_t)15;
     g.off_rootv = (uint32_t)o; o += (size_t)C * 16;
     g.hv_bytes = (((uint64_t)2 << p.Lt) - 1) * C * 16;
-    g.hv_global = (!g.whole && g.hv_bytes >= kHvGlobalMinBytes &&
+    g.hv_global = (!g.whole && g.hv_bytes >= kHvGlobalMinBytes && g.hv_bytes <= kHvGlobalMaxBytes &&
                    p.ws_bytes / ((uint64_t)sm_count * kHvGlobalBlocksPerSm) >= g.hv_bytes) ? 1u : 0u;
     g.off_hv = (uint32_t)o; if (!g.hv_global) o += (size_t)g.hv_bytes;
     g.off_bar = (uint32_t)o; o += (size_t)(kStagedMaxThreads / 32) * 4 * 8 + 8;      // room for any warps x nbuf, plus one
