@@ -260,10 +260,12 @@ struct SubHeap {
 constexpr int kStagedMaxThreads = 256;
 constexpr int kStagedLeanThreads = 64;      // lean variant: at most two warps, about 96 registers a thread
 constexpr int kStagedLeanMinBlocks = 10;
+constexpr int kStagedBatchedTag = 3;         // large blocks running the lean variant's code (small groups, exact operations)
 
 template <typename T, int OP, int XL, bool WHOLE, int MINB>
-__global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThreads : kStagedMaxThreads, MINB) staged_kernel(Params p, StagedGeom g) {
-    constexpr bool LEAN = MINB == kStagedLeanMinBlocks;
+__global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThreads : kStagedMaxThreads,
+                                  MINB == kStagedBatchedTag ? 2 : MINB) staged_kernel(Params p, StagedGeom g) {
+    constexpr bool LEAN = MINB == kStagedLeanMinBlocks || MINB == kStagedBatchedTag;
     extern __shared__ __align__(128) uint32_t smem[];
     char* sbase = reinterpret_cast<char*>(smem);
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
@@ -564,7 +566,14 @@ static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaS
     // SM's block limit and not the register file decides
     const bool lean = g.nwarps <= 2;
     if (g.whole) return lean ? launch_staged_w<T, OP, XL, true, 4>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, true, 2>(p, g, sm_count, st);
-    return lean ? launch_staged_w<T, OP, XL, false, kStagedLeanMinBlocks>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
+    if (lean) return launch_staged_w<T, OP, XL, false, kStagedLeanMinBlocks>(p, g, sm_count, st);
+    // Groups of at most 128 bytes: a row is so little data that the instructions around it count, so large blocks
+    // run the lean variant's code too (rows of a lane folded together, starting members rotated). Not for float32:
+    // its bank conflicts weigh more there than the saved instructions.
+    if constexpr (!Ordered<T>::value) {
+        if ((uint64_t)p.m * p.kbytes <= 128) return launch_staged_w<T, OP, XL, false, kStagedBatchedTag>(p, g, sm_count, st);
+    }
+    return launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
 }
 
 template <typename T, int OP>
