@@ -10,6 +10,7 @@
 // shuffles. Groups that are not "plain" (a missing member, a renumbered slot, the short last group) are folded
 // from global memory by the general routine; they are a handful per scenario.
 #pragma once
+#include <cuda.h>
 #include "ftc_tile_common.cuh"
 #include "ftc_kernels.h"
 
@@ -63,10 +64,25 @@ __device__ __forceinline__ uint32_t staged_row_offset(const Params& p, uint32_t 
     return WHOLE ? (grow * p.m + 1) * p.kbytes : trow * rowbytes;
 }
 
+// 16 bytes of a staged row. SW: the tile came in by tiled tensor copies with the 128-byte swizzle, which exchanges
+// the 16-byte chunks within each 128 bytes by the line number (bits 7-9 of the shared-memory address XORed into
+// bits 4-6); rows of different lane rows, 128 bytes or a multiple apart, then sit in different banks.
+template <bool SW>
+struct LdStaged {
+    __device__ __forceinline__ uint4 operator()(const char* q) const {
+        if (SW) {
+            uint32_t a = smem_addr(q);
+            a ^= (a >> 3) & 0x70u;
+            return *reinterpret_cast<const uint4*>(__cvta_shared_to_generic(a));
+        }
+        return *reinterpret_cast<const uint4*>(q);
+    }
+};
+
 // Fold of a plain group from its staged copy.
-template <typename T, int OP>
+template <typename T, int OP, bool SW = false>
 __device__ __forceinline__ uint4 fold_plain_staged(const Params& p, uint32_t sstar, const char* srow_lc) {
-    return fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdShared());
+    return fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdStaged<SW>());
 }
 
 // Fold of one group on the careful path: a full group without a renumbered slot comes from its staged copy
@@ -116,31 +132,31 @@ struct SubHeapPlain {
 // Fold of one group by every rule: a full group without a renumbered slot comes from its staged copy (`srow_lc`,
 // NULL when the row is not in the buffer) under its arrival mask; the others by the general routine from the
 // scenario in process order (`in_lc`: global memory, or the block-wide shared copy when WHOLE).
-template <typename T, int OP, bool WHOLE>
+template <typename T, int OP, bool WHOLE, bool SW = false>
 __device__ __noinline__ uint4 fold_staged_call(FoldShape fs, uint32_t root, uint32_t sstar, const uint32_t* inc,
                                                const char* in_lc, const char* srow_lc, uint32_t row) {
     const uint32_t vbase = row * fs.m + 1;
     if (srow_lc && row < fs.q && root - vbase >= fs.m)      // full group, no renumbered slot in it: its staged copy serves
-        return fold16_masked<T, OP>(srow_lc, fs.kbytes, fs.m, extract_bits(inc, vbase, fs.m), sstar, LdShared());
+        return fold16_masked<T, OP>(srow_lc, fs.kbytes, fs.m, extract_bits(inc, vbase, fs.m), sstar, LdStaged<SW>());
     if (WHOLE) return fold16_general<T, OP, 0, LdShared, FoldShape>(fs, root, sstar, inc, in_lc, row);
     return fold16_general<T, OP, 0, LdGlobal, FoldShape>(fs, root, sstar, inc, in_lc, row);
 }
 
 // A full group some of whose members' messages are missing, from its staged copy.
-template <typename T, int OP>
+template <typename T, int OP, bool SW = false>
 __device__ __noinline__ uint4 fold_masked_call(const char* srow_lc, uint32_t kbytes, uint32_t m, uint32_t mask, uint32_t sstar) {
-    return fold16_masked<T, OP>(srow_lc, kbytes, m, mask, sstar, LdShared());
+    return fold16_masked<T, OP>(srow_lc, kbytes, m, mask, sstar, LdStaged<SW>());
 }
 
 // One row from its staged copy; `masked`: the work item holds a group with a missing member, so look at the mask.
-template <typename T, int OP>
+template <typename T, int OP, bool SW = false>
 __device__ __forceinline__ uint4 fold_row_lean(const Params& p, uint32_t sstar, const uint32_t* inc, const char* srow_lc,
                                                uint32_t grow, bool masked) {
     if (masked) {
         const uint32_t mask = extract_bits(inc, grow * p.m + 1, p.m), full = p.m >= 32 ? 0xFFFFFFFFu : (1u << p.m) - 1u;
-        if (mask != full) return fold_masked_call<T, OP>(srow_lc, p.kbytes, p.m, mask, sstar);
+        if (mask != full) return fold_masked_call<T, OP, SW>(srow_lc, p.kbytes, p.m, mask, sstar);
     }
-    return fold_plain_staged<T, OP>(p, sstar, srow_lc);
+    return fold_plain_staged<T, OP, SW>(p, sstar, srow_lc);
 }
 
 __host__ __device__ constexpr int clog2(int v) { return v <= 1 ? 0 : 1 + clog2(v >> 1); }
@@ -173,12 +189,12 @@ struct SubComb {
 // of the selected subtree's member first, then the partners ascending: Algorithm "Up-correction"), so that the
 // loads and adds of different rows overlap; then the sub-heap is combined. The tile has no renumbered slot, no
 // short group and is complete down to its second-to-last level. `masked`: some group of the tile misses a member.
-template <typename T, int OP, int XL, bool WHOLE>
+template <typename T, int OP, int XL, bool WHOLE, bool SW = false>
 __device__ __forceinline__ void fold_tile_fast(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc, const char* in_lc,
                                                const char* buf_lc, uint32_t rowbytes, uint32_t j0, uint32_t lr, uint32_t rot, uint32_t rowB, bool hasB,
                                                uint32_t tA, uint32_t rowA, uint32_t G, bool masked, uint4& valA, uint4& valB) {
     constexpr int NS = 1 << XL;
-    const LdShared lds{};
+    const LdStaged<SW> lds{};
     uint32_t off[NS], grow[NS];
     const uint32_t off0 = staged_row_offset<WHOLE>(p, rowbytes, 0, j0);        // the tile's root: always there
     grow[0] = hasB ? rowB : j0;
@@ -238,20 +254,20 @@ __device__ __forceinline__ void fold_tile_fast(const Params& p, uint32_t root, u
 // trow/grow: tile-heap index and global row of the node. Its bytes sit at tile-heap position trow of the warp's
 // buffer, or (WHOLE) at their place in the block-wide copy of the scenario.
 // CALL: the fold is a function call (lean variant) instead of inline code.
-template <typename T, int OP, int XL, int U, bool WHOLE, bool CALL = false>
+template <typename T, int OP, int XL, int U, bool WHOLE, bool CALL = false, bool SW = false>
 struct SubHeap {
     static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc,
                                                  const char* in_lc, const char* buf_lc, uint32_t rowbytes,
                                                  uint32_t trow, uint32_t grow, uint32_t G) {
         // the deepest level of this recursion lies below the tile: its rows are not in the warp's buffer
         const char* srow = (WHOLE || U + 1 < XL) ? buf_lc + staged_row_offset<WHOLE>(p, rowbytes, trow, grow) : nullptr;
-        uint4 v = CALL ? fold_staged_call<T, OP, WHOLE>(fold_shape(p), root, sstar, inc, in_lc, srow, grow)
+        uint4 v = CALL ? fold_staged_call<T, OP, WHOLE, SW>(fold_shape(p), root, sstar, inc, in_lc, srow, grow)
                        : fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, grow);
         if (U + 1 < XL) {
             if (2 * grow + 1 < G)
-                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE, CALL>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
+                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE, CALL, SW>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
             if (2 * grow + 2 < G)
-                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE, CALL>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
+                v = comb16<T, OP>(v, SubHeap<T, OP, XL, (U + 1 < XL ? U + 1 : U), WHOLE, CALL, SW>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
         }
         return v;
     }
@@ -261,11 +277,18 @@ constexpr int kStagedMaxThreads = 256;
 constexpr int kStagedLeanThreads = 64;      // lean variant: at most two warps, about 96 registers a thread
 constexpr int kStagedLeanMinBlocks = 10;
 constexpr int kStagedBatchedTag = 3;         // large blocks running the lean variant's code (small groups, exact operations)
+constexpr int kStagedLeanSwzTag = 11;        // lean variant fed by swizzled tensor copies (float32, small vectors)
+constexpr int kStagedBatchedSwzTag = 5;      // the same in large blocks
+
+// Tensor maps of the swizzled variant: one per tile level (its box is that level's rows); unused otherwise.
+struct alignas(64) TmaMaps { CUtensorMap lvl[8]; };
 
 template <typename T, int OP, int XL, bool WHOLE, int MINB>
-__global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThreads : kStagedMaxThreads,
-                                  MINB == kStagedBatchedTag ? 2 : MINB) staged_kernel(Params p, StagedGeom g) {
-    constexpr bool LEAN = MINB == kStagedLeanMinBlocks || MINB == kStagedBatchedTag;
+__global__ void __launch_bounds__((MINB == kStagedLeanMinBlocks || MINB == kStagedLeanSwzTag) ? kStagedLeanThreads : kStagedMaxThreads,
+                                  (MINB == kStagedBatchedTag || MINB == kStagedBatchedSwzTag) ? 2 : (MINB == kStagedLeanSwzTag ? kStagedLeanMinBlocks : MINB))
+staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
+    constexpr bool SWZ = MINB == kStagedLeanSwzTag || MINB == kStagedBatchedSwzTag;
+    constexpr bool LEAN = MINB == kStagedLeanMinBlocks || MINB == kStagedBatchedTag || SWZ;
     extern __shared__ __align__(128) uint32_t smem[];
     char* sbase = reinterpret_cast<char*>(smem);
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
@@ -323,7 +346,28 @@ __global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThre
             const uint32_t j0 = ntop + it;
             if (j0 < p.Gmax) { first_row = ((j0 + 1) << lane) - 1; nrows = lvl_rows; dst_off = lvl_dst; }
         } else if (it < ntiles + ngroups) {
-            if (lane == 0) { first_row = (it - ntiles) << lw; nrows = min(RW, ntop - first_row); }
+            if (lane == 0) { first_row = (it - ntiles) << lw; nrows = SWZ ? RW : min(RW, ntop - first_row); }
+        }
+        if (SWZ) {
+            // Tiled tensor copies over the view [scenario][128-byte line][32 words] of the full groups: lane t brings
+            // level t with the map whose box is 2^t rows (rows above the tiles: the map of 2^lw rows). A box always
+            // delivers its full byte count; lines past the last full group arrive as zeros and are never read.
+            const uint32_t bytes = (nrows && first_row < p.q) ? nrows * rowbytes : 0u;
+            const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, bytes);
+            if (total) {
+                if (lane == 0) mbar_expect_tx(bar0 + b * 8, total);
+                __syncwarp();
+                if (bytes) {
+                    const CUtensorMap* map = &maps.lvl[it < ntiles ? lane : lw];
+                    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                                 ::"r"(smem_addr(tiles + (size_t)b * g.tile_cap + dst_off)), "l"(map), "r"(0),
+                                   "r"((int)(first_row * (rowbytes >> 7))), "r"((int)is_s), "r"(bar0 + b * 8) : "memory");
+                }
+                pending |= 1u << b;
+            }
+            if (++ibuf == g.nbuf) ibuf = 0;
+            if (++is_i == n_my) { is_i = 0; is_s += gridDim.x; is_src += (uint64_t)gridDim.x * scen_bytes; }
+            return;
         }
         // rows first_row .. first_row+nrows-1 are bytes [first_row*rowbytes + kbytes, ...) of the scenario, cut at its end
         const uint64_t b0 = (uint64_t)first_row * rowbytes + p.kbytes;
@@ -394,14 +438,14 @@ __global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThre
                     if (!careful) {
                         uint4 valA, valB;
                         const bool hasB = lr < RW - 1;
-                        fold_tile_fast<T, OP, XL, WHOLE>(p, root, sstar, inc, in_lc, buf_lc, rowbytes, j0, lr, rot, rowB, hasB, tA, rowA, G, masked, valA, valB);
+                        fold_tile_fast<T, OP, XL, WHOLE, SWZ>(p, root, sstar, inc, in_lc, buf_lc, rowbytes, j0, lr, rot, rowB, hasB, tA, rowA, G, masked, valA, valB);
                         valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                         if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                     } else if (j0 < G) {
                         uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
-                        if (rowA < G) valA = SubHeap<T, OP, XL + 1, 0, WHOLE, true>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, tA, rowA, G);
+                        if (rowA < G) valA = SubHeap<T, OP, XL + 1, 0, WHOLE, true, SWZ>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, tA, rowA, G);
                         const bool hasB = lr < RW - 1 && rowB < G;
-                        if (hasB) valB = fold_staged_call<T, OP, WHOLE>(fold_shape(p), root, sstar, inc, in_lc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB), rowB);
+                        if (hasB) valB = fold_staged_call<T, OP, WHOLE, SWZ>(fold_shape(p), root, sstar, inc, in_lc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB), rowB);
                         valB = tile_tree_phase<T, OP>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                         if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                     }
@@ -433,8 +477,8 @@ __global__ void __launch_bounds__(MINB == kStagedLeanMinBlocks ? kStagedLeanThre
                 const uint32_t row = ((it - ntiles) << lw) + lr;
                 const char* srow = buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, row);
                 if (LEAN) {
-                    if (!careful) hv[(size_t)row * p.C + lc] = fold_row_lean<T, OP>(p, sstar, inc, srow, row, masked);
-                    else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged_call<T, OP, WHOLE>(fold_shape(p), root, sstar, inc, in_lc, srow, row);
+                    if (!careful) hv[(size_t)row * p.C + lc] = fold_row_lean<T, OP, SWZ>(p, sstar, inc, srow, row, masked);
+                    else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged_call<T, OP, WHOLE, SWZ>(fold_shape(p), root, sstar, inc, in_lc, srow, row);
                 } else if (!careful && !masked) hv[(size_t)row * p.C + lc] = fold_plain_staged<T, OP>(p, sstar, srow);
                 else if (!careful) hv[(size_t)row * p.C + lc] = fold_fast_staged<T, OP, true>(p, sstar, inc, srow, row);
                 else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, row);
@@ -542,8 +586,13 @@ static uint32_t staged_xl(const Params& p) {
     return xl;
 }
 
+static const TmaMaps kNoMaps = {};
+
+// Tensor maps for the swizzled variant (host side, below).
+static bool staged_tensor_maps(const Params& p, uint32_t D, TmaMaps& maps);
+
 template <typename T, int OP, int XL, bool WHOLE, int MINB>
-static cudaError_t launch_staged_w(const Params& p, const StagedGeom& g, int sm_count, cudaStream_t st) {
+static cudaError_t launch_staged_w(const Params& p, const StagedGeom& g, int sm_count, cudaStream_t st, const TmaMaps& maps = kNoMaps) {
     cudaError_t e = cudaFuncSetAttribute(staged_kernel<T, OP, XL, WHOLE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
@@ -553,7 +602,7 @@ static cudaError_t launch_staged_w(const Params& p, const StagedGeom& g, int sm_
     if (g.hv_global && per_sm > kHvGlobalBlocksPerSm) per_sm = kHvGlobalBlocksPerSm;      // one workspace slice per block
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
-    staged_kernel<T, OP, XL, WHOLE, MINB><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
+    staged_kernel<T, OP, XL, WHOLE, MINB><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g, maps);
     return cudaGetLastError();
 }
 
@@ -566,6 +615,16 @@ static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaS
     // SM's block limit and not the register file decides
     const bool lean = g.nwarps <= 2;
     if (g.whole) return lean ? launch_staged_w<T, OP, XL, true, 4>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, true, 2>(p, g, sm_count, st);
+    // float32 with vectors of 16 or 32 bytes in groups of a multiple of 128 bytes: the fold order is fixed, so the
+    // rows of different lane rows would meet in the same banks (4- and 8-way conflicts); their tiles come in by
+    // tensor copies with the 128-byte swizzle instead
+    if constexpr (Ordered<T>::value) {
+        const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
+        TmaMaps maps;
+        if (p.C <= 2 && rowbytes % 128 == 0 && p.S < (1ull << 31) && staged_tensor_maps(p, (5 - p.cw_log2) + XL, maps))
+            return lean ? launch_staged_w<T, OP, XL, false, kStagedLeanSwzTag>(p, g, sm_count, st, maps)
+                        : launch_staged_w<T, OP, XL, false, kStagedBatchedSwzTag>(p, g, sm_count, st, maps);
+    }
     if (lean) return launch_staged_w<T, OP, XL, false, kStagedLeanMinBlocks>(p, g, sm_count, st);
     // Groups of at most 128 bytes: a row is so little data that the instructions around it count, so large blocks
     // run the lean variant's code too (rows of a lane folded together, starting members rotated). Not for float32:
@@ -574,6 +633,37 @@ static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaS
         if ((uint64_t)p.m * p.kbytes <= 128) return launch_staged_w<T, OP, XL, false, kStagedBatchedTag>(p, g, sm_count, st);
     }
     return launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
+}
+
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                      const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The scenario batch as a tensor [S][lines][32 x u32]: line = 128 bytes, counted from the first group of each scenario
+// (process 1), full groups only; consecutive scenarios lie P*k*e bytes apart. Map t has a box of 2^t rows. Returns
+// false when the driver entry point is missing or a map cannot be encoded (the caller then takes the untiled copies).
+static bool staged_tensor_maps(const Params& p, uint32_t D, TmaMaps& maps) {
+    static TensorMapEncodeFn encode = [] {
+        void* fn = nullptr; cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) fn = nullptr;
+        return reinterpret_cast<TensorMapEncodeFn>(fn);
+    }();
+    const uint64_t rowbytes = (uint64_t)p.m * p.kbytes, lines_per_row = rowbytes / 128, scen_bytes = (uint64_t)p.P * p.kbytes;
+    if (!encode || D > 8 || p.q == 0 || scen_bytes % 16) return false;
+    void* base = const_cast<char*>(static_cast<const char*>(p.in)) + p.kbytes;
+    const cuuint64_t dims[3] = {32, (cuuint64_t)p.q * lines_per_row, (cuuint64_t)p.S};
+    const cuuint64_t strides[2] = {128, scen_bytes};
+    const cuuint32_t elem_strides[3] = {1, 1, 1};
+    for (uint32_t t = 0; t < D; ++t) {
+        const uint64_t box_lines = lines_per_row << t;
+        if (box_lines > 256) return false;
+        const cuuint32_t box[3] = {32, (cuuint32_t)box_lines, 1};
+        if (encode(&maps.lvl[t], CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, base, dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return false;
+    }
+    for (uint32_t t = D; t < 8; ++t) maps.lvl[t] = maps.lvl[0];
+    return true;
 }
 
 template <typename T, int OP>

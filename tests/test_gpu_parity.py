@@ -414,3 +414,29 @@ def test_large_heap_array_in_the_workspace_and_without(P, f, k, dname, S):
         assert_same((to_host(d_out, x.dtype), d_st.cpu().numpy().view(np.uint32)), want, f"P={P} k={k} {dname} without workspace")
     else:
         assert rc == B.FTC_EWORKSPACE
+
+
+# ---------------------------------------------------------------------------------------------
+# float32 vectors of 16 and 32 bytes in groups of a multiple of 128 bytes: tiles arrive by swizzled tensor copies
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("P,f,k,S", [(16384, 3, 8, 6), (8200, 7, 4, 10), (1030, 3, 8, 40), (20000, 15, 4, 4), (4099, 1, 16, 12)])
+@pytest.mark.parametrize("allreduce", [False, True])
+def test_float32_small_vectors_swizzled_tiles(P, f, k, S, allreduce):
+    rng = np.random.Generator(np.random.PCG64(3 * P + k))
+    x = rng.standard_normal((S, P, k)).astype(np.float32)
+    pf = sc.picks_to_masks(sc.random_subsets(rng, S, P, rng.integers(0, f + 2, size=S)), P)
+    pf[0] = 0                                                        # one failure-free scenario
+    R = O.schedule(P, f)["rounds_attempt"]
+    inop = np.full((S, 2, 2), sc.UNUSED, dtype=np.uint32)
+    roots = rng.integers(0, P, size=S).astype(np.uint32)
+    roots[1 % S] = P - 1                                             # root in the last (short or full) group
+    for i in range(S):
+        for j in range(2):
+            if rng.random() < 0.5:
+                v = int(rng.integers(0, P))
+                if allreduce and (v - int(roots[i])) % P <= f:
+                    continue
+                inop[i, j] = (v, int(rng.integers(0, R + 2)))
+    got = run_gpu(x, f, "sum", pf, inop, roots, 0, allreduce)
+    assert B.ftc_kernel_name(got[2], allreduce) == "staged"
+    assert_same(got, run_oracle(x, f, "sum", pf, inop, roots, 0, allreduce), f"P={P} f={f} k={k} allreduce={allreduce}")
