@@ -31,6 +31,8 @@ struct Params {
     uint32_t C;        // 16-byte chunks per process vector
     uint32_t cw_log2;  // log2 of lanes along the chunk dimension (= log2 C)
     uint32_t Lt;       // heap level at which the warp tiles are rooted; levels above go through shared memory
+    uint32_t swz_mask; // swizzled tiles: XOR mask of the 16-byte chunk bits (0x70: 128-byte lines, 0x30: 64-byte lines)
+    uint32_t row_shift; // swizzled tiles of 64-byte groups: tile rows after the first sit one row further (128-byte aligned levels)
     uint32_t below;    // 1: the heap's sparsely filled last level lies below the tiles (its rows are folded one by one)
 };
 

@@ -59,20 +59,25 @@ struct StagedGeom {
 
 // Where a row's bytes sit: at tile-heap position trow of the warp's buffer, or (WHOLE) at their place in the
 // block-wide copy of the scenario (grow = global row).
-template <bool WHOLE>
+// SW (swizzled tiles): with 64-byte groups every tile row but the first sits one row further, so that each level
+// starts on a 128-byte boundary (tensor copies need that); p.row_shift is 0 otherwise.
+template <bool WHOLE, bool SW = false>
 __device__ __forceinline__ uint32_t staged_row_offset(const Params& p, uint32_t rowbytes, uint32_t trow, uint32_t grow) {
-    return WHOLE ? (grow * p.m + 1) * p.kbytes : trow * rowbytes;
+    if (WHOLE) return (grow * p.m + 1) * p.kbytes;
+    return SW ? (trow + (trow ? p.row_shift : 0u)) * rowbytes : trow * rowbytes;
 }
 
 // 16 bytes of a staged row. SW: the tile came in by tiled tensor copies with the 128-byte swizzle, which exchanges
-// the 16-byte chunks within each 128 bytes by the line number (bits 7-9 of the shared-memory address XORed into
-// bits 4-6); rows of different lane rows, 128 bytes or a multiple apart, then sit in different banks.
+// the 16-byte chunks within each line by the line number (128-byte lines: bits 7-9 of the shared-memory address
+// XORed into bits 4-6; 64-byte lines: bits 7-8 into bits 4-5); rows of different lane rows, 128 bytes or a multiple apart, then sit in different banks.
 template <bool SW>
 struct LdStaged {
+    uint32_t mask;        // 0x70 for 128-byte lines, 0x30 for 64-byte lines
+    __device__ __forceinline__ explicit LdStaged(uint32_t m) : mask(m) {}
     __device__ __forceinline__ uint4 operator()(const char* q) const {
         if (SW) {
             uint32_t a = smem_addr(q);
-            a ^= (a >> 3) & 0x70u;
+            a ^= (a >> 3) & mask;
             return *reinterpret_cast<const uint4*>(__cvta_shared_to_generic(a));
         }
         return *reinterpret_cast<const uint4*>(q);
@@ -82,7 +87,7 @@ struct LdStaged {
 // Fold of a plain group from its staged copy.
 template <typename T, int OP, bool SW = false>
 __device__ __forceinline__ uint4 fold_plain_staged(const Params& p, uint32_t sstar, const char* srow_lc) {
-    return fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdStaged<SW>());
+    return fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdStaged<SW>(p.swz_mask));
 }
 
 // Fold of one group on the careful path: a full group without a renumbered slot comes from its staged copy
@@ -137,15 +142,15 @@ __device__ __noinline__ uint4 fold_staged_call(FoldShape fs, uint32_t root, uint
                                                const char* in_lc, const char* srow_lc, uint32_t row) {
     const uint32_t vbase = row * fs.m + 1;
     if (srow_lc && row < fs.q && root - vbase >= fs.m)      // full group, no renumbered slot in it: its staged copy serves
-        return fold16_masked<T, OP>(srow_lc, fs.kbytes, fs.m, extract_bits(inc, vbase, fs.m), sstar, LdStaged<SW>());
+        return fold16_masked<T, OP>(srow_lc, fs.kbytes, fs.m, extract_bits(inc, vbase, fs.m), sstar, LdStaged<SW>(fs.swz_mask));
     if (WHOLE) return fold16_general<T, OP, 0, LdShared, FoldShape>(fs, root, sstar, inc, in_lc, row);
     return fold16_general<T, OP, 0, LdGlobal, FoldShape>(fs, root, sstar, inc, in_lc, row);
 }
 
 // A full group some of whose members' messages are missing, from its staged copy.
 template <typename T, int OP, bool SW = false>
-__device__ __noinline__ uint4 fold_masked_call(const char* srow_lc, uint32_t kbytes, uint32_t m, uint32_t mask, uint32_t sstar) {
-    return fold16_masked<T, OP>(srow_lc, kbytes, m, mask, sstar, LdStaged<SW>());
+__device__ __noinline__ uint4 fold_masked_call(const char* srow_lc, uint32_t kbytes, uint32_t m, uint32_t mask, uint32_t sstar, uint32_t swz_mask) {
+    return fold16_masked<T, OP>(srow_lc, kbytes, m, mask, sstar, LdStaged<SW>(swz_mask));
 }
 
 // One row from its staged copy; `masked`: the work item holds a group with a missing member, so look at the mask.
@@ -154,7 +159,7 @@ __device__ __forceinline__ uint4 fold_row_lean(const Params& p, uint32_t sstar, 
                                                uint32_t grow, bool masked) {
     if (masked) {
         const uint32_t mask = extract_bits(inc, grow * p.m + 1, p.m), full = p.m >= 32 ? 0xFFFFFFFFu : (1u << p.m) - 1u;
-        if (mask != full) return fold_masked_call<T, OP, SW>(srow_lc, p.kbytes, p.m, mask, sstar);
+        if (mask != full) return fold_masked_call<T, OP, SW>(srow_lc, p.kbytes, p.m, mask, sstar, p.swz_mask);
     }
     return fold_plain_staged<T, OP, SW>(p, sstar, srow_lc);
 }
@@ -194,17 +199,17 @@ __device__ __forceinline__ void fold_tile_fast(const Params& p, uint32_t root, u
                                                const char* buf_lc, uint32_t rowbytes, uint32_t j0, uint32_t lr, uint32_t rot, uint32_t rowB, bool hasB,
                                                uint32_t tA, uint32_t rowA, uint32_t G, bool masked, uint4& valA, uint4& valB) {
     constexpr int NS = 1 << XL;
-    const LdStaged<SW> lds{};
+    const LdStaged<SW> lds(p.swz_mask);
     uint32_t off[NS], grow[NS];
-    const uint32_t off0 = staged_row_offset<WHOLE>(p, rowbytes, 0, j0);        // the tile's root: always there
+    const uint32_t off0 = staged_row_offset<WHOLE, SW>(p, rowbytes, 0, j0);        // the tile's root: always there
     grow[0] = hasB ? rowB : j0;
-    off[0] = hasB ? staged_row_offset<WHOLE>(p, rowbytes, lr, rowB) : off0;
+    off[0] = hasB ? staged_row_offset<WHOLE, SW>(p, rowbytes, lr, rowB) : off0;
 #pragma unroll
     for (int b = 0; b < NS - 1; ++b) {
         const int u = clog2(b + 1), pos = b + 1 - (1 << u);
         const uint32_t t = ((tA + 1) << u) - 1 + pos, g = ((rowA + 1) << u) - 1 + pos;
         grow[1 + b] = g;
-        off[1 + b] = g < G ? staged_row_offset<WHOLE>(p, rowbytes, t, g) : off0;   // a missing row reads the root's bytes, unused
+        off[1 + b] = g < G ? staged_row_offset<WHOLE, SW>(p, rowbytes, t, g) : off0;   // a missing row reads the root's bytes, unused
     }
     uint4 acc[NS];
     if (!Ordered<T>::value && !masked) {
@@ -260,7 +265,7 @@ struct SubHeap {
                                                  const char* in_lc, const char* buf_lc, uint32_t rowbytes,
                                                  uint32_t trow, uint32_t grow, uint32_t G) {
         // the deepest level of this recursion lies below the tile: its rows are not in the warp's buffer
-        const char* srow = (WHOLE || U + 1 < XL) ? buf_lc + staged_row_offset<WHOLE>(p, rowbytes, trow, grow) : nullptr;
+        const char* srow = (WHOLE || U + 1 < XL) ? buf_lc + staged_row_offset<WHOLE, SW>(p, rowbytes, trow, grow) : nullptr;
         uint4 v = CALL ? fold_staged_call<T, OP, WHOLE, SW>(fold_shape(p), root, sstar, inc, in_lc, srow, grow)
                        : fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, grow);
         if (U + 1 < XL) {
@@ -359,9 +364,12 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
                 __syncwarp();
                 if (bytes) {
                     const CUtensorMap* map = &maps.lvl[it < ntiles ? lane : lw];
+                    // 64-byte groups: level t >= 1 of a tile starts at row slot 2^t (a 128-byte boundary), one further than usual
+                    if (p.row_shift && it < ntiles && lane) dst_off = rowbytes << lane;
+                    const uint32_t lines_per_row = p.swz_mask == 0x70u ? rowbytes >> 7 : 1u;
                     asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
                                  ::"r"(smem_addr(tiles + (size_t)b * g.tile_cap + dst_off)), "l"(map), "r"(0),
-                                   "r"((int)(first_row * (rowbytes >> 7))), "r"((int)is_s), "r"(bar0 + b * 8) : "memory");
+                                   "r"((int)(first_row * lines_per_row)), "r"((int)is_s), "r"(bar0 + b * 8) : "memory");
                 }
                 pending |= 1u << b;
             }
@@ -445,7 +453,7 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
                         uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
                         if (rowA < G) valA = SubHeap<T, OP, XL + 1, 0, WHOLE, true, SWZ>::eval(p, root, sstar, inc, in_lc, buf_lc, rowbytes, tA, rowA, G);
                         const bool hasB = lr < RW - 1 && rowB < G;
-                        if (hasB) valB = fold_staged_call<T, OP, WHOLE, SWZ>(fold_shape(p), root, sstar, inc, in_lc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB), rowB);
+                        if (hasB) valB = fold_staged_call<T, OP, WHOLE, SWZ>(fold_shape(p), root, sstar, inc, in_lc, buf_lc + staged_row_offset<WHOLE, SWZ>(p, rowbytes, lr, rowB), rowB);
                         valB = tile_tree_phase<T, OP>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                         if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                     }
@@ -535,7 +543,7 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
     p.below = (Heff < Hmax && Heff >= D) ? 1u : 0u;
     if (p.Lt > 16) return false;
     const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
-    const uint64_t cap = ((((uint64_t)1 << D) - 1) * rowbytes + 127) & ~(uint64_t)127;
+    const uint64_t cap = ((((uint64_t)1 << D) - 1 + p.row_shift) * rowbytes + 127) & ~(uint64_t)127;
     if (cap > 64 * 1024) return false;
     const uint32_t RW = 1u << lw, ntiles = 1u << p.Lt;
     const uint32_t nitems = ntiles + ((ntiles - 1 + RW - 1) >> lw) + 1;
@@ -609,21 +617,32 @@ static cudaError_t launch_staged_w(const Params& p, const StagedGeom& g, int sm_
 template <typename T, int OP, int XL>
 static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
     StagedGeom g;
-    if (!staged_geometry(p, smem_optin, sm_count, XL, g)) return cudaErrorInvalidConfiguration;
+    // float32 with vectors of 16 or 32 bytes: the fold order is fixed, so the rows of different lane rows would meet in
+    // the same banks when groups are a multiple of 128 bytes or 64 bytes (4- and 8-way conflicts); their tiles come in
+    // by tensor copies with the matching swizzle instead
+    const uint64_t gbytes = (uint64_t)p.m * p.kbytes;
+    bool swizzled = Ordered<T>::value && p.kbytes <= 32 && (gbytes % 128 == 0 || gbytes == 64) && p.S < (1ull << 31) &&
+                    (uint64_t)p.P * p.kbytes > 16 * 1024;
+    if (swizzled) { p.swz_mask = gbytes == 64 ? 0x30u : 0x70u; p.row_shift = gbytes == 64 ? 1u : 0u; }
+    if (!staged_geometry(p, smem_optin, sm_count, XL, g)) {
+        if (!swizzled) return cudaErrorInvalidConfiguration;
+        swizzled = false; p.swz_mask = 0; p.row_shift = 0;
+        if (!staged_geometry(p, smem_optin, sm_count, XL, g)) return cudaErrorInvalidConfiguration;
+    }
     // one- and two-warp blocks get the lean variant; its register cap (about 96) matches the blocks that fit by shared
     // memory. Scenarios staged whole are so small that many more blocks fit: for them 64 registers, so that the
     // SM's block limit and not the register file decides
     const bool lean = g.nwarps <= 2;
     if (g.whole) return lean ? launch_staged_w<T, OP, XL, true, 4>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, true, 2>(p, g, sm_count, st);
-    // float32 with vectors of 16 or 32 bytes in groups of a multiple of 128 bytes: the fold order is fixed, so the
-    // rows of different lane rows would meet in the same banks (4- and 8-way conflicts); their tiles come in by
-    // tensor copies with the 128-byte swizzle instead
     if constexpr (Ordered<T>::value) {
-        const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
         TmaMaps maps;
-        if (p.C <= 2 && rowbytes % 128 == 0 && p.S < (1ull << 31) && staged_tensor_maps(p, (5 - p.cw_log2) + XL, maps))
+        if (swizzled && !g.whole && staged_tensor_maps(p, (5 - p.cw_log2) + XL, maps))
             return lean ? launch_staged_w<T, OP, XL, false, kStagedLeanSwzTag>(p, g, sm_count, st, maps)
                         : launch_staged_w<T, OP, XL, false, kStagedBatchedSwzTag>(p, g, sm_count, st, maps);
+        if (swizzled) {               // no tensor maps: the plain layout after all
+            p.swz_mask = 0; p.row_shift = 0;
+            if (!staged_geometry(p, smem_optin, sm_count, XL, g)) return cudaErrorInvalidConfiguration;
+        }
     }
     if (lean) return launch_staged_w<T, OP, XL, false, kStagedLeanMinBlocks>(p, g, sm_count, st);
     // Groups of at most 128 bytes: a row is so little data that the instructions around it count, so large blocks
@@ -639,7 +658,7 @@ typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint3
                                       const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                       CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// The scenario batch as a tensor [S][lines][32 x u32]: line = 128 bytes, counted from the first group of each scenario
+// The scenario batch as a tensor [S][lines][line words]: line = 128 bytes (64 for 64-byte groups), counted from the first group of each scenario
 // (process 1), full groups only; consecutive scenarios lie P*k*e bytes apart. Map t has a box of 2^t rows. Returns
 // false when the driver entry point is missing or a map cannot be encoded (the caller then takes the untiled copies).
 static bool staged_tensor_maps(const Params& p, uint32_t D, TmaMaps& maps) {
@@ -648,18 +667,20 @@ static bool staged_tensor_maps(const Params& p, uint32_t D, TmaMaps& maps) {
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) fn = nullptr;
         return reinterpret_cast<TensorMapEncodeFn>(fn);
     }();
-    const uint64_t rowbytes = (uint64_t)p.m * p.kbytes, lines_per_row = rowbytes / 128, scen_bytes = (uint64_t)p.P * p.kbytes;
-    if (!encode || D > 8 || p.q == 0 || scen_bytes % 16) return false;
+    const uint64_t rowbytes = (uint64_t)p.m * p.kbytes, line = p.swz_mask == 0x70u ? 128 : 64;
+    const uint64_t lines_per_row = rowbytes / line, scen_bytes = (uint64_t)p.P * p.kbytes;
+    if (!encode || D > 8 || p.q == 0 || scen_bytes % 16 || rowbytes % line) return false;
     void* base = const_cast<char*>(static_cast<const char*>(p.in)) + p.kbytes;
-    const cuuint64_t dims[3] = {32, (cuuint64_t)p.q * lines_per_row, (cuuint64_t)p.S};
-    const cuuint64_t strides[2] = {128, scen_bytes};
+    const cuuint64_t dims[3] = {line / 4, (cuuint64_t)p.q * lines_per_row, (cuuint64_t)p.S};
+    const cuuint64_t strides[2] = {line, scen_bytes};
     const cuuint32_t elem_strides[3] = {1, 1, 1};
     for (uint32_t t = 0; t < D; ++t) {
         const uint64_t box_lines = lines_per_row << t;
         if (box_lines > 256) return false;
-        const cuuint32_t box[3] = {32, (cuuint32_t)box_lines, 1};
+        const cuuint32_t box[3] = {(cuuint32_t)(line / 4), (cuuint32_t)box_lines, 1};
         if (encode(&maps.lvl[t], CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, base, dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                   line == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return false;
     }
     for (uint32_t t = D; t < 8; ++t) maps.lvl[t] = maps.lvl[0];

@@ -136,8 +136,8 @@ __device__ __forceinline__ bool group_is_plain(const Params& p, uint32_t root, c
 }
 
 // The four numbers the general fold needs, for passing by value.
-struct FoldShape { uint32_t m, q, r, kbytes; };
-__device__ __forceinline__ FoldShape fold_shape(const Params& p) { return FoldShape{p.m, p.q, p.r, p.kbytes}; }
+struct FoldShape { uint32_t m, q, r, kbytes, swz_mask; };
+__device__ __forceinline__ FoldShape fold_shape(const Params& p) { return FoldShape{p.m, p.q, p.r, p.kbytes, p.swz_mask}; }
 
 // Any group, by the general routine (the careful path of the tiled kernels; rare). LD says where `in_lc`, the
 // scenario in process order, lives.

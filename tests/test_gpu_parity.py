@@ -419,7 +419,8 @@ def test_large_heap_array_in_the_workspace_and_without(P, f, k, dname, S):
 # ---------------------------------------------------------------------------------------------
 # float32 vectors of 16 and 32 bytes in groups of a multiple of 128 bytes: tiles arrive by swizzled tensor copies
 # ---------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("P,f,k,S", [(16384, 3, 8, 6), (8200, 7, 4, 10), (1030, 3, 8, 40), (20000, 15, 4, 4), (4099, 1, 16, 12)])
+@pytest.mark.parametrize("P,f,k,S", [(16384, 3, 8, 6), (8200, 7, 4, 10), (1030, 3, 8, 40), (20000, 15, 4, 4), (4099, 1, 16, 12),
+                                     (5000, 3, 4, 12), (20001, 1, 8, 5), (40000, 3, 4, 3), (1500, 3, 4, 30)])   # the last four: 64-byte groups
 @pytest.mark.parametrize("allreduce", [False, True])
 def test_float32_small_vectors_swizzled_tiles(P, f, k, S, allreduce):
     rng = np.random.Generator(np.random.PCG64(3 * P + k))
