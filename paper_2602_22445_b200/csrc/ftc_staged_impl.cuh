@@ -524,6 +524,8 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
 // ---- host side ----
 // The heap array moves to the workspace when it is at least this large and the workspace has a slice for every block
 // (at most kHvGlobalBlocksPerSm blocks per SM are launched then).
+// Scenarios up to this size are staged whole with one copy.
+constexpr uint64_t kWholeMaxBytes = 12 * 1024;
 constexpr size_t kHvGlobalMinBytes = 24 * 1024;
 constexpr size_t kHvGlobalMaxBytes = 512 * 1024;   // beyond this the slices of all blocks no longer stay in L2
 constexpr int kHvGlobalBlocksPerSm = 4;
@@ -556,9 +558,9 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
     uint32_t warps = 1;
     while (warps < max_warps && warps * 2 * per_warp <= nitems) warps *= 2;
     uint32_t nbuf = 1;
-    // tiny scenarios (up to 16 KB) are staged whole with one copy, larger ones tile by tile
+    // tiny scenarios are staged whole with one copy, larger ones tile by tile (at 16 KB the tiles already win)
     const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
-    g.whole = scen_bytes <= 16 * 1024 ? 1u : 0u;
+    g.whole = scen_bytes <= kWholeMaxBytes ? 1u : 0u;
     if (g.whole) nbuf = 0;
     size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
     o = (o + 15) & ~(size_t)15; g.off_special = (uint32_t)o;
@@ -622,7 +624,7 @@ static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaS
     // by tensor copies with the matching swizzle instead
     const uint64_t gbytes = (uint64_t)p.m * p.kbytes;
     bool swizzled = Ordered<T>::value && p.kbytes <= 32 && (gbytes % 128 == 0 || gbytes == 64) && p.S < (1ull << 31) &&
-                    (uint64_t)p.P * p.kbytes > 16 * 1024;
+                    (uint64_t)p.P * p.kbytes > kWholeMaxBytes;
     if (swizzled) { p.swz_mask = gbytes == 64 ? 0x30u : 0x70u; p.row_shift = gbytes == 64 ? 1u : 0u; }
     if (!staged_geometry(p, smem_optin, sm_count, XL, g)) {
         if (!swizzled) return cudaErrorInvalidConfiguration;
