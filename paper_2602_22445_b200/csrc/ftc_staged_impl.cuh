@@ -317,7 +317,11 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
     // and g different starting members (all < m) separate them.
     const uint32_t nq = p.C < 8 ? 8u / p.C : 1u, gq = min(nq, p.m & (0u - p.m));
     const uint32_t rot = (lr >> ilog2u(nq / gq)) & (gq - 1);
-    const uint32_t Lt = p.Lt, ntiles = 1u << Lt, ntop = ntiles - 1, ngroups = (ntop + RW - 1) >> lw;
+    // rows above the tiles come as work items of `grows` rows: as many per lane row as a tile's sub-heap has (one when
+    // the tiles are swizzled: the tensor map of that box is the one of a tile level)
+    const uint32_t Lt = p.Lt, ntiles = 1u << Lt, ntop = ntiles - 1;
+    const uint32_t GR = SWZ ? 1u : min((1u << XL) - 1, max(1u, (ntop + RW - 1) >> lw)), grows = RW * GR;
+    const uint32_t ngroups = (ntop + grows - 1) / grows;
     const uint32_t nitems = ntiles + ngroups + 1;
     const uint32_t rowbytes = p.m * p.kbytes;
     const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
@@ -351,7 +355,7 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
             const uint32_t j0 = ntop + it;
             if (j0 < p.Gmax) { first_row = ((j0 + 1) << lane) - 1; nrows = lvl_rows; dst_off = lvl_dst; }
         } else if (it < ntiles + ngroups) {
-            if (lane == 0) { first_row = (it - ntiles) << lw; nrows = SWZ ? RW : min(RW, ntop - first_row); }
+            if (lane == 0) { first_row = (it - ntiles) * grows; nrows = SWZ ? RW : min(grows, ntop - first_row); }
         }
         if (SWZ) {
             // Tiled tensor copies over the view [scenario][128-byte line][32 words] of the full groups: lane t brings
@@ -428,7 +432,7 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
             continue;
         }
         if (p.is_allreduce) count_holders(p, cx, pf, unr);
-        mark_special_items(p, cx, pf, tspec, tmask, Lt, lw, D, LEAN && p.below != 0);
+        mark_special_items(p, cx, pf, tspec, tmask, Lt, lw, D, LEAN && p.below != 0, grows, ngroups);
         const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
         const char* in_lc = (WHOLE ? wbuf : in_s) + lc * 16;      // the scenario in process order, for the general fold
 
@@ -482,14 +486,16 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
                     if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                 }
             } else if (it < ntiles + ngroups) {
-                const uint32_t row = ((it - ntiles) << lw) + lr;
-                const char* srow = buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, row);
-                if (LEAN) {
-                    if (!careful) hv[(size_t)row * p.C + lc] = fold_row_lean<T, OP, SWZ>(p, sstar, inc, srow, row, masked);
-                    else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged_call<T, OP, WHOLE, SWZ>(fold_shape(p), root, sstar, inc, in_lc, srow, row);
-                } else if (!careful && !masked) hv[(size_t)row * p.C + lc] = fold_plain_staged<T, OP>(p, sstar, srow);
-                else if (!careful) hv[(size_t)row * p.C + lc] = fold_fast_staged<T, OP, true>(p, sstar, inc, srow, row);
-                else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, row);
+                for (uint32_t gs = 0; gs < GR; ++gs) {
+                    const uint32_t rloc = gs * RW + lr, row = (it - ntiles) * grows + rloc;     // row rloc of the item's buffer
+                    const char* srow = buf_lc + staged_row_offset<WHOLE>(p, rowbytes, rloc, row);
+                    if (LEAN) {
+                        if (!careful) hv[(size_t)row * p.C + lc] = fold_row_lean<T, OP, SWZ>(p, sstar, inc, srow, row, masked);
+                        else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged_call<T, OP, WHOLE, SWZ>(fold_shape(p), root, sstar, inc, in_lc, srow, row);
+                    } else if (!careful && !masked) hv[(size_t)row * p.C + lc] = fold_plain_staged<T, OP>(p, sstar, srow);
+                    else if (!careful) hv[(size_t)row * p.C + lc] = fold_fast_staged<T, OP, true>(p, sstar, inc, srow, row);
+                    else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold_staged<T, OP, WHOLE>(p, root, sstar, inc, in_lc, srow, row);
+                }
             } else if (sstar >= p.r) {
                 if (lr == 0) rootv[lc] = WHOLE ? fold_root16<T, OP, LdShared>(p, root, inc, in_lc) : fold_root16<T, OP, LdGlobal>(p, root, inc, in_lc);
             }
@@ -548,7 +554,9 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
     const uint64_t cap = ((((uint64_t)1 << D) - 1 + p.row_shift) * rowbytes + 127) & ~(uint64_t)127;
     if (cap > 64 * 1024) return false;
     const uint32_t RW = 1u << lw, ntiles = 1u << p.Lt;
-    const uint32_t nitems = ntiles + ((ntiles - 1 + RW - 1) >> lw) + 1;
+    const uint32_t gr_max = (1u << XL) - 1, gr_need = (ntiles - 1 + RW - 1) >> lw;
+    const uint32_t grows = RW * (p.swz_mask ? 1u : (gr_need < 1 ? 1u : (gr_need < gr_max ? gr_need : gr_max)));
+    const uint32_t nitems = ntiles + (ntiles - 1 + grows - 1) / grows + 1;
     // Launch shape, from sweeps on B200: what limits the kernel is the number of resident warps doing the combine
     // work, and shared memory per warp decides that number. So: one buffer per warp, and blocks just large enough
     // to give every warp at least 16 work items per scenario (at most 8 warps).

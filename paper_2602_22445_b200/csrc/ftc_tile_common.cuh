@@ -180,23 +180,25 @@ __device__ __forceinline__ uint4 tile_tree_phase(uint4 valA, uint4 valB, uint32_
 // Work items (warp tiles, then groups of rows above the tiles) that need the careful path: those containing a
 // group that is not plain (a member failed or is an in-operation victim, a renumbered slot, the short last group)
 // and those that are incomplete above their last level. One bit per item in `tspec`; all threads call.
-// Item numbering: tile i (rooted at heap row 2^Lt - 1 + i, D levels) is item i; rows [g*RW, (g+1)*RW) above the
-// tiles are item 2^Lt + g.
+// Item numbering: tile i (rooted at heap row 2^Lt - 1 + i, D levels) is item i; rows [g*grows, (g+1)*grows) above the
+// tiles are item 2^Lt + g (grows = rows per such item, 0 = one per lane row).
 // `tmask` gets the items whose only peculiarity is a group with missing members (fold under the arrival mask, no
 // other checks needed); pass tmask = tspec to send those the careful way too.
 // `below`: rows under the tiles' last level (a sparsely filled last heap level) are folded one by one by the general
 // routine wherever a tile meets them, so they mark nothing.
 static __device__ void mark_special_items(const Params& p, const Ctx* cx, const uint32_t* pf, uint32_t* tspec,
-                                          uint32_t* tmask, uint32_t Lt, uint32_t lw, uint32_t D, bool below = false) {
+                                          uint32_t* tmask, uint32_t Lt, uint32_t lw, uint32_t D, bool below = false, uint32_t grows = 0,
+                                          uint32_t ngroups = 0) {
     const uint32_t tid = threadIdx.x, nt = blockDim.x;
-    const uint32_t ntiles = 1u << Lt, ntop = ntiles - 1, RW = 1u << lw, ngroups = (ntop + RW - 1) >> lw;
+    const uint32_t ntiles = 1u << Lt, ntop = ntiles - 1;
+    if (grows == 0) { grows = 1u << lw; ngroups = (ntop + grows - 1) >> lw; }      // callers with other sizes pass both
     const uint32_t nitems = ntiles + ngroups, root = cx->root, G = cx->G;
     for (uint32_t w = tid; w < (nitems + 31) / 32 + 1; w += nt) { tspec[w] = 0; tmask[w] = 0; }
     __syncthreads();
     auto mark_row = [&](uint32_t j, uint32_t* bm) {
         const uint32_t lvl = ilog2u(j + 1);
         if (below && lvl >= Lt + D) return;
-        const uint32_t it = lvl >= Lt ? ((j + 1) >> (lvl - Lt)) - ntiles : ntiles + (j >> lw);
+        const uint32_t it = lvl >= Lt ? ((j + 1) >> (lvl - Lt)) - ntiles : ntiles + j / grows;
         atomicOr(&bm[it >> 5], 1u << (it & 31));
     };
     for (uint32_t w = tid; w < p.W; w += nt) {
@@ -223,7 +225,7 @@ static __device__ void mark_special_items(const Params& p, const Ctx* cx, const 
         if (((ntop + it + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= G || (!below && ((ntop + it + 1) << D) - 1 < G))
             atomicOr(&tspec[it >> 5], 1u << (it & 31));
     for (uint32_t g = tid; g < ngroups; g += nt)
-        if (((g + 1) << lw) > ntop || ((g + 1) << lw) > G) atomicOr(&tspec[(ntiles + g) >> 5], 1u << ((ntiles + g) & 31));
+        if ((g + 1) * grows > ntop || (g + 1) * grows > G) atomicOr(&tspec[(ntiles + g) >> 5], 1u << ((ntiles + g) & 31));
     __syncthreads();
 }
 
