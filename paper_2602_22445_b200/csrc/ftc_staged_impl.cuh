@@ -282,7 +282,7 @@ constexpr int kStagedMaxThreads = 256;
 constexpr int kStagedLeanThreads = 64;      // lean variant: at most two warps, about 96 registers a thread
 constexpr int kStagedLeanMinBlocks = 10;
 constexpr int kStagedBatchedTag = 3;         // large blocks running the lean variant's code (small groups, exact operations)
-constexpr int kStagedLeanSwzTag = 11;        // lean variant fed by swizzled tensor copies (float32, small vectors)
+constexpr int kStagedLeanSwzTag = 21;        // lean variant fed by swizzled tensor copies (float32, small vectors)
 constexpr int kStagedBatchedSwzTag = 5;      // the same in large blocks
 
 // Tensor maps of the swizzled variant: one per tile level (its box is that level's rows); unused otherwise.
