@@ -568,7 +568,7 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
     uint32_t nbuf = 1;
     // tiny scenarios are staged whole with one copy, larger ones tile by tile (at 16 KB the tiles already win)
     const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
-    g.whole = scen_bytes <= kWholeMaxBytes ? 1u : 0u;
+    g.whole = scen_bytes <= (C >= 16 ? 16 * 1024 : kWholeMaxBytes) ? 1u : 0u;      // a few wide vectors: one copy up to 16 KB
     if (g.whole) nbuf = 0;
     size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
     o = (o + 15) & ~(size_t)15; g.off_special = (uint32_t)o;
