@@ -441,3 +441,20 @@ def test_float32_small_vectors_swizzled_tiles(P, f, k, S, allreduce):
     got = run_gpu(x, f, "sum", pf, inop, roots, 0, allreduce)
     assert B.ftc_kernel_name(got[2], allreduce) == "staged"
     assert_same(got, run_oracle(x, f, "sum", pf, inop, roots, 0, allreduce), f"P={P} f={f} k={k} allreduce={allreduce}")
+
+
+@pytest.mark.parametrize("P,f,k,dname,S", [(8200, 7, 4, "f32", 10), (16384, 5, 16, "u64", 5), (5000, 3, 4, "f32", 9)])
+def test_host_buffer_entry_point_on_swizzled_and_workspace_shapes(P, f, k, dname, S):
+    """The host-buffer call goes chunk by chunk through device staging: tensor maps are built per chunk, and the
+    staging holds the workspace for the tile results."""
+    import torch
+    rng = np.random.Generator(np.random.PCG64(P))
+    x = rng.standard_normal((S, P, k)).astype(np.float32) if dname == "f32" else rng.integers(0, 2**63, size=(S, P, k), dtype=np.uint64)
+    pf = sc.picks_to_masks(sc.random_subsets(rng, S, P, rng.integers(0, f + 1, size=S)), P)
+    roots = rng.integers(0, P, size=S).astype(np.uint32)
+    desc = B.make_desc(P, f, k, B.dtype_code(np.dtype(DT[dname])), "sum", root=-1)
+    out = np.zeros((S, k), dtype=DT[dname])
+    st = np.zeros((S, 4), dtype=np.uint32)
+    staging = torch.empty(B.ftc_host_staging_bytes(desc, 4), dtype=torch.uint8, device="cuda")     # several chunks
+    B.ftc_reduce_batch_host(desc, S, x, pf, None, roots, out, st, staging)
+    assert_same((out, st), run_oracle(x, f, "sum", pf, None, roots, 0, False), f"host variant P={P} k={k} {dname}")
