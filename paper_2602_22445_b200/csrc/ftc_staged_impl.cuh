@@ -1,14 +1,23 @@
-// Staged kernel: the main fast path. Same decomposition as the register-tiled kernel (one block per scenario,
-// the selected subtree's heap of up-correction groups cut into warp tiles, levels above the tiles combined in
-// shared memory), but the input bytes of a tile travel global -> shared memory as a few large asynchronous bulk
-// copies (one per heap level of the tile: each level of a sub-heap is one contiguous run of rows), tracked by an
-// mbarrier per buffer. A warp keeps one tile in flight per buffer while it works on another, so the bytes in
-// flight do not depend on registers, and no lane spends instructions on global addresses.
+// Staged kernel: the main fast path. One block plays one scenario at a time; the selected subtree's heap of
+// up-correction groups ("rows") is cut into warp tiles, and the levels above the tiles are combined in a heap array
+// (shared memory, or the caller's workspace when it is large). The input bytes of a tile travel global -> shared
+// memory asynchronously, one copy per heap level of the tile (each level of a sub-heap is one contiguous run of
+// rows), tracked by an mbarrier per buffer: untiled bulk copies, or tiled tensor copies with a swizzle where the
+// plain layout would put the rows of different lanes into the same banks. Each warp runs its own copy pipeline over
+// the flat sequence of its work items, across scenario boundaries, so the bytes in flight do not depend on
+// registers and no lane spends instructions on global addresses.
 //
 // A tile has lw + XL levels (lw = log2 of the lane rows, 32 / chunks per vector): each lane row evaluates a
-// sub-heap of XL levels by itself (post-order, values in registers), the lw levels above are combined with warp
-// shuffles. Groups that are not "plain" (a missing member, a renumbered slot, the short last group) are folded
-// from global memory by the general routine; they are a handful per scenario.
+// sub-heap of XL levels by itself (values in registers), the lw levels above are combined with warp shuffles.
+// Groups that are not "plain" (a missing member, a renumbered slot, the short last group) take slower folds; they
+// are a handful per scenario.
+//
+// Variants, chosen on the host (template parameter MINB is a tag, see the constants before the kernel):
+//   - large blocks (4-8 warps, 128 registers): rows folded one by one with fully inlined code -- C4, C5;
+//   - lean blocks (1-2 warps, ~96 registers) and large blocks with groups of at most 128 bytes: all rows of a lane
+//     folded together member by member, rare folds as function calls -- C3;
+//   - the same two fed by swizzled tensor copies: float32 vectors of 16 and 32 bytes;
+//   - scenarios staged whole by one copy (up to 12-16 KB): 64 registers.
 #pragma once
 #include <cuda.h>
 #include "ftc_tile_common.cuh"
