@@ -88,28 +88,28 @@ __global__ void __launch_bounds__(256, VEC ? 0 : 8) generic_kernel(Params p) {
         if (p.is_allreduce) count_holders(p, cx, pf, unr);
         const V* in_s = reinterpret_cast<const V*>(p.in) + s * (size_t)p.P * nu;
         const uint32_t G = cx->G, root = cx->root, sstar = cx->sstar;
-        // tree phase (Algorithm "reduce_non_root"): data <- data (op) child 1 (op) child 2 ..., leaves first
-        for (int lvl = (int)heap_level(p.arity, G - 1); lvl >= 0; --lvl) {
+        // tree phase (Algorithm "reduce_non_root"): data <- data (op) child 1 (op) child 2 ..., leaves first.
+        // The rows of the last level are leaves: their value is their group's fold, which the thread that handles
+        // the parent computes on the spot (most rows of a heap are leaves, so most values never touch the workspace).
+        const int last = (int)heap_level(p.arity, G - 1);
+        const uint32_t leaf_lo = (uint32_t)heap_level_start(p.arity, last);
+        for (int lvl = last > 0 ? last - 1 : 0; lvl >= 0; --lvl) {
             const uint32_t lo = (uint32_t)heap_level_start(p.arity, lvl);
             const uint32_t hi = (uint32_t)min(heap_level_start(p.arity, lvl + 1), (uint64_t)G);
+            auto node = [&](uint32_t j, uint32_t u) {
+                const uint64_t c0 = (uint64_t)p.arity * j + 1, c1 = min(c0 + p.arity, (uint64_t)G);
+                V v = fold_group_unit<U>(p, root, sstar, inc, in_s, nu, j, u);
+                for (uint64_t c = c0; c < c1; ++c)
+                    v = U::comb(v, (last > 0 && c >= leaf_lo) ? fold_group_unit<U>(p, root, sstar, inc, in_s, nu, (uint32_t)c, u)
+                                                              : ws[(size_t)c * nu + u]);
+                ws[(size_t)j * nu + u] = v;
+            };
             if (VEC) {
-                for (uint32_t j = lo + r0; j < hi; j += rows_per_pass) {
-                    const uint64_t c0 = (uint64_t)p.arity * j + 1, c1 = min(c0 + p.arity, (uint64_t)G);
-                    for (uint32_t u = u0; u < nu; u += upw) {
-                        V v = fold_group_unit<U>(p, root, sstar, inc, in_s, nu, j, u);
-                        for (uint64_t c = c0; c < c1; ++c) v = U::comb(v, ws[(size_t)c * nu + u]);
-                        ws[(size_t)j * nu + u] = v;
-                    }
-                }
+                for (uint32_t j = lo + r0; j < hi; j += rows_per_pass)
+                    for (uint32_t u = u0; u < nu; u += upw) node(j, u);
             } else {
                 // single elements: every thread takes the next (row, element) pair of the level, whatever k is
-                for (uint32_t x = tid; x < (hi - lo) * nu; x += nt) {
-                    const uint32_t j = lo + x / nu, u = x % nu;
-                    const uint64_t c0 = (uint64_t)p.arity * j + 1, c1 = min(c0 + p.arity, (uint64_t)G);
-                    V v = fold_group_unit<U>(p, root, sstar, inc, in_s, nu, j, u);
-                    for (uint64_t c = c0; c < c1; ++c) v = U::comb(v, ws[(size_t)c * nu + u]);
-                    ws[(size_t)j * nu + u] = v;
-                }
+                for (uint32_t x = tid; x < (hi - lo) * nu; x += nt) node(lo + x / nu, x % nu);
             }
             __syncthreads();
         }
