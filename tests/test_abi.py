@@ -40,6 +40,10 @@ def test_host_only_calls():
     assert (t["H"], t["rounds_reduce"], t["rounds_attempt"]) == (5, 8, 16)       # 256 rows: levels of 1, 4, 16, 64, 171
     assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(3))) == "generic"
     assert B.ftc_kernel_name(B.make_desc(8, 1, 1, B.FTC_I32, "sum", flags=B.FTC_TREE_ARITY(1))) == "invalid"
+    # many processes with wide vectors: the shared-memory kernel asks for a workspace for its array of tile results
+    wide = B.make_desc(16384, 5, 16, B.FTC_U64, "sum")
+    assert B.ftc_kernel_name(wide, True) == "staged" and B.ftc_workspace_bytes(wide, 1000, True) == 148 * 4 * 511 * 128
+    assert B.ftc_kernel_name(B.make_desc(65536, 4, 32, B.FTC_I32, "max"), True) == "staged"
     for code in (0, -1, -2, -3, -4, -5):
         assert B.ftc_strerror(code) and "unknown" not in B.ftc_strerror(code)
     assert "unknown" in B.ftc_strerror(-99)
