@@ -31,7 +31,8 @@
  *   - group partners are visited in ascending (renumbered) rank, skipping self;
  *   - below each root child the subtree is a heap on the local index
  *     j = floor((v-1)/(f+1)): binary by default (children 2j+1 and 2j+2), or
- *     a-ary on request (children a*j+1 .. a*j+a), received in ascending order;
+ *     a-ary on request (children a*j+1 .. a*j+a), or a binomial tree (parent of
+ *     j = j without its lowest set bit), children received in ascending order;
  *     the paper asks only for f+1 root children whose subtree sizes differ by
  *     at most one, which the interleaved numbering gives for any such shape;
  *   - the root examines its children in ascending order and takes the first
@@ -78,7 +79,7 @@ typedef struct {
     uint32_t max_inop;   /* in-operation failure slots per scenario */
     uint32_t sweep;      /* scheduler order: 0 descending rank, 1 ascending, >=2 seeded shuffle */
     uint32_t track_sets; /* carry a P-bit contribution set with every value (instrumentation) */
-    uint32_t arity;      /* children per node below the root's children: 0 or 2 = binary heap, a >= 2 = a-ary heap */
+    uint32_t arity;      /* shape below the root's children: 0 or 2 = binary heap, a >= 2 = a-ary heap, 1 = binomial tree */
 } orc_cfg_t;
 
 typedef struct { uint32_t victim, round; } orc_inop_t;
@@ -212,9 +213,17 @@ static uint32_t sub_of(const sim_t* s, uint32_t v) { return (v - 1) % s->m; }   
 static uint32_t rank_of(const sim_t* s, uint32_t j, uint32_t sidx) { return j * s->m + sidx + 1; }
 /* level of local index j in an a-ary heap: level l holds the a^l indices after those of the levels above */
 static uint32_t heap_level(uint32_t arity, uint32_t j) {
+    if (arity == 1) { uint32_t l = 0; for (; j; j &= j - 1) ++l; return l; }   /* binomial tree: depth = number of set bits */
     uint32_t l = 0; uint64_t start = 0, width = 1;
     while (j >= start + width) { start += width; width *= arity; ++l; }
     return l;
+}
+/* deepest level among the local indices 0..G-1 */
+static uint32_t deepest_level(uint32_t arity, uint32_t G) {
+    if (arity != 1) return heap_level(arity, G - 1);
+    uint32_t best = 0;
+    for (uint32_t j = 0; j < G; ++j) { uint32_t l = heap_level(1, j); if (l > best) best = l; }
+    return best;
 }
 static uint32_t depth_of(const sim_t* s, uint32_t v) { return v == 0 ? 0 : 1 + heap_level(s->arity, row_of(s, v)); }
 
@@ -243,6 +252,13 @@ static uint32_t children(const sim_t* s, uint32_t v, uint32_t* out) {
     uint32_t n = 0;
     if (v == 0) { for (uint32_t c = 1; c <= s->m && c < s->P; ++c) out[n++] = c; return n; }
     uint32_t j = row_of(s, v), sidx = sub_of(s, v);
+    if (s->arity == 1) {
+        /* binomial tree on the local index: the parent of j is j without its lowest set bit, so the children of j
+           are j + 2^i for every 2^i below that bit (all powers of two for j = 0), in ascending order */
+        for (uint64_t bit = 1; (j == 0 || bit < (j & (0u - j))) && (j + bit) * s->m + sidx + 1 < s->P; bit <<= 1)
+            out[n++] = rank_of(s, (uint32_t)(j + bit), sidx);
+        return n;
+    }
     for (uint32_t c = 1; c <= s->arity; ++c) {
         uint64_t jc = (uint64_t)s->arity * j + c;                 /* heap children of j: a*j+1 .. a*j+a */
         if (jc * s->m + sidx + 1 < s->P) out[n++] = rank_of(s, (uint32_t)jc, sidx);
@@ -251,6 +267,7 @@ static uint32_t children(const sim_t* s, uint32_t v, uint32_t* out) {
 }
 static uint32_t parent_of(const sim_t* s, uint32_t v) {
     uint32_t j = row_of(s, v);
+    if (s->arity == 1) return j == 0 ? 0 : rank_of(s, j & (j - 1), sub_of(s, v));
     return j == 0 ? 0 : rank_of(s, (j - 1) / s->arity, sub_of(s, v));
 }
 
@@ -482,7 +499,7 @@ int ftc_oracle_run(const orc_cfg_t* cfg, int is_allreduce, const void* in, const
     if (!cfg || !in || !prefail || !out) return -1;
     uint32_t P = cfg->P, f = cfg->f, k = cfg->k;
     if (k == 0 || P < f + 2 || f + 1 > 60 || root >= P || cfg->max_inop > 32) return -1;
-    if (cfg->arity == 1 || cfg->arity > 32) return -1;
+    if (cfg->arity > 32) return -1;
     if (cfg->dtype > DT_F32 || cfg->op > OP_XOR) return -1;
     if (cfg->dtype == DT_F32 && cfg->op != OP_SUM) return -1;
     sim_t S; memset(&S, 0, sizeof S);
@@ -492,7 +509,7 @@ int ftc_oracle_run(const orc_cfg_t* cfg, int is_allreduce, const void* in, const
     s->W = (P + 31) / 32;
     s->q = (P - 1) / s->m; s->r = (P - 1) % s->m;
     s->arity = cfg->arity ? cfg->arity : 2;
-    s->H = 1 + heap_level(s->arity, s->q + (s->r ? 1 : 0) - 1);     /* depth of the deepest node of the largest subtree */
+    s->H = 1 + deepest_level(s->arity, s->q + (s->r ? 1 : 0));      /* depth of the deepest node of the largest subtree */
     s->Rred = f + s->H; s->Ratt = 2 * s->Rred;
     s->is_allreduce = is_allreduce;
     size_t kb = (size_t)k * s->esz, fz = f ? f : 1;
@@ -655,8 +672,8 @@ int ftc_oracle_batch(const orc_cfg_t* cfg, int is_allreduce, uint64_t S, const v
 
 /* Schedule constants under the readings above: q, r, H, rounds of a reduce, rounds of an allreduce attempt. */
 int ftc_oracle_schedule(uint32_t P, uint32_t f, uint32_t arity, uint32_t* out5) {
-    if (P < f + 2 || arity == 1) return -1;
-    uint32_t m = f + 1, q = (P - 1) / m, r = (P - 1) % m, H = 1 + heap_level(arity ? arity : 2, q + (r ? 1 : 0) - 1);
+    if (P < f + 2) return -1;
+    uint32_t m = f + 1, q = (P - 1) / m, r = (P - 1) % m, H = 1 + deepest_level(arity ? arity : 2, q + (r ? 1 : 0));
     out5[0] = q; out5[1] = r; out5[2] = H; out5[3] = f + H; out5[4] = 2 * (f + H);
     return 0;
 }

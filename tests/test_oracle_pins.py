@@ -528,7 +528,7 @@ def test_failed_list_under_inop_failure_is_the_complement_of_the_contributions()
 # the I(f)-tree property (f+1 root children, subtree sizes within one of each other: definition before the
 # first theorem of section "Properties"), so every statement pinned above must hold for these shapes too.
 # ---------------------------------------------------------------------------------------------
-ARITIES = [3, 4, 5]
+ARITIES = [3, 4, 5, 1]          # 1 = binomial tree
 
 
 def test_arity_tree_structure_by_hand():
@@ -562,6 +562,34 @@ def test_arity_f32_children_combined_in_ascending_order():
     assert d["result"][0] == np.float32(np.float32(0.0) + acc) and d["result"][0] == np.float32(0.0)
     d2 = O.run(vals, f, "sum", [], arity=2)               # binary: 1 <- (1 + (2 + 4)) + 3: another rounding
     assert d2["result"][0] == np.float32(2.0)
+
+
+def test_binomial_tree_structure_by_hand():
+    """n = 14, f = 1, binomial: in subtree 0 (ranks 1,3,..,13; local index j = (v-1)/2) the parent of j is j without
+    its lowest set bit: 0 <- 1, 2, 4;  2 <- 3;  4 <- 5, 6. So rank 1 receives from ranks 3, 5, 9, rank 5 from 7,
+    rank 9 from 11 and 13; depth = 1 + number of set bits of j, the deepest being j = 3, 5, 6 at depth 3."""
+    n, f = 14, 1
+    x = (U64(1) << np.arange(n, dtype=np.uint64)).reshape(n, 1)
+    d = O.run(x, f, "sum", [], detail=True, track_sets=True, arity=1)
+    sets = {v: K.bits(d["tree_sets"][v], n) for v in range(1, n)}
+    assert sets[3] == [3, 4] and sets[7] == [7, 8] and sets[11] == [11, 12] and sets[13] == [0, 13]
+    assert sets[5] == [5, 6, 7, 8]                                  # j = 2 with its child j = 3
+    assert sets[9] == sorted([9, 10, 11, 12, 13, 0])                # j = 4 with j = 5 and j = 6 (short group: the root too)
+    assert sets[1] == list(range(n))
+    assert int(d["result"][0]) == (1 << n) - 1
+    assert O.schedule(14, 1, 1)["H"] == 3 and O.schedule(17, 0, 1)["H"] == 1 + 4     # 16 rows: j = 15 has four set bits
+    # a leaf that dies before its tree send (depth 3: round f+H-3 = 1) taints only its own chain: 7 -> 5 -> 1
+    d = O.run(x, f, "sum", [], inop=[(7, 1)], detail=True, track_sets=True, arity=1)
+    assert d["cand_flag"].tolist() == [1, 0] and d["subtree"] == 1
+
+
+def test_binomial_f32_children_in_ascending_order():
+    n, f = 5, 0                      # one subtree: ranks 1..4 = j 0..3; 0 <- 1, 2;  2 <- 3
+    vals = np.array([0.0, 1.0, 2.0**24, 1.0, -(2.0**24)], dtype=np.float32).reshape(n, 1)
+    d = O.run(vals, f, "sum", [], arity=1)
+    inner = np.float32(vals[3, 0] + vals[4, 0])                     # rank 3 (j = 2) takes rank 4 (j = 3)
+    want = np.float32(np.float32(np.float32(vals[1, 0] + vals[2, 0]) + inner))   # rank 1: its j = 1 child, then j = 2
+    assert d["result"][0] == np.float32(np.float32(0.0) + want)
 
 
 @pytest.mark.parametrize("arity", ARITIES)
