@@ -108,6 +108,9 @@ typedef struct { uint32_t victim; uint32_t round; } ftc_inop_t;
 #define FTC_OUT_EXPANDED   0x1u   /* allreduce: d_out is [S][P][k], zeros for processes that do not hold the result */
 #define FTC_TREE_ARITY(a)  (((uint32_t)(a) & 0xFFu) << 16)  /* subtrees below the root's children are a-ary heaps, 2 <= a <= FTC_MAX_ARITY (not given: binary) */
 #define FTC_MAX_ARITY 32u
+#define FTC_TREE_BINOMIAL   0x1000000u /* subtrees below the root's children are binomial trees on the local index j: parent of j =
+                                         j without its lowest set bit, children in ascending order, depth = 1 + set bits of j
+                                         (not together with FTC_TREE_ARITY; general kernel; not offered by ftc_candidates_batch) */
 #define FTC_KERNEL_GENERIC 0x100u /* force the general level-by-level kernel (needs the workspace) */
 #define FTC_KERNEL_DIRECT  0x200u /* force the register-tiled kernel (direct global loads) where the shape allows it */
 

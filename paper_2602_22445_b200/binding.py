@@ -26,6 +26,7 @@ FTC_INOP_UNUSED = 0xFFFFFFFF
 FTC_OUT_EXPANDED = 0x1
 FTC_KERNEL_GENERIC = 0x100
 FTC_MAX_ARITY = 32
+FTC_TREE_BINOMIAL = 0x1000000
 
 
 def FTC_TREE_ARITY(a: int) -> int:

@@ -13,10 +13,19 @@ static uint32_t heap_level_h(uint32_t arity, uint32_t j) {
     return l;
 }
 // children per node from the descriptor's flags: 0 = not given = binary; 1 and values above FTC_MAX_ARITY are invalid
+// (internally 1 stands for the binomial tree, which FTC_TREE_BINOMIAL asks for)
 static bool tree_arity(uint32_t flags, uint32_t& arity) {
     const uint32_t a = (flags >> 16) & 0xFFu;
+    if (flags & FTC_TREE_BINOMIAL) { arity = 1u; return a == 0; }
     arity = a ? a : 2u;
     return a != 1 && a <= FTC_MAX_ARITY;
+}
+// deepest level among the local indices 0..G-1 of a subtree
+static uint32_t deepest_level_h(uint32_t arity, uint32_t G) {
+    if (arity != 1) return heap_level_h(arity, G - 1);
+    const uint32_t M = G - 1;                 // most set bits of any index <= M
+    uint32_t b = 0; while (b < 32 && (M >> b)) ++b;
+    return (b && M == (uint32_t)((1ull << b) - 1)) ? b : (b ? b - 1 : 0);
 }
 
 static uint32_t elem_size(uint32_t dtype) { return (dtype == FTC_I32 || dtype == FTC_F32) ? 4u : 8u; }
@@ -46,7 +55,7 @@ static int fill_params(const ftc_desc_t* d, uint64_t S, int is_allreduce, Params
     p.P = d->P; p.f = d->f; p.m = d->f + 1; p.k = d->k; p.W = (d->P + 31) / 32;
     p.q = (d->P - 1) / p.m; p.r = (d->P - 1) % p.m;
     p.Gmax = p.q + (p.r ? 1u : 0u);
-    p.H = 1 + heap_level_h(p.arity, p.Gmax - 1);
+    p.H = 1 + deepest_level_h(p.arity, p.Gmax);
     p.Rred = p.f + p.H; p.Ratt = 2 * p.Rred;
     p.max_inop = d->max_inop; p.flags = d->flags; p.root = d->root; p.is_allreduce = is_allreduce;
     p.kbytes = d->k * elem_size(d->dtype);
@@ -234,6 +243,7 @@ int ftc_candidates_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, c
     Params p;
     int rc = fill_params(desc, S, is_allreduce ? 1 : 0, p);
     if (rc != FTC_OK) return rc;
+    if (p.arity == 1) return FTC_EUNSUPPORTED;                 // binomial subtrees: not in this call
     if (S == 0) return FTC_OK;
     if (!d_in || !d_prefail || !d_cand || !d_cand_info) return FTC_EINVAL;
     if (p.max_inop && !d_inop) return FTC_EINVAL;
@@ -310,7 +320,7 @@ int ftc_schedule_info(const ftc_desc_t* desc, ftc_sched_t* out) {
     if (!desc || !out || desc->f > FTC_MAX_F || desc->P < desc->f + 2 || !tree_arity(desc->flags, arity)) return FTC_EINVAL;
     const uint32_t m = desc->f + 1, q = (desc->P - 1) / m, r = (desc->P - 1) % m;
     out->q = q; out->r = r;
-    out->H = 1 + heap_level_h(arity, q + (r ? 1u : 0u) - 1);
+    out->H = 1 + deepest_level_h(arity, q + (r ? 1u : 0u));
     out->rounds_reduce = desc->f + out->H;
     out->rounds_attempt = 2 * out->rounds_reduce;
     out->msgs_upcorrection = (uint64_t)desc->f * m * q + (uint64_t)(r + 1) * r;

@@ -60,8 +60,12 @@ __device__ __forceinline__ bool test_bit(const uint32_t* bm, uint32_t i) { retur
 
 // ---- subtree shape: below each root child a heap on the local index j with p.arity children per node ----
 // Level l holds the arity^l indices that follow those of the levels above; node j has children a*j+1 .. a*j+a.
+// arity 1 stands for the binomial tree: the parent of j is j without its lowest set bit, so j's children are j + 2^i
+// for every 2^i below that bit (all of them for j = 0), its level is its number of set bits, and everything below
+// it is the index range (j, j + lowest set bit).
 __device__ __forceinline__ uint32_t heap_level(uint32_t arity, uint32_t j) {
     if (arity == 2) return ilog2u(j + 1);
+    if (arity == 1) return (uint32_t)__popc(j);
     uint32_t l = 0; uint64_t start = 0, width = 1;
     while (j >= start + width) { start += width; width *= arity; ++l; }
     return l;
@@ -77,6 +81,14 @@ __device__ __forceinline__ uint64_t heap_level_start(uint32_t arity, uint32_t l)
 // All lanes of a warp call it with the same arguments.
 __device__ __forceinline__ void mark_descendants(uint32_t arity, uint32_t m, uint32_t* bm, uint32_t j, uint32_t sv,
                                                  uint32_t Gs, uint32_t lane) {
+    if (arity == 1) {
+        const uint64_t end = j ? min((uint64_t)j + (j & (0u - j)), (uint64_t)Gs) : Gs;
+        for (uint64_t i = (uint64_t)j + 1 + lane; i < end; i += 32) {
+            const uint32_t u = (uint32_t)i * m + sv + 1;
+            atomicOr(&bm[u >> 5], 1u << (u & 31));
+        }
+        return;
+    }
     for (uint64_t lo = (uint64_t)arity * j + 1, n = arity; lo < Gs; lo = arity * lo + 1, n *= arity)
         for (uint64_t i = lane; i < n && lo + i < Gs; i += 32) {
             const uint32_t u = (uint32_t)(lo + i) * m + sv + 1;

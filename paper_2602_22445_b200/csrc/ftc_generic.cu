@@ -91,27 +91,48 @@ __global__ void __launch_bounds__(256, VEC ? 0 : 8) generic_kernel(Params p) {
         // tree phase (Algorithm "reduce_non_root"): data <- data (op) child 1 (op) child 2 ..., leaves first.
         // The rows of the last level are leaves: their value is their group's fold, which the thread that handles
         // the parent computes on the spot (most rows of a heap are leaves, so most values never touch the workspace).
-        const int last = (int)heap_level(p.arity, G - 1);
-        const uint32_t leaf_lo = (uint32_t)heap_level_start(p.arity, last);
-        for (int lvl = last > 0 ? last - 1 : 0; lvl >= 0; --lvl) {
-            const uint32_t lo = (uint32_t)heap_level_start(p.arity, lvl);
-            const uint32_t hi = (uint32_t)min(heap_level_start(p.arity, lvl + 1), (uint64_t)G);
-            auto node = [&](uint32_t j, uint32_t u) {
-                const uint64_t c0 = (uint64_t)p.arity * j + 1, c1 = min(c0 + p.arity, (uint64_t)G);
-                V v = fold_group_unit<U>(p, root, sstar, inc, in_s, nu, j, u);
-                for (uint64_t c = c0; c < c1; ++c)
-                    v = U::comb(v, (last > 0 && c >= leaf_lo) ? fold_group_unit<U>(p, root, sstar, inc, in_s, nu, (uint32_t)c, u)
-                                                              : ws[(size_t)c * nu + u]);
-                ws[(size_t)j * nu + u] = v;
-            };
-            if (VEC) {
-                for (uint32_t j = lo + r0; j < hi; j += rows_per_pass)
-                    for (uint32_t u = u0; u < nu; u += upw) node(j, u);
-            } else {
-                // single elements: every thread takes the next (row, element) pair of the level, whatever k is
-                for (uint32_t x = tid; x < (hi - lo) * nu; x += nt) node(lo + x / nu, x % nu);
+        if (p.arity == 1) {
+            // binomial subtrees: the nodes of one depth are scattered over the index range, so every level looks at
+            // all rows and takes those with that many set bits; children of j are j + 2^i below j's lowest set bit
+            for (int lvl = (int)p.H - 1; lvl >= 0; --lvl) {
+                auto node = [&](uint32_t j, uint32_t u) {
+                    V v = fold_group_unit<U>(p, root, sstar, inc, in_s, nu, j, u);
+                    for (uint64_t bit = 1; (j == 0 || bit < (j & (0u - j))) && j + bit < G; bit <<= 1)
+                        v = U::comb(v, ws[(size_t)(j + bit) * nu + u]);
+                    ws[(size_t)j * nu + u] = v;
+                };
+                if (VEC) {
+                    for (uint32_t j = r0; j < G; j += rows_per_pass)
+                        if (__popc(j) == lvl) for (uint32_t u = u0; u < nu; u += upw) node(j, u);
+                } else {
+                    for (uint32_t x = tid; x < G * nu; x += nt)
+                        if (__popc(x / nu) == lvl) node(x / nu, x % nu);
+                }
+                __syncthreads();
             }
-            __syncthreads();
+        } else {
+            const int last = (int)heap_level(p.arity, G - 1);
+            const uint32_t leaf_lo = (uint32_t)heap_level_start(p.arity, last);
+            for (int lvl = last > 0 ? last - 1 : 0; lvl >= 0; --lvl) {
+                const uint32_t lo = (uint32_t)heap_level_start(p.arity, lvl);
+                const uint32_t hi = (uint32_t)min(heap_level_start(p.arity, lvl + 1), (uint64_t)G);
+                auto node = [&](uint32_t j, uint32_t u) {
+                    const uint64_t c0 = (uint64_t)p.arity * j + 1, c1 = min(c0 + p.arity, (uint64_t)G);
+                    V v = fold_group_unit<U>(p, root, sstar, inc, in_s, nu, j, u);
+                    for (uint64_t c = c0; c < c1; ++c)
+                        v = U::comb(v, (last > 0 && c >= leaf_lo) ? fold_group_unit<U>(p, root, sstar, inc, in_s, nu, (uint32_t)c, u)
+                                                                  : ws[(size_t)c * nu + u]);
+                    ws[(size_t)j * nu + u] = v;
+                };
+                if (VEC) {
+                    for (uint32_t j = lo + r0; j < hi; j += rows_per_pass)
+                        for (uint32_t u = u0; u < nu; u += upw) node(j, u);
+                } else {
+                    // single elements: every thread takes the next (row, element) pair of the level, whatever k is
+                    for (uint32_t x = tid; x < (hi - lo) * nu; x += nt) node(lo + x / nu, x % nu);
+                }
+                __syncthreads();
+            }
         }
         // root (Algorithm "reduce_root"): the selected child's value, combined with the root's own data unless the
         // child's subtree already holds it (it does iff it contains a member of the root's group)

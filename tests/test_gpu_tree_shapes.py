@@ -1,5 +1,5 @@
-"""GPU parity for subtree shapes other than the binary heap (FTC_TREE_ARITY): a-ary heaps below the root's
-children, through every entry point, against the CPU oracle playing the same shape."""
+"""GPU parity for subtree shapes other than the binary heap: a-ary heaps (FTC_TREE_ARITY) and binomial trees
+(FTC_TREE_BINOMIAL) below the root's children, through every entry point, against the CPU oracle playing the same shape."""
 import numpy as np
 import pytest
 
@@ -10,7 +10,11 @@ from tests.gpu_util import assert_same, run_gpu, run_oracle, to_dev, to_host
 
 pytestmark = pytest.mark.gpu
 
-ARITIES = [3, 4, 7]
+ARITIES = [3, 4, 7, 1]            # 1 stands for the binomial tree (the oracle's code for it)
+
+
+def shape_flags(arity):
+    return B.FTC_TREE_BINOMIAL if arity == 1 else B.FTC_TREE_ARITY(arity)
 
 
 def random_case(rng, S, P, f, k, dtype, allreduce, arity):
@@ -38,7 +42,7 @@ def test_exhaustive_failure_sets_small_P(arity, allreduce):
             roots = rng.integers(0, P, size=len(sets)).astype(np.uint32)
             x = rng.integers(0, 2**64, size=(len(sets), P, 2), dtype=np.uint64)
             pf = sc.sets_to_masks(sets, P)
-            got = run_gpu(x, f, "sum", pf, None, roots, 0, allreduce, B.FTC_TREE_ARITY(arity))
+            got = run_gpu(x, f, "sum", pf, None, roots, 0, allreduce, shape_flags(arity))
             assert B.ftc_kernel_name(got[2], allreduce) == "generic"
             want = run_oracle(x, f, "sum", pf, None, roots, 0, allreduce, arity)
             assert_same(got, want, f"P={P} f={f} arity={arity}")
@@ -56,27 +60,27 @@ def test_exhaustive_inop_victim_and_round(arity, allreduce):
         inop = np.zeros((S, 1, 2), dtype=np.uint32)
         inop[:, 0, 0] = [c[1] for c in cases]
         inop[:, 0, 1] = [c[2] for c in cases]
-        got = run_gpu(x, f, "sum", pf, inop, None, 0, allreduce, B.FTC_TREE_ARITY(arity))
+        got = run_gpu(x, f, "sum", pf, inop, None, 0, allreduce, shape_flags(arity))
         want = run_oracle(x, f, "sum", pf, inop, None, 0, allreduce, arity)
         assert_same(got, want, f"P={P} f={f} arity={arity}")
 
 
-@pytest.mark.parametrize("arity", [3, 5])
+@pytest.mark.parametrize("arity", [3, 5, 1])
 def test_configuration_shapes(arity):
     """Samples of the large configurations on the other shapes: float32 bit for bit, in-operation failures,
     per-scenario roots at P = 65536."""
     w = sc.config3(S=64)
     x = w.host_inputs()
-    got = run_gpu(x, w.f, w.op, w.prefail, None, None, 0, True, B.FTC_TREE_ARITY(arity))
+    got = run_gpu(x, w.f, w.op, w.prefail, None, None, 0, True, shape_flags(arity))
     assert_same(got, run_oracle(x, w.f, w.op, w.prefail, None, None, 0, True, arity), f"C3 arity={arity}")
     w = sc.config4(O.schedule(4096, 4, arity)["rounds_attempt"], S=24)
     x = w.host_inputs()
-    got = run_gpu(x, w.f, w.op, w.prefail, w.inop, None, 0, True, B.FTC_TREE_ARITY(arity))
+    got = run_gpu(x, w.f, w.op, w.prefail, w.inop, None, 0, True, shape_flags(arity))
     assert_same(got, run_oracle(x, w.f, w.op, w.prefail, w.inop, None, 0, True, arity), f"C4 arity={arity}")
     for coll in ("reduce", "allreduce"):
         w = sc.config5(coll, "sum", S=3)
         x = w.host_inputs()
-        got = run_gpu(x, w.f, w.op, w.prefail, None, w.roots, 0, coll == "allreduce", B.FTC_TREE_ARITY(arity))
+        got = run_gpu(x, w.f, w.op, w.prefail, None, w.roots, 0, coll == "allreduce", shape_flags(arity))
         assert_same(got, run_oracle(x, w.f, w.op, w.prefail, None, w.roots, 0, coll == "allreduce", arity), f"C5 {coll}")
 
 
@@ -84,7 +88,7 @@ def test_configuration_shapes(arity):
 def test_expanded_candidates_messages_and_noalloc(arity):
     import torch
     rng = np.random.Generator(np.random.PCG64(300 + arity))
-    flags = B.FTC_TREE_ARITY(arity)
+    flags = shape_flags(arity)
     for P, f, k, dtype in ((10, 2, 4, np.uint64), (41, 1, 3, np.float32), (130, 3, 2, np.int32)):
         S = 50
         for allreduce in (False, True):
@@ -97,7 +101,9 @@ def test_expanded_candidates_messages_and_noalloc(arity):
             d_cand = torch.zeros((S, f + 1, k), dtype=d_x.dtype, device="cuda")
             d_info = torch.zeros((S, f + 1, 2), dtype=torch.int32, device="cuda")
             d_ws = torch.empty(B.ftc_candidates_workspace_bytes(desc, S), dtype=torch.uint8, device="cuda")
-            B.ftc_candidates_batch(desc, S, allreduce, d_x, to_dev(pf), to_dev(inop), to_dev(roots), d_cand, d_info, d_ws)
+            rc = B.ftc_candidates_batch(desc, S, allreduce, d_x, to_dev(pf), to_dev(inop), to_dev(roots), d_cand, d_info, d_ws,
+                                        check=False)
+            assert rc == (B.FTC_EUNSUPPORTED if arity == 1 else B.FTC_OK)        # binomial subtrees: not in this call
             # message counts
             d_msgs = torch.zeros((S, B.FTC_MSG_WORDS), dtype=torch.int64, device="cuda")
             B.ftc_message_counts_batch(desc, S, allreduce, to_dev(pf), to_dev(inop), to_dev(roots), d_msgs.view(torch.uint64))
@@ -105,7 +111,7 @@ def test_expanded_candidates_messages_and_noalloc(arity):
             cand, info, msgs = to_host(d_cand, x.dtype), d_info.cpu().numpy(), d_msgs.cpu().numpy().view(np.uint64)
             for i, d in enumerate(ref):
                 assert np.array_equal(msgs[i], d["msgs"]), (P, f, i, msgs[i], d["msgs"])
-                if d["attempts"] == 0:
+                if d["attempts"] == 0 or arity == 1:
                     continue
                 assert np.array_equal(info[i, :, 0], d["cand_flag"]) and np.array_equal(info[i, :, 1], d["cand_nfail"]), (P, f, i)
                 assert np.array_equal(cand[i].view(np.uint8), d["cand"].view(np.uint8)), (P, f, i)
@@ -138,6 +144,9 @@ def test_arity_in_the_descriptor():
     for bad in (1, 33, 255):
         d = B.make_desc(8, 1, 4, B.FTC_I32, "sum", flags=B.FTC_TREE_ARITY(bad))
         assert B.ftc_reduce_batch(d, 1, z, z, None, None, z, z, z, check=False) == B.FTC_EINVAL
+    both = B.make_desc(8, 1, 4, B.FTC_I32, "sum", flags=B.FTC_TREE_ARITY(3) | B.FTC_TREE_BINOMIAL)
+    assert B.ftc_reduce_batch(both, 1, z, z, None, None, z, z, z, check=False) == B.FTC_EINVAL
+    assert B.ftc_schedule_info(B.make_desc(65536, 8, 4, B.FTC_U64, "sum", flags=B.FTC_TREE_BINOMIAL))["H"] == O.schedule(65536, 8, 1)["H"]
     d2 = B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(2))
     assert B.ftc_kernel_name(d2, True) == "staged"                       # 2 is the default shape
     assert B.ftc_schedule_info(B.make_desc(65536, 8, 4, B.FTC_U64, "sum", flags=B.FTC_TREE_ARITY(3)))["H"] == O.schedule(65536, 8, 3)["H"]
