@@ -28,7 +28,8 @@
  *     next candidate if r had failed before the operation.
  *
  * Readings where the paper is silent (the same ones the documentation lists):
- *   - group partners are visited in ascending (renumbered) rank, skipping self;
+ *   - group partners are visited in ascending (renumbered) rank, skipping self,
+ *     the root first in the short last group (on request: the reverse order);
  *   - below each root child the subtree is a heap on the local index
  *     j = floor((v-1)/(f+1)): binary by default (children 2j+1 and 2j+2), or
  *     a-ary on request (children a*j+1 .. a*j+a), or a binomial tree (parent of
@@ -79,6 +80,7 @@ typedef struct {
     uint32_t max_inop;   /* in-operation failure slots per scenario */
     uint32_t sweep;      /* scheduler order: 0 descending rank, 1 ascending, >=2 seeded shuffle */
     uint32_t track_sets; /* carry a P-bit contribution set with every value (instrumentation) */
+    uint32_t partners_descending; /* 1: group partners are visited in descending rank, the root last (default: ascending, root first) */
     uint32_t arity;      /* shape below the root's children: 0 or 2 = binary heap, a >= 2 = a-ary heap, 1 = binomial tree */
 } orc_cfg_t;
 
@@ -227,8 +229,9 @@ static uint32_t deepest_level(uint32_t arity, uint32_t G) {
 }
 static uint32_t depth_of(const sim_t* s, uint32_t v) { return v == 0 ? 0 : 1 + heap_level(s->arity, row_of(s, v)); }
 
-/* members of the up-correction group of v in ascending rank, v excluded; returns their number */
-static uint32_t partners(const sim_t* s, uint32_t v, uint32_t* out) {
+/* members of the up-correction group of v in the order v visits them (ascending rank with the root first, or the
+   reverse), v excluded; returns their number */
+static uint32_t partners_ascending(const sim_t* s, uint32_t v, uint32_t* out) {
     uint32_t n = 0, lo, hi, u;
     if (v == 0) {
         if (s->r == 0) return 0;                       /* root belongs to no group */
@@ -240,6 +243,12 @@ static uint32_t partners(const sim_t* s, uint32_t v, uint32_t* out) {
     lo = j * s->m + 1; hi = lo + s->m - 1; if (hi > s->P - 1) hi = s->P - 1;
     if (j == s->q) out[n++] = 0;                        /* short last group: the root is a member, rank 0 first */
     for (u = lo; u <= hi; ++u) if (u != v) out[n++] = u;
+    return n;
+}
+static uint32_t partners(const sim_t* s, uint32_t v, uint32_t* out) {
+    uint32_t n = partners_ascending(s, v, out);
+    if (s->cfg->partners_descending)
+        for (uint32_t i = 0; i + 1 < n - i; ++i) { uint32_t t = out[i]; out[i] = out[n - 1 - i]; out[n - 1 - i] = t; }
     return n;
 }
 static uint32_t partner_index(const sim_t* s, uint32_t u, uint32_t v) {

@@ -23,7 +23,7 @@ UNUSED = 0xFFFFFFFF
 
 
 class Cfg(C.Structure):
-    _fields_ = [(n, C.c_uint32) for n in ("P", "f", "k", "dtype", "op", "max_inop", "sweep", "track_sets", "arity")]
+    _fields_ = [(n, C.c_uint32) for n in ("P", "f", "k", "dtype", "op", "max_inop", "sweep", "track_sets", "partners_descending", "arity")]
 
 
 class Out(C.Structure):
@@ -78,7 +78,8 @@ def _prep_inop(inop, max_inop):
 
 
 def run(x: np.ndarray, f: int, op: str, prefail, inop=None, root: int = 0, allreduce: bool = False,
-        sweep: int = 0, track_sets: bool = False, detail: bool = False, arity: int = 2) -> dict:
+        sweep: int = 0, track_sets: bool = False, detail: bool = False, arity: int = 2,
+        partners_descending: bool = False) -> dict:
     """Simulate one scenario. x: [P][k]; prefail: uint32 words or an iterable of failed ids;
     inop: [(victim, round), ...]. Returns result, status fields and (detail=True) instrumentation."""
     x = np.ascontiguousarray(x)
@@ -95,7 +96,7 @@ def run(x: np.ndarray, f: int, op: str, prefail, inop=None, root: int = 0, allre
     if inop is not None and len(inop):
         inop_a = np.ascontiguousarray(np.asarray(inop, dtype=np.uint32).reshape(-1, 2))
         max_inop = inop_a.shape[0]
-    cfg = Cfg(P, f, k, DTYPES[x.dtype], OPS[op], max_inop, sweep, 1 if track_sets else 0, arity)
+    cfg = Cfg(P, f, k, DTYPES[x.dtype], OPS[op], max_inop, sweep, 1 if track_sets else 0, int(partners_descending), arity)
     res = np.zeros(k, dtype=x.dtype)
     status = np.zeros(4, dtype=np.uint32)
     out = Out()
@@ -125,7 +126,7 @@ def run(x: np.ndarray, f: int, op: str, prefail, inop=None, root: int = 0, allre
 
 
 def batch(x: np.ndarray, f: int, op: str, prefail: np.ndarray, inop=None, roots=None, root: int = 0,
-          allreduce: bool = False, arity: int = 2):
+          allreduce: bool = False, arity: int = 2, partners_descending: bool = False):
     """Simulate S scenarios one after the other. x: [S][P][k]; prefail: [S][W] uint32;
     inop: [S][max_inop][2] uint32 or None; roots: [S] uint32 or None. Returns (result [S][k], status [S][4])."""
     x = np.ascontiguousarray(x)
@@ -137,7 +138,7 @@ def batch(x: np.ndarray, f: int, op: str, prefail: np.ndarray, inop=None, roots=
         max_inop = inop.shape[1]
     if roots is not None:
         roots = np.ascontiguousarray(roots, dtype=np.uint32)
-    cfg = Cfg(P, f, k, DTYPES[x.dtype], OPS[op], max_inop, 0, 0, arity)
+    cfg = Cfg(P, f, k, DTYPES[x.dtype], OPS[op], max_inop, 0, 0, int(partners_descending), arity)
     res = np.zeros((S, k), dtype=x.dtype)
     status = np.zeros((S, 4), dtype=np.uint32)
     rc = lib().ftc_oracle_batch(C.byref(cfg), 1 if allreduce else 0, S, _ptr(x), _ptr(prefail), _ptr(inop),

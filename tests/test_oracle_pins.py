@@ -643,3 +643,60 @@ def test_arity_inop_allowed_results_and_allreduce_consistency(n, f, arity):
                     assert holders == alive_end                  # at most f failures: every survivor holds the value
                     for p in holders:
                         assert np.array_equal(d["expanded"][p], d["result"])
+
+
+# ---------------------------------------------------------------------------------------------
+# The other partner order: Algorithm "Up-correction" leaves the order of "p in group \ {self}" open; besides the
+# ascending order (root first) the oracle plays the descending one (root last). Every semantic pin must hold for it.
+# ---------------------------------------------------------------------------------------------
+def test_descending_partner_order_decides_whom_a_dying_process_reached():
+    """The mirror image of the ascending case: n=6, f=2, short last group {4, 5, root}: process 5 now sends to 4 in
+    round 0 and to the root in round 1; process 3 of the full group {1,2,3} sends to 2 first, then to 1."""
+    x = (U64(1) << np.arange(6, dtype=np.uint64)).reshape(6, 1)
+    d = O.run(x, 2, "sum", [], inop=[(5, 1)], detail=True, track_sets=True, partners_descending=True)
+    assert d["subtree"] == 0 and K.bits(d["contrib"], 6) == [0, 1, 2, 3, 4, 5]      # 4 (subtree 0) got 5's value
+    d = O.run(x, 2, "sum", [1], inop=[(3, 1)], detail=True, track_sets=True, partners_descending=True)
+    assert d["subtree"] == 1 and K.bits(d["contrib"], 6) == [0, 2, 3, 4, 5]          # 2 got 3's value in round 0
+    d = O.run(x, 2, "sum", [2], inop=[(3, 1)], detail=True, track_sets=True, partners_descending=True)
+    assert d["subtree"] == 0 and K.bits(d["contrib"], 6) == [0, 1, 4, 5]             # the send to 2 was wasted, 1 got nothing
+
+
+def test_descending_partner_order_f32_fold():
+    """Group {1,2,3} (f=2, n=4, root 0 in no group): rank 1 folds own + x3 + x2, where ascending gives own + x2 + x3."""
+    vals = np.array([0.0, 1.0, 2.0**24, -(2.0**24)], dtype=np.float32).reshape(4, 1)
+    asc = O.run(vals, 2, "sum", [])
+    desc = O.run(vals, 2, "sum", [], partners_descending=True)
+    a = np.float32(np.float32(vals[1, 0] + vals[2, 0]) + vals[3, 0])      # (1 + 2^24) - 2^24 = 0
+    b = np.float32(np.float32(vals[1, 0] + vals[3, 0]) + vals[2, 0])      # (1 - 2^24) + 2^24 = 0 as well: use the root add
+    assert asc["result"][0] == np.float32(np.float32(0.0) + a)
+    assert desc["result"][0] == np.float32(np.float32(0.0) + b)
+    vals2 = np.array([0.0, 2.0**24, 1.0, 1.0 - 2.0**-23], dtype=np.float32).reshape(4, 1)   # order of the two small addends shows
+    asc, desc = O.run(vals2, 2, "sum", []), O.run(vals2, 2, "sum", [], partners_descending=True)
+    assert asc["result"][0] == np.float32(np.float32(vals2[1, 0] + vals2[2, 0]) + vals2[3, 0])
+    assert desc["result"][0] == np.float32(np.float32(vals2[1, 0] + vals2[3, 0]) + vals2[2, 0])
+
+
+@pytest.mark.parametrize("n,f", [(7, 1), (9, 2), (12, 2), (13, 3), (16, 3)])
+def test_descending_partner_order_semantics(n, f):
+    x = rand_u64(n, 2, 17 * n + f)
+    base = O.run(np.ones((n, 1), dtype=np.int32), f, "sum", [], allreduce=True, detail=True, partners_descending=True)
+    assert [int(v) for v in base["msgs"][:4]] == [uc_messages(n, f), n - 1, n - 1, uc_messages(n, f)]
+    for size in range(0, f + 1):
+        for dead in itertools.combinations(range(n), size):
+            for root in (0, n - 1):
+                d = O.run(x, f, "sum", dead, root=root, track_sets=True, detail=True, partners_descending=True)
+                live = [p for p in range(n) if p not in dead]
+                if root in dead:
+                    assert d["code"] == 1
+                    continue
+                assert d["code"] == 0 and np.array_equal(d["result"], K.reduce_over(x, live, "sum"))
+                assert K.bits(d["contrib"], n) == live
+    sch = O.schedule(n, f)
+    for victim in range(f + 1, n):
+        for t in range(1, sch["rounds_attempt"] + 2):
+            d = O.run(x, f, "sum", [], inop=[(victim, t)], allreduce=True, track_sets=True, detail=True, partners_descending=True)
+            C = K.bits(d["contrib"], n)
+            assert d["code"] == 0 and K.contribution_allowed(n, C, [], [victim])
+            assert np.array_equal(d["result"], K.reduce_over(x, C, "sum"))
+            alive_end = [p for p in range(n) if not (p == victim and t < sch["rounds_attempt"])]
+            assert K.bits(d["holders"], n) == alive_end
