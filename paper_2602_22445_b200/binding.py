@@ -27,6 +27,7 @@ FTC_OUT_EXPANDED = 0x1
 FTC_KERNEL_GENERIC = 0x100
 FTC_MAX_ARITY = 32
 FTC_TREE_BINOMIAL = 0x1000000
+FTC_PARTNERS_DESCENDING = 0x2000000
 
 
 def FTC_TREE_ARITY(a: int) -> int:

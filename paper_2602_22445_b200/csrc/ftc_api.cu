@@ -52,6 +52,7 @@ static int fill_params(const ftc_desc_t* d, uint64_t S, int is_allreduce, Params
     if (!tree_arity(d->flags, arity)) return FTC_EINVAL;
     std::memset(&p, 0, sizeof p);
     p.arity = arity;
+    p.pdesc = (d->flags & FTC_PARTNERS_DESCENDING) ? 1u : 0u;
     p.P = d->P; p.f = d->f; p.m = d->f + 1; p.k = d->k; p.W = (d->P + 31) / 32;
     p.q = (d->P - 1) / p.m; p.r = (d->P - 1) % p.m;
     p.Gmax = p.q + (p.r ? 1u : 0u);
@@ -77,7 +78,7 @@ static const DeviceInfo kB200 = {148, 232448};
 
 enum KernelKind { K_GENERIC = 0, K_TILED = 1, K_STAGED = 2 };
 static KernelKind pick_kernel(Params& p, const DeviceInfo& di) {
-    if ((p.flags & FTC_KERNEL_GENERIC) || p.arity != 2) return K_GENERIC;      // the tiled kernels are built on the binary heap
+    if ((p.flags & FTC_KERNEL_GENERIC) || p.arity != 2 || p.pdesc) return K_GENERIC;   // the tiled kernels are built on the binary heap and the ascending order
     if (!(p.flags & FTC_KERNEL_DIRECT) && staged_supported(p, di.smem_optin, di.sm_count)) return K_STAGED;
     return tiled_supported(p, di.smem_optin) ? K_TILED : K_GENERIC;
 }
@@ -243,7 +244,7 @@ int ftc_candidates_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, c
     Params p;
     int rc = fill_params(desc, S, is_allreduce ? 1 : 0, p);
     if (rc != FTC_OK) return rc;
-    if (p.arity == 1) return FTC_EUNSUPPORTED;                 // binomial subtrees: not in this call
+    if (p.arity == 1 || p.pdesc) return FTC_EUNSUPPORTED;      // binomial subtrees, descending partners: not in this call
     if (S == 0) return FTC_OK;
     if (!d_in || !d_prefail || !d_cand || !d_cand_info) return FTC_EINVAL;
     if (p.max_inop && !d_inop) return FTC_EINVAL;

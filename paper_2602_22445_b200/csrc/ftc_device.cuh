@@ -13,7 +13,8 @@ struct Params {
     uint32_t P, f, m, k, W;          // m = f+1 (group size = root children); W = mask words per scenario
     uint32_t q, r, H, Rred, Ratt;    // P-1 = q*m + r; deepest node; rounds of a reduce / of an allreduce attempt
     uint32_t Gmax;                   // nodes of the largest root subtree: q + (r > 0)
-    uint32_t arity;                  // children per node below the root's children (2: binary heap)
+    uint32_t arity;                  // children per node below the root's children (2: binary heap; 1: binomial tree)
+    uint32_t pdesc;                  // 1: group partners are visited in descending rank, the root last
     uint32_t max_inop, flags;
     int32_t  root;
     int32_t  is_allreduce;
@@ -126,11 +127,14 @@ __device__ __forceinline__ uint32_t local_round(uint32_t fr, uint32_t base) {
     return fr == kNever ? kNever : (fr <= base ? 0u : fr - base);
 }
 
-// Index of partner (row, sp) in the ascending partner list of member (row, sv), sv != sp. In the short last
-// group the root comes first.
+// Index of partner (row, sp) in the partner list of member (row, sv), sv != sp: ascending rank with the root first
+// in the short last group, or (p.pdesc) descending rank with the root last.
 __device__ __forceinline__ uint32_t partner_slot(const Params& p, uint32_t row, uint32_t sv, uint32_t sp) {
+    if (p.pdesc) return (row < p.q ? p.m : p.r) - 1 - sp - (sv > sp ? 1u : 0u);
     return (sp < sv ? sp : sp - 1) + (row == p.q ? 1u : 0u);
 }
+// Index of the root in the partner list of a member of the short last group.
+__device__ __forceinline__ uint32_t root_slot(const Params& p) { return p.pdesc ? p.r - 1 : 0u; }
 
 // Decode one scenario. All threads of the block call it. On return (after its last barrier) cx, pf (physical
 // pre-failure bits) and inc (bit v: the input of renumbered process v reaches the selected subtree's member of
@@ -242,7 +246,7 @@ static __device__ void decode_scenario(const Params& p, uint64_t s, Ctx* cx, uin
                     uint32_t t = local_round(cx->ir[lane], base);
                     bool member_in_subtree = j < p.q || sstar < p.r;   // does group j have a member below child sstar?
                     if (member_in_subtree) { if (sv != sstar) included = partner_slot(p, j, sv, sstar) < t; }
-                    else included = t >= 1;                            // the group's values reach the root itself: slot 0
+                    else included = t > root_slot(p);                  // the group's values reach the root itself
                 }
                 if (included) atomicOr(&cx->inop_incl, 1u << lane);
                 else {

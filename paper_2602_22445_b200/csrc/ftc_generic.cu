@@ -31,6 +31,12 @@ __device__ __forceinline__ typename U::V fold_group_unit(const Params& p, uint32
     const uint32_t mj = row < p.q ? p.m : p.r, vbase = row * p.m + 1;
     const uint32_t mask = extract_bits(inc, vbase, mj);
     typename U::V acc = U::ld(in_s + (size_t)renumber(vbase + sstar, root) * nu + u);
+    if (p.pdesc) {                       // the other partner order: descending rank, the root last
+        for (uint32_t sp = mj; sp-- > 0;)
+            if (sp != sstar && ((mask >> sp) & 1u)) acc = U::comb(acc, U::ld(in_s + (size_t)renumber(vbase + sp, root) * nu + u));
+        if (row == p.q) acc = U::comb(acc, U::ld(in_s + (size_t)root * nu + u));
+        return acc;
+    }
     if (row == p.q) acc = U::comb(acc, U::ld(in_s + (size_t)root * nu + u));
     for (uint32_t sp = 0; sp < mj; ++sp)
         if (sp != sstar && ((mask >> sp) & 1u)) acc = U::comb(acc, U::ld(in_s + (size_t)renumber(vbase + sp, root) * nu + u));
@@ -45,8 +51,10 @@ __device__ __forceinline__ typename U::V fold_root_unit(const Params& p, uint32_
     typename U::V acc = U::ld(in_s + (size_t)root * nu + u);
     if (p.r) {
         const uint32_t vbase = p.q * p.m + 1, mask = extract_bits(inc, vbase, p.r);
-        for (uint32_t sp = 0; sp < p.r; ++sp)
+        for (uint32_t i = 0; i < p.r; ++i) {
+            const uint32_t sp = p.pdesc ? p.r - 1 - i : i;
             if ((mask >> sp) & 1u) acc = U::comb(acc, U::ld(in_s + (size_t)renumber(vbase + sp, root) * nu + u));
+        }
     }
     return acc;
 }

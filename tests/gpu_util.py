@@ -54,8 +54,9 @@ def run_gpu(x, f, op, prefail, inop=None, roots=None, root=0, allreduce=False, f
     return to_host(d_out, np_dtype), d_status.cpu().numpy().view(np.uint32), desc
 
 
-def run_oracle(x, f, op, prefail, inop=None, roots=None, root=0, allreduce=False, arity=2):
-    return O.batch(x, f, op, prefail, inop=inop, roots=roots, root=root, allreduce=allreduce, arity=arity)
+def run_oracle(x, f, op, prefail, inop=None, roots=None, root=0, allreduce=False, arity=2, partners_descending=False):
+    return O.batch(x, f, op, prefail, inop=inop, roots=roots, root=root, allreduce=allreduce, arity=arity,
+                   partners_descending=partners_descending)
 
 
 def assert_same(got, want, what=""):

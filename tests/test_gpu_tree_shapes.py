@@ -150,3 +150,52 @@ def test_arity_in_the_descriptor():
     d2 = B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(2))
     assert B.ftc_kernel_name(d2, True) == "staged"                       # 2 is the default shape
     assert B.ftc_schedule_info(B.make_desc(65536, 8, 4, B.FTC_U64, "sum", flags=B.FTC_TREE_ARITY(3)))["H"] == O.schedule(65536, 8, 3)["H"]
+
+
+# ---------------------------------------------------------------------------------------------
+# the other partner order (FTC_PARTNERS_DESCENDING), alone and together with another subtree shape
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("arity", [2, 3, 1])
+@pytest.mark.parametrize("allreduce", [False, True])
+def test_descending_partners(arity, allreduce):
+    flags = B.FTC_PARTNERS_DESCENDING | (0 if arity == 2 else shape_flags(arity))
+    rng = np.random.Generator(np.random.PCG64(900 + arity))
+    # every (victim, round), alone and beside one pre-operation failure: the order decides whom a dying process reached
+    for P, f in ((6, 2), (11, 2), (20, 1), (29, 3)):
+        R = O.schedule(P, f, arity)["rounds_attempt" if allreduce else "rounds_reduce"]
+        cases = [(pre, v, t) for v in range(P) for t in range(0, R + 2) for pre in ((), ((v + 3) % P,))]
+        S = len(cases)
+        x = rng.integers(0, 2**64, size=(S, P, 2), dtype=np.uint64)
+        pf = sc.sets_to_masks([c[0] for c in cases], P)
+        inop = np.zeros((S, 1, 2), dtype=np.uint32)
+        inop[:, 0, 0] = [c[1] for c in cases]
+        inop[:, 0, 1] = [c[2] for c in cases]
+        got = run_gpu(x, f, "sum", pf, inop, None, 0, allreduce, flags)
+        assert B.ftc_kernel_name(got[2], allreduce) == "generic"
+        assert_same(got, run_oracle(x, f, "sum", pf, inop, None, 0, allreduce, arity, True), f"P={P} f={f} arity={arity}")
+    # float32 bit for bit, random failures and roots, expanded output and message counts
+    import torch
+    for P, f, k in ((41, 3, 4), (130, 2, 16), (1024, 3, 16)):
+        S = 40
+        x, pf, inop, roots = random_case(rng, S, P, f, k, np.float32, allreduce, arity)
+        got = run_gpu(x, f, "sum", pf, inop, roots, 0, allreduce, flags)
+        assert_same(got, run_oracle(x, f, "sum", pf, inop, roots, 0, allreduce, arity, True), f"f32 P={P} f={f} arity={arity}")
+        desc = B.make_desc(P, f, k, B.FTC_F32, "sum", root=-1, max_inop=2, flags=flags)
+        d_msgs = torch.zeros((S, B.FTC_MSG_WORDS), dtype=torch.int64, device="cuda")
+        B.ftc_message_counts_batch(desc, S, allreduce, to_dev(pf), to_dev(inop), to_dev(roots), d_msgs.view(torch.uint64))
+        torch.cuda.synchronize()
+        msgs = d_msgs.cpu().numpy().view(np.uint64)
+        ref = [O.run(x[i], f, "sum", pf[i], inop=[tuple(e) for e in inop[i]], root=int(roots[i]), allreduce=allreduce, detail=True,
+                     arity=arity, partners_descending=True) for i in range(S)]
+        for i, d in enumerate(ref):
+            assert np.array_equal(msgs[i], d["msgs"]), (P, f, i)
+        if allreduce:
+            desc_e = B.make_desc(P, f, k, B.FTC_F32, "sum", root=-1, max_inop=2, flags=flags | B.FTC_OUT_EXPANDED)
+            d_out = torch.zeros((S, P, k), dtype=torch.float32, device="cuda")
+            d_st = torch.zeros((S, 4), dtype=torch.int32, device="cuda")
+            d_ws = torch.empty(B.ftc_workspace_bytes(desc_e, S, True), dtype=torch.uint8, device="cuda")
+            B.ftc_allreduce_batch(desc_e, S, to_dev(x), to_dev(pf), to_dev(inop), to_dev(roots), d_out, d_st, d_ws)
+            torch.cuda.synchronize()
+            out, st = d_out.cpu().numpy(), d_st.cpu().numpy().view(np.uint32)
+            for i, d in enumerate(ref):
+                assert np.array_equal(st[i], d["status"]) and np.array_equal(out[i].view(np.uint8), d["expanded"].view(np.uint8)), (P, i)
