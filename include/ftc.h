@@ -110,10 +110,10 @@ typedef struct { uint32_t victim; uint32_t round; } ftc_inop_t;
 #define FTC_MAX_ARITY 32u
 #define FTC_TREE_BINOMIAL   0x1000000u /* subtrees below the root's children are binomial trees on the local index j: parent of j =
                                          j without its lowest set bit, children in ascending order, depth = 1 + set bits of j
-                                         (not together with FTC_TREE_ARITY; general kernel; not offered by ftc_candidates_batch) */
+                                         (not together with FTC_TREE_ARITY; general kernel) */
 #define FTC_PARTNERS_DESCENDING 0x2000000u /* up-correction (and the broadcast's correction) visits the group partners in descending
                                             rank, the root last, instead of ascending with the root first: the algorithm leaves the
-                                            order open (general kernel; not offered by ftc_candidates_batch) */
+                                            order open (general kernel) */
 #define FTC_KERNEL_GENERIC 0x100u /* force the general level-by-level kernel (needs the workspace) */
 #define FTC_KERNEL_DIRECT  0x200u /* force the register-tiled kernel (direct global loads) where the shape allows it */
 

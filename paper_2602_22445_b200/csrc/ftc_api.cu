@@ -244,7 +244,6 @@ int ftc_candidates_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, c
     Params p;
     int rc = fill_params(desc, S, is_allreduce ? 1 : 0, p);
     if (rc != FTC_OK) return rc;
-    if (p.arity == 1 || p.pdesc) return FTC_EUNSUPPORTED;      // binomial subtrees, descending partners: not in this call
     if (S == 0) return FTC_OK;
     if (!d_in || !d_prefail || !d_cand || !d_cand_info) return FTC_EINVAL;
     if (p.max_inop && !d_inop) return FTC_EINVAL;

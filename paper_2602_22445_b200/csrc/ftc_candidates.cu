@@ -90,29 +90,46 @@ __global__ void __launch_bounds__(256) candidates_kernel(Params p, T* cand, uint
             }
             __syncthreads();
             const uint32_t G = p.q + (sc < p.r ? 1u : 0u);
-            for (int lvl = (int)heap_level(p.arity, G - 1); lvl >= 0; --lvl) {
-                const uint32_t lo = (uint32_t)heap_level_start(p.arity, lvl);
-                const uint32_t hi = (uint32_t)min(heap_level_start(p.arity, lvl + 1), (uint64_t)G);
-                for (uint32_t u = tid; u < (hi - lo) * p.k; u += nt) {
-                    const uint32_t j = lo + u / p.k, e = u % p.k;
-                    const uint32_t v = j * p.m + sc + 1;
-                    if (!test_bit(snd, v)) { if (e == 0) { pres[j] = 0; fbit[j] = 0; nfl[j] = 0; } continue; }
-                    const uint32_t mj = j < p.q ? p.m : p.r, vbase = j * p.m + 1;
-                    const uint32_t mask = extract_bits(inc, vbase, mj);
-                    T acc = in_s[(size_t)renumber(v, root) * p.k + e];
-                    const bool from_root = j == p.q && sc < troot;
-                    if (from_root) acc = Comb<T, OP>::f(acc, in_s[(size_t)root * p.k + e]);
-                    for (uint32_t sp = 0; sp < mj; ++sp)
-                        if (sp != sc && ((mask >> sp) & 1u)) acc = Comb<T, OP>::f(acc, in_s[(size_t)renumber(vbase + sp, root) * p.k + e]);
-                    uint32_t fb = 0, nf = mj - __popc(mask) + ((j == p.q && !from_root) ? 1u : 0u);   // partners whose message did not arrive
-                    for (uint64_t c = (uint64_t)p.arity * j + 1; c <= (uint64_t)p.arity * j + p.arity && c < G; ++c) {
-                        if (pres[c]) { acc = Comb<T, OP>::f(acc, val[(size_t)c * p.k + e]); fb |= fbit[c]; nf += nfl[c]; }
-                        else { fb = 1; nf += 1; }
-                    }
-                    val[(size_t)j * p.k + e] = acc;
-                    if (e == 0) { pres[j] = 1; fbit[j] = fb; nfl[j] = nf; }
+            // one node: its group's fold as member sc holds it (own input, then what arrived, in the partner order),
+            // then its children in ascending order; a child that sent nothing sets the failed bit
+            auto node = [&](uint32_t j, uint32_t e) {
+                const uint32_t v = j * p.m + sc + 1;
+                if (!test_bit(snd, v)) { if (e == 0) { pres[j] = 0; fbit[j] = 0; nfl[j] = 0; } return; }
+                const uint32_t mj = j < p.q ? p.m : p.r, vbase = j * p.m + 1;
+                const uint32_t mask = extract_bits(inc, vbase, mj);
+                T acc = in_s[(size_t)renumber(v, root) * p.k + e];
+                // the root's up-correction send to member sc of its group is its send number sc (descending: r-1-sc)
+                const bool from_root = j == p.q && (p.pdesc ? p.r - 1 - sc : sc) < troot;
+                if (from_root && !p.pdesc) acc = Comb<T, OP>::f(acc, in_s[(size_t)root * p.k + e]);
+                for (uint32_t i = 0; i < mj; ++i) {
+                    const uint32_t sp = p.pdesc ? mj - 1 - i : i;
+                    if (sp != sc && ((mask >> sp) & 1u)) acc = Comb<T, OP>::f(acc, in_s[(size_t)renumber(vbase + sp, root) * p.k + e]);
                 }
-                __syncthreads();
+                if (from_root && p.pdesc) acc = Comb<T, OP>::f(acc, in_s[(size_t)root * p.k + e]);
+                uint32_t fb = 0, nf = mj - __popc(mask) + ((j == p.q && !from_root) ? 1u : 0u);   // partners whose message did not arrive
+                auto child = [&](uint64_t c) {
+                    if (pres[c]) { acc = Comb<T, OP>::f(acc, val[(size_t)c * p.k + e]); fb |= fbit[c]; nf += nfl[c]; }
+                    else { fb = 1; nf += 1; }
+                };
+                if (p.arity == 1) { for (uint64_t bit = 1; (j == 0 || bit < (j & (0u - j))) && j + bit < G; bit <<= 1) child(j + bit); }
+                else for (uint64_t c = (uint64_t)p.arity * j + 1; c <= (uint64_t)p.arity * j + p.arity && c < G; ++c) child(c);
+                val[(size_t)j * p.k + e] = acc;
+                if (e == 0) { pres[j] = 1; fbit[j] = fb; nfl[j] = nf; }
+            };
+            if (p.arity == 1) {
+                // binomial subtrees: a level's nodes are those with that many set bits
+                for (int lvl = (int)p.H - 1; lvl >= 0; --lvl) {
+                    for (uint32_t u = tid; u < G * p.k; u += nt)
+                        if (__popc(u / p.k) == lvl) node(u / p.k, u % p.k);
+                    __syncthreads();
+                }
+            } else {
+                for (int lvl = (int)heap_level(p.arity, G - 1); lvl >= 0; --lvl) {
+                    const uint32_t lo = (uint32_t)heap_level_start(p.arity, lvl);
+                    const uint32_t hi = (uint32_t)min(heap_level_start(p.arity, lvl + 1), (uint64_t)G);
+                    for (uint32_t u = tid; u < (hi - lo) * p.k; u += nt) node(lo + u / p.k, u % p.k);
+                    __syncthreads();
+                }
             }
             for (uint32_t e = tid; e < p.k; e += nt) cand_s[(size_t)sc * p.k + e] = pres[0] ? val[e] : T(0);
             if (tid == 0) { info_s[2 * sc] = pres[0] ? fbit[0] : 2u; info_s[2 * sc + 1] = pres[0] ? nfl[0] : 0u; }

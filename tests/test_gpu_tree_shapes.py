@@ -101,9 +101,7 @@ def test_expanded_candidates_messages_and_noalloc(arity):
             d_cand = torch.zeros((S, f + 1, k), dtype=d_x.dtype, device="cuda")
             d_info = torch.zeros((S, f + 1, 2), dtype=torch.int32, device="cuda")
             d_ws = torch.empty(B.ftc_candidates_workspace_bytes(desc, S), dtype=torch.uint8, device="cuda")
-            rc = B.ftc_candidates_batch(desc, S, allreduce, d_x, to_dev(pf), to_dev(inop), to_dev(roots), d_cand, d_info, d_ws,
-                                        check=False)
-            assert rc == (B.FTC_EUNSUPPORTED if arity == 1 else B.FTC_OK)        # binomial subtrees: not in this call
+            B.ftc_candidates_batch(desc, S, allreduce, d_x, to_dev(pf), to_dev(inop), to_dev(roots), d_cand, d_info, d_ws)
             # message counts
             d_msgs = torch.zeros((S, B.FTC_MSG_WORDS), dtype=torch.int64, device="cuda")
             B.ftc_message_counts_batch(desc, S, allreduce, to_dev(pf), to_dev(inop), to_dev(roots), d_msgs.view(torch.uint64))
@@ -111,7 +109,7 @@ def test_expanded_candidates_messages_and_noalloc(arity):
             cand, info, msgs = to_host(d_cand, x.dtype), d_info.cpu().numpy(), d_msgs.cpu().numpy().view(np.uint64)
             for i, d in enumerate(ref):
                 assert np.array_equal(msgs[i], d["msgs"]), (P, f, i, msgs[i], d["msgs"])
-                if d["attempts"] == 0 or arity == 1:
+                if d["attempts"] == 0:
                     continue
                 assert np.array_equal(info[i, :, 0], d["cand_flag"]) and np.array_equal(info[i, :, 1], d["cand_nfail"]), (P, f, i)
                 assert np.array_equal(cand[i].view(np.uint8), d["cand"].view(np.uint8)), (P, f, i)
@@ -187,8 +185,17 @@ def test_descending_partners(arity, allreduce):
         msgs = d_msgs.cpu().numpy().view(np.uint64)
         ref = [O.run(x[i], f, "sum", pf[i], inop=[tuple(e) for e in inop[i]], root=int(roots[i]), allreduce=allreduce, detail=True,
                      arity=arity, partners_descending=True) for i in range(S)]
+        d_cand = torch.zeros((S, f + 1, k), dtype=torch.float32, device="cuda")
+        d_info = torch.zeros((S, f + 1, 2), dtype=torch.int32, device="cuda")
+        d_cws = torch.empty(B.ftc_candidates_workspace_bytes(desc, S), dtype=torch.uint8, device="cuda")
+        B.ftc_candidates_batch(desc, S, allreduce, to_dev(x), to_dev(pf), to_dev(inop), to_dev(roots), d_cand, d_info, d_cws)
+        torch.cuda.synchronize()
+        cand, info = d_cand.cpu().numpy(), d_info.cpu().numpy()
         for i, d in enumerate(ref):
             assert np.array_equal(msgs[i], d["msgs"]), (P, f, i)
+            if d["attempts"]:
+                assert np.array_equal(info[i, :, 0], d["cand_flag"]) and np.array_equal(info[i, :, 1], d["cand_nfail"]), (P, f, i)
+                assert np.array_equal(cand[i].view(np.uint8), d["cand"].view(np.uint8)), (P, f, i)
         if allreduce:
             desc_e = B.make_desc(P, f, k, B.FTC_F32, "sum", root=-1, max_inop=2, flags=flags | B.FTC_OUT_EXPANDED)
             d_out = torch.zeros((S, P, k), dtype=torch.float32, device="cuda")
