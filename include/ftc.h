@@ -69,7 +69,8 @@ enum { FTC_SUM = 0, FTC_MAX = 1, FTC_XOR = 2 };   /* integer sums wrap; FTC_F32 
 enum {
     FTC_OK = 0,
     FTC_EINVAL = -1,        /* P < f+2, k = 0, root >= P, NULL or misaligned required pointer, f > 31, max_inop > 32, tree arity 1 or > 32 */
-    FTC_EUNSUPPORTED = -2,  /* unknown dtype/op, xor or max on f32 */
+    FTC_EUNSUPPORTED = -2,  /* unknown dtype/op, xor or max on f32, expanded output for so many processes that its bitmasks
+                               exceed shared memory */
     FTC_EWORKSPACE = -3,    /* workspace missing or smaller than ftc_workspace_bytes() */
     FTC_ECUDA = -4,         /* a CUDA call or launch failed */
     FTC_ETOOLARGE = -5      /* ftc_reduce_batch_noalloc: the shape does not fit the built-in scratch */
@@ -83,7 +84,8 @@ enum {
     FTC_ST_NO_LIVE_ROOT_CANDIDATE = 3,  /* allreduce: all f+1 candidates had failed before the operation */
     FTC_ST_PRECONDITION_INOP_ROOT = 4,  /* allreduce: a root candidate is listed as failing in-operation */
     FTC_ST_BAD_ROOT = 5,                /* d_roots[s] >= P */
-    FTC_ST_INTERNAL_TIMEOUT = 6         /* a bounded wait inside the kernel ran out; the scenario's result is not valid */
+    FTC_ST_INTERNAL_TIMEOUT = 6         /* a bounded wait for a copy inside the kernel ran out: this scenario and every later one
+                                           that the same thread block plays report this outcome; results are zero bytes */
 };
 
 /*
@@ -116,6 +118,10 @@ typedef struct { uint32_t victim; uint32_t round; } ftc_inop_t;
                                             order open (general kernel) */
 #define FTC_KERNEL_GENERIC 0x100u /* force the general level-by-level kernel (needs the workspace) */
 #define FTC_KERNEL_DIRECT  0x200u /* force the register-tiled kernel (direct global loads) where the shape allows it */
+#define FTC_DEBUG_ONE_POLL 0x4000000u /* testing aid: the kernel's bounded waits for its asynchronous copies look once instead of
+                                         polling, so most of them give up and the give-up path runs: affected scenarios report
+                                         FTC_ST_INTERNAL_TIMEOUT with zero bytes, nothing waits without a limit and nothing is read
+                                         or written out of bounds. Never set it in production calls */
 
 typedef struct {
     uint32_t P;         /* processes, P >= f+2 (the root needs f+1 children: definition of the I(f)-tree) */
@@ -146,7 +152,7 @@ typedef struct {
  *   d_inop    [S][max_inop] or NULL when max_inop = 0
  *   d_roots   [S] or NULL; read only when desc->root < 0
  *   d_out     [S][k]: the value delivered at the root (zeros unless the outcome is FTC_ST_OK); 16-byte aligned
- *   d_status  [S][FTC_STATUS_WORDS]
+ *   d_status  [S][FTC_STATUS_WORDS] uint32; 16-byte aligned (one record is stored as one 16-byte word)
  *   d_workspace, workspace_bytes: scratch of at least ftc_workspace_bytes(desc, S, 0) bytes (may be NULL if that is 0),
  *             16-byte aligned; contents are undefined afterwards; calls that share a workspace must not overlap on
  *             the device. Shapes that run on the shared-memory kernels also run with less or none (large process
@@ -186,7 +192,9 @@ FTC_API int ftc_allreduce_batch(const ftc_desc_t* desc, uint64_t S, const void* 
  *   - Limit: one block's slice, ceil((P-1)/(f+1)) * k * element size bytes, must fit the array; otherwise
  *     FTC_ETOOLARGE is returned and nothing is enqueued.
  *   - The first call on each device looks the array's device address up (one runtime query, with that device
- *     current). Make that first call before starting any stream capture on that device.
+ *     current) and keeps it for the life of the process. Make that first call before starting any stream capture
+ *     on that device. The address belongs to the device's primary context: a host program that destroys that
+ *     context (cudaDeviceReset) must not call this entry point on that device afterwards.
  *   - All calls on a device share the one array, which keeps whatever the previous call left in it. Nothing in it
  *     needs clearing: within a scenario every slot is written before it is read. But two calls whose kernels can
  *     overlap on the same GPU (different streams, or different host threads) race on it: serialise them.
@@ -275,6 +283,17 @@ FTC_API int ftc_fill_inputs(uint32_t kind, uint64_t seed, uint64_t first_scenari
 
 /* Name of the kernel family the batch calls would use for this descriptor: "staged", "tiled" or "generic". */
 FTC_API const char* ftc_kernel_name(const ftc_desc_t* desc, int is_allreduce);
+
+/* The same, down to the instantiation of the shared-memory kernel: "staged/whole" (scenario staged by one copy),
+ * "staged/lean" (blocks of one or two warps), "staged/large" (4-8 warps), "staged/batched-lean" (4-8 warps, groups of at
+ * most 128 bytes, exact operations), "staged/lean-swz" and "staged/batched-swz" (float32 vectors of 16 or 32 bytes, tiles
+ * by swizzled tensor copies), "staged/whole-large", "tiled", "generic"; assuming the workspace ftc_workspace_bytes() asks for. */
+FTC_API const char* ftc_kernel_variant(const ftc_desc_t* desc, int is_allreduce);
+
+/* Thread blocks the batch calls would launch for S scenarios on the current device (given the workspace
+ * ftc_workspace_bytes() asks for). Block b plays scenarios b, b + blocks, b + 2*blocks, ... one after the other; a batch
+ * keeps the whole GPU busy when S is a few times this number. Needs a device. Launches nothing. */
+FTC_API int ftc_launch_blocks(const ftc_desc_t* desc, uint64_t S, int is_allreduce, uint32_t* blocks);
 
 FTC_API const char* ftc_strerror(int code);
 FTC_API uint32_t ftc_version(void);

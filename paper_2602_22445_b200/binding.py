@@ -35,12 +35,13 @@ def FTC_TREE_ARITY(a: int) -> int:
     return (a & 0xFF) << 16
 
 FTC_KERNEL_DIRECT = 0x200
+FTC_DEBUG_ONE_POLL = 0x4000000
 OPS = {"sum": FTC_SUM, "max": FTC_MAX, "xor": FTC_XOR}
 
 EXPORTS = ["ftc_reduce_batch", "ftc_allreduce_batch", "ftc_reduce_batch_noalloc", "ftc_candidates_batch",
            "ftc_candidates_workspace_bytes", "ftc_message_counts_batch", "ftc_workspace_bytes", "ftc_reduce_batch_host",
            "ftc_allreduce_batch_host", "ftc_host_staging_bytes", "ftc_schedule_info", "ftc_fill_inputs",
-           "ftc_kernel_name", "ftc_strerror", "ftc_version"]
+           "ftc_kernel_name", "ftc_kernel_variant", "ftc_launch_blocks", "ftc_strerror", "ftc_version"]
 
 
 class ftc_desc_t(C.Structure):
@@ -95,6 +96,10 @@ def load():
     lib.ftc_fill_inputs.argtypes = [u32, u64, u64, u64, u32, u32, vp, vp]
     lib.ftc_kernel_name.restype = C.c_char_p
     lib.ftc_kernel_name.argtypes = [dp, C.c_int]
+    lib.ftc_kernel_variant.restype = C.c_char_p
+    lib.ftc_kernel_variant.argtypes = [dp, C.c_int]
+    lib.ftc_launch_blocks.restype = C.c_int
+    lib.ftc_launch_blocks.argtypes = [dp, u64, C.c_int, C.POINTER(u32)]
     lib.ftc_strerror.restype = C.c_char_p
     lib.ftc_strerror.argtypes = [C.c_int]
     lib.ftc_version.restype = u32
@@ -155,6 +160,18 @@ def ftc_version() -> int:
 
 def ftc_kernel_name(desc, is_allreduce=False) -> str:
     return load().ftc_kernel_name(C.byref(desc), int(is_allreduce)).decode()
+
+
+def ftc_kernel_variant(desc, is_allreduce=False) -> str:
+    return load().ftc_kernel_variant(C.byref(desc), int(is_allreduce)).decode()
+
+
+def ftc_launch_blocks(desc, S, is_allreduce=False) -> int:
+    out = C.c_uint32(0)
+    rc = load().ftc_launch_blocks(C.byref(desc), S, int(is_allreduce), C.byref(out))
+    if rc != FTC_OK:
+        raise FtcError(rc, "ftc_launch_blocks")
+    return out.value
 
 
 def ftc_workspace_bytes(desc, S, is_allreduce=False) -> int:

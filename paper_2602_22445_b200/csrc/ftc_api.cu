@@ -120,6 +120,7 @@ static int run_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const
     if ((rc = device_info(di)) != FTC_OK) return rc;
     const size_t front = compact_area(p);
     if (expanded && (!d_ws || ws_bytes < front || (reinterpret_cast<uintptr_t>(d_ws) & 255u))) return FTC_EWORKSPACE;
+    if (expanded && expand_smem_bytes(p) > (size_t)di.smem_optin) return FTC_EUNSUPPORTED;   // before anything is enqueued
     p.in = d_in; p.prefail = d_prefail; p.inop = d_inop; p.roots = d_roots; p.status = d_status;
     p.out = expanded ? d_ws : d_out;                            // compact results first, expanded afterwards
     if (expanded) { d_ws = static_cast<char*>(d_ws) + front; ws_bytes -= front; }
@@ -346,6 +347,35 @@ const char* ftc_kernel_name(const ftc_desc_t* desc, int is_allreduce) {
     p.ws_bytes = ~0ull;                                   // given the workspace ftc_workspace_bytes() asks for
     const KernelKind kind = pick_kernel(p, di);
     return kind == K_STAGED ? "staged" : kind == K_TILED ? "tiled" : "generic";
+}
+
+const char* ftc_kernel_variant(const ftc_desc_t* desc, int is_allreduce) {
+    Params p;
+    if (fill_params(desc, 1, is_allreduce, p) != FTC_OK) return "invalid";
+    DeviceInfo di;
+    if (device_info(di) != FTC_OK) di = kB200;
+    p.ws_bytes = ~0ull;
+    const KernelKind kind = pick_kernel(p, di);
+    if (kind == K_STAGED) return staged_variant(p, type_select(desc->dtype, desc->op), di.smem_optin, di.sm_count, nullptr);
+    return kind == K_TILED ? "tiled" : "generic";
+}
+
+int ftc_launch_blocks(const ftc_desc_t* desc, uint64_t S, int is_allreduce, uint32_t* blocks) {
+    Params p;
+    int rc = fill_params(desc, S, is_allreduce, p);
+    if (rc != FTC_OK) return rc;
+    if (!blocks) return FTC_EINVAL;
+    *blocks = 0;
+    if (S == 0) return FTC_OK;
+    DeviceInfo di;
+    if ((rc = device_info(di)) != FTC_OK) return rc;
+    p.ws_bytes = ~0ull;
+    p.grid_query = blocks;
+    const int tsel = type_select(desc->dtype, desc->op);
+    const KernelKind kind = pick_kernel(p, di);
+    cudaError_t e = kind == K_STAGED ? launch_staged(p, tsel, di.sm_count, di.smem_optin, nullptr)
+                  : kind == K_TILED ? launch_tiled(p, tsel, di.sm_count, nullptr) : launch_generic(p, tsel, di.sm_count, nullptr);
+    return e == cudaSuccess ? FTC_OK : FTC_ECUDA;
 }
 
 const char* ftc_strerror(int code) {

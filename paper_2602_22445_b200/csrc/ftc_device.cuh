@@ -35,6 +35,7 @@ struct Params {
     uint32_t swz_mask; // swizzled tiles: XOR mask of the 16-byte chunk bits (0x70: 128-byte lines, 0x30: 64-byte lines)
     uint32_t row_shift; // swizzled tiles of 64-byte groups: tile rows after the first sit one row further (128-byte aligned levels)
     uint32_t below;    // 1: the heap's sparsely filled last level lies below the tiles (its rows are folded one by one)
+    uint32_t* grid_query;  // host side only: when set, a launcher stores the number of blocks it would launch and launches nothing
 };
 
 // Per-scenario facts, in shared memory.
@@ -50,7 +51,7 @@ struct Ctx {
     uint32_t holders;
     uint32_t ndead_end; // in-operation victims (not pre-failed) that are dead at the end of the attempt
     uint32_t unreached_lost;
-    uint32_t pad;       // set when a bounded wait gave up
+    uint32_t reserved;
     uint32_t iv[FTC_MAX_INOP];   // victim (physical id) per slot, FTC_INOP_UNUSED if the slot does not count
     uint32_t ir[FTC_MAX_INOP];   // its failure round on the global clock (minimum over slots naming it)
     uint32_t ifirst;             // bit i: slot i is the first slot naming its victim
@@ -145,7 +146,7 @@ static __device__ void decode_scenario(const Params& p, uint64_t s, Ctx* cx, uin
     if (tid == 0) {
         cx->Fmask = 0; cx->npre = 0; cx->nexcl = 0; cx->inop_incl = 0; cx->holders = 0; cx->ndead_end = 0;
         cx->unreached_lost = 0; cx->code = FTC_ST_OK; cx->sstar = 0xFF; cx->attempts = 0; cx->base = 0; cx->root = 0;
-        cx->G = 0; cx->ifirst = 0; cx->pad = 0;
+        cx->G = 0; cx->ifirst = 0;
         pf[p.W] = 0; inc[p.W] = 0;
     }
     if (tid < FTC_MAX_INOP) {

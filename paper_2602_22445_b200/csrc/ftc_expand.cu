@@ -31,8 +31,10 @@ __global__ void __launch_bounds__(256) expand_kernel(Params p, const V* compact,
     }
 }
 
+size_t expand_smem_bytes(const Params& p) { return sizeof(Ctx) + 4 * (size_t)(p.W + 1) * 4; }
+
 cudaError_t launch_expand(const Params& p, const void* compact, void* out, int sm_count, cudaStream_t st) {
-    const size_t smem = sizeof(Ctx) + 4 * (size_t)(p.W + 1) * 4;
+    const size_t smem = expand_smem_bytes(p);
     const uint64_t cap = (uint64_t)sm_count * 8;
     const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
     cudaError_t e;

@@ -163,6 +163,7 @@ uint32_t generic_grid(const Params& p, int sm_count) {
 template <typename T, int OP, bool VEC>
 static cudaError_t launch_generic_v(const Params& p, uint32_t grid, cudaStream_t st) {
     size_t smem = generic_smem_bytes(p);
+    if (p.grid_query) { *p.grid_query = grid; return cudaSuccess; }
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(generic_kernel<T, OP, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;

@@ -30,6 +30,8 @@ cudaError_t launch_tiled(const Params& p, int tsel, int sm_count, cudaStream_t s
 bool staged_supported(Params& p, int smem_optin_bytes, int sm_count);
 size_t staged_workspace_bytes(Params p, int smem_optin_bytes, int sm_count);
 cudaError_t launch_staged(const Params& p, int tsel, int sm_count, int smem_optin_bytes, cudaStream_t st);
+// Name of the instantiation launch_staged would run ("staged/lean", ...); p.S and p.ws_bytes matter.
+const char* staged_variant(Params p, int tsel, int smem_optin_bytes, int sm_count, uint32_t* grid_cap_blocks_per_sm);
 
 // Every root child's delivery (value, flag, failed-list size): general kernel, workspace slices of candidates_slice_bytes().
 size_t candidates_slice_bytes(const Params& p);
@@ -40,6 +42,7 @@ size_t messages_smem_bytes(const Params& p);
 cudaError_t launch_messages(const Params& p, unsigned long long* out, int sm_count, cudaStream_t st);
 
 // Expanded allreduce output from the compact results (one value per scenario) left by the main kernel.
+size_t expand_smem_bytes(const Params& p);
 cudaError_t launch_expand(const Params& p, const void* compact, void* out, int sm_count, cudaStream_t st);
 
 cudaError_t launch_fill(uint32_t kind, uint64_t seed, uint64_t first, uint64_t S, uint32_t P, uint32_t k, void* out,

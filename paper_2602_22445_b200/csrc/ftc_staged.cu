@@ -25,6 +25,13 @@ size_t staged_workspace_bytes(Params p, int smem_optin_bytes, int sm_count) {
     return (size_t)sm_count * kHvGlobalBlocksPerSm * (size_t)g.hv_bytes;
 }
 
+const char* staged_variant(Params p, int tsel, int smem_optin_bytes, int sm_count, uint32_t* grid_cap_blocks_per_sm) {
+    StagedGeom g;
+    const StagedVariant v = staged_plan(p, tsel == TS_F32_SUM, true, staged_xl(p), smem_optin_bytes, sm_count, g);
+    if (grid_cap_blocks_per_sm) *grid_cap_blocks_per_sm = g.hv_global ? (uint32_t)kHvGlobalBlocksPerSm : 0u;
+    return staged_variant_name(v);
+}
+
 cudaError_t launch_staged(const Params& p, int tsel, int sm_count, int smem_optin, cudaStream_t st) {
     switch (tsel) {
     case TS_U32_SUM: return launch_staged_u32_sum(p, sm_count, smem_optin, st);

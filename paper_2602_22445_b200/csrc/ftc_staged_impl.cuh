@@ -43,11 +43,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after kWaitTries polls and reports it; the caller flags the scenario and carries on so
-// that block-wide barriers stay matched.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after `tries` polls and says so. A caller whose wait gave up never arms or waits on that
+// barrier again except for one last bounded wait before the block ends (the copy may still be in flight), marks the
+// block (sticky flag in shared memory) and lets every scenario the block still plays end as FTC_ST_INTERNAL_TIMEOUT.
+// tries = 1 (FTC_DEBUG_ONE_POLL) polls once without suspending, so that the give-up path can be exercised.
 constexpr uint32_t kWaitTries = 1u << 22;
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitTries; ++i)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t tries) {
+    if (tries == 1) return mbar_test_wait(bar, parity);
+    for (uint32_t i = 0; i < tries; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -61,7 +70,7 @@ __host__ __device__ inline uint32_t nitems_words(uint32_t Lt, uint32_t lw) {
 struct StagedGeom {
     uint32_t nwarps, nbuf, tile_cap;       // warps per block, buffers per warp, bytes per buffer (multiple of 128)
     uint32_t whole;                        // 1: the whole scenario is staged in one block-wide buffer
-    uint32_t off_special, off_rootv, off_hv, off_bar, off_tiles, smem_bytes;
+    uint32_t off_special, off_rootv, off_hv, off_bar, off_gaveup, off_tiles, smem_bytes;
     uint32_t hv_global;                    // 1: the heap array of tile roots and upper rows lives in the workspace
     uint64_t hv_bytes;                     // its size per block
 };
@@ -339,12 +348,18 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
     char* tiles = sbase + g.off_tiles + (size_t)wid * g.nbuf * g.tile_cap;
     const uint32_t cbar = smem_addr(sbase + g.off_bar) + g.nwarps * g.nbuf * 8;   // block-wide barrier (WHOLE)
     char* wbuf = sbase + g.off_tiles;                                            // block-wide scenario copy (WHOLE)
+    // set, and never cleared, once a bounded wait of this block gave up (decode_scenario does not touch it)
+    volatile uint32_t* gaveup = reinterpret_cast<volatile uint32_t*>(sbase + g.off_gaveup);
+    const uint32_t tries = (p.flags & FTC_DEBUG_ONE_POLL) ? 1u : kWaitTries;
     if (lane < g.nbuf) mbar_init(bar0 + lane * 8, 1);
     if (WHOLE && tid == 0) mbar_init(cbar, 1);
+    if (tid == 0) *gaveup = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
     uint32_t phase_bits = 0;                                      // bit b: parity to wait for on buffer b
     uint32_t cphase = 0;
+    bool cfail = false;                                           // WHOLE: this thread's wait for the block-wide copy gave up
+    bool stop = false;                                            // this warp issues no further copies (a wait of the block gave up)
 
     // ---- the copy pipeline of this warp: it runs over the flat sequence (scenario, work item) of everything the
     // warp will process, g.nbuf items ahead of the item being computed, across scenario boundaries. What is copied
@@ -357,7 +372,7 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
     // lane t copies level t of a tile: 2^t rows, placed after the 2^t - 1 rows of the levels above
     const uint32_t lvl_rows = lane < D ? 1u << lane : 0u, lvl_dst = (lvl_rows ? lvl_rows - 1 : 0u) * rowbytes;
     auto issue_next = [&]() {
-        if (WHOLE || n_my == 0 || is_s >= p.S) return;
+        if (WHOLE || n_my == 0 || is_s >= p.S || stop) return;
         const uint32_t it = wid + is_i * nw, b = ibuf;
         uint32_t first_row = 0, nrows = 0, dst_off = 0;
         if (it < ntiles) {
@@ -404,12 +419,20 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
         if (++ibuf == g.nbuf) ibuf = 0;
         if (++is_i == n_my) { is_i = 0; is_s += gridDim.x; is_src += (uint64_t)gridDim.x * scen_bytes; }
     };
-    // the buffer of the item about to be computed: wait for its copy if one was issued
+    // the buffer of the item about to be computed: wait for its copy if one was issued. A warp whose wait gave up
+    // keeps the buffer marked as in flight (its barrier's phase never completed: it is not armed or waited on again
+    // before the last wait at the end of the kernel), stops issuing and waiting, and marks the block.
     auto acquire = [&]() {
         const uint32_t b = WHOLE ? 0u : cbuf;
-        if (!WHOLE && ((pending >> b) & 1u)) {
-            if (!mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u)) { if (lane == 0) atomicOr(&cx->pad, 1u); }
-            phase_bits ^= 1u << b; pending &= ~(1u << b);
+        if (!WHOLE && ((pending >> b) & 1u) && !stop) {
+            bool ok = mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u, tries);
+            if (!__all_sync(0xFFFFFFFFu, ok)) {
+                // a lane that saw the phase complete proves the copy landed: the others look once more (returns at once)
+                if (__any_sync(0xFFFFFFFFu, ok) && !ok) ok = mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u, kWaitTries);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+            }
+            if (ok) { phase_bits ^= 1u << b; pending &= ~(1u << b); }
+            else { stop = true; if (lane == 0) atomicOr(const_cast<uint32_t*>(gaveup), 1u); }
         }
         return b;
     };
@@ -419,7 +442,10 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
 
     for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {
         const char* in_s = reinterpret_cast<const char*>(p.in) + s * scen_bytes;
-        if (WHOLE && wid == 0) {
+        // uniform: the flag is only written between the barriers of a scenario, and a barrier ended the previous one
+        const bool dead = *gaveup != 0;
+        if (dead) stop = true;
+        if (WHOLE && wid == 0 && !dead) {
             // the whole scenario, in pieces of at most 32 KB, lands while the masks are decoded
             if (lane == 0) mbar_expect_tx(cbar, (uint32_t)scen_bytes);
             __syncwarp();
@@ -428,15 +454,19 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
         }
         decode_scenario(p, s, cx, pf, inc);
         char* out_s = reinterpret_cast<char*>(p.out) + s * p.kbytes;
-        if (WHOLE) {
+        if (WHOLE && !dead) {
             // every thread sees the copy complete before it reads it or leaves the iteration
-            if (!mbar_wait_bounded(cbar, cphase)) atomicOr(&cx->pad, 1u);
-            cphase ^= 1u;
+            if (mbar_wait_bounded(cbar, cphase, tries)) cphase ^= 1u;
+            else { cfail = true; atomicOr(const_cast<uint32_t*>(gaveup), 1u); }
         }
-        if (cx->code != FTC_ST_OK) {
+        if (cx->code != FTC_ST_OK || dead) {
             if (tid < p.C) reinterpret_cast<uint4*>(out_s)[tid] = make_uint4(0, 0, 0, 0);
             for (uint32_t i = 0; i < n_my; ++i) { acquire(); release(); }        // its copies were issued: consume them unused
-            if (tid == 0) write_status_rec(p, s, cx);
+            __syncthreads();                                                     // a wait that gave up just now is seen by thread 0
+            if (tid == 0) {
+                if (*gaveup) cx->code = FTC_ST_INTERNAL_TIMEOUT;
+                write_status_rec(p, s, cx);
+            }
             __syncthreads();
             continue;
         }
@@ -524,16 +554,26 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
             __syncthreads();
         }
         // ---- the root (Algorithm "reduce_root") ----
+        // a wait that gave up during this scenario was flagged before the barrier that followed the work items:
+        // every thread reads the same value here; the result is then not valid and zero bytes are written instead
+        const bool bad = *gaveup != 0;
         if (tid < p.C) {
             uint4 recv = hv[tid];
-            reinterpret_cast<uint4*>(out_s)[tid] = sstar < p.r ? recv : comb16<T, OP>(rootv[tid], recv);
+            recv = sstar < p.r ? recv : comb16<T, OP>(rootv[tid], recv);
+            reinterpret_cast<uint4*>(out_s)[tid] = bad ? make_uint4(0, 0, 0, 0) : recv;
         }
         if (tid == 0) {
-            if (cx->pad) cx->code = FTC_ST_INTERNAL_TIMEOUT;
+            if (bad) cx->code = FTC_ST_INTERNAL_TIMEOUT;
             write_status_rec(p, s, cx);
         }
         __syncthreads();
     }
+    // Only after a wait gave up: a copy may still be in flight toward this block's shared memory. One more bounded
+    // wait per such buffer before the block ends and the SM hands the memory to another block.
+    if (!WHOLE) {
+        for (uint32_t b = 0; b < g.nbuf; ++b)
+            if ((pending >> b) & 1u) mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u, kWaitTries);
+    } else if (cfail) mbar_wait_bounded(cbar, cphase, kWaitTries);
 }
 
 // ---- host side ----
@@ -588,6 +628,7 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
                    p.ws_bytes / ((uint64_t)sm_count * kHvGlobalBlocksPerSm) >= g.hv_bytes) ? 1u : 0u;
     g.off_hv = (uint32_t)o; if (!g.hv_global) o += (size_t)g.hv_bytes;
     g.off_bar = (uint32_t)o; o += (size_t)(kStagedMaxThreads / 32) * 4 * 8 + 8;      // room for any warps x nbuf, plus one
+    g.off_gaveup = (uint32_t)o; o += 8;
     o = (o + 127) & ~(size_t)127; g.off_tiles = (uint32_t)o;
     if (g.whole) {
         o += (size_t)((scen_bytes + 127) & ~(uint64_t)127);
@@ -629,48 +670,86 @@ static cudaError_t launch_staged_w(const Params& p, const StagedGeom& g, int sm_
     if (g.hv_global && per_sm > kHvGlobalBlocksPerSm) per_sm = kHvGlobalBlocksPerSm;      // one workspace slice per block
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
+    if (p.grid_query) { *p.grid_query = grid; return cudaSuccess; }
     staged_kernel<T, OP, XL, WHOLE, MINB><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g, maps);
     return cudaGetLastError();
+}
+
+// Which instantiation plays a shape. The names are what ftc_kernel_variant() reports.
+enum StagedVariant { SV_NONE = 0, SV_WHOLE, SV_WHOLE_LARGE, SV_LEAN, SV_LEAN_SWZ, SV_BATCHED_LEAN, SV_BATCHED_SWZ, SV_LARGE };
+static inline const char* staged_variant_name(StagedVariant v) {
+    switch (v) {
+    case SV_WHOLE: return "staged/whole";
+    case SV_WHOLE_LARGE: return "staged/whole-large";
+    case SV_LEAN: return "staged/lean";
+    case SV_LEAN_SWZ: return "staged/lean-swz";
+    case SV_BATCHED_LEAN: return "staged/batched-lean";
+    case SV_BATCHED_SWZ: return "staged/batched-swz";
+    case SV_LARGE: return "staged/large";
+    default: return "none";
+    }
+}
+
+// Can the batch be described by the tensor maps of the swizzled variant (everything but the driver's own checks)?
+static inline bool staged_tensor_maps_possible(const Params& p, uint32_t D) {
+    const uint64_t rowbytes = (uint64_t)p.m * p.kbytes, line = p.swz_mask == 0x70u ? 128 : 64;
+    const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
+    if (D > 8 || p.q == 0 || scen_bytes % 16 || rowbytes % line) return false;
+    return ((rowbytes / line) << (D - 1)) <= 256;
+}
+
+// Geometry and instantiation for a shape; `ordered`: the combine order is observable (float32); `allow_swz`: the
+// swizzled variants may be chosen (the launch retries without them when the driver refuses a tensor map).
+static StagedVariant staged_plan(Params& p, bool ordered, bool allow_swz, uint32_t XL, int smem_optin, int sm_count, StagedGeom& g) {
+    // float32 with vectors of 16 or 32 bytes: the fold order is fixed, so the rows of different lane rows would meet in
+    // the same banks when groups are a multiple of 128 bytes or 64 bytes (4- and 8-way conflicts); their tiles come in
+    // by tensor copies with the matching swizzle instead
+    const uint64_t gbytes = (uint64_t)p.m * p.kbytes;
+    bool swizzled = allow_swz && ordered && p.kbytes <= 32 && (gbytes % 128 == 0 || gbytes == 64) && p.S < (1ull << 31) &&
+                    (uint64_t)p.P * p.kbytes > kWholeMaxBytes;
+    p.swz_mask = 0; p.row_shift = 0;
+    if (swizzled) { p.swz_mask = gbytes == 64 ? 0x30u : 0x70u; p.row_shift = gbytes == 64 ? 1u : 0u; }
+    if (swizzled && !(staged_geometry(p, smem_optin, sm_count, XL, g) && !g.whole && staged_tensor_maps_possible(p, (5 - p.cw_log2) + XL))) {
+        swizzled = false; p.swz_mask = 0; p.row_shift = 0;
+    }
+    if (!swizzled && !staged_geometry(p, smem_optin, sm_count, XL, g)) return SV_NONE;
+    // one- and two-warp blocks get the lean variant; its register cap (about 96) matches the blocks that fit by shared
+    // memory. Scenarios staged whole are so small that many more blocks fit: for them 64 registers, so that the
+    // SM's block limit and not the register file decides
+    const bool lean = g.nwarps <= 2;
+    if (g.whole) return lean ? SV_WHOLE : SV_WHOLE_LARGE;
+    if (swizzled) return lean ? SV_LEAN_SWZ : SV_BATCHED_SWZ;
+    if (lean) return SV_LEAN;
+    // Groups of at most 128 bytes: a row is so little data that the instructions around it count, so large blocks
+    // run the lean variant's code too (rows of a lane folded together, starting members rotated). Not for float32:
+    // its bank conflicts weigh more there than the saved instructions.
+    if (!ordered && gbytes <= 128) return SV_BATCHED_LEAN;
+    return SV_LARGE;
 }
 
 template <typename T, int OP, int XL>
 static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
     StagedGeom g;
-    // float32 with vectors of 16 or 32 bytes: the fold order is fixed, so the rows of different lane rows would meet in
-    // the same banks when groups are a multiple of 128 bytes or 64 bytes (4- and 8-way conflicts); their tiles come in
-    // by tensor copies with the matching swizzle instead
-    const uint64_t gbytes = (uint64_t)p.m * p.kbytes;
-    bool swizzled = Ordered<T>::value && p.kbytes <= 32 && (gbytes % 128 == 0 || gbytes == 64) && p.S < (1ull << 31) &&
-                    (uint64_t)p.P * p.kbytes > kWholeMaxBytes;
-    if (swizzled) { p.swz_mask = gbytes == 64 ? 0x30u : 0x70u; p.row_shift = gbytes == 64 ? 1u : 0u; }
-    if (!staged_geometry(p, smem_optin, sm_count, XL, g)) {
-        if (!swizzled) return cudaErrorInvalidConfiguration;
-        swizzled = false; p.swz_mask = 0; p.row_shift = 0;
-        if (!staged_geometry(p, smem_optin, sm_count, XL, g)) return cudaErrorInvalidConfiguration;
-    }
-    // one- and two-warp blocks get the lean variant; its register cap (about 96) matches the blocks that fit by shared
-    // memory. Scenarios staged whole are so small that many more blocks fit: for them 64 registers, so that the
-    // SM's block limit and not the register file decides
-    const bool lean = g.nwarps <= 2;
-    if (g.whole) return lean ? launch_staged_w<T, OP, XL, true, 4>(p, g, sm_count, st) : launch_staged_w<T, OP, XL, true, 2>(p, g, sm_count, st);
+    StagedVariant v = staged_plan(p, Ordered<T>::value, true, XL, smem_optin, sm_count, g);
     if constexpr (Ordered<T>::value) {
-        TmaMaps maps;
-        if (swizzled && !g.whole && staged_tensor_maps(p, (5 - p.cw_log2) + XL, maps))
-            return lean ? launch_staged_w<T, OP, XL, false, kStagedLeanSwzTag>(p, g, sm_count, st, maps)
-                        : launch_staged_w<T, OP, XL, false, kStagedBatchedSwzTag>(p, g, sm_count, st, maps);
-        if (swizzled) {               // no tensor maps: the plain layout after all
-            p.swz_mask = 0; p.row_shift = 0;
-            if (!staged_geometry(p, smem_optin, sm_count, XL, g)) return cudaErrorInvalidConfiguration;
+        if (v == SV_LEAN_SWZ || v == SV_BATCHED_SWZ) {
+            TmaMaps maps = kNoMaps;
+            if (p.grid_query || staged_tensor_maps(p, (5 - p.cw_log2) + XL, maps))
+                return v == SV_LEAN_SWZ ? launch_staged_w<T, OP, XL, false, kStagedLeanSwzTag>(p, g, sm_count, st, maps)
+                                        : launch_staged_w<T, OP, XL, false, kStagedBatchedSwzTag>(p, g, sm_count, st, maps);
+            v = staged_plan(p, true, false, XL, smem_optin, sm_count, g);      // no tensor maps: the plain layout after all
         }
     }
-    if (lean) return launch_staged_w<T, OP, XL, false, kStagedLeanMinBlocks>(p, g, sm_count, st);
-    // Groups of at most 128 bytes: a row is so little data that the instructions around it count, so large blocks
-    // run the lean variant's code too (rows of a lane folded together, starting members rotated). Not for float32:
-    // its bank conflicts weigh more there than the saved instructions.
-    if constexpr (!Ordered<T>::value) {
-        if ((uint64_t)p.m * p.kbytes <= 128) return launch_staged_w<T, OP, XL, false, kStagedBatchedTag>(p, g, sm_count, st);
+    switch (v) {
+    case SV_WHOLE: return launch_staged_w<T, OP, XL, true, 4>(p, g, sm_count, st);
+    case SV_WHOLE_LARGE: return launch_staged_w<T, OP, XL, true, 2>(p, g, sm_count, st);
+    case SV_LEAN: return launch_staged_w<T, OP, XL, false, kStagedLeanMinBlocks>(p, g, sm_count, st);
+    case SV_BATCHED_LEAN:
+        if constexpr (!Ordered<T>::value) return launch_staged_w<T, OP, XL, false, kStagedBatchedTag>(p, g, sm_count, st);
+        return cudaErrorInvalidConfiguration;
+    case SV_LARGE: return launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
+    default: return cudaErrorInvalidConfiguration;
     }
-    return launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
 }
 
 typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -688,7 +767,7 @@ static bool staged_tensor_maps(const Params& p, uint32_t D, TmaMaps& maps) {
     }();
     const uint64_t rowbytes = (uint64_t)p.m * p.kbytes, line = p.swz_mask == 0x70u ? 128 : 64;
     const uint64_t lines_per_row = rowbytes / line, scen_bytes = (uint64_t)p.P * p.kbytes;
-    if (!encode || D > 8 || p.q == 0 || scen_bytes % 16 || rowbytes % line) return false;
+    if (!encode || !staged_tensor_maps_possible(p, D)) return false;
     void* base = const_cast<char*>(static_cast<const char*>(p.in)) + p.kbytes;
     const cuuint64_t dims[3] = {line / 4, (cuuint64_t)p.q * lines_per_row, (cuuint64_t)p.S};
     const cuuint64_t strides[2] = {line, scen_bytes};

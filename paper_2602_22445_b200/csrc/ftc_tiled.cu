@@ -145,6 +145,7 @@ static cudaError_t launch_tiled_t(const Params& p, int sm_count, cudaStream_t st
     if (per_sm < 1) per_sm = 1;
     uint64_t g = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < g ? p.S : g);
+    if (p.grid_query) { *p.grid_query = grid; return cudaSuccess; }
     tiled_kernel<T, OP, MCAP, MINB><<<grid, threads, smem, st>>>(p);
     return cudaGetLastError();
 }

@@ -59,6 +59,26 @@ def run_oracle(x, f, op, prefail, inop=None, roots=None, root=0, allreduce=False
                    partners_descending=partners_descending)
 
 
+def run_oracle_mt(x, f, op, prefail, inop=None, roots=None, root=0, allreduce=False, chunk=None):
+    """run_oracle over chunks of scenarios on all host cores (threads: the C call releases the interpreter lock)."""
+    import os
+    from concurrent.futures import ThreadPoolExecutor
+    S = x.shape[0]
+    cores = os.cpu_count() or 1
+    chunk = chunk or max(1, (S + 4 * cores - 1) // (4 * cores))
+    O.lib()
+    cuts = [(a, min(a + chunk, S)) for a in range(0, S, chunk)]
+
+    def work(ab):
+        a, b = ab
+        return O.batch(x[a:b], f, op, prefail[a:b], inop=None if inop is None else inop[a:b],
+                       roots=None if roots is None else roots[a:b], root=root, allreduce=allreduce)
+
+    with ThreadPoolExecutor(max_workers=cores) as ex:
+        parts = list(ex.map(work, cuts))
+    return np.concatenate([q[0] for q in parts]), np.concatenate([q[1] for q in parts])
+
+
 def assert_same(got, want, what=""):
     g_out, g_st = got[0], got[1]
     w_out, w_st = want

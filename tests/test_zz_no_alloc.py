@@ -5,19 +5,20 @@ that cannot afford the device-wide stall of an allocation, or a plug-in living i
 memory budget. For them ftc_reduce_batch_noalloc keeps the general kernel's scratch inside the library.
 The test calls it through the C ABI twice in a row -- the second call finds the first call's leftovers in
 the array -- and wants bit-identical results and status records to ftc_reduce_batch on the same inputs
-(integer and float32 alike: both run the same kernel, so no tolerance is needed).
+(integer and float32 alike: both run the same kernel, so no tolerance is needed), and to the CPU oracle,
+which shares no code with either. The second round also checks that the call took no device memory.
 """
 import numpy as np
 import pytest
 
 from paper_2602_22445_b200 import binding as B
 from paper_2602_22445_b200 import scenarios as sc
-from tests.gpu_util import run_gpu, to_dev, to_host
+from tests.gpu_util import run_gpu, run_oracle, to_dev, to_host
 
 pytestmark = pytest.mark.gpu
 
 
-def run_noalloc(x, f, op, prefail, inop=None, roots=None, root=0):
+def run_noalloc(x, f, op, prefail, inop=None, roots=None, root=0, free_unchanged=False):
     import torch
     d_x = to_dev(x)
     S, P, k = d_x.shape
@@ -29,8 +30,12 @@ def run_noalloc(x, f, op, prefail, inop=None, roots=None, root=0):
     d_out = torch.empty((S, k), dtype=d_x.dtype, device="cuda")
     d_out.view(torch.uint8).fill_(0xA5)
     d_st = torch.full((S, 4), 0x7FFFFFFF, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
     B.ftc_reduce_batch_noalloc(desc, S, d_x, d_pf, d_inop, d_roots, d_out, d_st)
     torch.cuda.synchronize()
+    if free_unchanged:                                   # the device's free memory as the driver reports it
+        assert torch.cuda.mem_get_info()[0] == free_before
     return to_host(d_out, x.dtype), d_st.cpu().numpy().view(np.uint32)
 
 
@@ -58,9 +63,12 @@ def test_noalloc_matches_workspace_entry_point_twice_in_a_row():
             f = {333: 2, 1024: 3, 4096: 4}[x.shape[1]]
             op = "sum" if x.dtype == np.float32 else ("max" if x.shape[1] == 4096 else "sum")
             want_out, want_st, _ = run_gpu(x, f, op, pf, inop, roots, flags=B.FTC_KERNEL_GENERIC)
-            got_out, got_st = run_noalloc(x, f, op, pf, inop, roots)
+            got_out, got_st = run_noalloc(x, f, op, pf, inop, roots, free_unchanged=rep == 1)
             assert np.array_equal(got_st, want_st), (rep, x.shape)
             assert np.array_equal(got_out.view(np.uint8), want_out.view(np.uint8)), (rep, x.shape)
+            orc_out, orc_st = run_oracle(x, f, op, pf, inop, roots)
+            assert np.array_equal(got_st, orc_st), (rep, x.shape)
+            assert np.array_equal(got_out.view(np.uint8), orc_out.view(np.uint8)), (rep, x.shape)
 
 
 def test_noalloc_rejects_shapes_beyond_the_built_in_scratch():
