@@ -35,6 +35,12 @@ def make_batch(P, f, k, dname, allreduce, S, seed):
     roots = rng.integers(0, P, size=S).astype(np.uint32)
     roots[rng.random(S) < 0.1] = P - 1                                # the root in the last group
     roots[rng.random(S) < 0.1] = 0
+    for i in range(7, S, 50):                                         # a failed root: no-op reduce, second allreduce attempt
+        pf[i, roots[i] >> 5] |= np.uint32(1 << (roots[i] & 31))
+    for i in range(11, S, 100):                                       # every root candidate failed
+        for c in range(f + 1):
+            v = (int(roots[i]) + c) % P
+            pf[i, v >> 5] |= np.uint32(1 << (v & 31))
     R = O.schedule(P, f)["rounds_attempt"]
     inop = np.full((S, 2, 2), sc.UNUSED, dtype=np.uint32)
     vic = rng.integers(0, P, size=(S, 2))
