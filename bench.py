@@ -8,7 +8,13 @@ configuration (f=4, k=32 int32, max, pre- and in-operation failures), a batch of
 (16 GiB of inputs, far larger than L2, so no flush is needed between steps).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c4|c5|c5r] [--batch S]
+    python bench.py --full-config [--workload cN]   # every batch of the configuration, every scenario checked
     python bench.py --impl reference ...      # times the CPU oracle on a bounded sample of the same workload
+
+Beside the K timed steps of the headline workload the line carries: the same step repeated for about two seconds
+with the SM clocks sampled meanwhile (roofline.sustained), the bandwidth of the library's read-only streaming
+kernels over the same buffer (roofline.read_only_gbs), and one record per other configuration, timed the same way
+(workloads: c5, c5r, c3).
 
 Prints ONE JSON line (rank 0). With N > 1 (torchrun) every rank runs its own batch: scenarios are
 independent, there is no collective on the data path ("weak" scaling).
@@ -49,8 +55,9 @@ def make_workload(name: str, S: int, first: int, rounds_attempt_c4: int):
 
 
 DEFAULT_BATCH = {"c3": 1 << 18, "c4": 1 << 15, "c5": 1 << 13, "c5r": 1 << 13}     # 16 GiB of inputs each
+CONFIG_SCENARIOS = {"c3": 1 << 20, "c4": 1 << 18, "c5": 1 << 14, "c5r": 1 << 14}    # scenarios of the whole configuration
 DESCRIPTION = {
-    "c3": "allreduce P=1024 f=3 k=16 float32 sum, 0..3 pre-operation failures",
+    "c3": "allreduce P=1024 f=3 k=16 float32 (Irwin-Hall stand-in for N(0,1)) sum, 0..3 pre-operation failures",
     "c4": "allreduce P=4096 f=4 k=32 int32 max, 0..2 pre-operation + 0..2 in-operation failures",
     "c5": "allreduce P=65536 f=8 k=4 uint64 sum, 0..8 pre-operation failures, per-scenario first root",
     "c5r": "reduce P=65536 f=8 k=4 uint64 xor, 0..8 pre-operation failures, per-scenario root",
@@ -106,6 +113,7 @@ class ClockSampler:
         self.first = self.lines()
 
     def stop(self) -> dict:
+        """Ends the sampling; returns the record of everything since mark()."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -113,9 +121,20 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
+        self.proc = None
+        rec = self.window(getattr(self, "first", 0), 1 << 60)
+        os.unlink(self.path)
+        return rec
+
+    def window(self, lo: int, hi: int) -> dict:
+        """Clock record of the samples lo <= line < hi (at least the last sample before hi)."""
+        if not os.path.exists(self.path):
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        if hi <= lo:
+            lo = max(0, hi - 1)
         sm, mx, reasons = [], [], set()
         for ln, line in enumerate(open(self.path)):
-            if ln < getattr(self, "first", 0):
+            if ln < lo or ln >= hi:
                 continue
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 9:
@@ -127,7 +146,6 @@ class ClockSampler:
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
-        os.unlink(self.path)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "samples": len(sm), "reasons": sorted(reasons)}
 
@@ -163,7 +181,7 @@ def time_oracle(w, prepared):
     return n_scen / dt, dt, min(cores, len(ids))
 
 
-ORACLE_SAMPLE = {"c3": (32768, 256), "c4": (8192, 64), "c5": (192, 2), "c5r": (192, 2)}
+ORACLE_SAMPLE = {"c3": (32768, 256), "c4": (4096, 32), "c5": (192, 2), "c5r": (192, 2)}
 
 
 def run_reference(args):
@@ -254,6 +272,190 @@ def upload(w, torch):
     return d_pf, d_inop, d_roots
 
 
+def measured_peak():
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        return float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class Leg:
+    """One workload resident on the device: inputs generated there, failure patterns uploaded, outputs and workspace."""
+
+    def __init__(self, name, S, first, args, B, torch, sched_rounds):
+        self.name, self.S, self.B, self.torch = name, S, B, torch
+        w = make_workload(name, S, first, sched_rounds)
+        if args.collective:
+            w.collective = args.collective
+        if args.failure_free:
+            w.prefail[:] = 0
+            if w.inop is not None:
+                w.inop[:, :, 0] = sc.UNUSED
+        self.w = w
+        self.allred = w.collective == "allreduce"
+        self.tdt = getattr(torch, np.dtype(w.dtype).name)
+        kflags = {"auto": 0, "direct": B.FTC_KERNEL_DIRECT, "generic": B.FTC_KERNEL_GENERIC}[args.kernel]
+        self.desc = B.make_desc(w.P, w.f, w.k, B.dtype_code(self.tdt), w.op, root=-1 if w.roots is not None else 0,
+                                max_inop=0 if w.inop is None else w.inop.shape[1], flags=kflags)
+        self.fn = B.ftc_allreduce_batch if self.allred else B.ftc_reduce_batch
+        self.d_x = torch.empty((S, w.P, w.k), dtype=self.tdt, device="cuda")
+        B.ftc_fill_inputs(w.kind, w.seed, w.first_scenario, S, w.P, w.k, self.d_x)
+        self.d_pf, self.d_inop, self.d_roots = upload(w, torch)
+        self.d_out = torch.empty((S, w.k), dtype=self.tdt, device="cuda")
+        self.d_st = torch.empty((S, 4), dtype=torch.int32, device="cuda")
+        self.d_ws = torch.empty(max(B.ftc_workspace_bytes(self.desc, S, self.allred), 16), dtype=torch.uint8, device="cuda")
+        self.sched = B.ftc_schedule_info(self.desc)
+        self.esz = ESZ[np.dtype(w.dtype).name]
+        self.bytes_per_launch = S * bytes_per_scenario(w)
+        torch.cuda.synchronize()
+
+    def regenerate(self, first, sched_rounds):
+        """The next batch of the same workload in the same buffers (scenarios first .. first+S-1)."""
+        w = make_workload(self.name, self.S, first, sched_rounds)
+        w.collective = self.w.collective
+        self.w = w
+        self.B.ftc_fill_inputs(w.kind, w.seed, w.first_scenario, self.S, w.P, w.k, self.d_x)
+        self.d_pf, self.d_inop, self.d_roots = upload(w, self.torch)
+        self.torch.cuda.synchronize()
+
+    def step(self):
+        self.fn(self.desc, self.S, self.d_x, self.d_pf, self.d_inop, self.d_roots, self.d_out, self.d_st, self.d_ws)
+
+    def rounds(self):
+        return self.sched["rounds_attempt"] if self.allred else self.sched["rounds_reduce"]
+
+    def status(self):
+        return self.d_st.cpu().numpy().view(np.uint32)
+
+    def free(self):
+        for n in ("d_x", "d_pf", "d_inop", "d_roots", "d_out", "d_st", "d_ws"):
+            setattr(self, n, None)
+        self.torch.cuda.empty_cache()
+
+
+def time_steps(torch, fn, steps):
+    """CUDA events on the launching stream (torch's current stream: the binding passes exactly that stream to the
+    library) around every step; returns (per-step ms, total ms)."""
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    torch.cuda.synchronize()
+    ev[0].record()
+    for i in range(steps):
+        fn()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    return [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)], ev[0].elapsed_time(ev[-1])
+
+
+def time_sustained(torch, fn, ms_per_step, seconds, sampler):
+    """The same step back to back for about `seconds` of GPU time: (steps, ms per step, clocks during it)."""
+    n = max(10, int(seconds * 1e3 / max(ms_per_step, 1e-3)))
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    m0 = sampler.lines() if sampler else 0
+    a.record()
+    for _ in range(n):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    clocks = sampler.window(m0, sampler.lines()) if sampler else None
+    return n, a.elapsed_time(b) / n, clocks
+
+
+def roofline_record(name, bytes_launch, per_launch_ms, S, peak, peak_kind):
+    avg = sum(per_launch_ms) / len(per_launch_ms)
+    achieved = bytes_launch / (avg / 1e3) / 1e9
+    return {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "peak_kind": peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": kernel_traffic(name, S),
+            "bytes_per_launch": bytes_launch, "avg_launch_ms": avg, "min_launch_ms": min(per_launch_ms)}
+
+
+def add_sustained(roof, leg, torch, sampler, seconds):
+    n, ms, clocks = time_sustained(torch, leg.step, roof["avg_launch_ms"], seconds, sampler)
+    ach = leg.bytes_per_launch / (ms / 1e3) / 1e9
+    mhz = clocks["sm_mhz"] if clocks else None
+    roof["sustained"] = {"steps": n, "seconds": n * ms / 1e3, "ms_per_step": ms, "achieved": ach, "frac": ach / roof["peak"],
+                         "sm_mhz_median": mhz, "ms_x_mhz": (ms * mhz) if mhz else None, "clocks": clocks}
+
+
+def run_side_leg(name, args, B, torch, sampler, peak, peak_kind):
+    """One more workload, timed like the headline one: K steps, then a sustained run; its own roofline record."""
+    S = DEFAULT_BATCH[name]
+    leg = Leg(name, S, 0, args, B, torch, 28)
+    for _ in range(max(args.warmup, 3)):
+        leg.step()
+    m0 = sampler.lines() if sampler else 0
+    per_ms, total_ms = time_steps(torch, leg.step, args.steps)
+    clocks = sampler.window(m0, sampler.lines()) if sampler else None
+    roof = roofline_record(name, leg.bytes_per_launch, per_ms, S, peak, peak_kind)
+    add_sustained(roof, leg, torch, sampler, args.sustain_seconds / 2)
+    ms = total_ms / args.steps
+    st = leg.status()
+    rec = {"workload": f"{name}: {DESCRIPTION[name]}", "value": S / (ms / 1e3), "unit": "scenarios/s", "ms_per_step": ms,
+           "steps": args.steps, "scenarios_per_step": S, "process_rounds_per_sec": S / (ms / 1e3) * leg.w.P * leg.rounds(),
+           "kernel": B.ftc_kernel_variant(leg.desc, leg.allred), "dtype": np.dtype(leg.w.dtype).name,
+           "ok_scenarios": int(((st[:, 0] & 0xFF) == 0).sum()), "roofline": roof, "clocks": clocks}
+    leg.free()
+    return rec
+
+
+def read_only_ceiling(B, torch, d_x, steps):
+    """The library's streaming kernels over the same buffer: what a kernel that only reads can reach here."""
+    nbytes = (d_x.numel() * d_x.element_size()) // 16384 * 16384
+    sink = torch.zeros(2, dtype=torch.int64, device="cuda")
+    out = {}
+    for mode, label in ((0, "loads_128bit"), (1, "bulk_copies_to_shared")):
+        for _ in range(3):
+            B.ftc_read_bandwidth_probe(mode, d_x, nbytes, sink)
+        per_ms, _ = time_steps(torch, lambda: B.ftc_read_bandwidth_probe(mode, d_x, nbytes, sink), max(5, min(steps, 20)))
+        out[label] = nbytes / (sum(per_ms) / len(per_ms) / 1e3) / 1e9
+    out["gave_up"] = int(sink[1].item())
+    return out
+
+
+def run_full_config(args, B, torch, sampler, peak, peak_kind):
+    """Every batch of the configuration at its stated scenario count: per batch the inputs are regenerated on the device,
+    K steps are timed, and the batch is checked against the any-size properties; times are summed over the batches."""
+    from paper_2602_22445_b200 import verify
+    name = args.workload
+    S = args.batch or DEFAULT_BATCH[name]
+    total = CONFIG_SCENARIOS[name]
+    nb = (total + S - 1) // S
+    leg = Leg(name, S, 0, args, B, torch, 28)
+    sum_ms, all_ms, checks = 0.0, [], {"ok_scenarios": 0, "noop_scenarios": 0, "retried": 0, "excluded_pairs": 0}
+    m0 = sampler.lines() if sampler else 0
+    for b in range(nb):
+        if b:
+            leg.regenerate(b * S, 28)
+        for _ in range(max(args.warmup, 3)):
+            leg.step()
+        per_ms, total_ms = time_steps(torch, leg.step, args.steps)
+        sum_ms += total_ms / args.steps
+        all_ms += per_ms
+        st = leg.status()
+        for k, v in verify.check_status_fields(leg.w, st).items():
+            checks[k] += v
+        rep = verify.check_results_by_definition(leg.w, leg.d_x, leg.d_out, st)
+        checks["excluded_pairs"] += rep["excluded_pairs"]
+        if "worst_relative_error" in rep:
+            checks["worst_relative_error"] = max(checks.get("worst_relative_error", 0.0), rep["worst_relative_error"])
+    clocks = sampler.stop() if sampler else None
+    roof = roofline_record(name, leg.bytes_per_launch, all_ms, S, peak, peak_kind)
+    value = nb * S / (sum_ms / 1e3)
+    line = {
+        "metric": "scenarios_per_sec", "value": value, "unit": "scenarios/s", "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": sum_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": {"int32": "i32", "int64": "i64", "uint64": "u64", "float32": "f32"}[np.dtype(leg.w.dtype).name], "data": "synthetic",
+        "process_rounds_per_sec": value * leg.w.P * leg.rounds(),
+        "config": {"workload": f"{name}: {DESCRIPTION[name]} [whole configuration]", "scenarios_total": nb * S, "batches": nb,
+                   "scenarios_per_batch": S, "step": "one pass over all batches (times of the batches summed)",
+                   "cache": "inputs larger than L2, no flush", "kernel": B.ftc_kernel_variant(leg.desc, leg.allred),
+                   "rounds_per_scenario": leg.rounds(), "subtrees_played": f"1 of {leg.w.f + 1}",
+                   "checked": "every scenario: outcome and counts from the masks, result by the plain definition (torch)", **checks},
+        "roofline": roof, "cpu_baseline": None, "e2e": None, "gpu_launches": args.steps * nb, "clocks": clocks,
+    }
+    print(json.dumps(line))
+
+
 def run_gpu(args):
     import torch
     from paper_2602_22445_b200 import binding as B
@@ -270,41 +472,24 @@ def run_gpu(args):
         dist = dist_mod
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     B.load()
-
-    name = args.workload
-    S = args.batch or DEFAULT_BATCH[name]
-    probe = make_workload(name, 1, 0, 28)
-    tdt = getattr(torch, np.dtype(probe.dtype).name)
-    desc0 = B.make_desc(probe.P, probe.f, probe.k, B.dtype_code(tdt), probe.op)
-    sched = B.ftc_schedule_info(desc0)
-    w = make_workload(name, S, rank * S, sched["rounds_attempt"])          # each rank its own scenarios
-    if args.collective:
-        w.collective = args.collective
-    if args.failure_free:
-        w.prefail[:] = 0
-        if w.inop is not None:
-            w.inop[:, :, 0] = sc.UNUSED
-    allred = w.collective == "allreduce"
-    kflags = {"auto": 0, "direct": B.FTC_KERNEL_DIRECT, "generic": B.FTC_KERNEL_GENERIC}[args.kernel]
-    desc = B.make_desc(w.P, w.f, w.k, B.dtype_code(tdt), w.op, root=-1 if w.roots is not None else 0,
-                       max_inop=0 if w.inop is None else w.inop.shape[1], flags=kflags)
-    fn = B.ftc_allreduce_batch if allred else B.ftc_reduce_batch
-
-    d_x = torch.empty((S, w.P, w.k), dtype=tdt, device="cuda")
-    B.ftc_fill_inputs(w.kind, w.seed, w.first_scenario, S, w.P, w.k, d_x)
-    d_pf, d_inop, d_roots = upload(w, torch)
-    d_out = torch.empty((S, w.k), dtype=tdt, device="cuda")
-    d_st = torch.empty((S, 4), dtype=torch.int32, device="cuda")
-    wsb = B.ftc_workspace_bytes(desc, S, allred)
-    d_ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device="cuda")
-    torch.cuda.synchronize()
-
-    def step():
-        fn(desc, S, d_x, d_pf, d_inop, d_roots, d_out, d_st, d_ws)
-
+    peak, peak_kind = measured_peak()
     sampler = ClockSampler(local) if rank == 0 else None
     if sampler:
         sampler.wait_ready()
+    if args.full_config:
+        if world > 1:
+            raise SystemExit("--full-config runs on one GPU")
+        run_full_config(args, B, torch, sampler, peak, peak_kind)
+        return
+
+    name = args.workload
+    S = args.batch or DEFAULT_BATCH[name]
+    leg = Leg(name, S, rank * S, args, B, torch, 28)                       # each rank its own scenarios
+    w, desc, allred, tdt = leg.w, leg.desc, leg.allred, leg.tdt
+    sched = leg.sched
+    d_x, d_out, d_st = leg.d_x, leg.d_out, leg.d_st
+    step = leg.step
+
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
@@ -312,21 +497,15 @@ def run_gpu(args):
         dist.barrier()
     if sampler:
         sampler.mark()
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    torch.cuda.synchronize()
-    ev[0].record()
-    for i in range(args.steps):
-        step()
-        ev[i + 1].record()
-    torch.cuda.synchronize()
+    per_launch_ms, total_ms = time_steps(torch, step, args.steps)
     if dist:
         dist.barrier()
-    clocks = sampler.stop() if sampler else None
-    per_launch_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    total_ms = ev[0].elapsed_time(ev[-1])
+    clocks = sampler.window(sampler.first, sampler.lines()) if sampler else None
     total_ms = max_over_ranks(total_ms, dist, torch.device("cuda", local))
     ms_per_step = total_ms / args.steps
     value = whole_job_value(world, S, ms_per_step)
+    roof = roofline_record(name, leg.bytes_per_launch, per_launch_ms, S, peak, peak_kind)
+    status = leg.status()
 
     e2e = None
     if not args.kernel_only:
@@ -359,33 +538,50 @@ def run_gpu(args):
 
         e2e = {"value": world * Se / e2e_s, "unit": "scenarios/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "scenarios_per_step": Se, "matches_device_run": same}
+        del h_x, staging
     if rank != 0:
         if dist:
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the one kernel a step launches ----
-    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(peaks_path):
-        peak, peak_kind = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
-    else:
-        peak, peak_kind = 6650.0, "fallback"
-    bytes_launch = S * bytes_per_scenario(w)
-    avg_launch_ms = sum(per_launch_ms) / len(per_launch_ms)
-    achieved = bytes_launch / (avg_launch_ms / 1e3) / 1e9
-    traffic = kernel_traffic(name, S)
-
-    # ---- the oracle beside it, on a bounded sample ----
+    launches = args.steps
+    workloads = {}
     cpu = None
-    if not (args.no_cpu_baseline or args.kernel_only):
-        n, chunk = ORACLE_SAMPLE[name]
-        wo = make_workload(name, n, 0, sched["rounds_attempt"])
-        rate, dt, cores = time_oracle(wo, prepare_oracle(wo, n, chunk))
-        cpu = {"value": rate, "unit": "scenarios/s", "cores": cores, "kind": "oracle",
-               "sample": f"first {n} scenarios of the workload ({dt:.1f} s wall on {cores} threads)"}
+    if not args.kernel_only:
+        # ---- the same step for seconds, with the clocks it ran at; and what a kernel that only reads can reach ----
+        add_sustained(roof, leg, torch, sampler, args.sustain_seconds)
+        launches += roof["sustained"]["steps"]
+        roof["read_only_gbs"] = read_only_ceiling(B, torch, d_x, args.steps)
+        roof["read_only_gbs"]["best"] = max(roof["read_only_gbs"]["loads_128bit"], roof["read_only_gbs"]["bulk_copies_to_shared"])
+        roof["frac_of_read_only"] = roof["achieved"] / roof["read_only_gbs"]["best"]
 
-    status = d_st.cpu().numpy().view(np.uint32)
-    R = rounds_of(w, sched)
+        # ---- the oracle beside it, on a bounded sample played until about 4 s of wall time on all cores are done ----
+        if not args.no_cpu_baseline:
+            n, chunk = ORACLE_SAMPLE[name]
+            n = min(n, S)
+            ids = [np.arange(s, min(s + chunk, n)) for s in range(0, n, chunk)]
+            xh = d_x[:n].cpu()
+            xh = xh.view(torch.int64).numpy().view(np.uint64) if tdt == torch.uint64 else xh.numpy()
+            prepared = (ids, [xh[i[0]:i[-1] + 1] for i in ids])
+            plays, secs, cores = 0, 0.0, 1
+            while secs < 4.0 and plays < 64:
+                _, dt, cores = time_oracle(w, prepared)
+                plays += 1
+                secs += dt
+            cpu = {"value": plays * n / secs, "unit": "scenarios/s", "cores": cores, "kind": "oracle",
+                   "sample": f"first {n} scenarios of the workload, played {plays} times ({secs:.1f} s wall on {cores} threads)"}
+        leg.free()
+        del d_x, d_out, d_st
+
+        # ---- the other configurations the target names, each timed the same way (one GPU only) ----
+        if world == 1 and not args.no_legs:
+            for other in [x for x in ("c5", "c5r", "c3", "c4") if x != name]:
+                workloads[other] = run_side_leg(other, args, B, torch, sampler, peak, peak_kind)
+                launches += args.steps + workloads[other]["roofline"]["sustained"]["steps"]
+    if sampler:
+        sampler.stop()
+
+    R = leg.rounds()
     line = {
         "metric": "scenarios_per_sec", "value": value, "unit": "scenarios/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -395,15 +591,17 @@ def run_gpu(args):
         "config": {"workload": f"{name}: {DESCRIPTION[name]}" + (f" [collective={args.collective}]" if args.collective else "")
                    + (" [failure-free]" if args.failure_free else ""), "scenarios_per_step_per_gpu": S,
                    "input_bytes_per_step_per_gpu": S * w.P * w.k * ESZ[np.dtype(w.dtype).name],
-                   "cache": "inputs larger than L2, no flush", "kernel": B.ftc_kernel_name(desc, allred),
-                   "rounds_per_scenario": R, "ok_scenarios": int(((status[:, 0] & 0xFF) == 0).sum())},
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": peak_kind, "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": traffic,
-                     "bytes_per_launch": bytes_launch, "avg_launch_ms": avg_launch_ms,
-                     "min_launch_ms": min(per_launch_ms)},
+                   "cache": "inputs larger than L2, no flush", "kernel": B.ftc_kernel_variant(desc, allred),
+                   "rounds_per_scenario": R, "subtrees_played": f"1 of {w.f + 1} (the child the root selects; "
+                   "process_rounds_per_sec counts P x rounds per scenario as the schedule has them)",
+                   "scenarios_of_the_configuration": CONFIG_SCENARIOS[name],
+                   "ok_scenarios": int(((status[:, 0] & 0xFF) == 0).sum())},
+        "roofline": roof,
+        "workloads": workloads,
         "cpu_baseline": cpu,
         "e2e": e2e,
         "gpu_launches": args.steps,
+        "launches_all_legs": launches,
         "clocks": clocks,
     }
     print(json.dumps(line))
@@ -424,7 +622,11 @@ def main():
     ap.add_argument("--collective", default="", choices=["", "reduce", "allreduce"], help="override the workload's collective")
     ap.add_argument("--failure-free", action="store_true", help="clear every failure of the workload (diagnostic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end and CPU legs (for profiler runs)")
+    ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end, sustained, CPU and other-workload legs (for profiler runs)")
+    ap.add_argument("--no-legs", action="store_true", help="skip the legs over the other configurations")
+    ap.add_argument("--sustain-seconds", type=float, default=2.0, help="GPU time of the sustained run of the headline workload")
+    ap.add_argument("--full-config", action="store_true",
+                    help="play every batch of the configuration (its stated scenario count), checking every scenario")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

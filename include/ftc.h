@@ -281,6 +281,15 @@ FTC_API int ftc_schedule_info(const ftc_desc_t* desc, ftc_sched_t* out);
 FTC_API int ftc_fill_inputs(uint32_t kind, uint64_t seed, uint64_t first_scenario, uint64_t S, uint32_t P, uint32_t k,
                     void* d_out, void* cuda_stream);
 
+/*
+ * Measurement aid (not part of the paper's method): reads `bytes` bytes (a multiple of 16 KiB) at d_buf (16-byte
+ * aligned) once and does nothing else. mode 0: 128-bit loads folded with xor in registers; mode 1: asynchronous bulk
+ * copies into shared memory, the way the batch kernels stage their inputs. Timed over the buffer a batch call reads,
+ * it gives the bandwidth a read-only kernel can reach on this GPU (a copy benchmark reads and writes).
+ * d_sink: two uint64 words, zeroed by the caller; word 1 counts warps whose bounded wait for a copy gave up (0 in a valid run).
+ */
+FTC_API int ftc_read_bandwidth_probe(uint32_t mode, const void* d_buf, uint64_t bytes, uint64_t* d_sink, void* cuda_stream);
+
 /* Name of the kernel family the batch calls would use for this descriptor: "staged", "tiled" or "generic". */
 FTC_API const char* ftc_kernel_name(const ftc_desc_t* desc, int is_allreduce);
 

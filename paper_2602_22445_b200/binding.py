@@ -41,7 +41,7 @@ OPS = {"sum": FTC_SUM, "max": FTC_MAX, "xor": FTC_XOR}
 EXPORTS = ["ftc_reduce_batch", "ftc_allreduce_batch", "ftc_reduce_batch_noalloc", "ftc_candidates_batch",
            "ftc_candidates_workspace_bytes", "ftc_message_counts_batch", "ftc_workspace_bytes", "ftc_reduce_batch_host",
            "ftc_allreduce_batch_host", "ftc_host_staging_bytes", "ftc_schedule_info", "ftc_fill_inputs",
-           "ftc_kernel_name", "ftc_kernel_variant", "ftc_launch_blocks", "ftc_strerror", "ftc_version"]
+           "ftc_kernel_name", "ftc_kernel_variant", "ftc_launch_blocks", "ftc_read_bandwidth_probe", "ftc_strerror", "ftc_version"]
 
 
 class ftc_desc_t(C.Structure):
@@ -100,6 +100,8 @@ def load():
     lib.ftc_kernel_variant.argtypes = [dp, C.c_int]
     lib.ftc_launch_blocks.restype = C.c_int
     lib.ftc_launch_blocks.argtypes = [dp, u64, C.c_int, C.POINTER(u32)]
+    lib.ftc_read_bandwidth_probe.restype = C.c_int
+    lib.ftc_read_bandwidth_probe.argtypes = [u32, vp, u64, vp, vp]
     lib.ftc_strerror.restype = C.c_char_p
     lib.ftc_strerror.argtypes = [C.c_int]
     lib.ftc_version.restype = u32
@@ -266,6 +268,13 @@ def ftc_allreduce_batch_host(desc, S, h_in, h_prefail, h_inop, h_roots, h_out, h
                              check=True) -> int:
     return _batch_host("ftc_allreduce_batch_host", desc, S, h_in, h_prefail, h_inop, h_roots, h_out, h_status,
                        d_staging, stream, check)
+
+
+def ftc_read_bandwidth_probe(mode, d_buf, nbytes, d_sink, stream=None) -> int:
+    rc = load().ftc_read_bandwidth_probe(mode, _dev_ptr(d_buf), nbytes, _dev_ptr(d_sink), _stream(stream))
+    if rc != FTC_OK:
+        raise FtcError(rc, "ftc_read_bandwidth_probe")
+    return rc
 
 
 def ftc_fill_inputs(kind, seed, first_scenario, S, P, k, d_out, stream=None) -> int:

@@ -339,6 +339,15 @@ int ftc_fill_inputs(uint32_t kind, uint64_t seed, uint64_t first_scenario, uint6
                ? FTC_OK : FTC_ECUDA;
 }
 
+int ftc_read_bandwidth_probe(uint32_t mode, const void* d_buf, uint64_t bytes, uint64_t* d_sink, void* cuda_stream) {
+    if (mode > 1 || !d_buf || !d_sink || !aligned16(d_buf) || (reinterpret_cast<uintptr_t>(d_sink) & 7u) || bytes % (16 * 1024)) return FTC_EINVAL;
+    DeviceInfo di;
+    int rc = device_info(di);
+    if (rc != FTC_OK) return rc;
+    return launch_probe(mode, d_buf, bytes, reinterpret_cast<unsigned long long*>(d_sink), di.sm_count,
+                        static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? FTC_OK : FTC_ECUDA;
+}
+
 const char* ftc_kernel_name(const ftc_desc_t* desc, int is_allreduce) {
     Params p;
     if (fill_params(desc, 1, is_allreduce, p) != FTC_OK) return "invalid";

@@ -45,6 +45,9 @@ cudaError_t launch_messages(const Params& p, unsigned long long* out, int sm_cou
 size_t expand_smem_bytes(const Params& p);
 cudaError_t launch_expand(const Params& p, const void* compact, void* out, int sm_count, cudaStream_t st);
 
+// Read-bandwidth probe: mode 0 = 128-bit loads, mode 1 = bulk copies into shared memory; sink = two 64-bit words.
+cudaError_t launch_probe(uint32_t mode, const void* buf, uint64_t bytes, unsigned long long* sink, int sm_count, cudaStream_t st);
+
 cudaError_t launch_fill(uint32_t kind, uint64_t seed, uint64_t first, uint64_t S, uint32_t P, uint32_t k, void* out,
                         int sm_count, cudaStream_t st);
 
