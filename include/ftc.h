@@ -225,6 +225,24 @@ FTC_API int ftc_candidates_batch(const ftc_desc_t* desc, uint64_t S, int is_allr
 FTC_API size_t ftc_candidates_workspace_bytes(const ftc_desc_t* desc, uint64_t S);
 
 /*
+ * The list of failed processes that the root holds when it delivers (section "Failure information", first scheme:
+ * in the up-correction phase and in the tree phase every process appends the ids of the processes it could not
+ * receive a value from; the lists travel up the tree with the values; "the root receives a complete list of failed
+ * processes from each child ... that does not contain a failed process in the subtree spanned by it"). It is the list
+ * that came with the value of the child the root selected, plus, when that child's subtree holds no member of the
+ * root's own up-correction group, what the root noted itself. Under in-operation failures it lists exactly the
+ * processes whose input is not part of the delivered result. is_allreduce != 0: the reduce of the attempt that counts.
+ *   d_failed [S][ceil(P/32)] uint32: bit p of a scenario's words set = process p (the caller's numbering) is on the list
+ *   d_nfail  [S] uint32: the size of the list (the second scheme sends only this); equals the number of set bits,
+ *            since concatenated lists come from disjoint sets
+ * Scenarios whose outcome is not FTC_ST_OK deliver nothing: all zero. Only the failure pattern is read; desc->k, dtype
+ * and op must be valid but do not matter. Other arguments as for ftc_reduce_batch. No workspace.
+ */
+FTC_API int ftc_failed_list_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const uint32_t* d_prefail,
+                                  const ftc_inop_t* d_inop, const uint32_t* d_roots, uint32_t* d_failed, uint32_t* d_nfail,
+                                  void* cuda_stream);
+
+/*
  * Messages sent in each scenario (theorem on the number of messages of the reduce and theorem on the messages of
  * the allreduce, section "Properties": failure-free f(f+1)q + a(a-1) up-correction and P-1 tree messages; no
  * process sends more when processes fail; an allreduce whose first candidates had failed repeats the reduce).

@@ -39,7 +39,7 @@ FTC_DEBUG_ONE_POLL = 0x4000000
 OPS = {"sum": FTC_SUM, "max": FTC_MAX, "xor": FTC_XOR}
 
 EXPORTS = ["ftc_reduce_batch", "ftc_allreduce_batch", "ftc_reduce_batch_noalloc", "ftc_candidates_batch",
-           "ftc_candidates_workspace_bytes", "ftc_message_counts_batch", "ftc_workspace_bytes", "ftc_reduce_batch_host",
+           "ftc_candidates_workspace_bytes", "ftc_message_counts_batch", "ftc_failed_list_batch", "ftc_workspace_bytes", "ftc_reduce_batch_host",
            "ftc_allreduce_batch_host", "ftc_host_staging_bytes", "ftc_schedule_info", "ftc_fill_inputs",
            "ftc_kernel_name", "ftc_kernel_variant", "ftc_launch_blocks", "ftc_read_bandwidth_probe", "ftc_strerror", "ftc_version"]
 
@@ -86,6 +86,8 @@ def load():
     lib.ftc_candidates_workspace_bytes.argtypes = [dp, u64]
     lib.ftc_message_counts_batch.restype = C.c_int
     lib.ftc_message_counts_batch.argtypes = [dp, u64, C.c_int, vp, vp, vp, vp, vp]
+    lib.ftc_failed_list_batch.restype = C.c_int
+    lib.ftc_failed_list_batch.argtypes = [dp, u64, C.c_int, vp, vp, vp, vp, vp, vp]
     lib.ftc_workspace_bytes.restype = sz
     lib.ftc_workspace_bytes.argtypes = [dp, u64, C.c_int]
     lib.ftc_host_staging_bytes.restype = sz
@@ -245,6 +247,14 @@ def ftc_message_counts_batch(desc, S, is_allreduce, d_prefail, d_inop, d_roots, 
                                          _dev_ptr(d_roots), _dev_ptr(d_msgs), _stream(stream))
     if check and rc != FTC_OK:
         raise FtcError(rc, "ftc_message_counts_batch")
+    return rc
+
+
+def ftc_failed_list_batch(desc, S, is_allreduce, d_prefail, d_inop, d_roots, d_failed, d_nfail, stream=None, check=True) -> int:
+    rc = load().ftc_failed_list_batch(C.byref(desc), S, int(is_allreduce), _dev_ptr(d_prefail), _dev_ptr(d_inop),
+                                      _dev_ptr(d_roots), _dev_ptr(d_failed), _dev_ptr(d_nfail), _stream(stream))
+    if check and rc != FTC_OK:
+        raise FtcError(rc, "ftc_failed_list_batch")
     return rc
 
 

@@ -280,6 +280,24 @@ int ftc_message_counts_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduc
     return e == cudaSuccess ? FTC_OK : FTC_ECUDA;
 }
 
+int ftc_failed_list_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const uint32_t* d_prefail,
+                          const ftc_inop_t* d_inop, const uint32_t* d_roots, uint32_t* d_failed, uint32_t* d_nfail,
+                          void* cuda_stream) {
+    Params p;
+    int rc = fill_params(desc, S, is_allreduce ? 1 : 0, p);
+    if (rc != FTC_OK) return rc;
+    if (S == 0) return FTC_OK;
+    if (!d_prefail || !d_failed || !d_nfail) return FTC_EINVAL;
+    if (p.max_inop && !d_inop) return FTC_EINVAL;
+    if (p.root < 0 && !d_roots) return FTC_EINVAL;
+    DeviceInfo di;
+    if ((rc = device_info(di)) != FTC_OK) return rc;
+    if (messages_smem_bytes(p) > (size_t)di.smem_optin) return FTC_EUNSUPPORTED;
+    p.prefail = d_prefail; p.inop = d_inop; p.roots = d_roots;
+    cudaError_t e = launch_failed_list(p, d_failed, d_nfail, di.sm_count, static_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? FTC_OK : FTC_ECUDA;
+}
+
 size_t ftc_candidates_workspace_bytes(const ftc_desc_t* desc, uint64_t S) {
     Params p;
     if (fill_params(desc, S, 0, p) != FTC_OK || S == 0) return 0;

@@ -41,6 +41,9 @@ cudaError_t launch_candidates(const Params& p, int tsel, void* cand, uint32_t* i
 size_t messages_smem_bytes(const Params& p);
 cudaError_t launch_messages(const Params& p, unsigned long long* out, int sm_count, cudaStream_t st);
 
+// The failed-process list the root ends up with (bitmask over process ids, and its size); reads the failure pattern only.
+cudaError_t launch_failed_list(const Params& p, uint32_t* failed, uint32_t* nfail, int sm_count, cudaStream_t st);
+
 // Expanded allreduce output from the compact results (one value per scenario) left by the main kernel.
 size_t expand_smem_bytes(const Params& p);
 cudaError_t launch_expand(const Params& p, const void* compact, void* out, int sm_count, cudaStream_t st);

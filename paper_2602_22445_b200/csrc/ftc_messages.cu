@@ -159,6 +159,61 @@ __global__ void __launch_bounds__(kMsgThreads) messages_kernel(Params p, unsigne
     }
 }
 
+// The list of failed processes that reaches the root with the value it delivers (first scheme of section "Failure
+// information"): every process appends the ids of those it could not receive a value from, in the up-correction
+// phase and in the tree phase, and the lists travel up the tree with the values. The child the root selects has no
+// failed process in its subtree, so its list holds exactly the up-correction partners whose message did not reach
+// the subtree's member of their group; when that subtree holds no member of the root's own (short, last) group the
+// root adds those it noted itself. Group by group that is the complement of the arrival mask the decode builds.
+// Output: the list as a bitmask over the caller's process ids, and its size.
+__global__ void __launch_bounds__(kMsgThreads) failed_list_kernel(Params p, uint32_t* failed, uint32_t* nfail) {
+    extern __shared__ __align__(16) uint32_t smem[];
+    Ctx* cx = reinterpret_cast<Ctx*>(smem);
+    uint32_t* pf = smem + sizeof(Ctx) / 4;
+    uint32_t* inc = pf + p.W + 1;
+    __shared__ uint32_t total;
+    const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
+    for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {
+        decode_scenario(p, s, cx, pf, inc);
+        if (tid == 0) total = 0;
+        __syncthreads();
+        const bool ok = cx->code == FTC_ST_OK;
+        const uint32_t root = cx->root;
+        // bit `root` of the renumbered mask belongs to process 0, bit 0 to the root (which delivers, so it is alive)
+        const uint32_t b0 = ok && root != 0 ? ((~inc[root >> 5]) >> (root & 31)) & 1u : 0u;
+        uint32_t cnt = 0;
+        for (uint32_t w = tid; w < p.W; w += nt) {
+            uint32_t word = 0;
+            if (ok) {
+                word = ~inc[w];
+                if (w == p.W - 1 && (p.P & 31)) word &= (1u << (p.P & 31)) - 1u;
+                if (w == 0) word &= ~1u;
+                cnt += __popc(word);
+                if (root != 0) {
+                    if (w == (root >> 5)) word &= ~(1u << (root & 31));
+                    if (w == 0) word |= b0;
+                }
+            }
+            failed[s * p.W + w] = word;
+        }
+        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+        if (lane == 0 && cnt) atomicAdd(&total, cnt);
+        __syncthreads();
+        if (tid == 0) nfail[s] = total;
+        __syncthreads();
+    }
+}
+
+cudaError_t launch_failed_list(const Params& p, uint32_t* failed, uint32_t* nfail, int sm_count, cudaStream_t st) {
+    const size_t smem = sizeof(Ctx) + 2 * (size_t)(p.W + 1) * 4;
+    cudaError_t e = cudaFuncSetAttribute(failed_list_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const uint64_t cap = (uint64_t)sm_count * 8;
+    const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
+    failed_list_kernel<<<grid, kMsgThreads, smem, st>>>(p, failed, nfail);
+    return cudaGetLastError();
+}
+
 size_t messages_smem_bytes(const Params& p) { return sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4; }
 
 cudaError_t launch_messages(const Params& p, unsigned long long* out, int sm_count, cudaStream_t st) {
