@@ -33,6 +33,11 @@ cudaError_t launch_staged(const Params& p, int tsel, int sm_count, int smem_opti
 // Name of the instantiation launch_staged would run ("staged/lean", ...); p.S and p.ws_bytes matter.
 const char* staged_variant(Params p, int tsel, int smem_optin_bytes, int sm_count, uint32_t* grid_cap_blocks_per_sm);
 
+// Warp kernel (scenarios of a few KB, one warp per scenario): shape check and launch. The staged launcher and the
+// variant query route to it when the shape fits.
+bool warp_supported(Params p, int smem_optin_bytes);
+cudaError_t launch_warp(const Params& p, int tsel, int sm_count, int smem_optin_bytes, cudaStream_t st);
+
 // Every root child's delivery (value, flag, failed-list size): general kernel, workspace slices of candidates_slice_bytes().
 size_t candidates_slice_bytes(const Params& p);
 cudaError_t launch_candidates(const Params& p, int tsel, void* cand, uint32_t* info, int sm_count, cudaStream_t st);

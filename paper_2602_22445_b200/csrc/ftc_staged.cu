@@ -26,6 +26,8 @@ size_t staged_workspace_bytes(Params p, int smem_optin_bytes, int sm_count) {
 }
 
 const char* staged_variant(Params p, int tsel, int smem_optin_bytes, int sm_count, uint32_t* grid_cap_blocks_per_sm) {
+    if (grid_cap_blocks_per_sm) *grid_cap_blocks_per_sm = 0;
+    if (warp_supported(p, smem_optin_bytes)) return "staged/warp";
     StagedGeom g;
     const StagedVariant v = staged_plan(p, tsel == TS_F32_SUM, true, staged_xl(p), smem_optin_bytes, sm_count, g);
     if (grid_cap_blocks_per_sm) *grid_cap_blocks_per_sm = g.hv_global ? (uint32_t)kHvGlobalBlocksPerSm : 0u;
@@ -33,6 +35,7 @@ const char* staged_variant(Params p, int tsel, int smem_optin_bytes, int sm_coun
 }
 
 cudaError_t launch_staged(const Params& p, int tsel, int sm_count, int smem_optin, cudaStream_t st) {
+    if (warp_supported(p, smem_optin)) return launch_warp(p, tsel, sm_count, smem_optin, st);
     switch (tsel) {
     case TS_U32_SUM: return launch_staged_u32_sum(p, sm_count, smem_optin, st);
     case TS_I32_MAX: return launch_staged_i32_max(p, sm_count, smem_optin, st);

@@ -1,0 +1,234 @@
+// Warp kernel: scenarios of a few KB, one warp (= one block) per scenario at a time. For such scenarios the work
+// per scenario that is not combining -- decoding the masks, barriers between the threads of a block, setting up
+// copies -- outweighs the combining, so everything here is warp-local: the masks are decoded in registers
+// (ftc_decode_warp.cuh), consecutive scenarios arrive several at a time by one bulk copy into the warp's own double
+// buffer, their masks, in-operation entries and roots are fetched one group ahead into registers, and the whole
+// subtree heap of a scenario is one warp tile (lanes = lane rows x 16-byte chunks, lane-local sub-heaps below,
+// shuffles above), evaluated by the same routines as the tiles of the staged kernel.
+// Before the evaluation the warp exchanges the vectors of process 0 and of the root in its copy of the scenario, so
+// that the copy is in renumbered order (section "Reduce": the root swaps numbers with process 0) and no group needs
+// special addressing. Scenarios the register decode leaves out (more failures than tolerated, a root out of range)
+// go through decode_scenario()/count_holders(), which a one-warp block can call as they are.
+#pragma once
+#include "ftc_staged_impl.cuh"
+#include "ftc_decode_warp.cuh"
+
+namespace ftc {
+
+struct WarpGeom {
+    uint32_t group;        // scenarios per buffer (consecutive scenarios, one bulk copy)
+    uint32_t buf_bytes;    // bytes per buffer (multiple of 128)
+    uint32_t off_bar, off_buf, smem_bytes;
+};
+
+constexpr int kWarpMinBlocks = 16;
+
+template <typename T, int OP, int XL>
+__global__ void __launch_bounds__(32, kWarpMinBlocks) warp_kernel(Params p, WarpGeom g) {
+    extern __shared__ __align__(128) uint32_t smem[];
+    char* sbase = reinterpret_cast<char*>(smem);
+    Ctx* cx = reinterpret_cast<Ctx*>(smem);
+    uint32_t* pf = smem + sizeof(Ctx) / 4;
+    uint32_t* inc = pf + p.W + 1;
+    uint32_t* unr = inc + p.W + 1;
+    const uint32_t lane = threadIdx.x;
+    const uint32_t cwl = p.cw_log2, lw = 5 - cwl, RW = 1u << lw;
+    const uint32_t lr = lane >> cwl, lc = lane & (p.C - 1);
+    const uint32_t D = lw + XL;
+    const uint32_t nq = p.C < 8 ? 8u / p.C : 1u, gq = min(nq, p.m & (0u - p.m));
+    const uint32_t rot = (lr >> ilog2u(nq / gq)) & (gq - 1);          // starting member of this lane row's folds (bank spread)
+    const uint32_t rowbytes = p.m * p.kbytes;
+    const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
+    const uint32_t tries = (p.flags & FTC_DEBUG_ONE_POLL) ? 1u : kWaitTries;
+    const uint32_t bar0 = smem_addr(sbase + g.off_bar);
+    char* bufs = sbase + g.off_buf;
+    if (lane < 2) mbar_init(bar0 + lane * 8, 1);
+    if (lane == 0) { pf[p.W] = 0; inc[p.W] = 0; }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+
+    const uint64_t ngroups = (p.S + g.group - 1) / g.group;
+    uint32_t phase_bits = 0, pending = 0;
+    bool dead = false;                  // a bounded wait gave up: no further copies or waits, every later scenario reports it
+    auto group_size = [&](uint64_t grp) { return (uint32_t)min((uint64_t)g.group, p.S - grp * g.group); };
+    auto issue = [&](uint64_t grp, uint32_t b) {
+        if (dead) return;
+        const uint32_t bytes = group_size(grp) * (uint32_t)scen_bytes;
+        if (lane == 0) {
+            mbar_expect_tx(bar0 + b * 8, bytes);
+            bulk_g2s(smem_addr(bufs + (size_t)b * g.buf_bytes), reinterpret_cast<const char*>(p.in) + grp * g.group * scen_bytes,
+                     bytes, bar0 + b * 8);
+        }
+        pending |= 1u << b;
+    };
+    // masks, in-operation entries and roots of a group, one register each (group * W, group * max_inop and group are at most 32)
+    struct Small { uint32_t pfw, vic, rnd, root; };
+    auto fetch = [&](uint64_t grp) {
+        Small s{0, FTC_INOP_UNUSED, 0, 0};
+        const uint32_t n = group_size(grp);
+        const uint64_t s0 = grp * g.group;
+        if (lane < n * p.W) s.pfw = __ldg(p.prefail + s0 * p.W + lane);
+        if (lane < n * p.max_inop) { const ftc_inop_t* e = p.inop + s0 * p.max_inop + lane; s.vic = __ldg(&e->victim); s.rnd = __ldg(&e->round); }
+        if (p.root < 0 && lane < n) s.root = __ldg(p.roots + s0 + lane);
+        return s;
+    };
+
+    uint64_t grp = blockIdx.x;
+    uint32_t b = 0;
+    Small cur{0, FTC_INOP_UNUSED, 0, 0};
+    if (grp < ngroups) { issue(grp, 0); cur = fetch(grp); }
+    for (; grp < ngroups; grp += gridDim.x, b ^= 1u) {
+        const uint64_t nxt = grp + gridDim.x;
+        Small nx{0, FTC_INOP_UNUSED, 0, 0};
+        if (nxt < ngroups) { issue(nxt, b ^ 1u); nx = fetch(nxt); }
+        if (!dead && ((pending >> b) & 1u)) {
+            bool ok = mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u, tries);
+            if (!__all_sync(kFullWarp, ok)) {
+                if (__any_sync(kFullWarp, ok) && !ok) ok = mbar_wait_bounded(bar0 + b * 8, (phase_bits >> b) & 1u, kWaitTries);
+                ok = __all_sync(kFullWarp, ok);
+            }
+            if (ok) { phase_bits ^= 1u << b; pending &= ~(1u << b); }
+            else dead = true;
+        }
+        const uint32_t n = group_size(grp);
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint64_t s = grp * g.group + i;
+            char* out_s = reinterpret_cast<char*>(p.out) + s * p.kbytes;
+            uint32_t pfw = __shfl_sync(kFullWarp, cur.pfw, lane < p.W ? i * p.W + lane : 0u);
+            if (lane >= p.W) pfw = 0;
+            else if (lane == p.W - 1 && (p.P & 31)) pfw &= (1u << (p.P & 31)) - 1u;
+            const uint32_t src = lane < p.max_inop ? i * p.max_inop + lane : 0u;
+            const uint32_t ev = __shfl_sync(kFullWarp, cur.vic, src), er = __shfl_sync(kFullWarp, cur.rnd, src);
+            const uint32_t first_root = p.root >= 0 ? (uint32_t)p.root : __shfl_sync(kFullWarp, cur.root, i);
+            WarpScen w;
+            if (decode_warp(p, pfw, ev, er, first_root, w)) {
+                if (lane <= p.W) inc[lane] = w.incw;
+                if (p.W == 32 && lane == 0) inc[32] = 0;
+                __syncwarp();
+            } else {
+                // the general routines (a block of one warp may call them): everything outside the register decode
+                decode_scenario(p, s, cx, pf, inc);
+                if (cx->code == FTC_ST_OK && p.is_allreduce) count_holders(p, cx, pf, unr);
+                w.code = cx->code; w.sstar = cx->sstar; w.attempts = cx->attempts; w.root = cx->root; w.base = cx->base;
+                w.npre = cx->npre; w.nexcl = cx->nexcl; w.inop_incl = cx->inop_incl; w.holders = cx->holders; w.G = cx->G;
+                w.any_victim = 1;
+                __syncwarp();
+            }
+            const bool okc = w.code == FTC_ST_OK && !dead;
+            if (!okc) {
+                if (lane < p.C) reinterpret_cast<uint4*>(out_s)[lane] = make_uint4(0, 0, 0, 0);
+            } else {
+                char* sc = bufs + (size_t)b * g.buf_bytes + (size_t)i * scen_bytes;
+                // renumbered order: the vectors of process 0 and of the root change places (the copy is the warp's own)
+                if (w.root != 0) {
+                    if (lane < p.C) {
+                        uint4* a = reinterpret_cast<uint4*>(sc) + lane;
+                        uint4* c = reinterpret_cast<uint4*>(sc + (size_t)w.root * p.kbytes) + lane;
+                        const uint4 va = *a, vc = *c;
+                        *a = vc; *c = va;
+                    }
+                    __syncwarp();
+                }
+                const uint32_t sstar = w.sstar, G = w.G;
+                const char* in_lc = sc + lc * 16;
+                // the one tile: heap rows 0 .. 2^D - 2; lane row lr owns row lr of the upper levels and the sub-heap under row RW-1+lr
+                const uint32_t tA = RW - 1 + lr, rowA = tA, tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB), rowB = lr;
+                const bool masked = w.npre != 0 || w.any_victim != 0;
+                // the short last group and a heap that does not fill the tile down to its second-to-last level take the careful folds
+                const bool careful = G > p.q || ((2u << (D >= 2 ? D - 2 : 0)) - 2 >= G);
+                uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
+                if (!careful) {
+                    const bool hasB = lr < RW - 1;
+                    fold_tile_fast<T, OP, XL, true, false>(p, 0u, sstar, inc, in_lc, in_lc, rowbytes, 0u, lr, rot, rowB, hasB, tA, rowA, G, masked, valA, valB);
+                    valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
+                } else {
+                    if (rowA < G) valA = SubHeap<T, OP, XL, 0, true, true, false>::eval(p, 0u, sstar, inc, in_lc, in_lc, rowbytes, tA, rowA, G);
+                    const bool hasB = lr < RW - 1 && rowB < G;
+                    if (hasB) valB = fold_staged_call<T, OP, true, false>(fold_shape(p), 0u, sstar, inc, in_lc, in_lc + staged_row_offset<true>(p, rowbytes, lr, rowB), rowB);
+                    valB = tile_tree_phase<T, OP>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
+                }
+                // the root (Algorithm "reduce_root"): its own data on the left unless the child's subtree holds it already
+                if (lr == 0) {
+                    uint4 recv = lw ? valB : valA;
+                    if (sstar >= p.r) recv = comb16<T, OP>(fold_root16<T, OP, LdShared>(p, 0u, inc, in_lc), recv);
+                    reinterpret_cast<uint4*>(out_s)[lc] = recv;
+                }
+            }
+            if (lane == 0) {
+                uint4 rec;
+                const uint32_t code = dead ? (uint32_t)FTC_ST_INTERNAL_TIMEOUT : w.code;
+                rec.x = code | ((okc ? w.sstar : 0xFFu) << 8) | (w.attempts << 16);
+                rec.y = okc ? p.P - w.npre - w.nexcl : 0u;
+                rec.z = okc ? w.inop_incl : 0u;
+                rec.w = (okc && p.is_allreduce) ? w.holders : 0u;
+                *reinterpret_cast<uint4*>(p.status + s * FTC_STATUS_WORDS) = rec;
+            }
+            __syncwarp();
+        }
+        cur = nx;
+    }
+    // only after a wait gave up: a copy may still be in flight toward this block's shared memory
+    for (uint32_t bb = 0; bb < 2; ++bb)
+        if ((pending >> bb) & 1u) mbar_wait_bounded(bar0 + bb * 8, (phase_bits >> bb) & 1u, kWaitTries);
+}
+
+// ---- host side ----
+// Shapes: 16-byte chunks, a power-of-two chunk count of at most 32, at most 1024 processes (one mask word per lane), a
+// subtree heap that fits one warp tile with a lane-local sub-heap of at most three levels, scenarios of at most
+// kWarpMaxBytes. XL: the shallowest sub-heap that holds the heap.
+constexpr uint64_t kWarpMaxBytes = 8 * 1024;
+constexpr uint32_t kWarpBufTarget = 4 * 1024;       // a buffer holds as many consecutive scenarios as fit in this (at least one)
+
+static bool warp_geometry(Params& p, int smem_optin, uint32_t& XL, WarpGeom& g) {
+    if (p.kbytes % 16 || p.W > 32) return false;
+    const uint32_t C = p.kbytes / 16;
+    if (C == 0 || C > 32 || (C & (C - 1))) return false;
+    const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
+    if (scen_bytes > kWarpMaxBytes) return false;
+    uint32_t cwl = 0; while ((1u << cwl) < C) ++cwl;
+    const uint32_t lw = 5 - cwl;
+    uint32_t Hmax = 1; while ((1u << Hmax) <= p.Gmax) ++Hmax;
+    if (Hmax > lw + 3) return false;
+    XL = Hmax > lw + 1 ? Hmax - lw : 1u;
+    p.C = C; p.cw_log2 = cwl; p.Lt = 0; p.below = 0; p.swz_mask = 0; p.row_shift = 0;
+    uint32_t group = (uint32_t)(kWarpBufTarget / scen_bytes);
+    if (group < 1) group = 1;
+    while (group > 1 && (group * p.W > 32 || group * p.max_inop > 32 || group > 32)) --group;
+    if (p.max_inop > 32) return false;
+    g.group = group;
+    g.buf_bytes = (uint32_t)((group * scen_bytes + 127) & ~(uint64_t)127);
+    size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
+    o = (o + 15) & ~(size_t)15; g.off_bar = (uint32_t)o; o += 16;
+    o = (o + 127) & ~(size_t)127; g.off_buf = (uint32_t)o;
+    o += 2 * (size_t)g.buf_bytes;
+    g.smem_bytes = (uint32_t)o;
+    return o <= (size_t)smem_optin - 1024;
+}
+
+template <typename T, int OP, int XL>
+static cudaError_t launch_warp_x(const Params& p, const WarpGeom& g, int sm_count, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(warp_kernel<T, OP, XL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, warp_kernel<T, OP, XL>, 32, g.smem_bytes);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    const uint64_t ngroups = (p.S + g.group - 1) / g.group, cap = (uint64_t)sm_count * per_sm;
+    const uint32_t grid = (uint32_t)(ngroups < cap ? ngroups : cap);
+    if (p.grid_query) { *p.grid_query = grid; return cudaSuccess; }
+    warp_kernel<T, OP, XL><<<grid, 32, g.smem_bytes, st>>>(p, g);
+    return cudaGetLastError();
+}
+
+template <typename T, int OP>
+static cudaError_t launch_warp_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
+    WarpGeom g; uint32_t XL = 1;
+    if (!warp_geometry(p, smem_optin, XL, g)) return cudaErrorInvalidConfiguration;
+    switch (XL) {
+    case 1: return launch_warp_x<T, OP, 1>(p, g, sm_count, st);
+    case 2: return launch_warp_x<T, OP, 2>(p, g, sm_count, st);
+    default: return launch_warp_x<T, OP, 3>(p, g, sm_count, st);
+    }
+}
+
+}  // namespace ftc

@@ -69,8 +69,17 @@ CASES = [
     ("staged/lean-swz", 5000, 3, 4, "f32", "sum", False),             # 64-byte groups
     ("staged/batched-swz", 16384, 3, 8, "f32", "sum", False),
     ("staged/batched-swz", 40000, 3, 4, "f32", "sum", True),          # 64-byte groups in large blocks
-    ("staged/whole", 64, 2, 8, "i64", "sum", False),                  # the P=64 configuration's shape
-    ("staged/whole", 150, 3, 4, "f32", "sum", True),
+    ("staged/whole", 150, 3, 16, "f32", "sum", True),                 # 9.6 KB per scenario
+    ("staged/whole", 700, 6, 4, "i32", "xor", False),                 # 11 KB, a heap too deep for one warp tile
+    ("staged/warp", 64, 2, 8, "i64", "sum", False),                   # the P=64 configuration's shape
+    ("staged/warp", 150, 3, 4, "f32", "sum", True),                   # short last group, 16-byte vectors
+    ("staged/warp", 64, 3, 4, "i32", "max", True),                    # a heap shallower than the warp tile
+    ("staged/warp", 500, 1, 4, "i32", "xor", False),                  # 8 KB, lane-local sub-heaps of three levels
+    ("staged/warp", 40, 4, 32, "i32", "max", True),                   # 128-byte vectors
+    ("staged/warp", 12, 0, 64, "f32", "sum", False),                  # no tolerance: groups of one, 256-byte vectors
+    ("staged/warp", 9, 1, 128, "i32", "sum", True),                   # 512-byte vectors: one lane row
+    ("staged/warp", 100, 5, 4, "u64", "sum", True),
+    ("staged/warp", 1024, 7, 2, "i32", "sum", False),                 # kbytes = 8: not this kernel (checked below)
     ("tiled", 4096, 4, 32, "i32", "max", True),
 ]
 
@@ -79,6 +88,9 @@ CASES = [
 def test_every_variant_with_several_scenarios_per_block(variant, P, f, k, dname, op, allreduce):
     flags = B.FTC_KERNEL_DIRECT if variant == "tiled" else 0
     desc = B.make_desc(P, f, k, B.dtype_code(np.dtype(DT[dname])), op, root=-1, max_inop=2, flags=flags)
+    if k * np.dtype(DT[dname]).itemsize % 16:
+        assert B.ftc_kernel_variant(desc, allreduce) == "generic"
+        return
     assert B.ftc_kernel_variant(desc, allreduce) == variant
     blocks = B.ftc_launch_blocks(desc, 1 << 30, allreduce)
     assert blocks >= 148
@@ -122,7 +134,7 @@ def test_seeded_random_shapes(P, f, k, dname, op, allreduce):
 # ---------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("P,f,k,dname,op,allreduce", [(1024, 3, 16, "f32", "sum", True), (4096, 4, 32, "i32", "max", True),
                                                       (16384, 3, 8, "f32", "sum", False), (16384, 1, 8, "i32", "sum", True),
-                                                      (64, 2, 8, "i64", "sum", False)])
+                                                      (64, 2, 8, "i64", "sum", False), (150, 3, 16, "f32", "sum", True)])
 def test_a_wait_that_gives_up_poisons_its_block_and_nothing_else(P, f, k, dname, op, allreduce):
     """With FTC_DEBUG_ONE_POLL the waits for the asynchronous copies look once and give up. Then: a scenario is either
     played correctly (bit-equal to the oracle) or reports FTC_ST_INTERNAL_TIMEOUT with zero bytes; once a block has
@@ -145,6 +157,6 @@ def test_a_wait_that_gives_up_poisons_its_block_and_nothing_else(P, f, k, dname,
     for b in range(blocks):                                           # sticky per block
         seq = timed_out[b::blocks]
         assert np.array_equal(seq, np.sort(seq)), (b, seq)
-    if variant != "staged/whole":                                     # tile copies are waited for right after their issue
+    if variant not in ("staged/whole", "staged/warp"):               # tile copies are waited for right after their issue
         assert timed_out.any()
     assert_same(run_gpu(None, f, op, pf, inop, roots, 0, allreduce, 0, d_x=d_x), want, f"normal call after the give-up run, {variant}")
