@@ -55,6 +55,7 @@ static int fill_params(const ftc_desc_t* d, uint64_t S, int is_allreduce, Params
     p.pdesc = (d->flags & FTC_PARTNERS_DESCENDING) ? 1u : 0u;
     p.P = d->P; p.f = d->f; p.m = d->f + 1; p.k = d->k; p.W = (d->P + 31) / 32;
     p.q = (d->P - 1) / p.m; p.r = (d->P - 1) % p.m;
+    p.m_magic = (uint32_t)((0x100000000ull + p.m - 1) / p.m);
     p.Gmax = p.q + (p.r ? 1u : 0u);
     p.H = 1 + deepest_level_h(p.arity, p.Gmax);
     p.Rred = p.f + p.H; p.Ratt = 2 * p.Rred;

@@ -19,6 +19,10 @@ struct WarpScen {
 
 constexpr uint32_t kFullWarp = 0xFFFFFFFFu;
 
+// x / m and x % m for x below 2^26 without a division (p.m_magic = ceil(2^32 / m), m <= 32: the rounding error of the
+// reciprocal times x stays below one unit of the quotient's last place)
+__device__ __forceinline__ uint32_t div_m(const Params& p, uint32_t x) { return p.m == 1 ? x : __umulhi(x, p.m_magic); }
+
 // Failure round (global clock) of process `proc`, which may differ from lane to lane. pfw: this lane's word of
 // the pre-operation mask; iv / ir: this lane's in-operation slot (victim or FTC_INOP_UNUSED, merged round).
 __device__ __forceinline__ uint32_t fail_round_lanes(uint32_t pfw, uint32_t iv, uint32_t ir, uint32_t max_inop, uint32_t proc) {
@@ -35,6 +39,8 @@ __device__ __forceinline__ uint32_t fail_round_lanes(uint32_t pfw, uint32_t iv, 
 // ev / er: in-operation slot `lane` as the caller passed it (lanes >= max_inop: anything).
 // Returns false when the scenario is left to the general routines: a root out of range, or more failed processes
 // (before and during the operation) than the f the schedule tolerates. All lanes call; all get the same answer.
+// ALLRED / INOP: compile-time copies of p.is_allreduce != 0 and p.max_inop != 0 (code that cannot run is left out).
+template <bool ALLRED, bool INOP>
 __device__ __forceinline__ bool decode_warp(const Params& p, uint32_t pfw, uint32_t ev, uint32_t er, uint32_t first_root, WarpScen& o) {
     const uint32_t lane = threadIdx.x & 31;
     if (first_root >= p.P) return false;
@@ -42,10 +48,11 @@ __device__ __forceinline__ bool decode_warp(const Params& p, uint32_t pfw, uint3
 
     // in-operation slots: a victim out of range or failed before the operation does not count; slots naming the
     // same victim merge into the earliest round; the first of them stands for the victim
-    uint32_t v = (lane < p.max_inop && ev < p.P) ? ev : FTC_INOP_UNUSED;
-    uint32_t rmin = lane < p.max_inop ? er : 0u;
-    uint32_t ifirst;
-    {
+    uint32_t v = (INOP && lane < p.max_inop && ev < p.P) ? ev : FTC_INOP_UNUSED;
+    uint32_t rmin = (INOP && lane < p.max_inop) ? er : 0u;
+    uint32_t ifirst = 0;
+    o.any_victim = 0;
+    if (INOP) {
         const uint32_t word = __shfl_sync(kFullWarp, pfw, v == FTC_INOP_UNUSED ? 0u : v >> 5);
         const bool pre = v != FTC_INOP_UNUSED && ((word >> (v & 31)) & 1u);
         bool first = true;
@@ -57,19 +64,19 @@ __device__ __forceinline__ bool decode_warp(const Params& p, uint32_t pfw, uint3
         if (pre) v = FTC_INOP_UNUSED;
         o.any_victim = __ballot_sync(kFullWarp, v != FTC_INOP_UNUSED);
         ifirst = __ballot_sync(kFullWarp, v != FTC_INOP_UNUSED && first);
-        if (npre + __popc(ifirst) > p.f) return false;
     }
+    if (npre + __popc(ifirst) > p.f) return false;
     const uint32_t iv = v, ir = rmin;
 
     // the root of the attempt that counts (Algorithm "Allreduce": the first candidate that had not failed beforehand)
     uint32_t code = FTC_ST_OK, root = first_root, base = 0, attempts = 1;
-    if (!p.is_allreduce) {
+    if (!ALLRED) {
         // the root must be alive when the last tree messages arrive (round f+H-1)
-        if (fail_round_lanes(pfw, iv, ir, p.max_inop, first_root) < p.Rred) code = FTC_ST_ROOT_FAILED;
+        if (fail_round_lanes(pfw, iv, ir, INOP ? p.max_inop : 0u, first_root) < p.Rred) code = FTC_ST_ROOT_FAILED;
     } else {
         uint32_t c = first_root + (lane < p.m ? lane : 0u);
         if (c >= p.P) c -= p.P;
-        const uint32_t fr = fail_round_lanes(pfw, iv, ir, p.max_inop, c);
+        const uint32_t fr = fail_round_lanes(pfw, iv, ir, INOP ? p.max_inop : 0u, c);
         const uint32_t inopc = __ballot_sync(kFullWarp, lane < p.m && fr != 0 && fr != kNever);
         const uint32_t alive = __ballot_sync(kFullWarp, lane < p.m && fr != 0);
         if (inopc) { code = FTC_ST_PRECONDITION_INOP_ROOT; attempts = 0; }
@@ -88,13 +95,13 @@ __device__ __forceinline__ bool decode_warp(const Params& p, uint32_t pfw, uint3
     uint32_t F = 0;
     for (uint32_t word = pfw; word; word &= word - 1) {
         const uint32_t vr = renumber((lane << 5) + (__ffs(word) - 1), root);
-        if (vr) F |= 1u << ((vr - 1) % p.m);
+        if (vr) F |= 1u << ((vr - 1) - div_m(p, vr - 1) * p.m);
     }
-    const uint32_t vren = iv != FTC_INOP_UNUSED ? renumber(iv, root) : 0u;
-    const uint32_t t = local_round(ir, base);
+    const uint32_t vren = (INOP && iv != FTC_INOP_UNUSED) ? renumber(iv, root) : 0u;
+    const uint32_t t = INOP ? local_round(ir, base) : kNever;
     uint32_t j = 0, sv = 0;
-    if (vren) {
-        j = (vren - 1) / p.m; sv = (vren - 1) - j * p.m;
+    if (INOP && vren) {
+        j = div_m(p, vren - 1); sv = (vren - 1) - j * p.m;
         const uint32_t d = 1 + ilog2u(j + 1);
         if (!(p.f + p.H - d < t)) F |= 1u << sv;                        // tree send of depth d is round f+H-d
     }
@@ -121,23 +128,25 @@ __device__ __forceinline__ bool decode_warp(const Params& p, uint32_t pfw, uint3
     // an in-operation victim is included iff its up-correction message to the selected subtree's member of its group
     // (or to the root, when the group has no member there) was still sent
     bool included = true;
-    if (vren) {
+    if (INOP && vren) {
         const bool member_in_subtree = j < p.q || sstar < p.r;
         if (member_in_subtree) { if (sv != sstar) included = partner_slot(p, j, sv, sstar) < t; }
         else included = t > root_slot(p);
     }
-    o.inop_incl = __ballot_sync(kFullWarp, iv != FTC_INOP_UNUSED && included);
-    const uint32_t excl = __ballot_sync(kFullWarp, iv != FTC_INOP_UNUSED && !included);
-    o.nexcl = __popc(excl & ifirst);
-    for (uint32_t e = excl; e; e &= e - 1) {                            // the same in every lane
-        const uint32_t vj = __shfl_sync(kFullWarp, vren, __ffs(e) - 1);
-        if (lane == (vj >> 5)) incw &= ~(1u << (vj & 31));
+    if (INOP) {
+        o.inop_incl = __ballot_sync(kFullWarp, iv != FTC_INOP_UNUSED && included);
+        const uint32_t excl = __ballot_sync(kFullWarp, iv != FTC_INOP_UNUSED && !included);
+        o.nexcl = __popc(excl & ifirst);
+        for (uint32_t e = excl; e; e &= e - 1) {                        // the same in every lane
+            const uint32_t vj = __shfl_sync(kFullWarp, vren, __ffs(e) - 1);
+            if (lane == (vj >> 5)) incw &= ~(1u << (vj & 31));
+        }
     }
     o.incw = incw;
     // broadcast: with at most f failures a failure-free subtree carries the value to every group, so everybody
     // alive at the end of the attempt holds it
-    if (p.is_allreduce) {
-        const uint32_t dead_end = __ballot_sync(kFullWarp, iv != FTC_INOP_UNUSED && t < p.Ratt) & ifirst;
+    if (ALLRED) {
+        const uint32_t dead_end = INOP ? (__ballot_sync(kFullWarp, iv != FTC_INOP_UNUSED && t < p.Ratt) & ifirst) : 0u;
         o.holders = p.P - npre - __popc(dead_end);
     }
     return true;

@@ -35,6 +35,7 @@ struct Params {
     uint32_t swz_mask; // swizzled tiles: XOR mask of the 16-byte chunk bits (0x70: 128-byte lines, 0x30: 64-byte lines)
     uint32_t row_shift; // swizzled tiles of 64-byte groups: tile rows after the first sit one row further (128-byte aligned levels)
     uint32_t below;    // 1: the heap's sparsely filled last level lies below the tiles (its rows are folded one by one)
+    uint32_t m_magic;  // ceil(2^32 / m): floor(x / m) = (x * m_magic) >> 32 for every x below 2^26 (m <= 32)
     uint32_t* grid_query;  // host side only: when set, a launcher stores the number of blocks it would launch and launches nothing
 };
 

@@ -212,10 +212,13 @@ struct SubComb {
 // of the selected subtree's member first, then the partners ascending: Algorithm "Up-correction"), so that the
 // loads and adds of different rows overlap; then the sub-heap is combined. The tile has no renumbered slot, no
 // short group and is complete down to its second-to-last level. `masked`: some group of the tile misses a member.
-template <typename T, int OP, int XL, bool WHOLE, bool SW = false>
+// SHORT: the tile may hold the short last group (row `short_row`; its members end before a full group's would, the
+// bytes behind them are readable): whatever the common fold made of that row is replaced by the general fold.
+template <typename T, int OP, int XL, bool WHOLE, bool SW = false, bool SHORT = false>
 __device__ __forceinline__ void fold_tile_fast(const Params& p, uint32_t root, uint32_t sstar, const uint32_t* inc, const char* in_lc,
                                                const char* buf_lc, uint32_t rowbytes, uint32_t j0, uint32_t lr, uint32_t rot, uint32_t rowB, bool hasB,
-                                               uint32_t tA, uint32_t rowA, uint32_t G, bool masked, uint4& valA, uint4& valB) {
+                                               uint32_t tA, uint32_t rowA, uint32_t G, bool masked, uint4& valA, uint4& valB,
+                                               uint32_t short_row = 0xFFFFFFFFu) {
     constexpr int NS = 1 << XL;
     const LdStaged<SW> lds(p.swz_mask);
     uint32_t off[NS], grow[NS];
@@ -268,6 +271,11 @@ __device__ __forceinline__ void fold_tile_fast(const Params& p, uint32_t root, u
                     if ((mask[s] >> sp) & 1u) acc[s] = comb16<T, OP>(acc[s], lds(mem + off[s]));
             }
         }
+    }
+    if (SHORT) {
+#pragma unroll
+        for (int s = 0; s < NS; ++s)
+            if (grow[s] == short_row) acc[s] = fold_staged_call<T, OP, WHOLE, SW>(fold_shape(p), root, sstar, inc, in_lc, nullptr, short_row);
     }
     valB = acc[0];
     valA = SubComb<T, OP, XL, 0, WHOLE>::eval(p, root, sstar, inc, in_lc, acc, grow, G);

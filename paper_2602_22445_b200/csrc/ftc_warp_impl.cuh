@@ -4,7 +4,10 @@
 // (ftc_decode_warp.cuh), consecutive scenarios arrive several at a time by one bulk copy into the warp's own double
 // buffer, their masks, in-operation entries and roots are fetched one group ahead into registers, and the whole
 // subtree heap of a scenario is one warp tile (lanes = lane rows x 16-byte chunks, lane-local sub-heaps below,
-// shuffles above), evaluated by the same routines as the tiles of the staged kernel.
+// shuffles above), evaluated by the same routines as the tiles of the staged kernel. The tile has exactly as many
+// levels as the heap (fewer lane rows are used when the heap is shallow), so it is complete down to its
+// second-to-last level and the check-free folds serve every scenario; only the short last group, one row, is
+// folded by the general routine.
 // Before the evaluation the warp exchanges the vectors of process 0 and of the root in its copy of the scenario, so
 // that the copy is in renumbered order (section "Reduce": the root swaps numbers with process 0) and no group needs
 // special addressing. Scenarios the register decode leaves out (more failures than tolerated, a root out of range)
@@ -16,15 +19,19 @@
 namespace ftc {
 
 struct WarpGeom {
+    uint32_t lw;           // levels of the tile combined with shuffles: 2^lw lane rows are used
     uint32_t group;        // scenarios per buffer (consecutive scenarios, one bulk copy)
     uint32_t buf_bytes;    // bytes per buffer (multiple of 128)
     uint32_t off_bar, off_buf, smem_bytes;
 };
 
-constexpr int kWarpMinBlocks = 16;
+// blocks (= warps) per SM the register budget allows: sub-heaps of three levels keep eight rows per lane in registers
+template <int XL> struct WarpMinBlocks { static constexpr int value = XL >= 3 ? 16 : 32; };
 
-template <typename T, int OP, int XL>
-__global__ void __launch_bounds__(32, kWarpMinBlocks) warp_kernel(Params p, WarpGeom g) {
+// MODE: bit 0 = allreduce, bit 1 = the call has in-operation slots.
+template <typename T, int OP, int XL, int MODE>
+__global__ void __launch_bounds__(32, WarpMinBlocks<XL>::value) warp_kernel(Params p, WarpGeom g) {
+    constexpr bool ALLRED = (MODE & 1) != 0, INOP = (MODE & 2) != 0;
     extern __shared__ __align__(128) uint32_t smem[];
     char* sbase = reinterpret_cast<char*>(smem);
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
@@ -32,9 +39,9 @@ __global__ void __launch_bounds__(32, kWarpMinBlocks) warp_kernel(Params p, Warp
     uint32_t* inc = pf + p.W + 1;
     uint32_t* unr = inc + p.W + 1;
     const uint32_t lane = threadIdx.x;
-    const uint32_t cwl = p.cw_log2, lw = 5 - cwl, RW = 1u << lw;
-    const uint32_t lr = lane >> cwl, lc = lane & (p.C - 1);
-    const uint32_t D = lw + XL;
+    const uint32_t cwl = p.cw_log2, lw = g.lw, RW = 1u << lw;
+    const uint32_t lr_real = lane >> cwl, lc = lane & (p.C - 1);
+    const uint32_t lr = lr_real < RW ? lr_real : 0u;                    // lane rows beyond the tile repeat lane row 0 (their results are unused)
     const uint32_t nq = p.C < 8 ? 8u / p.C : 1u, gq = min(nq, p.m & (0u - p.m));
     const uint32_t rot = (lr >> ilog2u(nq / gq)) & (gq - 1);          // starting member of this lane row's folds (bank spread)
     const uint32_t rowbytes = p.m * p.kbytes;
@@ -97,18 +104,21 @@ __global__ void __launch_bounds__(32, kWarpMinBlocks) warp_kernel(Params p, Warp
             uint32_t pfw = __shfl_sync(kFullWarp, cur.pfw, lane < p.W ? i * p.W + lane : 0u);
             if (lane >= p.W) pfw = 0;
             else if (lane == p.W - 1 && (p.P & 31)) pfw &= (1u << (p.P & 31)) - 1u;
-            const uint32_t src = lane < p.max_inop ? i * p.max_inop + lane : 0u;
-            const uint32_t ev = __shfl_sync(kFullWarp, cur.vic, src), er = __shfl_sync(kFullWarp, cur.rnd, src);
+            uint32_t ev = FTC_INOP_UNUSED, er = 0;
+            if (INOP) {
+                const uint32_t src = lane < p.max_inop ? i * p.max_inop + lane : 0u;
+                ev = __shfl_sync(kFullWarp, cur.vic, src); er = __shfl_sync(kFullWarp, cur.rnd, src);
+            }
             const uint32_t first_root = p.root >= 0 ? (uint32_t)p.root : __shfl_sync(kFullWarp, cur.root, i);
             WarpScen w;
-            if (decode_warp(p, pfw, ev, er, first_root, w)) {
+            if (decode_warp<ALLRED, INOP>(p, pfw, ev, er, first_root, w)) {
                 if (lane <= p.W) inc[lane] = w.incw;
                 if (p.W == 32 && lane == 0) inc[32] = 0;
                 __syncwarp();
             } else {
                 // the general routines (a block of one warp may call them): everything outside the register decode
                 decode_scenario(p, s, cx, pf, inc);
-                if (cx->code == FTC_ST_OK && p.is_allreduce) count_holders(p, cx, pf, unr);
+                if (cx->code == FTC_ST_OK && ALLRED) count_holders(p, cx, pf, unr);
                 w.code = cx->code; w.sstar = cx->sstar; w.attempts = cx->attempts; w.root = cx->root; w.base = cx->base;
                 w.npre = cx->npre; w.nexcl = cx->nexcl; w.inop_incl = cx->inop_incl; w.holders = cx->holders; w.G = cx->G;
                 w.any_victim = 1;
@@ -134,21 +144,13 @@ __global__ void __launch_bounds__(32, kWarpMinBlocks) warp_kernel(Params p, Warp
                 // the one tile: heap rows 0 .. 2^D - 2; lane row lr owns row lr of the upper levels and the sub-heap under row RW-1+lr
                 const uint32_t tA = RW - 1 + lr, rowA = tA, tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB), rowB = lr;
                 const bool masked = w.npre != 0 || w.any_victim != 0;
-                // the short last group and a heap that does not fill the tile down to its second-to-last level take the careful folds
-                const bool careful = G > p.q || ((2u << (D >= 2 ? D - 2 : 0)) - 2 >= G);
-                uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
-                if (!careful) {
-                    const bool hasB = lr < RW - 1;
-                    fold_tile_fast<T, OP, XL, true, false>(p, 0u, sstar, inc, in_lc, in_lc, rowbytes, 0u, lr, rot, rowB, hasB, tA, rowA, G, masked, valA, valB);
-                    valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
-                } else {
-                    if (rowA < G) valA = SubHeap<T, OP, XL, 0, true, true, false>::eval(p, 0u, sstar, inc, in_lc, in_lc, rowbytes, tA, rowA, G);
-                    const bool hasB = lr < RW - 1 && rowB < G;
-                    if (hasB) valB = fold_staged_call<T, OP, true, false>(fold_shape(p), 0u, sstar, inc, in_lc, in_lc + staged_row_offset<true>(p, rowbytes, lr, rowB), rowB);
-                    valB = tile_tree_phase<T, OP>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
-                }
+                uint4 valA, valB;
+                const bool hasB = lr < RW - 1;
+                fold_tile_fast<T, OP, XL, true, false, true>(p, 0u, sstar, inc, in_lc, in_lc, rowbytes, 0u, lr, rot, rowB, hasB, tA, rowA, G, masked, valA, valB,
+                                                             G > p.q ? p.q : 0xFFFFFFFFu);
+                valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                 // the root (Algorithm "reduce_root"): its own data on the left unless the child's subtree holds it already
-                if (lr == 0) {
+                if (lr_real == 0) {
                     uint4 recv = lw ? valB : valA;
                     if (sstar >= p.r) recv = comb16<T, OP>(fold_root16<T, OP, LdShared>(p, 0u, inc, in_lc), recv);
                     reinterpret_cast<uint4*>(out_s)[lc] = recv;
@@ -160,7 +162,7 @@ __global__ void __launch_bounds__(32, kWarpMinBlocks) warp_kernel(Params p, Warp
                 rec.x = code | ((okc ? w.sstar : 0xFFu) << 8) | (w.attempts << 16);
                 rec.y = okc ? p.P - w.npre - w.nexcl : 0u;
                 rec.z = okc ? w.inop_incl : 0u;
-                rec.w = (okc && p.is_allreduce) ? w.holders : 0u;
+                rec.w = (okc && ALLRED) ? w.holders : 0u;
                 *reinterpret_cast<uint4*>(p.status + s * FTC_STATUS_WORDS) = rec;
             }
             __syncwarp();
@@ -177,7 +179,7 @@ __global__ void __launch_bounds__(32, kWarpMinBlocks) warp_kernel(Params p, Warp
 // subtree heap that fits one warp tile with a lane-local sub-heap of at most three levels, scenarios of at most
 // kWarpMaxBytes. XL: the shallowest sub-heap that holds the heap.
 constexpr uint64_t kWarpMaxBytes = 8 * 1024;
-constexpr uint32_t kWarpBufTarget = 4 * 1024;       // a buffer holds as many consecutive scenarios as fit in this (at least one)
+constexpr uint32_t kWarpBufTarget = 2560;       // a buffer holds as many consecutive scenarios as fit in this (at least one)
 
 static bool warp_geometry(Params& p, int smem_optin, uint32_t& XL, WarpGeom& g) {
     if (p.kbytes % 16 || p.W > 32) return false;
@@ -189,14 +191,16 @@ static bool warp_geometry(Params& p, int smem_optin, uint32_t& XL, WarpGeom& g) 
     const uint32_t lw = 5 - cwl;
     uint32_t Hmax = 1; while ((1u << Hmax) <= p.Gmax) ++Hmax;
     if (Hmax > lw + 3) return false;
-    XL = Hmax > lw + 1 ? Hmax - lw : 1u;
+    g.lw = Hmax - 1 < lw ? Hmax - 1 : lw;                      // a shallow heap uses fewer lane rows
+    XL = Hmax - g.lw;
     p.C = C; p.cw_log2 = cwl; p.Lt = 0; p.below = 0; p.swz_mask = 0; p.row_shift = 0;
     uint32_t group = (uint32_t)(kWarpBufTarget / scen_bytes);
     if (group < 1) group = 1;
     while (group > 1 && (group * p.W > 32 || group * p.max_inop > 32 || group > 32)) --group;
     if (p.max_inop > 32) return false;
     g.group = group;
-    g.buf_bytes = (uint32_t)((group * scen_bytes + 127) & ~(uint64_t)127);
+    // behind the last scenario: room for the bytes a full group would have beyond the short last group (read, not used)
+    g.buf_bytes = (uint32_t)((group * scen_bytes + (uint64_t)p.m * p.kbytes + 127) & ~(uint64_t)127);
     size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
     o = (o + 15) & ~(size_t)15; g.off_bar = (uint32_t)o; o += 16;
     o = (o + 127) & ~(size_t)127; g.off_buf = (uint32_t)o;
@@ -205,19 +209,29 @@ static bool warp_geometry(Params& p, int smem_optin, uint32_t& XL, WarpGeom& g) 
     return o <= (size_t)smem_optin - 1024;
 }
 
-template <typename T, int OP, int XL>
-static cudaError_t launch_warp_x(const Params& p, const WarpGeom& g, int sm_count, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(warp_kernel<T, OP, XL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
+template <typename T, int OP, int XL, int MODE>
+static cudaError_t launch_warp_m(const Params& p, const WarpGeom& g, int sm_count, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(warp_kernel<T, OP, XL, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, warp_kernel<T, OP, XL>, 32, g.smem_bytes);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, warp_kernel<T, OP, XL, MODE>, 32, g.smem_bytes);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     const uint64_t ngroups = (p.S + g.group - 1) / g.group, cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(ngroups < cap ? ngroups : cap);
     if (p.grid_query) { *p.grid_query = grid; return cudaSuccess; }
-    warp_kernel<T, OP, XL><<<grid, 32, g.smem_bytes, st>>>(p, g);
+    warp_kernel<T, OP, XL, MODE><<<grid, 32, g.smem_bytes, st>>>(p, g);
     return cudaGetLastError();
+}
+
+template <typename T, int OP, int XL>
+static cudaError_t launch_warp_x(const Params& p, const WarpGeom& g, int sm_count, cudaStream_t st) {
+    switch ((p.is_allreduce ? 1 : 0) | (p.max_inop ? 2 : 0)) {
+    case 0: return launch_warp_m<T, OP, XL, 0>(p, g, sm_count, st);
+    case 1: return launch_warp_m<T, OP, XL, 1>(p, g, sm_count, st);
+    case 2: return launch_warp_m<T, OP, XL, 2>(p, g, sm_count, st);
+    default: return launch_warp_m<T, OP, XL, 3>(p, g, sm_count, st);
+    }
 }
 
 template <typename T, int OP>
