@@ -15,6 +15,7 @@ struct WarpScen {
     uint32_t any_victim;     // some in-operation slot counts (its victim is in range and had not failed before the operation)
     // per lane
     uint32_t incw;           // word `lane` of the arrival mask over renumbered ranks (0 beyond the mask)
+    uint32_t iv;             // in-operation slot `lane`: its victim, or FTC_INOP_UNUSED when the slot does not count
 };
 
 constexpr uint32_t kFullWarp = 0xFFFFFFFFu;
@@ -39,9 +40,12 @@ __device__ __forceinline__ uint32_t fail_round_lanes(uint32_t pfw, uint32_t iv, 
 // ev / er: in-operation slot `lane` as the caller passed it (lanes >= max_inop: anything).
 // Returns false when the scenario is left to the general routines: a root out of range, or more failed processes
 // (before and during the operation) than the f the schedule tolerates. All lanes call; all get the same answer.
-// ALLRED / INOP: compile-time copies of p.is_allreduce != 0 and p.max_inop != 0 (code that cannot run is left out).
-template <bool ALLRED, bool INOP>
+// ALLRED_ / INOP_: 0 or 1 = compile-time copies of p.is_allreduce != 0 and p.max_inop != 0 (code that cannot run is
+// left out); 2 = look at p when running.
+template <int ALLRED_, int INOP_>
 __device__ __forceinline__ bool decode_warp(const Params& p, uint32_t pfw, uint32_t ev, uint32_t er, uint32_t first_root, WarpScen& o) {
+    const bool ALLRED = ALLRED_ == 2 ? p.is_allreduce != 0 : ALLRED_ != 0;
+    const bool INOP = INOP_ == 2 ? p.max_inop != 0 : INOP_ != 0;
     const uint32_t lane = threadIdx.x & 31;
     if (first_root >= p.P) return false;
     const uint32_t npre = __reduce_add_sync(kFullWarp, __popc(pfw));
@@ -88,7 +92,7 @@ __device__ __forceinline__ bool decode_warp(const Params& p, uint32_t pfw, uint3
         }
     }
     o.code = code; o.root = root; o.base = base; o.attempts = attempts; o.npre = npre;
-    o.sstar = 0xFF; o.nexcl = 0; o.inop_incl = 0; o.holders = 0; o.G = 0; o.incw = 0;
+    o.sstar = 0xFF; o.nexcl = 0; o.inop_incl = 0; o.holders = 0; o.G = 0; o.incw = 0; o.iv = iv;
     if (code != FTC_ST_OK) return true;
 
     // failed bits of the root's children: a subtree is unclean iff one of its processes does not send up the tree
@@ -150,6 +154,37 @@ __device__ __forceinline__ bool decode_warp(const Params& p, uint32_t pfw, uint3
         o.holders = p.P - npre - __popc(dead_end);
     }
     return true;
+}
+
+// Work items of the staged kernel that need the careful path or the masked folds, for a block of one warp whose
+// tiles and groups of upper rows number at most 32: the same marks as mark_special_items(), as two words.
+// pfw: this lane's word of the pre-operation mask; iv: this lane's in-operation slot (victim or FTC_INOP_UNUSED).
+__device__ __forceinline__ void mark_special_warp(const Params& p, uint32_t pfw, uint32_t iv, uint32_t root, uint32_t G, uint32_t Lt,
+                                                  uint32_t D, bool below, uint32_t grows, uint32_t ngroups, uint32_t& spec, uint32_t& mask) {
+    const uint32_t lane = threadIdx.x & 31, ntiles = 1u << Lt, ntop = ntiles - 1;
+    auto item_bit = [&](uint32_t j) -> uint32_t {
+        const uint32_t lvl = ilog2u(j + 1);
+        if (below && lvl >= Lt + D) return 0u;                      // rows under the tiles are folded one by one anyway
+        return 1u << (lvl >= Lt ? ((j + 1) >> (lvl - Lt)) - ntiles : ntiles + j / grows);
+    };
+    uint32_t mk = 0, sp = 0;
+    for (uint32_t word = pfw; word; word &= word - 1) {
+        const uint32_t v = renumber((lane << 5) + (__ffs(word) - 1), root);
+        if (v) { const uint32_t j = div_m(p, v - 1); if (j < G) mk |= item_bit(j); }
+    }
+    if (iv != FTC_INOP_UNUSED) {
+        const uint32_t v = renumber(iv, root);
+        if (v) { const uint32_t j = div_m(p, v - 1); if (j < G) mk |= item_bit(j); }
+    }
+    if (lane == 0) {
+        if (root != 0 && div_m(p, root - 1) < G) sp |= item_bit(div_m(p, root - 1));   // the slot that holds process 0's input
+        if (G > p.q) sp |= item_bit(p.q);                                              // the short last group
+    }
+    if (lane < ntiles && ((((ntop + lane + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= G) || (!below && ((ntop + lane + 1) << D) - 1 < G)))
+        sp |= 1u << lane;
+    if (lane < ngroups && ((lane + 1) * grows > ntop || (lane + 1) * grows > G)) sp |= 1u << (ntiles + lane);
+    mask = __reduce_or_sync(kFullWarp, mk);
+    spec = __reduce_or_sync(kFullWarp, sp);
 }
 
 }  // namespace ftc

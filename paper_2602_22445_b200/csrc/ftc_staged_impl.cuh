@@ -21,6 +21,7 @@
 #pragma once
 #include <cuda.h>
 #include "ftc_tile_common.cuh"
+#include "ftc_decode_warp.cuh"
 #include "ftc_kernels.h"
 
 namespace ftc {
@@ -448,6 +449,19 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
     auto release = [&]() { __syncwarp(); if (!WHOLE && ++cbuf == g.nbuf) cbuf = 0; issue_next(); };
     if (!WHOLE) for (uint32_t i = 0; i < g.nbuf; ++i) issue_next();
 
+    // Blocks of one warp whose masks are one word per lane decode in registers (ftc_decode_warp.cuh) and fetch the next
+    // scenario's mask word, in-operation entry and root while the current scenario is played.
+    const bool warp_decode = LEAN && !WHOLE && nw == 1 && p.W <= 32 && ntiles + ngroups <= 32;
+    uint32_t nx_pf = 0, nx_vic = FTC_INOP_UNUSED, nx_rnd = 0, nx_root = 0;
+    auto fetch_small = [&](uint64_t s) {
+        nx_pf = 0; nx_vic = FTC_INOP_UNUSED; nx_rnd = 0; nx_root = 0;
+        if (s >= p.S) return;
+        if (lane < p.W) nx_pf = __ldg(p.prefail + s * p.W + lane);
+        if (lane < p.max_inop) { const ftc_inop_t* e = p.inop + s * p.max_inop + lane; nx_vic = __ldg(&e->victim); nx_rnd = __ldg(&e->round); }
+        if (p.root < 0) nx_root = __ldg(p.roots + s);
+    };
+    if (LEAN && warp_decode) fetch_small(blockIdx.x);
+
     for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {
         const char* in_s = reinterpret_cast<const char*>(p.in) + s * scen_bytes;
         // uniform: the flag is only written between the barriers of a scenario, and a barrier ended the previous one
@@ -460,7 +474,31 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
             for (uint64_t o = (uint64_t)lane * 32768; o < scen_bytes; o += 32u * 32768)
                 bulk_g2s(smem_addr(wbuf + o), in_s + o, (uint32_t)min((uint64_t)32768, scen_bytes - o), cbar);
         }
-        decode_scenario(p, s, cx, pf, inc);
+        bool marked = false;
+        if (LEAN && warp_decode) {
+            uint32_t pfw = nx_pf;
+            if (lane == p.W - 1 && (p.P & 31)) pfw &= (1u << (p.P & 31)) - 1u;
+            const uint32_t ev = nx_vic, er = nx_rnd, first_root = p.root >= 0 ? (uint32_t)p.root : nx_root;
+            fetch_small(s + gridDim.x);
+            WarpScen w;
+            if (decode_warp<2, 2>(p, pfw, ev, er, first_root, w)) {
+                if (lane == 0) {
+                    cx->code = w.code; cx->sstar = w.sstar; cx->attempts = w.attempts; cx->root = w.root; cx->base = w.base;
+                    cx->npre = w.npre; cx->nexcl = w.nexcl; cx->inop_incl = w.inop_incl; cx->holders = w.holders; cx->G = w.G;
+                    pf[p.W] = 0;
+                }
+                if (lane < p.W) pf[lane] = pfw;
+                if (lane <= p.W) inc[lane] = w.incw;
+                if (p.W == 32 && lane == 0) inc[32] = 0;
+                if (w.code == FTC_ST_OK) {
+                    uint32_t spec, mask;
+                    mark_special_warp(p, pfw, w.iv, w.root, w.G, Lt, D, p.below != 0, grows, ngroups, spec, mask);
+                    if (lane == 0) { tspec[0] = spec; tspec[1] = 0; tmask[0] = mask; tmask[1] = 0; }
+                }
+                marked = true;
+                __syncwarp();
+            } else decode_scenario(p, s, cx, pf, inc);
+        } else decode_scenario(p, s, cx, pf, inc);
         char* out_s = reinterpret_cast<char*>(p.out) + s * p.kbytes;
         if (WHOLE && !dead) {
             // every thread sees the copy complete before it reads it or leaves the iteration
@@ -478,8 +516,10 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
             __syncthreads();
             continue;
         }
-        if (p.is_allreduce) count_holders(p, cx, pf, unr);
-        mark_special_items(p, cx, pf, tspec, tmask, Lt, lw, D, LEAN && p.below != 0, grows, ngroups);
+        if (!marked) {                 // warp-uniform, and the block is one warp when it is set
+            if (p.is_allreduce) count_holders(p, cx, pf, unr);
+            mark_special_items(p, cx, pf, tspec, tmask, Lt, lw, D, LEAN && p.below != 0, grows, ngroups);
+        }
         const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
         const char* in_lc = (WHOLE ? wbuf : in_s) + lc * 16;      // the scenario in process order, for the general fold
 

@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(32, WarpMinBlocks<XL>::value) warp_kernel(Para
             }
             const uint32_t first_root = p.root >= 0 ? (uint32_t)p.root : __shfl_sync(kFullWarp, cur.root, i);
             WarpScen w;
-            if (decode_warp<ALLRED, INOP>(p, pfw, ev, er, first_root, w)) {
+            if (decode_warp<(ALLRED ? 1 : 0), (INOP ? 1 : 0)>(p, pfw, ev, er, first_root, w)) {
                 if (lane <= p.W) inc[lane] = w.incw;
                 if (p.W == 32 && lane == 0) inc[32] = 0;
                 __syncwarp();
