@@ -79,7 +79,7 @@ static const DeviceInfo kB200 = {148, 232448};
 
 enum KernelKind { K_GENERIC = 0, K_TILED = 1, K_STAGED = 2 };
 static KernelKind pick_kernel(Params& p, const DeviceInfo& di) {
-    if ((p.flags & FTC_KERNEL_GENERIC) || p.arity != 2 || p.pdesc) return K_GENERIC;   // the tiled kernels are built on the binary heap and the ascending order
+    if ((p.flags & FTC_KERNEL_GENERIC) || p.arity != 2) return K_GENERIC;   // the tiled kernels are built on the binary heap
     if (!(p.flags & FTC_KERNEL_DIRECT) && staged_supported(p, di.smem_optin, di.sm_count)) return K_STAGED;
     return tiled_supported(p, di.smem_optin) ? K_TILED : K_GENERIC;
 }

@@ -106,7 +106,7 @@ struct LdStaged {
 // Fold of a plain group from its staged copy.
 template <typename T, int OP, bool SW = false>
 __device__ __forceinline__ uint4 fold_plain_staged(const Params& p, uint32_t sstar, const char* srow_lc) {
-    return fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdStaged<SW>(p.swz_mask));
+    return fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdStaged<SW>(p.swz_mask), p.pdesc != 0);
 }
 
 // Fold of one group on the careful path: a full group without a renumbered slot comes from its staged copy
@@ -117,7 +117,7 @@ __device__ __forceinline__ uint4 fold_staged(const Params& p, uint32_t root, uin
                                              const char* in_lc, const char* srow_lc, uint32_t row) {
     const uint32_t vbase = row * p.m + 1;
     if (srow_lc && row < p.q && root - vbase >= p.m)      // full group, no renumbered slot in it: its staged copy serves
-        return fold16_masked<T, OP>(srow_lc, p.kbytes, p.m, extract_bits(inc, vbase, p.m), sstar, LdShared());
+        return fold16_masked<T, OP>(srow_lc, p.kbytes, p.m, extract_bits(inc, vbase, p.m), sstar, LdShared(), p.pdesc != 0);
     if (WHOLE) return fold16_careful<T, OP, LdShared>(p, root, sstar, inc, in_lc, row);
     return fold16_careful<T, OP, LdGlobal>(p, root, sstar, inc, in_lc, row);
 }
@@ -127,7 +127,7 @@ __device__ __forceinline__ uint4 fold_staged(const Params& p, uint32_t root, uin
 // MASKED: groups may miss members (fold under the arrival mask in `inc`), otherwise the same.
 template <typename T, int OP, bool MASKED>
 __device__ __forceinline__ uint4 fold_fast_staged(const Params& p, uint32_t sstar, const uint32_t* inc, const char* srow_lc, uint32_t grow) {
-    if (MASKED) return fold16_masked<T, OP>(srow_lc, p.kbytes, p.m, extract_bits(inc, grow * p.m + 1, p.m), sstar, LdShared());
+    if (MASKED) return fold16_masked<T, OP>(srow_lc, p.kbytes, p.m, extract_bits(inc, grow * p.m + 1, p.m), sstar, LdShared(), p.pdesc != 0);
     return fold_plain_staged<T, OP>(p, sstar, srow_lc);
 }
 
@@ -161,15 +161,15 @@ __device__ __noinline__ uint4 fold_staged_call(FoldShape fs, uint32_t root, uint
                                                const char* in_lc, const char* srow_lc, uint32_t row) {
     const uint32_t vbase = row * fs.m + 1;
     if (srow_lc && row < fs.q && root - vbase >= fs.m)      // full group, no renumbered slot in it: its staged copy serves
-        return fold16_masked<T, OP>(srow_lc, fs.kbytes, fs.m, extract_bits(inc, vbase, fs.m), sstar, LdStaged<SW>(fs.swz_mask));
+        return fold16_masked<T, OP>(srow_lc, fs.kbytes, fs.m, extract_bits(inc, vbase, fs.m), sstar, LdStaged<SW>(fs.swz_mask), fs.pdesc != 0);
     if (WHOLE) return fold16_general<T, OP, 0, LdShared, FoldShape>(fs, root, sstar, inc, in_lc, row);
     return fold16_general<T, OP, 0, LdGlobal, FoldShape>(fs, root, sstar, inc, in_lc, row);
 }
 
 // A full group some of whose members' messages are missing, from its staged copy.
 template <typename T, int OP, bool SW = false>
-__device__ __noinline__ uint4 fold_masked_call(const char* srow_lc, uint32_t kbytes, uint32_t m, uint32_t mask, uint32_t sstar, uint32_t swz_mask) {
-    return fold16_masked<T, OP>(srow_lc, kbytes, m, mask, sstar, LdStaged<SW>(swz_mask));
+__device__ __noinline__ uint4 fold_masked_call(const char* srow_lc, uint32_t kbytes, uint32_t m, uint32_t mask, uint32_t sstar, uint32_t swz_mask, bool desc) {
+    return fold16_masked<T, OP>(srow_lc, kbytes, m, mask, sstar, LdStaged<SW>(swz_mask), desc);
 }
 
 // One row from its staged copy; `masked`: the work item holds a group with a missing member, so look at the mask.
@@ -178,7 +178,7 @@ __device__ __forceinline__ uint4 fold_row_lean(const Params& p, uint32_t sstar, 
                                                uint32_t grow, bool masked) {
     if (masked) {
         const uint32_t mask = extract_bits(inc, grow * p.m + 1, p.m), full = p.m >= 32 ? 0xFFFFFFFFu : (1u << p.m) - 1u;
-        if (mask != full) return fold_masked_call<T, OP, SW>(srow_lc, p.kbytes, p.m, mask, sstar, p.swz_mask);
+        if (mask != full) return fold_masked_call<T, OP, SW>(srow_lc, p.kbytes, p.m, mask, sstar, p.swz_mask, p.pdesc != 0);
     }
     return fold_plain_staged<T, OP, SW>(p, sstar, srow_lc);
 }
@@ -252,24 +252,30 @@ __device__ __forceinline__ void fold_tile_fast(const Params& p, uint32_t root, u
         const char* own = buf_lc + sstar * p.kbytes;
 #pragma unroll
         for (int s = 0; s < NS; ++s) acc[s] = lds(own + off[s]);
+        // the partners in the schedule's order (ascending rank, or descending), own skipped: one pointer walks the group
+        const bool desc = Ordered<T>::value && p.pdesc != 0;
+        const int32_t step = desc ? -(int32_t)p.kbytes : (int32_t)p.kbytes;
+        const char* mem = desc ? buf_lc + (p.m - 1) * p.kbytes : buf_lc;
         if (!masked) {
 #pragma unroll 1
             for (uint32_t i = 1; i < p.m; ++i) {
-                const char* mem = buf_lc + (i - (i <= sstar ? 1u : 0u)) * p.kbytes;      // partners ascending, own skipped
+                if (mem == own) mem += step;
 #pragma unroll
                 for (int s = 0; s < NS; ++s) acc[s] = comb16<T, OP>(acc[s], lds(mem + off[s]));
+                mem += step;
             }
         } else {
             uint32_t mask[NS];
 #pragma unroll
             for (int s = 0; s < NS; ++s) mask[s] = grow[s] < G ? extract_bits(inc, grow[s] * p.m + 1, p.m) : 0u;
+            uint32_t sp = desc ? p.m - 1 : 0u;
 #pragma unroll 1
             for (uint32_t i = 1; i < p.m; ++i) {
-                const uint32_t sp = i - (i <= sstar ? 1u : 0u);
-                const char* mem = buf_lc + sp * p.kbytes;
+                if (mem == own) { mem += step; sp += desc ? 0xFFFFFFFFu : 1u; }
 #pragma unroll
                 for (int s = 0; s < NS; ++s)
                     if ((mask[s] >> sp) & 1u) acc[s] = comb16<T, OP>(acc[s], lds(mem + off[s]));
+                mem += step; sp += desc ? 0xFFFFFFFFu : 1u;
             }
         }
     }

@@ -47,6 +47,17 @@ __device__ __forceinline__ uint4 fold16_general(const SHAPE& p, uint32_t root, u
     const uint32_t mj = row < p.q ? p.m : p.r, vbase = row * p.m + 1;
     const uint32_t mask = extract_bits(inc, vbase, mj);
     uint4 acc = make_uint4(0, 0, 0, 0);
+    if (Ordered<T>::value && p.pdesc) {
+        // the other partner order: own input, then the partners whose message arrived in descending rank, the root last
+        const uint32_t vo = vbase + sstar;
+        acc = ld(in_lc + (size_t)(vo == root ? 0u : vo) * p.kbytes);
+        for (uint32_t sp = mj; sp-- > 0;) {
+            const uint32_t vr = vbase + sp;
+            if (sp != sstar && ((mask >> sp) & 1u)) acc = comb16<T, OP>(acc, ld(in_lc + (size_t)(vr == root ? 0u : vr) * p.kbytes));
+        }
+        if (row == p.q) acc = comb16<T, OP>(acc, ld(in_lc + (size_t)root * p.kbytes));
+        return acc;
+    }
     if (MCAP > 0) {
         uint4 v[MCAP > 0 ? MCAP : 1];
 #pragma unroll
@@ -88,22 +99,25 @@ __device__ __forceinline__ uint4 fold16_general(const SHAPE& p, uint32_t root, u
 }
 
 // Position in memory of the i-th operand of a full group's fold: for float the member of the selected subtree
-// comes first, then the others ascending; for the exactly associative operations simply ascending.
+// comes first, then the others ascending (desc: descending); for the exactly associative operations simply ascending.
 template <typename T>
-__device__ __forceinline__ uint32_t fold_member(uint32_t i, uint32_t sstar) {
-    return Ordered<T>::value ? (i == 0 ? sstar : i - (i <= sstar ? 1u : 0u)) : i;
+__device__ __forceinline__ uint32_t fold_member(uint32_t i, uint32_t sstar, uint32_t m = 0, bool desc = false) {
+    if (!Ordered<T>::value) return i;
+    if (i == 0) return sstar;
+    if (desc) { const uint32_t c = m - i; return c - (c <= sstar ? 1u : 0u); }
+    return i - (i <= sstar ? 1u : 0u);
 }
 
 // Fold of a full group all of whose members' messages are present, from m vectors `stride` bytes apart starting
 // at `ptr` (global or shared memory, LD loads 16 bytes). MCAP > 0: all loads issued together.
 template <typename T, int OP, int MCAP, typename LD>
-__device__ __forceinline__ uint4 fold16_full(const char* ptr, uint32_t stride, uint32_t m, uint32_t sstar, LD ld) {
+__device__ __forceinline__ uint4 fold16_full(const char* ptr, uint32_t stride, uint32_t m, uint32_t sstar, LD ld, bool desc = false) {
     uint4 acc;
     if (MCAP > 0) {
         uint4 v[MCAP > 0 ? MCAP : 1];
 #pragma unroll
         for (int i = 0; i < MCAP; ++i)
-            if ((uint32_t)i < m) v[i] = ld(ptr + fold_member<T>(i, sstar) * stride);
+            if ((uint32_t)i < m) v[i] = ld(ptr + fold_member<T>(i, sstar, m, desc) * stride);
         acc = v[0];
 #pragma unroll
         for (int i = 1; i < MCAP; ++i)
@@ -111,7 +125,7 @@ __device__ __forceinline__ uint4 fold16_full(const char* ptr, uint32_t stride, u
     } else {
         acc = ld(ptr + fold_member<T>(0, sstar) * stride);
 #pragma unroll 4
-        for (uint32_t i = 1; i < m; ++i) acc = comb16<T, OP>(acc, ld(ptr + fold_member<T>(i, sstar) * stride));
+        for (uint32_t i = 1; i < m; ++i) acc = comb16<T, OP>(acc, ld(ptr + fold_member<T>(i, sstar, m, desc) * stride));
     }
     return acc;
 }
@@ -119,11 +133,13 @@ __device__ __forceinline__ uint4 fold16_full(const char* ptr, uint32_t stride, u
 // Fold of a full-size group some of whose members' messages may be missing (`mask`), from a copy in which the
 // members sit `stride` bytes apart in rank order: own input first, then the arrived ones ascending.
 template <typename T, int OP, typename LD>
-__device__ __forceinline__ uint4 fold16_masked(const char* ptr, uint32_t stride, uint32_t m, uint32_t mask, uint32_t sstar, LD ld) {
+__device__ __forceinline__ uint4 fold16_masked(const char* ptr, uint32_t stride, uint32_t m, uint32_t mask, uint32_t sstar, LD ld, bool desc = false) {
     uint4 acc = ld(ptr + sstar * stride);
 #pragma unroll 2
-    for (uint32_t sp = 0; sp < m; ++sp)
+    for (uint32_t i = 0; i < m; ++i) {
+        const uint32_t sp = (Ordered<T>::value && desc) ? m - 1 - i : i;
         if (sp != sstar && ((mask >> sp) & 1u)) acc = comb16<T, OP>(acc, ld(ptr + sp * stride));
+    }
     return acc;
 }
 
@@ -136,8 +152,8 @@ __device__ __forceinline__ bool group_is_plain(const Params& p, uint32_t root, c
 }
 
 // The four numbers the general fold needs, for passing by value.
-struct FoldShape { uint32_t m, q, r, kbytes, swz_mask; };
-__device__ __forceinline__ FoldShape fold_shape(const Params& p) { return FoldShape{p.m, p.q, p.r, p.kbytes, p.swz_mask}; }
+struct FoldShape { uint32_t m, q, r, kbytes, swz_mask, pdesc; };
+__device__ __forceinline__ FoldShape fold_shape(const Params& p) { return FoldShape{p.m, p.q, p.r, p.kbytes, p.swz_mask, p.pdesc}; }
 
 // Any group, by the general routine (the careful path of the tiled kernels; rare). LD says where `in_lc`, the
 // scenario in process order, lives.
@@ -237,8 +253,8 @@ __device__ __forceinline__ uint4 fold_root16(const Params& p, uint32_t root, con
     uint4 acc = ld(in_lc + (size_t)root * p.kbytes);
     if (p.r) {
         const uint32_t vbase = p.q * p.m + 1, mask = extract_bits(inc, vbase, p.r);
-        for (uint32_t sp = 0; sp < p.r; ++sp) {
-            const uint32_t vr = vbase + sp;
+        for (uint32_t i = 0; i < p.r; ++i) {
+            const uint32_t sp = (Ordered<T>::value && p.pdesc) ? p.r - 1 - i : i, vr = vbase + sp;
             if ((mask >> sp) & 1u) acc = comb16<T, OP>(acc, ld(in_lc + (size_t)(vr == root ? 0u : vr) * p.kbytes));
         }
     }

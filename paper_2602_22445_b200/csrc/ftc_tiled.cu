@@ -60,9 +60,9 @@ __global__ void __launch_bounds__(kTiledMaxThreads, MINB) tiled_kernel(Params p)
                 const uint32_t rowB = ((j0 + 1) << tB) - 1 + idxB;            // this lane's row of the upper levels
                 if (!careful) {
                     // all rows plain, the levels above the bottom complete: constant strides; only the bottom may be ragged
-                    if (rowA < G) valA = fold16_full<T, OP, MCAP>(in_lc + (size_t)(rowA * p.m + 1) * p.kbytes, p.kbytes, p.m, sstar, LdGlobal());
+                    if (rowA < G) valA = fold16_full<T, OP, MCAP>(in_lc + (size_t)(rowA * p.m + 1) * p.kbytes, p.kbytes, p.m, sstar, LdGlobal(), p.pdesc != 0);
                     const bool hasBp = lr < RW - 1;
-                    if (hasBp) valB = fold16_full<T, OP, MCAP>(in_lc + (size_t)(rowB * p.m + 1) * p.kbytes, p.kbytes, p.m, sstar, LdGlobal());
+                    if (hasBp) valB = fold16_full<T, OP, MCAP>(in_lc + (size_t)(rowB * p.m + 1) * p.kbytes, p.kbytes, p.m, sstar, LdGlobal(), p.pdesc != 0);
                     valB = tile_tree_phase<T, OP, false, true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasBp, G);
                     if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                     continue;
@@ -76,7 +76,7 @@ __global__ void __launch_bounds__(kTiledMaxThreads, MINB) tiled_kernel(Params p)
             } else if (it < ntiles + ngroups) {
                 // ---- rows above the tiles: fold now, combine later ----
                 const uint32_t row = ((it - ntiles) << lw) + lr;
-                if (!careful) hv[(size_t)row * p.C + lc] = fold16_full<T, OP, MCAP>(in_lc + (size_t)(row * p.m + 1) * p.kbytes, p.kbytes, p.m, sstar, LdGlobal());
+                if (!careful) hv[(size_t)row * p.C + lc] = fold16_full<T, OP, MCAP>(in_lc + (size_t)(row * p.m + 1) * p.kbytes, p.kbytes, p.m, sstar, LdGlobal(), p.pdesc != 0);
                 else if (row < ntop && row < G) hv[(size_t)row * p.C + lc] = fold16_careful<T, OP, LdGlobal>(p, root, sstar, inc, in_lc, row);
             } else if (sstar >= p.r) {
                 if (lr == 0) rootv[lc] = fold_root16<T, OP>(p, root, inc, in_lc);

@@ -105,6 +105,28 @@ def test_every_variant_with_several_scenarios_per_block(variant, P, f, k, dname,
     assert (codes == 0).sum() > S // 2 and (codes != 0).any()         # most scenarios succeed, some do not
 
 
+DESC_CASES = [c for c in CASES if c[4] == "f32"] + [("staged/large", 4096, 4, 32, "i32", "max", True), ("staged/warp", 64, 2, 8, "i64", "sum", False),
+                                                    ("tiled", 1024, 3, 16, "f32", "sum", True), ("tiled", 300, 2, 8, "f32", "sum", False)]
+
+
+@pytest.mark.parametrize("variant,P,f,k,dname,op,allreduce", DESC_CASES)
+def test_descending_partner_order_on_every_variant(variant, P, f, k, dname, op, allreduce):
+    """The other partner order (Algorithm "Up-correction" leaves it open): which partners a dying process reached and the
+    float32 fold order change with it; the shared-memory kernels play it too."""
+    flags = B.FTC_PARTNERS_DESCENDING | (B.FTC_KERNEL_DIRECT if variant == "tiled" else 0)
+    desc = B.make_desc(P, f, k, B.dtype_code(np.dtype(DT[dname])), op, root=-1, max_inop=2, flags=flags)
+    assert B.ftc_kernel_variant(desc, allreduce) == variant
+    blocks = B.ftc_launch_blocks(desc, 1 << 30, allreduce)
+    S = min(2 * blocks + 3, max(8, (1 << 30) // (P * k * np.dtype(DT[dname]).itemsize)))
+    d_x, x, pf, inop, roots = make_batch(P, f, k, dname, allreduce, S, seed=31 * P + k)
+    got = run_gpu(None, f, op, pf, inop, roots, 0, allreduce, flags, d_x=d_x)
+    want = run_oracle_mt(x, f, op, pf, inop, roots, 0, allreduce, partners_descending=True)
+    assert_same(got, want, f"descending {variant} P={P} f={f} k={k} {dname} {op} allreduce={allreduce}")
+    if dname == "f32" and f >= 2:                                     # the order is observable: ascending gives other bits somewhere
+        other = run_oracle_mt(x, f, op, pf, inop, roots, 0, allreduce)
+        assert not np.array_equal(other[0].view(np.uint8), want[0].view(np.uint8))
+
+
 # Shapes and failure patterns drawn at random once (seeded), kept as a fixed list: mid-size and large process counts,
 # every element type, vector widths of 16 to 512 bytes, group sizes of 1 to 16.
 def fuzz_cases():
