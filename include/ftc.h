@@ -213,16 +213,22 @@ FTC_API int ftc_reduce_batch_noalloc(const ftc_desc_t* desc, uint64_t S, const v
  * included. is_allreduce != 0: the reduce of the allreduce attempt that counts (the last one if no candidate is alive).
  *   d_cand      [S][f+1][k]: the value child s delivers (zeros if it delivers nothing); 16-byte aligned
  *   d_cand_info [S][f+1][2] uint32: [0] 0 = delivered with the failed bit clear, 1 = delivered with the failed bit set,
- *               2 = nothing delivered; [1] size of the list of failed processes that came with the value
- *   workspace of at least ftc_candidates_workspace_bytes(desc, S) bytes, 16-byte aligned
+ *               2 = nothing delivered, 3 = a bounded wait inside the kernel ran out (no value; as FTC_ST_INTERNAL_TIMEOUT);
+ *               [1] size of the list of failed processes that came with the value
+ *   workspace of at least ftc_candidates_workspace_bytes(desc, S) bytes, 256-byte aligned
  * Other arguments as for ftc_reduce_batch. Scenarios whose root is invalid or violates the allreduce precondition
- * play no attempt: zeros and "nothing delivered". Always runs on the general kernel (any k).
+ * play no attempt: zeros and "nothing delivered".
+ * Two kernels (ftc_candidates_kernel_name): "staged" for the exactly associative operations (integer sum, max, xor) on
+ * binary heaps with vectors of 16..512 bytes (a power-of-two number of 16-byte chunks) and scenarios above 12 KB -- one pass
+ * over the inputs on the tiles of the shared-memory kernel, a group without a failed member being folded once for all
+ * children; "generic" (any k, float32, other subtree shapes, FTC_KERNEL_GENERIC) plays child after child.
  */
 FTC_API int ftc_candidates_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const void* d_in,
                                  const uint32_t* d_prefail, const ftc_inop_t* d_inop, const uint32_t* d_roots,
                                  void* d_cand, uint32_t* d_cand_info, void* d_workspace, size_t workspace_bytes,
                                  void* cuda_stream);
 FTC_API size_t ftc_candidates_workspace_bytes(const ftc_desc_t* desc, uint64_t S);
+FTC_API const char* ftc_candidates_kernel_name(const ftc_desc_t* desc);
 
 /*
  * The list of failed processes that the root holds when it delivers (section "Failure information", first scheme:

@@ -39,7 +39,7 @@ FTC_DEBUG_ONE_POLL = 0x4000000
 OPS = {"sum": FTC_SUM, "max": FTC_MAX, "xor": FTC_XOR}
 
 EXPORTS = ["ftc_reduce_batch", "ftc_allreduce_batch", "ftc_reduce_batch_noalloc", "ftc_candidates_batch",
-           "ftc_candidates_workspace_bytes", "ftc_message_counts_batch", "ftc_failed_list_batch", "ftc_workspace_bytes", "ftc_reduce_batch_host",
+           "ftc_candidates_workspace_bytes", "ftc_candidates_kernel_name", "ftc_message_counts_batch", "ftc_failed_list_batch", "ftc_workspace_bytes", "ftc_reduce_batch_host",
            "ftc_allreduce_batch_host", "ftc_host_staging_bytes", "ftc_schedule_info", "ftc_fill_inputs",
            "ftc_kernel_name", "ftc_kernel_variant", "ftc_launch_blocks", "ftc_read_bandwidth_probe", "ftc_strerror", "ftc_version"]
 
@@ -84,6 +84,8 @@ def load():
     lib.ftc_candidates_batch.argtypes = [dp, u64, C.c_int, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.ftc_candidates_workspace_bytes.restype = sz
     lib.ftc_candidates_workspace_bytes.argtypes = [dp, u64]
+    lib.ftc_candidates_kernel_name.restype = C.c_char_p
+    lib.ftc_candidates_kernel_name.argtypes = [dp]
     lib.ftc_message_counts_batch.restype = C.c_int
     lib.ftc_message_counts_batch.argtypes = [dp, u64, C.c_int, vp, vp, vp, vp, vp]
     lib.ftc_failed_list_batch.restype = C.c_int
@@ -225,6 +227,10 @@ def ftc_reduce_batch_noalloc(desc, S, d_in, d_prefail, d_inop, d_roots, d_out, d
     if check and rc != FTC_OK:
         raise FtcError(rc, "ftc_reduce_batch_noalloc")
     return rc
+
+
+def ftc_candidates_kernel_name(desc) -> str:
+    return load().ftc_candidates_kernel_name(C.byref(desc)).decode()
 
 
 def ftc_candidates_workspace_bytes(desc, S) -> int:

@@ -253,12 +253,18 @@ int ftc_candidates_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, c
     if (!aligned16(d_in) || !aligned16(d_cand) || !aligned16(d_cand_info)) return FTC_EINVAL;
     DeviceInfo di;
     if ((rc = device_info(di)) != FTC_OK) return rc;
+    const int tsel = type_select(desc->dtype, desc->op);
+    p.in = d_in; p.prefail = d_prefail; p.inop = d_inop; p.roots = d_roots; p.ws = d_workspace;
+    if (cand_fast_supported(p, tsel, di.smem_optin, di.sm_count)) {
+        const size_t need = cand_fast_workspace_bytes(p, tsel, di.smem_optin, di.sm_count);
+        if (!d_workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return FTC_EWORKSPACE;
+        return launch_cand_fast(p, tsel, d_cand, d_cand_info, di.sm_count, di.smem_optin, static_cast<cudaStream_t>(cuda_stream), nullptr)
+                   == cudaSuccess ? FTC_OK : FTC_ECUDA;
+    }
     const size_t need = (size_t)generic_grid(p, di.sm_count) * candidates_slice_bytes(p);
     if (!d_workspace || workspace_bytes < need || !aligned16(d_workspace)) return FTC_EWORKSPACE;
     if (generic_smem_bytes(p) > (size_t)di.smem_optin) return FTC_EUNSUPPORTED;
-    p.in = d_in; p.prefail = d_prefail; p.inop = d_inop; p.roots = d_roots; p.ws = d_workspace;
-    cudaError_t e = launch_candidates(p, type_select(desc->dtype, desc->op), d_cand, d_cand_info, di.sm_count,
-                                      static_cast<cudaStream_t>(cuda_stream));
+    cudaError_t e = launch_candidates(p, tsel, d_cand, d_cand_info, di.sm_count, static_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? FTC_OK : FTC_ECUDA;
 }
 
@@ -299,11 +305,23 @@ int ftc_failed_list_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, 
     return e == cudaSuccess ? FTC_OK : FTC_ECUDA;
 }
 
+const char* ftc_candidates_kernel_name(const ftc_desc_t* desc) {
+    Params p;
+    if (fill_params(desc, 1, 0, p) != FTC_OK) return "invalid";
+    DeviceInfo di;
+    if (device_info(di) != FTC_OK) di = kB200;
+    return cand_fast_supported(p, type_select(desc->dtype, desc->op), di.smem_optin, di.sm_count) ? "staged" : "generic";
+}
+
 size_t ftc_candidates_workspace_bytes(const ftc_desc_t* desc, uint64_t S) {
     Params p;
     if (fill_params(desc, S, 0, p) != FTC_OK || S == 0) return 0;
     DeviceInfo di;
-    if (device_info(di) != FTC_OK) di = kB200;
+    const bool have_device = device_info(di) == FTC_OK;
+    if (!have_device) di = kB200;
+    const int tsel = type_select(desc->dtype, desc->op);
+    if (have_device && cand_fast_supported(p, tsel, di.smem_optin, di.sm_count))
+        return cand_fast_workspace_bytes(p, tsel, di.smem_optin, di.sm_count);
     return (size_t)generic_grid(p, di.sm_count) * candidates_slice_bytes(p);
 }
 

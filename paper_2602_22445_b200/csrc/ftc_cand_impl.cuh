@@ -1,0 +1,416 @@
+// What every root child delivers (Algorithm "reduce_root": "receive from any child (data, failure information)";
+// section "Failure information", second and third scheme), on the tiles of the staged kernel, for the exactly
+// associative operations (integer sum, max, xor). The batch kernels evaluate only the child the root selects;
+// here all f+1 subtrees are played, nodes that deliver nothing included, in one pass over the inputs.
+//
+// What makes one pass cheap: a group none of whose members failed, before or during the operation, has the same
+// value at every member after up-correction when the operation is exactly associative and commutative (every
+// member folds the same f+1 inputs). So a warp tile without a failed process, a renumbered slot or the short last
+// group is evaluated once and its value serves all f+1 subtrees; only the few tiles that hold such a row are played
+// child by child with the full rules: a node that does not send delivers nothing, its parent sets the failed bit
+// and counts it, the list sizes add up.
+//
+// Per node and child the kernel carries a value and a word: exists | present | failed bit | size of the failed list.
+// The values of the tile roots and of the rows above the tiles live in a per-block slice of the workspace, one heap
+// array per root child (they stay in L2), and are combined level by level as in the staged kernel.
+#pragma once
+#include "ftc_staged_impl.cuh"
+
+namespace ftc {
+
+constexpr uint32_t kMetaExists = 1u << 31, kMetaPresent = 1u << 30, kMetaFailed = 1u << 29, kMetaCount = (1u << 29) - 1;
+
+// A node takes one child's delivery: a child that sent is combined, its failed bit and list size taken over; a child
+// that sent nothing sets the failed bit and is noted (Algorithm "reduce_non_root" with the second scheme's size).
+template <typename T, int OP>
+__device__ __forceinline__ void take_child(uint4& acc, uint32_t& meta, uint4 cv, uint32_t cm) {
+    if (!(cm & kMetaExists)) return;
+    if (cm & kMetaPresent) { acc = comb16<T, OP>(acc, cv); meta = (meta | (cm & kMetaFailed)) + (cm & kMetaCount); }
+    else meta = (meta | kMetaFailed) + 1u;
+}
+
+// Facts of the scenario the child-by-child folds need (shared memory).
+struct CandScen {
+    const Ctx* cx;
+    const uint32_t* alive;   // bit v (renumbered): v had not failed before the operation
+    const uint32_t* snd;     // bit v (renumbered): v performs its tree send
+    uint32_t root, base, troot;
+};
+
+// Node (row, sc) of root subtree sc after up-correction (Algorithm "Up-correction"): own input, the root's if it is a
+// partner and its message was sent, then the partners whose message arrived. `in_lc`: the scenario in the caller's
+// process order (global memory) at this lane's chunk. The caller guarantees that the node exists (sc < members of the row).
+template <typename T, int OP>
+__device__ __noinline__ uint4 cand_fold(const Params& p, CandScen cs, const char* in_lc, uint32_t row, uint32_t sc, uint32_t& meta) {
+    const uint32_t mj = row < p.q ? p.m : p.r, vbase = row * p.m + 1, v = vbase + sc;
+    if (!test_bit(cs.snd, v)) { meta = kMetaExists; return make_uint4(0, 0, 0, 0); }
+    uint32_t mask = extract_bits(cs.alive, vbase, mj);
+    for (uint32_t i = 0; i < p.max_inop; ++i) {              // a dying partner's message arrives iff it was still sent
+        const uint32_t vic = cs.cx->iv[i];
+        if (vic == FTC_INOP_UNUSED) continue;
+        const uint32_t vr = renumber(vic, cs.root);
+        if (vr < vbase || vr >= vbase + mj || vr == v) continue;
+        const uint32_t sv = vr - vbase, t = local_round(cs.cx->ir[i], cs.base);
+        if (!(partner_slot(p, row, sv, sc) < t)) mask &= ~(1u << sv);
+    }
+    uint4 acc = ld_stream(in_lc + (size_t)(v == cs.root ? 0u : v) * p.kbytes);
+    // the root's up-correction send to member sc of its group is its send number sc (descending order: r-1-sc)
+    const bool from_root = row == p.q && (p.pdesc ? p.r - 1 - sc : sc) < cs.troot;
+    if (from_root) acc = comb16<T, OP>(acc, ld_stream(in_lc + (size_t)cs.root * p.kbytes));
+    for (uint32_t sp = 0; sp < mj; ++sp) {
+        const uint32_t vr = vbase + sp;
+        if (sp != sc && ((mask >> sp) & 1u)) acc = comb16<T, OP>(acc, ld_stream(in_lc + (size_t)(vr == cs.root ? 0u : vr) * p.kbytes));
+    }
+    meta = kMetaExists | kMetaPresent | (mj - __popc(mask) + ((row == p.q && !from_root) ? 1u : 0u));
+    return acc;
+}
+
+// A lane's sub-heap of XL levels for child sc: node, then child 1, then child 2. Rows >= G do not exist.
+template <typename T, int OP, int XL, int U>
+struct SubHeapCand {
+    static __device__ __forceinline__ uint4 eval(const Params& p, const CandScen& cs, const char* in_lc, uint32_t grow, uint32_t G, uint32_t sc, uint32_t& meta) {
+        if (grow >= G) { meta = 0; return make_uint4(0, 0, 0, 0); }
+        uint4 v = cand_fold<T, OP>(p, cs, in_lc, grow, sc, meta);
+        if (U + 1 < XL && (meta & kMetaPresent)) {           // what the children of a node that does not send deliver is lost
+            constexpr int UN = (U + 1 < XL ? U + 1 : U);
+            uint32_t cm;
+            uint4 cv = SubHeapCand<T, OP, XL, UN>::eval(p, cs, in_lc, 2 * grow + 1, G, sc, cm);
+            take_child<T, OP>(v, meta, cv, cm);
+            cv = SubHeapCand<T, OP, XL, UN>::eval(p, cs, in_lc, 2 * grow + 2, G, sc, cm);
+            take_child<T, OP>(v, meta, cv, cm);
+        }
+        return v;
+    }
+};
+
+// Tree phase inside a warp tile with the words riding along (see tile_tree_phase for the lane roles).
+template <typename T, int OP>
+__device__ __forceinline__ uint4 tile_tree_phase_cand(uint4 valA, uint32_t mA, uint4 valB, uint32_t& mB, uint32_t lw, uint32_t cwl, uint32_t C,
+                                                      uint32_t lane, uint32_t lc, uint32_t tB, uint32_t idxB, bool hasB) {
+    if (lw) {
+        const bool mine = hasB && tB == lw - 1;
+        const uint32_t src1 = mine ? (((2 * idxB) << cwl) | lc) : lane, src2 = mine ? src1 + C : lane;
+        const uint4 c1 = shfl16(valA, src1), c2 = shfl16(valA, src2);
+        const uint32_t m1 = __shfl_sync(0xFFFFFFFFu, mA, src1), m2 = __shfl_sync(0xFFFFFFFFu, mA, src2);
+        if (mine && (mB & kMetaPresent)) { take_child<T, OP>(valB, mB, c1, m1); take_child<T, OP>(valB, mB, c2, m2); }
+    }
+    for (int t = (int)lw - 2; t >= 0; --t) {
+        const bool mine = hasB && tB == (uint32_t)t;
+        const uint32_t src1 = mine ? ((((2u << t) - 1 + 2 * idxB) << cwl) | lc) : lane, src2 = mine ? src1 + C : lane;
+        const uint4 c1 = shfl16(valB, src1), c2 = shfl16(valB, src2);
+        const uint32_t m1 = __shfl_sync(0xFFFFFFFFu, mB, src1), m2 = __shfl_sync(0xFFFFFFFFu, mB, src2);
+        if (mine && (mB & kMetaPresent)) { take_child<T, OP>(valB, mB, c1, m1); take_child<T, OP>(valB, mB, c2, m2); }
+    }
+    return valB;
+}
+
+struct CandGeom {
+    StagedGeom st;
+    uint64_t slice_bytes;       // workspace per block: f+1 heap arrays of values, then the words
+    uint32_t nheap, ntop;       // rows of a heap array (tile roots and above): 2^(Lt+1) - 1; rows above the tiles: 2^Lt - 1
+};
+
+template <typename T, int OP, int XL>
+__global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, CandGeom cg, T* cand, uint32_t* info) {
+    const StagedGeom& g = cg.st;
+    extern __shared__ __align__(128) uint32_t smem[];
+    char* sbase = reinterpret_cast<char*>(smem);
+    Ctx* cx = reinterpret_cast<Ctx*>(smem);
+    uint32_t* pf = smem + sizeof(Ctx) / 4;
+    uint32_t* alive = pf + p.W + 1;
+    uint32_t* snd = alive + p.W + 1;
+    uint32_t* tspec = reinterpret_cast<uint32_t*>(sbase + g.off_special);
+    volatile uint32_t* gaveup = reinterpret_cast<volatile uint32_t*>(sbase + g.off_gaveup);
+    // per block: values hv[sc][row][chunk], combined words hm[sc][row], own words of the rows above the tiles hmo[sc][row]
+    char* slice = static_cast<char*>(p.ws) + (size_t)blockIdx.x * cg.slice_bytes;
+    uint4* hv = reinterpret_cast<uint4*>(slice);
+    uint32_t* hm = reinterpret_cast<uint32_t*>(slice + (size_t)p.m * cg.nheap * p.C * 16);
+    uint32_t* hmo = hm + (size_t)p.m * cg.nheap;
+
+    const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
+    const uint32_t cwl = p.cw_log2, lw = 5 - cwl, RW = 1u << lw, Cmask = p.C - 1;
+    const uint32_t lr = lane >> cwl, lc = lane & Cmask;
+    const uint32_t D = lw + XL;
+    const uint32_t Lt = p.Lt, ntiles = 1u << Lt, ntop = ntiles - 1;
+    const uint32_t GR = min((1u << XL) - 1, max(1u, (ntop + RW - 1) >> lw)), grows = RW * GR;
+    const uint32_t ngroups = (ntop + grows - 1) / grows;
+    const uint32_t nitems = ntiles + ngroups;
+    const uint32_t rowbytes = p.m * p.kbytes;
+    const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
+    const uint32_t tries = (p.flags & FTC_DEBUG_ONE_POLL) ? 1u : kWaitTries;
+    const uint32_t Gc = p.q;                                       // rows every root subtree has; row q exists below children s < r only
+
+    const uint32_t bar0 = smem_addr(sbase + g.off_bar) + wid * 8;
+    char* tile = sbase + g.off_tiles + (size_t)wid * g.tile_cap;
+    if (lane == 0) mbar_init(bar0, 1);
+    if (tid == 0) *gaveup = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    uint32_t phase = 0;
+    bool pending = false, stop = false;
+
+    // ---- this warp's copy pipeline over the flat sequence (scenario, work item), one buffer, one item ahead ----
+    const uint32_t n_my = wid < nitems ? (nitems - wid + nw - 1) / nw : 0;
+    uint64_t is_s = blockIdx.x;
+    const char* is_src = reinterpret_cast<const char*>(p.in) + is_s * scen_bytes;
+    uint32_t is_i = 0;
+    const uint32_t lvl_rows = lane < D ? 1u << lane : 0u, lvl_dst = (lvl_rows ? lvl_rows - 1 : 0u) * rowbytes;
+    auto issue_next = [&]() {
+        if (n_my == 0 || is_s >= p.S || stop) return;
+        const uint32_t it = wid + is_i * nw;
+        uint32_t first_row = 0, nrows = 0, dst_off = 0;
+        if (it < ntiles) {
+            const uint32_t j0 = ntop + it;
+            if (j0 < p.Gmax) { first_row = ((j0 + 1) << lane) - 1; nrows = lvl_rows; dst_off = lvl_dst; }
+        } else if (lane == 0) { first_row = (it - ntiles) * grows; nrows = min(grows, ntop - first_row); }
+        const uint64_t b0 = (uint64_t)first_row * rowbytes + p.kbytes;
+        uint32_t bytes = 0;
+        if (nrows && b0 < scen_bytes) bytes = (uint32_t)min((uint64_t)nrows * rowbytes, scen_bytes - b0);
+        const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, bytes);
+        if (total) {
+            if (lane == 0) mbar_expect_tx(bar0, total);
+            __syncwarp();
+            if (bytes) bulk_g2s(smem_addr(tile + dst_off), is_src + b0, bytes, bar0);
+            pending = true;
+        }
+        if (++is_i == n_my) { is_i = 0; is_s += gridDim.x; is_src += (uint64_t)gridDim.x * scen_bytes; }
+    };
+    auto acquire = [&]() {
+        if (pending && !stop) {
+            bool ok = mbar_wait_bounded(bar0, phase, tries);
+            if (!__all_sync(0xFFFFFFFFu, ok)) {
+                if (__any_sync(0xFFFFFFFFu, ok) && !ok) ok = mbar_wait_bounded(bar0, phase, kWaitTries);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+            }
+            if (ok) { phase ^= 1u; pending = false; }
+            else { stop = true; if (lane == 0) atomicOr(const_cast<uint32_t*>(gaveup), 1u); }
+        }
+    };
+    auto release = [&]() { __syncwarp(); issue_next(); };
+    issue_next();
+
+    for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {
+        const char* in_s = reinterpret_cast<const char*>(p.in) + s * scen_bytes;
+        const bool dead = *gaveup != 0;
+        if (dead) stop = true;
+        decode_scenario(p, s, cx, pf, alive);                      // `alive` is scratch for its arrival mask here
+        T* cand_s = cand + s * (uint64_t)p.m * p.k;
+        uint32_t* info_s = info + s * (uint64_t)p.m * 2;
+        const uint32_t code = cx->code;
+        if (code == FTC_ST_BAD_ROOT || code == FTC_ST_PRECONDITION_INOP_ROOT || dead) {    // no attempt is played
+            for (uint32_t u = tid; u < p.m * p.C; u += nt) reinterpret_cast<uint4*>(cand_s)[u] = make_uint4(0, 0, 0, 0);
+            for (uint32_t u = tid; u < p.m; u += nt) { info_s[2 * u] = dead ? 3u : 2u; info_s[2 * u + 1] = 0; }
+            for (uint32_t i = 0; i < n_my; ++i) { acquire(); release(); }
+            __syncthreads();
+            continue;
+        }
+        uint32_t root = cx->root, base = cx->base;
+        if (code == FTC_ST_NO_LIVE_ROOT_CANDIDATE) {                // the last attempt, toward a dead root
+            const uint32_t first = p.root >= 0 ? (uint32_t)p.root : p.roots[s];
+            root = (first + p.f) % p.P; base = p.f * p.Ratt;
+        }
+        const uint32_t troot = local_round(fail_round(p, cx, pf, root), base);
+        __syncthreads();                                           // decode's arrival mask is no longer read
+        // who had not failed beforehand and who sends up the tree, over renumbered ranks
+        for (uint32_t w = tid; w <= p.W; w += nt) {
+            uint32_t word = w < p.W ? ~pf[w] : 0u;
+            if (w == p.W - 1 && (p.P & 31)) word &= (1u << (p.P & 31)) - 1u;
+            alive[w] = word; snd[w] = word;
+        }
+        __syncthreads();
+        if (tid == 0 && root != 0) {                               // bit `root` is process 0, bit 0 the root
+            const uint32_t b0 = alive[0] & 1u, bit = 1u << (root & 31);
+            alive[0] |= 1u;
+            if (b0) { alive[root >> 5] |= bit; snd[root >> 5] |= bit; } else { alive[root >> 5] &= ~bit; snd[root >> 5] &= ~bit; }
+        }
+        __syncthreads();
+        if (tid < p.max_inop && cx->iv[tid] != FTC_INOP_UNUSED) {
+            const uint32_t v = renumber(cx->iv[tid], root);
+            if (v) {
+                const uint32_t d = 1 + ilog2u((v - 1) / p.m + 1), t = local_round(cx->ir[tid], base);
+                if (!(p.f + p.H - d < t)) atomicAnd(&snd[v >> 5], ~(1u << (v & 31)));      // tree send of depth d is round f+H-d
+            }
+        }
+        // ---- work items that are played child by child: those with a failed process, a renumbered slot, the short last
+        // group, or not complete above their last level. One bit per item (tile i, then groups of rows above the tiles).
+        for (uint32_t w = tid; w < (nitems + 31) / 32 + 1; w += nt) tspec[w] = 0;
+        __syncthreads();
+        {
+            auto mark_row = [&](uint32_t j) {
+                const uint32_t lvl = ilog2u(j + 1);
+                const uint32_t it = lvl >= Lt ? ((j + 1) >> (lvl - Lt)) - ntiles : ntiles + j / grows;
+                atomicOr(&tspec[it >> 5], 1u << (it & 31));
+            };
+            for (uint32_t w = tid; w < p.W; w += nt) {
+                uint32_t word = pf[w];
+                while (word) {
+                    const uint32_t b = __ffs(word) - 1; word &= word - 1;
+                    const uint32_t v = renumber((w << 5) + b, root);
+                    if (v) mark_row((v - 1) / p.m);
+                }
+            }
+            if (tid < p.max_inop && cx->iv[tid] != FTC_INOP_UNUSED) {
+                const uint32_t v = renumber(cx->iv[tid], root);
+                if (v) mark_row((v - 1) / p.m);
+            }
+            if (tid == 0) {
+                if (root != 0) mark_row((root - 1) / p.m);          // the slot that holds process 0's input
+                if (p.r) mark_row(p.q);                             // the short last group
+            }
+            for (uint32_t it = tid; it < ntiles; it += nt)
+                if (((ntop + it + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= Gc) atomicOr(&tspec[it >> 5], 1u << (it & 31));
+            for (uint32_t gi = tid; gi < ngroups; gi += nt)
+                if ((gi + 1) * grows > ntop || (gi + 1) * grows > Gc) atomicOr(&tspec[(ntiles + gi) >> 5], 1u << ((ntiles + gi) & 31));
+        }
+        __syncthreads();
+        const CandScen cs{cx, alive, snd, root, base, troot};
+        const char* in_lc = in_s + lc * 16;
+
+        for (uint32_t i = 0; i < n_my; ++i) {
+            const uint32_t it = wid + i * nw;
+            acquire();
+            const char* buf_lc = tile + lc * 16;
+            const bool special = test_bit(tspec, it);              // warp-uniform
+            if (it < ntiles) {
+                const uint32_t j0 = ntop + it;
+                const uint32_t tA = RW - 1 + lr, rowA = ((j0 + 1) << lw) - 1 + lr;
+                const uint32_t tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB);
+                const uint32_t rowB = ((j0 + 1) << tB) - 1 + idxB;
+                if (!special) {
+                    // every group of the tile is whole: one value per row serves all children (exact operations)
+                    uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
+                    if (XL > 1 || rowA < Gc) valA = SubHeapPlain<T, OP, XL, 0, false, false>::eval(p, 0u, alive, buf_lc, rowbytes, tA, rowA, Gc);
+                    const bool hasB = lr < RW - 1;
+                    if (hasB) valB = fold_plain_staged<T, OP>(p, 0u, buf_lc + staged_row_offset<false>(p, rowbytes, lr, rowB));
+                    valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, Gc);
+                    release();
+                    if (lr == 0) {
+                        const uint4 v = lw ? valB : valA;
+                        for (uint32_t sc = 0; sc < p.m; ++sc) {
+                            hv[((size_t)sc * cg.nheap + j0) * p.C + lc] = v;
+                            if (lc == 0) hm[(size_t)sc * cg.nheap + j0] = kMetaExists | kMetaPresent;
+                        }
+                    }
+                } else {
+                    release();                                     // these few tiles read the scenario itself
+                    for (uint32_t sc = 0; sc < p.m; ++sc) {
+                        const uint32_t G = p.q + (sc < p.r ? 1u : 0u);
+                        uint32_t mA = 0, mB = 0;
+                        uint4 valA = SubHeapCand<T, OP, XL, 0>::eval(p, cs, in_lc, rowA, G, sc, mA), valB = make_uint4(0, 0, 0, 0);
+                        const bool hasB = lr < RW - 1;
+                        if (hasB && rowB < G) valB = cand_fold<T, OP>(p, cs, in_lc, rowB, sc, mB);
+                        valB = tile_tree_phase_cand<T, OP>(valA, mA, valB, mB, lw, cwl, p.C, lane, lc, tB, idxB, hasB);
+                        if (lr == 0) {
+                            hv[((size_t)sc * cg.nheap + j0) * p.C + lc] = lw ? valB : valA;
+                            if (lc == 0) hm[(size_t)sc * cg.nheap + j0] = lw ? mB : mA;
+                        }
+                    }
+                }
+            } else {
+                // ---- rows above the tiles: fold now, combine later ----
+                if (!special) {
+                    uint4 v[7];
+#pragma unroll
+                    for (uint32_t gs = 0; gs < 7; ++gs)
+                        if (gs < GR) v[gs] = fold_plain_staged<T, OP>(p, 0u, buf_lc + (size_t)(gs * RW + lr) * rowbytes);
+                    release();
+#pragma unroll
+                    for (uint32_t gs = 0; gs < 7; ++gs) {
+                        if (gs >= GR) continue;
+                        const uint32_t row = (it - ntiles) * grows + gs * RW + lr;
+                        for (uint32_t sc = 0; sc < p.m; ++sc) {
+                            hv[((size_t)sc * cg.nheap + row) * p.C + lc] = v[gs];
+                            if (lc == 0) hmo[(size_t)sc * cg.ntop + row] = kMetaExists | kMetaPresent;
+                        }
+                    }
+                } else {
+                    release();
+                    for (uint32_t gs = 0; gs < GR; ++gs) {
+                        const uint32_t row = (it - ntiles) * grows + gs * RW + lr;
+                        if (row >= ntop) continue;
+                        for (uint32_t sc = 0; sc < p.m; ++sc) {
+                            const uint32_t G = p.q + (sc < p.r ? 1u : 0u);
+                            uint32_t mo = 0;
+                            uint4 v = make_uint4(0, 0, 0, 0);
+                            if (row < G) v = cand_fold<T, OP>(p, cs, in_lc, row, sc, mo);
+                            hv[((size_t)sc * cg.nheap + row) * p.C + lc] = v;
+                            if (lc == 0) hmo[(size_t)sc * cg.ntop + row] = mo;
+                        }
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        // ---- levels above the tiles, leaves first (Algorithm "reduce_non_root"), all root children in one sweep ----
+        for (int lvl = (int)Lt - 1; lvl >= 0; --lvl) {
+            const uint32_t lo = (1u << lvl) - 1u, n = lo + 1u;
+            for (uint32_t u = tid; u < n * p.m * p.C; u += nt) {
+                const uint32_t c = u & Cmask, x = u >> cwl, sc = x % p.m, row = lo + x / p.m;
+                uint32_t meta = hmo[(size_t)sc * cg.ntop + row];
+                uint4 v = hv[((size_t)sc * cg.nheap + row) * p.C + c];
+                if (meta & kMetaPresent) {
+                    const size_t c1 = (size_t)sc * cg.nheap + 2 * row + 1;
+                    take_child<T, OP>(v, meta, hv[c1 * p.C + c], hm[c1]);
+                    take_child<T, OP>(v, meta, hv[(c1 + 1) * p.C + c], hm[c1 + 1]);
+                    hv[((size_t)sc * cg.nheap + row) * p.C + c] = v;
+                }
+                if (c == 0) hm[(size_t)sc * cg.nheap + row] = meta;
+            }
+            __syncthreads();
+        }
+        // ---- what the root receives from each child ----
+        const bool bad = *gaveup != 0;
+        for (uint32_t u = tid; u < p.m * p.C; u += nt) {
+            const uint32_t sc = u >> cwl, c = u & Cmask, meta = hm[(size_t)sc * cg.nheap];
+            const bool got = (meta & kMetaPresent) && !bad;
+            reinterpret_cast<uint4*>(cand_s)[u] = got ? hv[((size_t)sc * cg.nheap) * p.C + c] : make_uint4(0, 0, 0, 0);
+            if (c == 0) {
+                info_s[2 * sc] = bad ? 3u : (meta & kMetaPresent) ? ((meta & kMetaFailed) ? 1u : 0u) : 2u;
+                info_s[2 * sc + 1] = got ? (meta & kMetaCount) : 0u;
+            }
+        }
+        __syncthreads();
+    }
+    if (pending) mbar_wait_bounded(bar0, phase, kWaitTries);      // only after a wait gave up: a copy may still be in flight
+}
+
+// ---- host side ----
+static bool cand_geometry(Params& p, int smem_optin, int sm_count, uint32_t& XL, CandGeom& cg) {
+    if (p.arity != 2) return false;
+    XL = staged_xl(p);
+    p.ws_bytes = 0; p.swz_mask = 0; p.row_shift = 0;               // its own slices; plain tiles
+    if (!staged_geometry(p, smem_optin, sm_count, XL, cg.st, /*all_children=*/true)) return false;
+    if (cg.st.whole || cg.st.nbuf != 1) return false;
+    cg.nheap = (2u << p.Lt) - 1; cg.ntop = (1u << p.Lt) - 1;
+    cg.slice_bytes = (((uint64_t)p.m * cg.nheap * p.C * 16 + (uint64_t)p.m * (cg.nheap + cg.ntop) * 4) + 255) & ~(uint64_t)255;
+    return true;
+}
+
+template <typename T, int OP, int XL>
+static cudaError_t launch_cand_x(const Params& p, const CandGeom& cg, T* cand, uint32_t* info, int sm_count, cudaStream_t st, uint32_t* grid_out) {
+    cudaError_t e = cudaFuncSetAttribute(cand_kernel<T, OP, XL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cg.st.smem_bytes);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, cand_kernel<T, OP, XL>, (int)cg.st.nwarps * 32, cg.st.smem_bytes);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    if (per_sm > 2) per_sm = 2;                                   // slices of all blocks stay in L2
+    const uint64_t cap = (uint64_t)sm_count * per_sm;
+    const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
+    if (grid_out) { *grid_out = (uint32_t)cap; return cudaSuccess; }
+    cand_kernel<T, OP, XL><<<grid, cg.st.nwarps * 32, cg.st.smem_bytes, st>>>(p, cg, cand, info);
+    return cudaGetLastError();
+}
+
+template <typename T, int OP>
+static cudaError_t launch_cand_t(Params p, void* cand, uint32_t* info, int sm_count, int smem_optin, cudaStream_t st, uint32_t* grid_out) {
+    CandGeom cg; uint32_t XL;
+    if (!cand_geometry(p, smem_optin, sm_count, XL, cg)) return cudaErrorInvalidConfiguration;
+    switch (XL) {
+    case 2: return launch_cand_x<T, OP, 2>(p, cg, static_cast<T*>(cand), info, sm_count, st, grid_out);
+    case 3: return launch_cand_x<T, OP, 3>(p, cg, static_cast<T*>(cand), info, sm_count, st, grid_out);
+    default: return launch_cand_x<T, OP, 1>(p, cg, static_cast<T*>(cand), info, sm_count, st, grid_out);
+    }
+}
+
+}  // namespace ftc

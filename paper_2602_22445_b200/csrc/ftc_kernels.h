@@ -42,6 +42,12 @@ cudaError_t launch_warp(const Params& p, int tsel, int sm_count, int smem_optin_
 size_t candidates_slice_bytes(const Params& p);
 cudaError_t launch_candidates(const Params& p, int tsel, void* cand, uint32_t* info, int sm_count, cudaStream_t st);
 
+// The same on the staged tiles, all root children in one pass over the inputs (exactly associative operations).
+// grid_out != NULL: store the blocks a launch may use (the workspace holds one slice per block) and launch nothing.
+bool cand_fast_supported(Params p, int tsel, int smem_optin_bytes, int sm_count);
+size_t cand_fast_workspace_bytes(Params p, int tsel, int smem_optin_bytes, int sm_count);
+cudaError_t launch_cand_fast(const Params& p, int tsel, void* cand, uint32_t* info, int sm_count, int smem_optin_bytes, cudaStream_t st, uint32_t* grid_out);
+
 // Message counts per scenario (FTC_MSG_WORDS 64-bit words each); reads the failure pattern only.
 size_t messages_smem_bytes(const Params& p);
 cudaError_t launch_messages(const Params& p, unsigned long long* out, int sm_count, cudaStream_t st);

@@ -639,7 +639,9 @@ constexpr size_t kHvGlobalMinBytes = 24 * 1024;
 constexpr size_t kHvGlobalMaxBytes = 512 * 1024;   // beyond this the slices of all blocks no longer stay in L2
 constexpr int kHvGlobalBlocksPerSm = 4;
 
-static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL, StagedGeom& g) {
+// all_children: geometry for the kernel that plays every root child (ftc_cand_impl.cuh): every heap level is tiled and
+// the heap arrays live in the workspace, never in shared memory.
+static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL, StagedGeom& g, bool all_children = false) {
     if (p.kbytes % 16) return false;
     const uint32_t C = p.kbytes / 16;
     if (C == 0 || C > 32 || (C & (C - 1))) return false;
@@ -649,7 +651,7 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
     // a last level filled to less than an eighth stays out of the tiles (its few rows go the careful way), so that
     // the tiles, and with them the copy buffers, are full
     const uint32_t last_rows = p.Gmax - ((1u << (Hmax - 1)) - 1);
-    const uint32_t Heff = (Hmax >= 2 && last_rows * 8 < (1u << (Hmax - 1))) ? Hmax - 1 : Hmax;
+    const uint32_t Heff = (!all_children && Hmax >= 2 && last_rows * 8 < (1u << (Hmax - 1))) ? Hmax - 1 : Hmax;
     p.C = C; p.cw_log2 = cwl; p.Lt = Heff > D ? Heff - D : 0;
     p.below = (Heff < Hmax && Heff >= D) ? 1u : 0u;
     if (p.Lt > 16) return false;
@@ -680,7 +682,8 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
     g.hv_bytes = (((uint64_t)2 << p.Lt) - 1) * C * 16;
     g.hv_global = (!g.whole && g.hv_bytes >= kHvGlobalMinBytes && g.hv_bytes <= kHvGlobalMaxBytes &&
                    p.ws_bytes / ((uint64_t)sm_count * kHvGlobalBlocksPerSm) >= g.hv_bytes) ? 1u : 0u;
-    g.off_hv = (uint32_t)o; if (!g.hv_global) o += (size_t)g.hv_bytes;
+    if (all_children) g.hv_global = 0;
+    g.off_hv = (uint32_t)o; if (!g.hv_global && !all_children) o += (size_t)g.hv_bytes;
     g.off_bar = (uint32_t)o; o += (size_t)(kStagedMaxThreads / 32) * 4 * 8 + 8;      // room for any warps x nbuf, plus one
     g.off_gaveup = (uint32_t)o; o += 8;
     o = (o + 127) & ~(size_t)127; g.off_tiles = (uint32_t)o;
