@@ -282,8 +282,9 @@ def measured_peak():
 class Leg:
     """One workload resident on the device: inputs generated there, failure patterns uploaded, outputs and workspace."""
 
-    def __init__(self, name, S, first, args, B, torch, sched_rounds):
+    def __init__(self, name, S, first, args, B, torch, sched_rounds, candidates=False):
         self.name, self.S, self.B, self.torch = name, S, B, torch
+        self.candidates = candidates
         w = make_workload(name, S, first, sched_rounds)
         if args.collective:
             w.collective = args.collective
@@ -303,10 +304,17 @@ class Leg:
         self.d_pf, self.d_inop, self.d_roots = upload(w, torch)
         self.d_out = torch.empty((S, w.k), dtype=self.tdt, device="cuda")
         self.d_st = torch.empty((S, 4), dtype=torch.int32, device="cuda")
-        self.d_ws = torch.empty(max(B.ftc_workspace_bytes(self.desc, S, self.allred), 16), dtype=torch.uint8, device="cuda")
         self.sched = B.ftc_schedule_info(self.desc)
         self.esz = ESZ[np.dtype(w.dtype).name]
         self.bytes_per_launch = S * bytes_per_scenario(w)
+        if candidates:
+            # every root child's delivery: f+1 values and (flag, list size) pairs per scenario instead of one result and status
+            self.d_out = torch.empty((S, w.f + 1, w.k), dtype=self.tdt, device="cuda")
+            self.d_st = torch.empty((S, w.f + 1, 2), dtype=torch.int32, device="cuda")
+            self.d_ws = torch.empty(max(B.ftc_candidates_workspace_bytes(self.desc, S), 256), dtype=torch.uint8, device="cuda")
+            self.bytes_per_launch += S * w.f * (w.k * self.esz + 8) - S * 8
+        else:
+            self.d_ws = torch.empty(max(B.ftc_workspace_bytes(self.desc, S, self.allred), 16), dtype=torch.uint8, device="cuda")
         torch.cuda.synchronize()
 
     def regenerate(self, first, sched_rounds):
@@ -319,7 +327,11 @@ class Leg:
         self.torch.cuda.synchronize()
 
     def step(self):
-        self.fn(self.desc, self.S, self.d_x, self.d_pf, self.d_inop, self.d_roots, self.d_out, self.d_st, self.d_ws)
+        if self.candidates:
+            self.B.ftc_candidates_batch(self.desc, self.S, self.allred, self.d_x, self.d_pf, self.d_inop, self.d_roots, self.d_out,
+                                        self.d_st, self.d_ws)
+        else:
+            self.fn(self.desc, self.S, self.d_x, self.d_pf, self.d_inop, self.d_roots, self.d_out, self.d_st, self.d_ws)
 
     def rounds(self):
         return self.sched["rounds_attempt"] if self.allred else self.sched["rounds_reduce"]
@@ -377,23 +389,35 @@ def add_sustained(roof, leg, torch, sampler, seconds):
                          "sm_mhz_median": mhz, "ms_x_mhz": (ms * mhz) if mhz else None, "clocks": clocks}
 
 
-def run_side_leg(name, args, B, torch, sampler, peak, peak_kind):
-    """One more workload, timed like the headline one: K steps, then a sustained run; its own roofline record."""
+def run_side_leg(name, args, B, torch, sampler, peak, peak_kind, candidates=False):
+    """One more workload, timed like the headline one: K steps, then a sustained run; its own roofline record.
+    candidates: what every root child delivers (ftc_candidates_batch) instead of the batch call."""
     S = DEFAULT_BATCH[name]
-    leg = Leg(name, S, 0, args, B, torch, 28)
+    leg = Leg(name, S, 0, args, B, torch, 28, candidates=candidates)
     for _ in range(max(args.warmup, 3)):
         leg.step()
     m0 = sampler.lines() if sampler else 0
     per_ms, total_ms = time_steps(torch, leg.step, args.steps)
     clocks = sampler.window(m0, sampler.lines()) if sampler else None
     roof = roofline_record(name, leg.bytes_per_launch, per_ms, S, peak, peak_kind)
+    if candidates:
+        roof["traffic"] = None
     add_sustained(roof, leg, torch, sampler, args.sustain_seconds / 2)
     ms = total_ms / args.steps
-    st = leg.status()
-    rec = {"workload": f"{name}: {DESCRIPTION[name]}", "value": S / (ms / 1e3), "unit": "scenarios/s", "ms_per_step": ms,
+    rec = {"workload": f"{name}: {DESCRIPTION[name]}" + (" [what every root child delivers: all f+1 subtrees played]" if candidates else ""),
+           "value": S / (ms / 1e3), "unit": "scenarios/s", "ms_per_step": ms,
            "steps": args.steps, "scenarios_per_step": S, "process_rounds_per_sec": S / (ms / 1e3) * leg.w.P * leg.rounds(),
-           "kernel": B.ftc_kernel_variant(leg.desc, leg.allred), "dtype": np.dtype(leg.w.dtype).name,
-           "ok_scenarios": int(((st[:, 0] & 0xFF) == 0).sum()), "roofline": roof, "clocks": clocks}
+           "dtype": np.dtype(leg.w.dtype).name, "roofline": roof, "clocks": clocks}
+    if candidates:
+        info = leg.d_st.cpu().numpy()
+        rec["kernel"] = "candidates/" + B.ftc_candidates_kernel_name(leg.desc)
+        rec["subtrees_played"] = f"{leg.w.f + 1} of {leg.w.f + 1}"
+        rec["children_delivering_clean"] = int((info[:, :, 0] == 0).sum())
+        rec["children_with_failed_bit_or_silent"] = int((info[:, :, 0] != 0).sum())
+    else:
+        st = leg.status()
+        rec["kernel"] = B.ftc_kernel_variant(leg.desc, leg.allred)
+        rec["ok_scenarios"] = int(((st[:, 0] & 0xFF) == 0).sum())
     leg.free()
     return rec
 
@@ -480,6 +504,19 @@ def run_gpu(args):
         if world > 1:
             raise SystemExit("--full-config runs on one GPU")
         run_full_config(args, B, torch, sampler, peak, peak_kind)
+        return
+    if args.candidates:
+        if world > 1:
+            raise SystemExit("--candidates runs on one GPU")
+        rec = run_side_leg(args.workload, args, B, torch, sampler, peak, peak_kind, candidates=True)
+        sampler.stop()
+        line = {"metric": "scenarios_per_sec", "value": rec["value"], "unit": "scenarios/s", "n_gpus": 1, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": rec["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": rec["dtype"], "data": "synthetic", "process_rounds_per_sec": rec["process_rounds_per_sec"],
+                "config": {"workload": rec["workload"], "scenarios_per_step_per_gpu": rec["scenarios_per_step"], "kernel": rec["kernel"],
+                           "subtrees_played": rec["subtrees_played"], "cache": "inputs larger than L2, no flush"},
+                "roofline": rec["roofline"], "cpu_baseline": None, "e2e": None, "gpu_launches": args.steps, "clocks": rec["clocks"]}
+        print(json.dumps(line))
         return
 
     name = args.workload
@@ -578,6 +615,10 @@ def run_gpu(args):
             for other in [x for x in ("c5", "c5r", "c3", "c4") if x != name]:
                 workloads[other] = run_side_leg(other, args, B, torch, sampler, peak, peak_kind)
                 launches += args.steps + workloads[other]["roofline"]["sustained"]["steps"]
+            for other in ("c4", "c5"):                      # all f+1 root children played (integer configurations)
+                key = other + "_all_children"
+                workloads[key] = run_side_leg(other, args, B, torch, sampler, peak, peak_kind, candidates=True)
+                launches += args.steps + workloads[key]["roofline"]["sustained"]["steps"]
     if sampler:
         sampler.stop()
 
@@ -625,6 +666,8 @@ def main():
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end, sustained, CPU and other-workload legs (for profiler runs)")
     ap.add_argument("--no-legs", action="store_true", help="skip the legs over the other configurations")
     ap.add_argument("--sustain-seconds", type=float, default=2.0, help="GPU time of the sustained run of the headline workload")
+    ap.add_argument("--candidates", action="store_true",
+                    help="time ftc_candidates_batch (what every root child delivers: all f+1 subtrees) on the workload")
     ap.add_argument("--full-config", action="store_true",
                     help="play every batch of the configuration (its stated scenario count), checking every scenario")
     args = ap.parse_args()

@@ -11,8 +11,10 @@
 // and counts it, the list sizes add up.
 //
 // Per node and child the kernel carries a value and a word: exists | present | failed bit | size of the failed list.
-// The values of the tile roots and of the rows above the tiles live in a per-block slice of the workspace, one heap
-// array per root child (they stay in L2), and are combined level by level as in the staged kernel.
+// Above the tiles the same split holds: the heap array of tile roots and upper rows is combined once in shared memory
+// for all children ("common" values, as in the staged kernel); only the nodes that have a specially played row
+// somewhere below them ("dirty": the ancestors of the few special rows) carry one value and word per child, in a
+// per-block slice of the workspace that is touched at those nodes only.
 #pragma once
 #include "ftc_staged_impl.cuh"
 
@@ -39,9 +41,14 @@ struct CandScen {
 
 // Node (row, sc) of root subtree sc after up-correction (Algorithm "Up-correction"): own input, the root's if it is a
 // partner and its message was sent, then the partners whose message arrived. `in_lc`: the scenario in the caller's
-// process order (global memory) at this lane's chunk. The caller guarantees that the node exists (sc < members of the row).
+// process order (global memory) at this lane's chunk; `srow_lc`: the row's staged copy in shared memory (its first
+// member, this lane's chunk), which serves every member but the one whose input sits in the renumbered slot.
+// The caller guarantees that the node exists (sc < members of the row).
 template <typename T, int OP>
-__device__ __noinline__ uint4 cand_fold(const Params& p, CandScen cs, const char* in_lc, uint32_t row, uint32_t sc, uint32_t& meta) {
+__device__ __noinline__ uint4 cand_fold(const Params& p, CandScen cs, const char* in_lc, const char* srow_lc, uint32_t row, uint32_t sc, uint32_t& meta) {
+    auto member = [&](uint32_t sp, uint32_t vr) -> uint4 {
+        return vr == cs.root ? ld_stream(in_lc) : *reinterpret_cast<const uint4*>(srow_lc + (size_t)sp * p.kbytes);
+    };
     const uint32_t mj = row < p.q ? p.m : p.r, vbase = row * p.m + 1, v = vbase + sc;
     if (!test_bit(cs.snd, v)) { meta = kMetaExists; return make_uint4(0, 0, 0, 0); }
     uint32_t mask = extract_bits(cs.alive, vbase, mj);
@@ -53,13 +60,13 @@ __device__ __noinline__ uint4 cand_fold(const Params& p, CandScen cs, const char
         const uint32_t sv = vr - vbase, t = local_round(cs.cx->ir[i], cs.base);
         if (!(partner_slot(p, row, sv, sc) < t)) mask &= ~(1u << sv);
     }
-    uint4 acc = ld_stream(in_lc + (size_t)(v == cs.root ? 0u : v) * p.kbytes);
+    uint4 acc = member(sc, v);
     // the root's up-correction send to member sc of its group is its send number sc (descending order: r-1-sc)
     const bool from_root = row == p.q && (p.pdesc ? p.r - 1 - sc : sc) < cs.troot;
     if (from_root) acc = comb16<T, OP>(acc, ld_stream(in_lc + (size_t)cs.root * p.kbytes));
     for (uint32_t sp = 0; sp < mj; ++sp) {
         const uint32_t vr = vbase + sp;
-        if (sp != sc && ((mask >> sp) & 1u)) acc = comb16<T, OP>(acc, ld_stream(in_lc + (size_t)(vr == cs.root ? 0u : vr) * p.kbytes));
+        if (sp != sc && ((mask >> sp) & 1u)) acc = comb16<T, OP>(acc, member(sp, vr));
     }
     meta = kMetaExists | kMetaPresent | (mj - __popc(mask) + ((row == p.q && !from_root) ? 1u : 0u));
     return acc;
@@ -68,15 +75,16 @@ __device__ __noinline__ uint4 cand_fold(const Params& p, CandScen cs, const char
 // A lane's sub-heap of XL levels for child sc: node, then child 1, then child 2. Rows >= G do not exist.
 template <typename T, int OP, int XL, int U>
 struct SubHeapCand {
-    static __device__ __forceinline__ uint4 eval(const Params& p, const CandScen& cs, const char* in_lc, uint32_t grow, uint32_t G, uint32_t sc, uint32_t& meta) {
+    static __device__ __forceinline__ uint4 eval(const Params& p, const CandScen& cs, const char* in_lc, const char* buf_lc, uint32_t rowbytes,
+                                                 uint32_t trow, uint32_t grow, uint32_t G, uint32_t sc, uint32_t& meta) {
         if (grow >= G) { meta = 0; return make_uint4(0, 0, 0, 0); }
-        uint4 v = cand_fold<T, OP>(p, cs, in_lc, grow, sc, meta);
+        uint4 v = cand_fold<T, OP>(p, cs, in_lc, buf_lc + (size_t)trow * rowbytes, grow, sc, meta);
         if (U + 1 < XL && (meta & kMetaPresent)) {           // what the children of a node that does not send deliver is lost
             constexpr int UN = (U + 1 < XL ? U + 1 : U);
             uint32_t cm;
-            uint4 cv = SubHeapCand<T, OP, XL, UN>::eval(p, cs, in_lc, 2 * grow + 1, G, sc, cm);
+            uint4 cv = SubHeapCand<T, OP, XL, UN>::eval(p, cs, in_lc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G, sc, cm);
             take_child<T, OP>(v, meta, cv, cm);
-            cv = SubHeapCand<T, OP, XL, UN>::eval(p, cs, in_lc, 2 * grow + 2, G, sc, cm);
+            cv = SubHeapCand<T, OP, XL, UN>::eval(p, cs, in_lc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G, sc, cm);
             take_child<T, OP>(v, meta, cv, cm);
         }
         return v;
@@ -120,6 +128,9 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
     uint32_t* alive = pf + p.W + 1;
     uint32_t* snd = alive + p.W + 1;
     uint32_t* tspec = reinterpret_cast<uint32_t*>(sbase + g.off_special);
+    uint32_t* dirty = reinterpret_cast<uint32_t*>(sbase + g.off_dirty);          // bit n: node n of the heap array is played per child
+    uint32_t* rspec = dirty + ((cg.nheap + 31) / 32 + 1);                        // bit j: row j above the tiles is a special row
+    uint4* hvc = reinterpret_cast<uint4*>(sbase + g.off_hv);                     // common values, heap order
     volatile uint32_t* gaveup = reinterpret_cast<volatile uint32_t*>(sbase + g.off_gaveup);
     // per block: values hv[sc][row][chunk], combined words hm[sc][row], own words of the rows above the tiles hmo[sc][row]
     char* slice = static_cast<char*>(p.ws) + (size_t)blockIdx.x * cg.slice_bytes;
@@ -232,14 +243,21 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
             }
         }
         // ---- work items that are played child by child: those with a failed process, a renumbered slot, the short last
-        // group, or not complete above their last level. One bit per item (tile i, then groups of rows above the tiles).
+        // group, or not complete above their last level. One bit per item (tile i, then groups of rows above the tiles);
+        // and the nodes of the heap array whose value differs from child to child: the ancestors of every special row.
         for (uint32_t w = tid; w < (nitems + 31) / 32 + 1; w += nt) tspec[w] = 0;
+        for (uint32_t w = tid; w < (cg.nheap + 31) / 32 + 1 + (cg.ntop + 31) / 32 + 1; w += nt) dirty[w] = 0;      // dirty and rspec
         __syncthreads();
         {
+            auto mark_dirty_from = [&](uint32_t n) {
+                for (;;) { atomicOr(&dirty[n >> 5], 1u << (n & 31)); if (n == 0) break; n = (n - 1) >> 1; }
+            };
             auto mark_row = [&](uint32_t j) {
                 const uint32_t lvl = ilog2u(j + 1);
                 const uint32_t it = lvl >= Lt ? ((j + 1) >> (lvl - Lt)) - ntiles : ntiles + j / grows;
                 atomicOr(&tspec[it >> 5], 1u << (it & 31));
+                if (lvl < Lt) atomicOr(&rspec[j >> 5], 1u << (j & 31));
+                mark_dirty_from(lvl >= Lt ? ((j + 1) >> (lvl - Lt)) - 1 : j);
             };
             for (uint32_t w = tid; w < p.W; w += nt) {
                 uint32_t word = pf[w];
@@ -257,8 +275,12 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
                 if (root != 0) mark_row((root - 1) / p.m);          // the slot that holds process 0's input
                 if (p.r) mark_row(p.q);                             // the short last group
             }
+            // tiles that exist but are not complete down to their second-to-last level: the check-free folds do not fit them
             for (uint32_t it = tid; it < ntiles; it += nt)
-                if (((ntop + it + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= Gc) atomicOr(&tspec[it >> 5], 1u << (it & 31));
+                if (ntop + it < Gc && ((ntop + it + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= Gc) {
+                    atomicOr(&tspec[it >> 5], 1u << (it & 31));
+                    mark_dirty_from(ntop + it);
+                }
             for (uint32_t gi = tid; gi < ngroups; gi += nt)
                 if ((gi + 1) * grows > ntop || (gi + 1) * grows > Gc) atomicOr(&tspec[(ntiles + gi) >> 5], 1u << ((ntiles + gi) & 31));
         }
@@ -278,92 +300,106 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
                 const uint32_t rowB = ((j0 + 1) << tB) - 1 + idxB;
                 if (!special) {
                     // every group of the tile is whole: one value per row serves all children (exact operations)
-                    uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
-                    if (XL > 1 || rowA < Gc) valA = SubHeapPlain<T, OP, XL, 0, false, false>::eval(p, 0u, alive, buf_lc, rowbytes, tA, rowA, Gc);
-                    const bool hasB = lr < RW - 1;
-                    if (hasB) valB = fold_plain_staged<T, OP>(p, 0u, buf_lc + staged_row_offset<false>(p, rowbytes, lr, rowB));
-                    valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, Gc);
-                    release();
-                    if (lr == 0) {
-                        const uint4 v = lw ? valB : valA;
-                        for (uint32_t sc = 0; sc < p.m; ++sc) {
-                            hv[((size_t)sc * cg.nheap + j0) * p.C + lc] = v;
-                            if (lc == 0) hm[(size_t)sc * cg.nheap + j0] = kMetaExists | kMetaPresent;
-                        }
+                    if (j0 < Gc) {
+                        uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
+                        if (XL > 1 || rowA < Gc) valA = SubHeapPlain<T, OP, XL, 0, false, false>::eval(p, 0u, alive, buf_lc, rowbytes, tA, rowA, Gc);
+                        const bool hasB = lr < RW - 1;
+                        if (hasB) valB = fold_plain_staged<T, OP>(p, 0u, buf_lc + staged_row_offset<false>(p, rowbytes, lr, rowB));
+                        valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, Gc);
+                        if (lr == 0) hvc[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                     }
+                    release();
                 } else {
-                    release();                                     // these few tiles read the scenario itself
                     for (uint32_t sc = 0; sc < p.m; ++sc) {
                         const uint32_t G = p.q + (sc < p.r ? 1u : 0u);
                         uint32_t mA = 0, mB = 0;
-                        uint4 valA = SubHeapCand<T, OP, XL, 0>::eval(p, cs, in_lc, rowA, G, sc, mA), valB = make_uint4(0, 0, 0, 0);
+                        uint4 valA = SubHeapCand<T, OP, XL, 0>::eval(p, cs, in_lc, buf_lc, rowbytes, tA, rowA, G, sc, mA), valB = make_uint4(0, 0, 0, 0);
                         const bool hasB = lr < RW - 1;
-                        if (hasB && rowB < G) valB = cand_fold<T, OP>(p, cs, in_lc, rowB, sc, mB);
+                        if (hasB && rowB < G) valB = cand_fold<T, OP>(p, cs, in_lc, buf_lc + (size_t)lr * rowbytes, rowB, sc, mB);
                         valB = tile_tree_phase_cand<T, OP>(valA, mA, valB, mB, lw, cwl, p.C, lane, lc, tB, idxB, hasB);
                         if (lr == 0) {
                             hv[((size_t)sc * cg.nheap + j0) * p.C + lc] = lw ? valB : valA;
                             if (lc == 0) hm[(size_t)sc * cg.nheap + j0] = lw ? mB : mA;
                         }
                     }
+                    release();
                 }
             } else {
                 // ---- rows above the tiles: fold now, combine later ----
                 if (!special) {
-                    uint4 v[7];
-#pragma unroll
-                    for (uint32_t gs = 0; gs < 7; ++gs)
-                        if (gs < GR) v[gs] = fold_plain_staged<T, OP>(p, 0u, buf_lc + (size_t)(gs * RW + lr) * rowbytes);
-                    release();
-#pragma unroll
-                    for (uint32_t gs = 0; gs < 7; ++gs) {
-                        if (gs >= GR) continue;
-                        const uint32_t row = (it - ntiles) * grows + gs * RW + lr;
-                        for (uint32_t sc = 0; sc < p.m; ++sc) {
-                            hv[((size_t)sc * cg.nheap + row) * p.C + lc] = v[gs];
-                            if (lc == 0) hmo[(size_t)sc * cg.ntop + row] = kMetaExists | kMetaPresent;
-                        }
+                    for (uint32_t gs = 0; gs < GR; ++gs) {
+                        const uint32_t rloc = gs * RW + lr;
+                        hvc[(size_t)((it - ntiles) * grows + rloc) * p.C + lc] = fold_plain_staged<T, OP>(p, 0u, buf_lc + (size_t)rloc * rowbytes);
                     }
                 } else {
-                    release();
                     for (uint32_t gs = 0; gs < GR; ++gs) {
-                        const uint32_t row = (it - ntiles) * grows + gs * RW + lr;
+                        const uint32_t rloc = gs * RW + lr, row = (it - ntiles) * grows + rloc;
                         if (row >= ntop) continue;
+                        if (!test_bit(rspec, row)) {               // an ordinary row of a group that holds a special one, or a ragged end
+                            if (row < Gc) hvc[(size_t)row * p.C + lc] = fold_plain_staged<T, OP>(p, 0u, buf_lc + (size_t)rloc * rowbytes);
+                            continue;
+                        }
                         for (uint32_t sc = 0; sc < p.m; ++sc) {
                             const uint32_t G = p.q + (sc < p.r ? 1u : 0u);
                             uint32_t mo = 0;
                             uint4 v = make_uint4(0, 0, 0, 0);
-                            if (row < G) v = cand_fold<T, OP>(p, cs, in_lc, row, sc, mo);
+                            if (row < G) v = cand_fold<T, OP>(p, cs, in_lc, buf_lc + (size_t)rloc * rowbytes, row, sc, mo);
                             hv[((size_t)sc * cg.nheap + row) * p.C + lc] = v;
                             if (lc == 0) hmo[(size_t)sc * cg.ntop + row] = mo;
                         }
                     }
                 }
+                release();
             }
         }
         __syncthreads();
-        // ---- levels above the tiles, leaves first (Algorithm "reduce_non_root"), all root children in one sweep ----
+        // ---- levels above the tiles, leaves first (Algorithm "reduce_non_root") ----
         for (int lvl = (int)Lt - 1; lvl >= 0; --lvl) {
             const uint32_t lo = (1u << lvl) - 1u, n = lo + 1u;
+            // nodes played per child: own value (a special row's per-child fold, else the row's common fold), then each
+            // child's delivery (per child if that node is played per child, else its common value)
             for (uint32_t u = tid; u < n * p.m * p.C; u += nt) {
-                const uint32_t c = u & Cmask, x = u >> cwl, sc = x % p.m, row = lo + x / p.m;
-                uint32_t meta = hmo[(size_t)sc * cg.ntop + row];
-                uint4 v = hv[((size_t)sc * cg.nheap + row) * p.C + c];
+                const uint32_t c = u & Cmask, x = u >> cwl, row = lo + x / p.m;
+                if (!test_bit(dirty, row)) continue;
+                const uint32_t sc = x % p.m;
+                const size_t me = (size_t)sc * cg.nheap + row;
+                uint32_t meta = kMetaExists | kMetaPresent;
+                uint4 v;
+                if (test_bit(rspec, row)) { meta = hmo[(size_t)sc * cg.ntop + row]; v = hv[me * p.C + c]; }
+                else v = hvc[(size_t)row * p.C + c];
                 if (meta & kMetaPresent) {
-                    const size_t c1 = (size_t)sc * cg.nheap + 2 * row + 1;
-                    take_child<T, OP>(v, meta, hv[c1 * p.C + c], hm[c1]);
-                    take_child<T, OP>(v, meta, hv[(c1 + 1) * p.C + c], hm[c1 + 1]);
-                    hv[((size_t)sc * cg.nheap + row) * p.C + c] = v;
+#pragma unroll
+                    for (uint32_t k2 = 1; k2 <= 2; ++k2) {
+                        const uint32_t ch = 2 * row + k2;
+                        if (test_bit(dirty, ch)) take_child<T, OP>(v, meta, hv[((size_t)sc * cg.nheap + ch) * p.C + c], hm[(size_t)sc * cg.nheap + ch]);
+                        else if (ch < Gc) take_child<T, OP>(v, meta, hvc[(size_t)ch * p.C + c], kMetaExists | kMetaPresent);
+                    }
                 }
-                if (c == 0) hm[(size_t)sc * cg.nheap + row] = meta;
+                hv[me * p.C + c] = v;
+                if (c == 0) hm[me] = meta;
+            }
+            __syncthreads();
+            // common values
+            for (uint32_t u = tid; u < n * p.C; u += nt) {
+                const uint32_t row = lo + (u >> cwl), c = u & Cmask;
+                if (row >= Gc) continue;
+                uint4 v = hvc[(size_t)row * p.C + c];
+                if (2 * row + 1 < Gc) v = comb16<T, OP>(v, hvc[(size_t)(2 * row + 1) * p.C + c]);
+                if (2 * row + 2 < Gc) v = comb16<T, OP>(v, hvc[(size_t)(2 * row + 2) * p.C + c]);
+                hvc[(size_t)row * p.C + c] = v;
             }
             __syncthreads();
         }
         // ---- what the root receives from each child ----
         const bool bad = *gaveup != 0;
+        const bool per_child = test_bit(dirty, 0u);                // else: nothing failed anywhere, every child delivers the common value
         for (uint32_t u = tid; u < p.m * p.C; u += nt) {
-            const uint32_t sc = u >> cwl, c = u & Cmask, meta = hm[(size_t)sc * cg.nheap];
+            const uint32_t sc = u >> cwl, c = u & Cmask;
+            const uint32_t meta = per_child ? hm[(size_t)sc * cg.nheap] : (kMetaExists | kMetaPresent);
             const bool got = (meta & kMetaPresent) && !bad;
-            reinterpret_cast<uint4*>(cand_s)[u] = got ? hv[((size_t)sc * cg.nheap) * p.C + c] : make_uint4(0, 0, 0, 0);
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (got) v = per_child ? hv[((size_t)sc * cg.nheap) * p.C + c] : hvc[c];
+            reinterpret_cast<uint4*>(cand_s)[u] = v;
             if (c == 0) {
                 info_s[2 * sc] = bad ? 3u : (meta & kMetaPresent) ? ((meta & kMetaFailed) ? 1u : 0u) : 2u;
                 info_s[2 * sc + 1] = got ? (meta & kMetaCount) : 0u;
@@ -394,10 +430,10 @@ static cudaError_t launch_cand_x(const Params& p, const CandGeom& cg, T* cand, u
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, cand_kernel<T, OP, XL>, (int)cg.st.nwarps * 32, cg.st.smem_bytes);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
-    if (per_sm > 2) per_sm = 2;                                   // slices of all blocks stay in L2
+    if (per_sm > 4) per_sm = 4;
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
-    if (grid_out) { *grid_out = (uint32_t)cap; return cudaSuccess; }
+    if (grid_out) { *grid_out = (uint32_t)cap; return cudaSuccess; }      // one workspace slice per block
     cand_kernel<T, OP, XL><<<grid, cg.st.nwarps * 32, cg.st.smem_bytes, st>>>(p, cg, cand, info);
     return cudaGetLastError();
 }
