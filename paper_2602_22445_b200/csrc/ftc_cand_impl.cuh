@@ -20,6 +20,7 @@
 
 namespace ftc {
 
+constexpr uint32_t kNoRow = 0xFFFFFFFFu, kManyRows = 0xFFFFFFFEu;
 constexpr uint32_t kMetaExists = 1u << 31, kMetaPresent = 1u << 30, kMetaFailed = 1u << 29, kMetaCount = (1u << 29) - 1;
 
 // A node takes one child's delivery: a child that sent is combined, its failed bit and list size taken over; a child
@@ -112,6 +113,114 @@ __device__ __forceinline__ uint4 tile_tree_phase_cand(uint4 valA, uint32_t mA, u
     return valB;
 }
 
+// What the out-of-line tile routines need.
+struct TileJob {
+    CandScen cs;
+    const char* in_s;        // the scenario in global memory (process order)
+    char* tile;              // the warp's staged copy of the tile's rows (tile-heap order); the out-of-line routines overwrite it
+    uint4* hv; uint32_t* hm; // per-child values and words of the heap array (workspace slice)
+    uint4* hvc;              // common values of the heap array (shared memory)
+    uint32_t nheap, j0, srow, Lt, D, Gc, rowbytes;
+};
+
+// Several special rows in one tile (rare): the whole tile child by child.
+template <typename T, int OP, int XL>
+__device__ __forceinline__ void cand_tile_many(const Params& p, const TileJob& jb) {
+    const uint32_t lane = threadIdx.x & 31, cwl = p.cw_log2, lw = 5 - cwl, RW = 1u << lw;
+    const uint32_t lr = lane >> cwl, lc = lane & (p.C - 1), j0 = jb.j0;
+    const uint32_t tA = RW - 1 + lr, rowA = ((j0 + 1) << lw) - 1 + lr;
+    const uint32_t tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB), rowB = ((j0 + 1) << tB) - 1 + idxB;
+    const char* in_lc = jb.in_s + lc * 16;
+    const char* buf_lc = jb.tile + lc * 16;
+    for (uint32_t sc = 0; sc < p.m; ++sc) {
+        const uint32_t G = p.q + (sc < p.r ? 1u : 0u);
+        uint32_t mA = 0, mB = 0;
+        uint4 valA = SubHeapCand<T, OP, XL, 0>::eval(p, jb.cs, in_lc, buf_lc, jb.rowbytes, tA, rowA, G, sc, mA), valB = make_uint4(0, 0, 0, 0);
+        const bool hasB = lr < RW - 1;
+        if (hasB && rowB < G) valB = cand_fold<T, OP>(p, jb.cs, in_lc, buf_lc + (size_t)lr * jb.rowbytes, rowB, sc, mB);
+        valB = tile_tree_phase_cand<T, OP>(valA, mA, valB, mB, lw, cwl, p.C, lane, lc, tB, idxB, hasB);
+        if (lr == 0) {
+            jb.hv[((size_t)sc * jb.nheap + j0) * p.C + lc] = lw ? valB : valA;
+            if (lc == 0) jb.hm[(size_t)sc * jb.nheap + j0] = lw ? mB : mA;
+        }
+    }
+}
+
+// A ragged tile, or one special row in it. First the common value of every node's subtree, by the plain definition
+// (valid wherever no special row lies below): own folds, then level by level. The value of a node takes the place of
+// its row's first member in the staged copy (no further shared memory is needed); the special row and its ancestors
+// keep their inputs, their values are not common anyway. Then, for one special row, its path to the tile's root, one
+// lane per (child, chunk): what hangs off the path is common.
+template <typename T, int OP>
+__device__ __forceinline__ void cand_tile_one(const Params& p, const TileJob& jb) {
+    const uint32_t lane = threadIdx.x & 31, cwl = p.cw_log2, Cmask = p.C - 1, j0 = jb.j0, Gc = jb.Gc, D = jb.D, rowbytes = jb.rowbytes;
+    char* tile = jb.tile;
+    const uint32_t nnodes = (1u << D) - 1;
+    const uint32_t srow = jb.srow;
+    // tile-heap index of the special row (none: beyond every node)
+    const uint32_t su = srow == kNoRow ? 0u : ilog2u(srow + 1) - jb.Lt;
+    const uint32_t st0 = srow == kNoRow ? 0xFFFFFFFFu : (1u << su) - 1 + (srow + 1 - ((j0 + 1) << su));
+    auto row_of_node = [&](uint32_t t) { const uint32_t u = ilog2u(t + 1); return ((j0 + 1) << u) - 1 + (t + 1 - (1u << u)); };
+    auto on_path = [&](uint32_t t) {                              // t is the special row's node or one of its ancestors
+        const uint32_t u = ilog2u(t + 1);
+        return srow != kNoRow && u <= su && ((st0 + 1) >> (su - u)) == t + 1;
+    };
+    auto tsub = [&](uint32_t t, uint32_t c) -> uint4& { return *reinterpret_cast<uint4*>(tile + (size_t)t * rowbytes + c * 16); };
+    for (uint32_t u = lane; u < nnodes * p.C; u += 32) {
+        const uint32_t t = u >> cwl, c = u & Cmask;
+        if (row_of_node(t) < Gc && !on_path(t)) tsub(t, c) = fold_plain_staged<T, OP>(p, 0u, tile + (size_t)t * rowbytes + c * 16);
+    }
+    __syncwarp();
+    for (int lv = (int)D - 2; lv >= 0; --lv) {
+        const uint32_t t0 = (1u << lv) - 1;
+        for (uint32_t u = lane; u < (t0 + 1) * p.C; u += 32) {
+            const uint32_t t = t0 + (u >> cwl), c = u & Cmask, row = row_of_node(t);
+            if (row >= Gc || on_path(t)) continue;
+            uint4 v = tsub(t, c);
+            if (2 * row + 1 < Gc) v = comb16<T, OP>(v, tsub(2 * t + 1, c));
+            if (2 * row + 2 < Gc) v = comb16<T, OP>(v, tsub(2 * t + 2, c));
+            tsub(t, c) = v;
+        }
+        __syncwarp();
+    }
+    if (srow == kNoRow) {                          // ragged only: the same for every child
+        if (lane < p.C && j0 < Gc) jb.hvc[(size_t)j0 * p.C + lane] = tsub(0, lane);
+        return;
+    }
+    for (uint32_t base_u = 0; base_u < p.m * p.C; base_u += 32) {
+        const uint32_t unit = base_u + lane;
+        if (unit >= p.m * p.C) continue;
+        const uint32_t sc = unit >> cwl, c = unit & Cmask;
+        const uint32_t G = p.q + (sc < p.r ? 1u : 0u);
+        const char* in_c = jb.in_s + c * 16;
+        uint32_t t = st0, row = srow, meta = 0;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (row < G) {
+            v = cand_fold<T, OP>(p, jb.cs, in_c, tile + (size_t)t * rowbytes + c * 16, row, sc, meta);
+            if ((meta & kMetaPresent) && su + 1 < D) {          // its own children are common
+                if (2 * row + 1 < Gc) take_child<T, OP>(v, meta, tsub(2 * t + 1, c), kMetaExists | kMetaPresent);
+                if (2 * row + 2 < Gc) take_child<T, OP>(v, meta, tsub(2 * t + 2, c), kMetaExists | kMetaPresent);
+            }
+        }
+        while (t > 0) {
+            const uint32_t tp = (t - 1) >> 1, rp = (row - 1) >> 1;
+            uint32_t pm;
+            uint4 pv = cand_fold<T, OP>(p, jb.cs, in_c, tile + (size_t)tp * rowbytes + c * 16, rp, sc, pm);
+            if (pm & kMetaPresent) {
+                const bool first = (t & 1u) != 0;                  // the path's node is child 1 of its parent
+                const uint32_t ts = first ? t + 1 : t - 1, rs = first ? row + 1 : row - 1;
+                const uint4 sv = tsub(ts, c);
+                const uint32_t sm = rs < Gc ? (kMetaExists | kMetaPresent) : 0u;
+                if (first) { take_child<T, OP>(pv, pm, v, meta); take_child<T, OP>(pv, pm, sv, sm); }
+                else { take_child<T, OP>(pv, pm, sv, sm); take_child<T, OP>(pv, pm, v, meta); }
+            }
+            v = pv; meta = pm; t = tp; row = rp;
+        }
+        jb.hv[((size_t)sc * jb.nheap + j0) * p.C + c] = v;
+        if (c == 0) jb.hm[(size_t)sc * jb.nheap + j0] = meta;
+    }
+}
+
 struct CandGeom {
     StagedGeom st;
     uint64_t slice_bytes;       // workspace per block: f+1 heap arrays of values, then the words
@@ -130,6 +239,7 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
     uint32_t* tspec = reinterpret_cast<uint32_t*>(sbase + g.off_special);
     uint32_t* dirty = reinterpret_cast<uint32_t*>(sbase + g.off_dirty);          // bit n: node n of the heap array is played per child
     uint32_t* rspec = dirty + ((cg.nheap + 31) / 32 + 1);                        // bit j: row j above the tiles is a special row
+    uint32_t* trowv = rspec + ((cg.ntop + 31) / 32 + 1);                        // per tile: its one special row, kNoRow or kManyRows
     uint4* hvc = reinterpret_cast<uint4*>(sbase + g.off_hv);                     // common values, heap order
     volatile uint32_t* gaveup = reinterpret_cast<volatile uint32_t*>(sbase + g.off_gaveup);
     // per block: values hv[sc][row][chunk], combined words hm[sc][row], own words of the rows above the tiles hmo[sc][row]
@@ -247,6 +357,7 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
         // and the nodes of the heap array whose value differs from child to child: the ancestors of every special row.
         for (uint32_t w = tid; w < (nitems + 31) / 32 + 1; w += nt) tspec[w] = 0;
         for (uint32_t w = tid; w < (cg.nheap + 31) / 32 + 1 + (cg.ntop + 31) / 32 + 1; w += nt) dirty[w] = 0;      // dirty and rspec
+        for (uint32_t w = tid; w < ntiles; w += nt) trowv[w] = kNoRow;
         __syncthreads();
         {
             auto mark_dirty_from = [&](uint32_t n) {
@@ -257,6 +368,10 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
                 const uint32_t it = lvl >= Lt ? ((j + 1) >> (lvl - Lt)) - ntiles : ntiles + j / grows;
                 atomicOr(&tspec[it >> 5], 1u << (it & 31));
                 if (lvl < Lt) atomicOr(&rspec[j >> 5], 1u << (j & 31));
+                else {                                              // the tile remembers its special row while it is the only one
+                    const uint32_t old = atomicCAS(&trowv[it], kNoRow, j);
+                    if (old != kNoRow && old != j) trowv[it] = kManyRows;
+                }
                 mark_dirty_from(lvl >= Lt ? ((j + 1) >> (lvl - Lt)) - 1 : j);
             };
             for (uint32_t w = tid; w < p.W; w += nt) {
@@ -277,10 +392,7 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
             }
             // tiles that exist but are not complete down to their second-to-last level: the check-free folds do not fit them
             for (uint32_t it = tid; it < ntiles; it += nt)
-                if (ntop + it < Gc && ((ntop + it + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= Gc) {
-                    atomicOr(&tspec[it >> 5], 1u << (it & 31));
-                    mark_dirty_from(ntop + it);
-                }
+                if (ntop + it < Gc && ((ntop + it + 2) << (D >= 2 ? D - 2 : 0)) - 2 >= Gc) atomicOr(&tspec[it >> 5], 1u << (it & 31));
             for (uint32_t gi = tid; gi < ngroups; gi += nt)
                 if ((gi + 1) * grows > ntop || (gi + 1) * grows > Gc) atomicOr(&tspec[(ntiles + gi) >> 5], 1u << ((ntiles + gi) & 31));
         }
@@ -310,18 +422,10 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
                     }
                     release();
                 } else {
-                    for (uint32_t sc = 0; sc < p.m; ++sc) {
-                        const uint32_t G = p.q + (sc < p.r ? 1u : 0u);
-                        uint32_t mA = 0, mB = 0;
-                        uint4 valA = SubHeapCand<T, OP, XL, 0>::eval(p, cs, in_lc, buf_lc, rowbytes, tA, rowA, G, sc, mA), valB = make_uint4(0, 0, 0, 0);
-                        const bool hasB = lr < RW - 1;
-                        if (hasB && rowB < G) valB = cand_fold<T, OP>(p, cs, in_lc, buf_lc + (size_t)lr * rowbytes, rowB, sc, mB);
-                        valB = tile_tree_phase_cand<T, OP>(valA, mA, valB, mB, lw, cwl, p.C, lane, lc, tB, idxB, hasB);
-                        if (lr == 0) {
-                            hv[((size_t)sc * cg.nheap + j0) * p.C + lc] = lw ? valB : valA;
-                            if (lc == 0) hm[(size_t)sc * cg.nheap + j0] = lw ? mB : mA;
-                        }
-                    }
+                    // the few tiles with a special row or a ragged end: out of line, so that the common path stays compact
+                    const TileJob job{cs, in_s, tile, hv, hm, hvc, cg.nheap, j0, trowv[it], Lt, D, Gc, rowbytes};
+                    if (job.srow == kManyRows) cand_tile_many<T, OP, XL>(p, job);
+                    else cand_tile_one<T, OP>(p, job);
                     release();
                 }
             } else {

@@ -72,7 +72,7 @@ struct StagedGeom {
     uint32_t nwarps, nbuf, tile_cap;       // warps per block, buffers per warp, bytes per buffer (multiple of 128)
     uint32_t whole;                        // 1: the whole scenario is staged in one block-wide buffer
     uint32_t off_special, off_rootv, off_hv, off_bar, off_gaveup, off_tiles, smem_bytes;
-    uint32_t off_dirty;                    // all-children kernel: bitmaps over the rows of the heap array
+    uint32_t off_dirty;                    // all-children kernel: bitmaps over the rows of the heap array, then one word per tile
     uint32_t hv_global;                    // 1: the heap array of tile roots and upper rows lives in the workspace
     uint64_t hv_bytes;                     // its size per block
 };
@@ -659,6 +659,7 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
     const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
     const uint64_t cap = ((((uint64_t)1 << D) - 1 + p.row_shift) * rowbytes + 127) & ~(uint64_t)127;
     if (cap > 64 * 1024) return false;
+
     const uint32_t RW = 1u << lw, ntiles = 1u << p.Lt;
     const uint32_t gr_max = (1u << XL) - 1, gr_need = (ntiles - 1 + RW - 1) >> lw;
     const uint32_t grows = RW * (p.swz_mask ? 1u : (gr_need < 1 ? 1u : (gr_need < gr_max ? gr_need : gr_max)));
@@ -685,7 +686,7 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
                    p.ws_bytes / ((uint64_t)sm_count * kHvGlobalBlocksPerSm) >= g.hv_bytes) ? 1u : 0u;
     g.off_hv = (uint32_t)o; if (!g.hv_global) o += (size_t)g.hv_bytes;
     g.off_dirty = (uint32_t)o;
-    if (all_children) o += (((((size_t)3 << p.Lt) + 31) / 32 + 4) * 4 + 15) & ~(size_t)15;      // keeps the barriers behind it 8-byte aligned
+    if (all_children) o += ((((((size_t)3 << p.Lt) + 31) / 32 + 4) + ((size_t)1 << p.Lt)) * 4 + 15) & ~(size_t)15;   // keeps the barriers behind it 8-byte aligned
     g.off_bar = (uint32_t)o; o += (size_t)(kStagedMaxThreads / 32) * 4 * 8 + 8;      // room for any warps x nbuf, plus one
     g.off_gaveup = (uint32_t)o; o += 8;
     o = (o + 127) & ~(size_t)127; g.off_tiles = (uint32_t)o;
