@@ -7,14 +7,14 @@ ftc_allreduce_batch / ftc_reduce_batch = one kernel launch. Default workload: th
 configuration (f=4, k=32 int32, max, pre- and in-operation failures), a batch of 32768 scenarios
 (16 GiB of inputs, far larger than L2, so no flush is needed between steps).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3|c4|c5|c5r] [--batch S]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|c5|c5r] [--batch S]
     python bench.py --full-config [--workload cN]   # every batch of the configuration, every scenario checked
     python bench.py --impl reference ...      # times the CPU oracle on a bounded sample of the same workload
 
 Beside the K timed steps of the headline workload the line carries: the same step repeated for about two seconds
 with the SM clocks sampled meanwhile (roofline.sustained), the bandwidth of the library's read-only streaming
 kernels over the same buffer (roofline.read_only_gbs), and one record per other configuration, timed the same way
-(workloads: c5, c5r, c3).
+(workloads: c5, c5r, c3, c2, and what every root child delivers on c4 and c5).
 
 Prints ONE JSON line (rank 0). With N > 1 (torchrun) every rank runs its own batch: scenarios are
 independent, there is no collective on the data path ("weak" scaling).
@@ -43,6 +43,13 @@ ESZ = {"int32": 4, "int64": 8, "uint64": 8, "float32": 4}
 
 
 def make_workload(name: str, S: int, first: int, rounds_attempt_c4: int):
+    if name == "c2":
+        # all 2081 failure sets of size <= 2, each under S / 2081 input draws (the configuration has 16 draws: 33 296 scenarios)
+        if S % 2081:
+            raise SystemExit("a c2 batch is a multiple of 2081 scenarios (every failure set of size <= 2 once per draw)")
+        w = sc.config2(draws=S // 2081)
+        w.first_scenario = first
+        return w
     if name == "c3":
         return sc.config3(S=S, first=first)
     if name == "c4":
@@ -54,9 +61,11 @@ def make_workload(name: str, S: int, first: int, rounds_attempt_c4: int):
     raise SystemExit(f"unknown workload {name}")
 
 
-DEFAULT_BATCH = {"c3": 1 << 18, "c4": 1 << 15, "c5": 1 << 13, "c5r": 1 << 13}     # 16 GiB of inputs each
-CONFIG_SCENARIOS = {"c3": 1 << 20, "c4": 1 << 18, "c5": 1 << 14, "c5r": 1 << 14}    # scenarios of the whole configuration
+DEFAULT_BATCH = {"c3": 1 << 18, "c4": 1 << 15, "c5": 1 << 13, "c5r": 1 << 13,      # 16 GiB of inputs each
+                 "c2": 2081 * 1024}                                                  # 8 GiB: the configuration's sets under 1024 draws
+CONFIG_SCENARIOS = {"c3": 1 << 20, "c4": 1 << 18, "c5": 1 << 14, "c5r": 1 << 14, "c2": 2081 * 16}    # scenarios of the whole configuration
 DESCRIPTION = {
+    "c2": "reduce P=64 f=2 k=8 int64 sum, every pre-operation failure set of size <= 2, root 0 (64x the configuration's 16 input draws)",
     "c3": "allreduce P=1024 f=3 k=16 float32 (Irwin-Hall stand-in for N(0,1)) sum, 0..3 pre-operation failures",
     "c4": "allreduce P=4096 f=4 k=32 int32 max, 0..2 pre-operation + 0..2 in-operation failures",
     "c5": "allreduce P=65536 f=8 k=4 uint64 sum, 0..8 pre-operation failures, per-scenario first root",
@@ -181,7 +190,7 @@ def time_oracle(w, prepared):
     return n_scen / dt, dt, min(cores, len(ids))
 
 
-ORACLE_SAMPLE = {"c3": (32768, 256), "c4": (4096, 32), "c5": (192, 2), "c5r": (192, 2)}
+ORACLE_SAMPLE = {"c3": (32768, 256), "c4": (4096, 32), "c5": (192, 2), "c5r": (192, 2), "c2": (2081 * 128, 2081)}
 
 
 def run_reference(args):
@@ -189,7 +198,7 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import oracle as orc
-    sched = orc.schedule(*{"c3": (1024, 3), "c4": (4096, 4), "c5": (65536, 8), "c5r": (65536, 8)}[args.workload])
+    sched = orc.schedule(*{"c2": (64, 2), "c3": (1024, 3), "c4": (4096, 4), "c5": (65536, 8), "c5r": (65536, 8)}[args.workload])
     n_max, chunk = ORACLE_SAMPLE[args.workload]
     w = make_workload(args.workload, n_max, 0, sched["rounds_attempt"])
     cores = os.cpu_count() or 1
@@ -209,7 +218,7 @@ def run_reference(args):
     line = {
         "impl": "reference", "metric": "scenarios_per_sec", "value": value, "unit": "scenarios/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": {"c3": "f32", "c4": "i32", "c5": "u64", "c5r": "u64"}[args.workload],
+        "vs_baseline": None, "dtype": {"c2": "i64", "c3": "f32", "c4": "i32", "c5": "u64", "c5r": "u64"}[args.workload],
         "data": "synthetic", "process_rounds_per_sec": value * w.P * rounds_of(w, sched),
         "config": {"workload": f"{args.workload}: {DESCRIPTION[args.workload]}", "scenarios_per_step": n,
                    "note": "CPU oracle (literal message-by-message simulation) on a bounded sample per step"},
@@ -225,14 +234,14 @@ def run_reference(args):
 # GPU arm
 # ------------------------------------------------------------------------------------------------
 def kernel_source_hash() -> str:
-    """Hash of the sources of the staged kernel (the one the traffic figures belong to): ncu counters taken from
-    an older kernel must not be quoted for a newer one."""
+    """Hash of the sources of the staged and warp kernels (the ones the traffic figures belong to): ncu counters
+    taken from an older kernel must not be quoted for a newer one."""
     import glob
     import hashlib
     h = hashlib.sha256()
     base = os.path.join(ROOT, "paper_2602_22445_b200", "csrc")
-    files = glob.glob(os.path.join(base, "ftc_staged*.cu")) + glob.glob(os.path.join(base, "ftc_staged*.cuh")) + \
-        [os.path.join(base, n) for n in ("ftc_tile_common.cuh", "ftc_device.cuh")]
+    files = [f for pat in ("ftc_staged*.cu", "ftc_staged*.cuh", "ftc_warp*.cu", "ftc_warp*.cuh") for f in glob.glob(os.path.join(base, pat))] + \
+        [os.path.join(base, n) for n in ("ftc_tile_common.cuh", "ftc_device.cuh", "ftc_decode_warp.cuh")]
     for f in sorted(files):
         h.update(open(f, "rb").read())
     return h.hexdigest()[:16]
@@ -392,7 +401,7 @@ def add_sustained(roof, leg, torch, sampler, seconds):
 def run_side_leg(name, args, B, torch, sampler, peak, peak_kind, candidates=False):
     """One more workload, timed like the headline one: K steps, then a sustained run; its own roofline record.
     candidates: what every root child delivers (ftc_candidates_batch) instead of the batch call."""
-    S = DEFAULT_BATCH[name]
+    S = (args.batch if args.candidates and args.batch else 0) or DEFAULT_BATCH[name]
     leg = Leg(name, S, 0, args, B, torch, 28, candidates=candidates)
     for _ in range(max(args.warmup, 3)):
         leg.step()
@@ -441,8 +450,8 @@ def run_full_config(args, B, torch, sampler, peak, peak_kind):
     K steps are timed, and the batch is checked against the any-size properties; times are summed over the batches."""
     from paper_2602_22445_b200 import verify
     name = args.workload
-    S = args.batch or DEFAULT_BATCH[name]
     total = CONFIG_SCENARIOS[name]
+    S = args.batch or min(DEFAULT_BATCH[name], total)
     nb = (total + S - 1) // S
     leg = Leg(name, S, 0, args, B, torch, 28)
     sum_ms, all_ms, checks = 0.0, [], {"ok_scenarios": 0, "noop_scenarios": 0, "retried": 0, "excluded_pairs": 0}
@@ -612,7 +621,7 @@ def run_gpu(args):
 
         # ---- the other configurations the target names, each timed the same way (one GPU only) ----
         if world == 1 and not args.no_legs:
-            for other in [x for x in ("c5", "c5r", "c3", "c4") if x != name]:
+            for other in [x for x in ("c5", "c5r", "c3", "c4", "c2") if x != name]:
                 workloads[other] = run_side_leg(other, args, B, torch, sampler, peak, peak_kind)
                 launches += args.steps + workloads[other]["roofline"]["sustained"]["steps"]
             for other in ("c4", "c5"):                      # all f+1 root children played (integer configurations)
