@@ -20,10 +20,12 @@ __device__ __forceinline__ uint4 ld_stream(const char* ptr) {
     return __ldg(reinterpret_cast<const uint4*>(ptr));
 }
 
+// WIDTH < 32: the warp is cut into groups of WIDTH lanes and `src` counts within the caller's group.
+template <int WIDTH = 32>
 __device__ __forceinline__ uint4 shfl16(uint4 v, uint32_t src) {
     uint4 r;
-    r.x = __shfl_sync(0xFFFFFFFFu, v.x, src); r.y = __shfl_sync(0xFFFFFFFFu, v.y, src);
-    r.z = __shfl_sync(0xFFFFFFFFu, v.z, src); r.w = __shfl_sync(0xFFFFFFFFu, v.w, src);
+    r.x = __shfl_sync(0xFFFFFFFFu, v.x, src, WIDTH); r.y = __shfl_sync(0xFFFFFFFFu, v.y, src, WIDTH);
+    r.z = __shfl_sync(0xFFFFFFFFu, v.z, src, WIDTH); r.w = __shfl_sync(0xFFFFFFFFu, v.w, src, WIDTH);
     return r;
 }
 
@@ -168,14 +170,15 @@ __device__ __forceinline__ uint4 fold16_careful(const Params& p, uint32_t root, 
 // index lr, level tB, position idxB; rowB its global row, hasB whether it exists). Returns the updated valB.
 // FULL: every row of the tile's upper levels and of its bottom level exists (no existence checks at all);
 // FULL_ABOVE: only the bottom level may be ragged (checked), everything above exists.
-template <typename T, int OP, bool FULL = false, bool FULL_ABOVE = false>
+// WIDTH < 32: one tile per group of WIDTH lanes; `lane` is then the lane within the group.
+template <typename T, int OP, bool FULL = false, bool FULL_ABOVE = false, int WIDTH = 32>
 __device__ __forceinline__ uint4 tile_tree_phase(uint4 valA, uint4 valB, uint32_t lw, uint32_t cwl, uint32_t C,
                                                  uint32_t lane, uint32_t lc, uint32_t tB, uint32_t idxB, uint32_t rowB,
                                                  bool hasB, uint32_t G) {
     if (lw) {
         const bool mine = hasB && tB == lw - 1;
         const uint32_t src1 = mine ? (((2 * idxB) << cwl) | lc) : lane;
-        const uint4 c1 = shfl16(valA, src1), c2 = shfl16(valA, mine ? src1 + C : lane);
+        const uint4 c1 = shfl16<WIDTH>(valA, src1), c2 = shfl16<WIDTH>(valA, mine ? src1 + C : lane);
         if (mine) {
             if (FULL || 2 * rowB + 1 < G) valB = comb16<T, OP>(valB, c1);
             if (FULL || 2 * rowB + 2 < G) valB = comb16<T, OP>(valB, c2);
@@ -184,7 +187,7 @@ __device__ __forceinline__ uint4 tile_tree_phase(uint4 valA, uint4 valB, uint32_
     for (int t = (int)lw - 2; t >= 0; --t) {
         const bool mine = hasB && tB == (uint32_t)t;
         const uint32_t src1 = mine ? ((((2u << t) - 1 + 2 * idxB) << cwl) | lc) : lane;
-        const uint4 c1 = shfl16(valB, src1), c2 = shfl16(valB, mine ? src1 + C : lane);
+        const uint4 c1 = shfl16<WIDTH>(valB, src1), c2 = shfl16<WIDTH>(valB, mine ? src1 + C : lane);
         if (mine) {
             if (FULL || FULL_ABOVE || 2 * rowB + 1 < G) valB = comb16<T, OP>(valB, c1);
             if (FULL || FULL_ABOVE || 2 * rowB + 2 < G) valB = comb16<T, OP>(valB, c2);

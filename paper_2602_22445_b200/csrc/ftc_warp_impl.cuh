@@ -19,6 +19,7 @@
 namespace ftc {
 
 struct WarpGeom {
+    uint32_t lanes;        // lanes that play one scenario: 32, or 16 / 8 when the tile needs no more (several scenarios per warp)
     uint32_t lw;           // levels of the tile combined with shuffles: 2^lw lane rows are used
     uint32_t group;        // scenarios per buffer (consecutive scenarios, one bulk copy)
     uint32_t buf_bytes;    // bytes per buffer (multiple of 128)
@@ -26,21 +27,29 @@ struct WarpGeom {
 };
 
 // blocks (= warps) per SM the register budget allows: sub-heaps of three levels keep eight rows per lane in registers
-template <int XL> struct WarpMinBlocks { static constexpr int value = XL >= 3 ? 16 : 32; };
+// (several scenarios per warp need a few more registers: 24 warps then)
+template <int XL, int L = 32> struct WarpMinBlocks { static constexpr int value = XL >= 3 ? 16 : (L < 32 ? 24 : 32); };
 
 // MODE: bit 0 = allreduce, bit 1 = the call has in-operation slots.
-template <typename T, int OP, int XL, int MODE>
-__global__ void __launch_bounds__(32, WarpMinBlocks<XL>::value) warp_kernel(Params p, WarpGeom g) {
+// L: lanes per scenario. L < 32: the warp plays 32 / L scenarios at a time, one per group of L lanes, with one
+// instruction stream: the decode is decode_group<L>, the tile's shuffles stay inside the group, and what used to be
+// the same for the whole warp (root, selected child, masks) is the same within a group. A pair that holds a scenario
+// for the general routines is played one scenario after the other, all groups on the same scenario.
+template <typename T, int OP, int XL, int MODE, int L>
+__global__ void __launch_bounds__(32, WarpMinBlocks<XL, L>::value) warp_kernel(Params p, WarpGeom g) {
     constexpr bool ALLRED = (MODE & 1) != 0, INOP = (MODE & 2) != 0;
+    constexpr uint32_t NS = 32 / L;
     extern __shared__ __align__(128) uint32_t smem[];
     char* sbase = reinterpret_cast<char*>(smem);
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
     uint32_t* pf = smem + sizeof(Ctx) / 4;
     uint32_t* inc = pf + p.W + 1;
     uint32_t* unr = inc + p.W + 1;
+    uint32_t* ginc = unr + p.W + 1;                                     // L < 32: one arrival mask (W + 1 words) per group
     const uint32_t lane = threadIdx.x;
+    const uint32_t lg = lane & (L - 1), gi = lane / L;                  // lane within its group, group within the warp
     const uint32_t cwl = p.cw_log2, lw = g.lw, RW = 1u << lw;
-    const uint32_t lr_real = lane >> cwl, lc = lane & (p.C - 1);
+    const uint32_t lr_real = lg >> cwl, lc = lg & (p.C - 1);
     const uint32_t lr = lr_real < RW ? lr_real : 0u;                    // lane rows beyond the tile repeat lane row 0 (their results are unused)
     const uint32_t nq = p.C < 8 ? 8u / p.C : 1u, gq = min(nq, p.m & (0u - p.m));
     const uint32_t rot = (lr >> ilog2u(nq / gq)) & (gq - 1);          // starting member of this lane row's folds (bank spread)
@@ -98,74 +107,159 @@ __global__ void __launch_bounds__(32, WarpMinBlocks<XL>::value) warp_kernel(Para
             else dead = true;
         }
         const uint32_t n = group_size(grp);
+        if constexpr (L == 32) {
         for (uint32_t i = 0; i < n; ++i) {
-            const uint64_t s = grp * g.group + i;
-            char* out_s = reinterpret_cast<char*>(p.out) + s * p.kbytes;
-            uint32_t pfw = __shfl_sync(kFullWarp, cur.pfw, lane < p.W ? i * p.W + lane : 0u);
-            if (lane >= p.W) pfw = 0;
-            else if (lane == p.W - 1 && (p.P & 31)) pfw &= (1u << (p.P & 31)) - 1u;
-            uint32_t ev = FTC_INOP_UNUSED, er = 0;
-            if (INOP) {
-                const uint32_t src = lane < p.max_inop ? i * p.max_inop + lane : 0u;
-                ev = __shfl_sync(kFullWarp, cur.vic, src); er = __shfl_sync(kFullWarp, cur.rnd, src);
-            }
-            const uint32_t first_root = p.root >= 0 ? (uint32_t)p.root : __shfl_sync(kFullWarp, cur.root, i);
-            WarpScen w;
-            if (decode_warp<(ALLRED ? 1 : 0), (INOP ? 1 : 0)>(p, pfw, ev, er, first_root, w)) {
-                if (lane <= p.W) inc[lane] = w.incw;
-                if (p.W == 32 && lane == 0) inc[32] = 0;
-                __syncwarp();
-            } else {
-                // the general routines (a block of one warp may call them): everything outside the register decode
-                decode_scenario(p, s, cx, pf, inc);
-                if (cx->code == FTC_ST_OK && ALLRED) count_holders(p, cx, pf, unr);
-                w.code = cx->code; w.sstar = cx->sstar; w.attempts = cx->attempts; w.root = cx->root; w.base = cx->base;
-                w.npre = cx->npre; w.nexcl = cx->nexcl; w.inop_incl = cx->inop_incl; w.holders = cx->holders; w.G = cx->G;
-                w.any_victim = 1;
-                __syncwarp();
-            }
-            const bool okc = w.code == FTC_ST_OK && !dead;
-            if (!okc) {
-                if (lane < p.C) reinterpret_cast<uint4*>(out_s)[lane] = make_uint4(0, 0, 0, 0);
-            } else {
-                char* sc = bufs + (size_t)b * g.buf_bytes + (size_t)i * scen_bytes;
-                // renumbered order: the vectors of process 0 and of the root change places (the copy is the warp's own)
-                if (w.root != 0) {
-                    if (lane < p.C) {
-                        uint4* a = reinterpret_cast<uint4*>(sc) + lane;
-                        uint4* c = reinterpret_cast<uint4*>(sc + (size_t)w.root * p.kbytes) + lane;
-                        const uint4 va = *a, vc = *c;
-                        *a = vc; *c = va;
-                    }
+                const uint64_t s = grp * g.group + i;
+                char* out_s = reinterpret_cast<char*>(p.out) + s * p.kbytes;
+                uint32_t pfw = __shfl_sync(kFullWarp, cur.pfw, lane < p.W ? i * p.W + lane : 0u);
+                if (lane >= p.W) pfw = 0;
+                else if (lane == p.W - 1 && (p.P & 31)) pfw &= (1u << (p.P & 31)) - 1u;
+                uint32_t ev = FTC_INOP_UNUSED, er = 0;
+                if (INOP) {
+                    const uint32_t src = lane < p.max_inop ? i * p.max_inop + lane : 0u;
+                    ev = __shfl_sync(kFullWarp, cur.vic, src); er = __shfl_sync(kFullWarp, cur.rnd, src);
+                }
+                const uint32_t first_root = p.root >= 0 ? (uint32_t)p.root : __shfl_sync(kFullWarp, cur.root, i);
+                WarpScen w;
+                if (decode_warp<(ALLRED ? 1 : 0), (INOP ? 1 : 0)>(p, pfw, ev, er, first_root, w)) {
+                    if (lane <= p.W) inc[lane] = w.incw;
+                    if (p.W == 32 && lane == 0) inc[32] = 0;
+                    __syncwarp();
+                } else {
+                    // the general routines (a block of one warp may call them): everything outside the register decode
+                    decode_scenario(p, s, cx, pf, inc);
+                    if (cx->code == FTC_ST_OK && ALLRED) count_holders(p, cx, pf, unr);
+                    w.code = cx->code; w.sstar = cx->sstar; w.attempts = cx->attempts; w.root = cx->root; w.base = cx->base;
+                    w.npre = cx->npre; w.nexcl = cx->nexcl; w.inop_incl = cx->inop_incl; w.holders = cx->holders; w.G = cx->G;
+                    w.any_victim = 1;
                     __syncwarp();
                 }
-                const uint32_t sstar = w.sstar, G = w.G;
+                const bool okc = w.code == FTC_ST_OK && !dead;
+                if (!okc) {
+                    if (lane < p.C) reinterpret_cast<uint4*>(out_s)[lane] = make_uint4(0, 0, 0, 0);
+                } else {
+                    char* sc = bufs + (size_t)b * g.buf_bytes + (size_t)i * scen_bytes;
+                    // renumbered order: the vectors of process 0 and of the root change places (the copy is the warp's own)
+                    if (w.root != 0) {
+                        if (lane < p.C) {
+                            uint4* a = reinterpret_cast<uint4*>(sc) + lane;
+                            uint4* c = reinterpret_cast<uint4*>(sc + (size_t)w.root * p.kbytes) + lane;
+                            const uint4 va = *a, vc = *c;
+                            *a = vc; *c = va;
+                        }
+                        __syncwarp();
+                    }
+                    const uint32_t sstar = w.sstar, G = w.G;
+                    const char* in_lc = sc + lc * 16;
+                    // the one tile: heap rows 0 .. 2^D - 2; lane row lr owns row lr of the upper levels and the sub-heap under row RW-1+lr
+                    const uint32_t tA = RW - 1 + lr, rowA = tA, tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB), rowB = lr;
+                    const bool masked = w.npre != 0 || w.any_victim != 0;
+                    uint4 valA, valB;
+                    const bool hasB = lr < RW - 1;
+                    fold_tile_fast<T, OP, XL, true, false, true>(p, 0u, sstar, inc, in_lc, in_lc, rowbytes, 0u, lr, rot, rowB, hasB, tA, rowA, G, masked, valA, valB,
+                                                                 G > p.q ? p.q : 0xFFFFFFFFu);
+                    valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
+                    // the root (Algorithm "reduce_root"): its own data on the left unless the child's subtree holds it already
+                    if (lr_real == 0) {
+                        uint4 recv = lw ? valB : valA;
+                        if (sstar >= p.r) recv = comb16<T, OP>(fold_root16<T, OP, LdShared>(p, 0u, inc, in_lc), recv);
+                        reinterpret_cast<uint4*>(out_s)[lc] = recv;
+                    }
+                }
+                if (lane == 0) {
+                    uint4 rec;
+                    const uint32_t code = dead ? (uint32_t)FTC_ST_INTERNAL_TIMEOUT : w.code;
+                    rec.x = code | ((okc ? w.sstar : 0xFFu) << 8) | (w.attempts << 16);
+                    rec.y = okc ? p.P - w.npre - w.nexcl : 0u;
+                    rec.z = okc ? w.inop_incl : 0u;
+                    rec.w = (okc && ALLRED) ? w.holders : 0u;
+                    *reinterpret_cast<uint4*>(p.status + s * FTC_STATUS_WORDS) = rec;
+                }
+                __syncwarp();
+            }
+        } else {
+            // ---- 32 / L scenarios at a time, one per group of L lanes ----
+            auto evaluate = [&](const WarpScen& w, const uint32_t* incp, char* sc, bool writer, uint64_t s) {
+                const bool okc = w.code == FTC_ST_OK && !dead;
+                // renumbered order: the vectors of process 0 and of the root change places (the copy is the warp's own)
+                if (okc && writer && w.root != 0 && lg < p.C) {
+                    uint4* a = reinterpret_cast<uint4*>(sc) + lg;
+                    uint4* c = reinterpret_cast<uint4*>(sc + (size_t)w.root * p.kbytes) + lg;
+                    const uint4 va = *a, vc = *c;
+                    *a = vc; *c = va;
+                }
+                __syncwarp();
+                const uint32_t sstar = okc ? w.sstar : 0u, G = okc ? w.G : 0u;   // G = 0: every fold reads row 0, results unused
                 const char* in_lc = sc + lc * 16;
-                // the one tile: heap rows 0 .. 2^D - 2; lane row lr owns row lr of the upper levels and the sub-heap under row RW-1+lr
                 const uint32_t tA = RW - 1 + lr, rowA = tA, tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB), rowB = lr;
-                const bool masked = w.npre != 0 || w.any_victim != 0;
+                const bool masked = okc && (w.npre != 0 || w.any_victim != 0);
                 uint4 valA, valB;
                 const bool hasB = lr < RW - 1;
-                fold_tile_fast<T, OP, XL, true, false, true>(p, 0u, sstar, inc, in_lc, in_lc, rowbytes, 0u, lr, rot, rowB, hasB, tA, rowA, G, masked, valA, valB,
-                                                             G > p.q ? p.q : 0xFFFFFFFFu);
-                valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
-                // the root (Algorithm "reduce_root"): its own data on the left unless the child's subtree holds it already
-                if (lr_real == 0) {
-                    uint4 recv = lw ? valB : valA;
-                    if (sstar >= p.r) recv = comb16<T, OP>(fold_root16<T, OP, LdShared>(p, 0u, inc, in_lc), recv);
-                    reinterpret_cast<uint4*>(out_s)[lc] = recv;
+                fold_tile_fast<T, OP, XL, true, false, true>(p, 0u, sstar, incp, in_lc, in_lc, rowbytes, 0u, lr, rot, rowB, hasB, tA, rowA, G, masked, valA, valB,
+                                                             (okc && G > p.q) ? p.q : 0xFFFFFFFFu);
+                valB = tile_tree_phase<T, OP, (XL > 1), true, L>(valA, valB, lw, cwl, p.C, lg, lc, tB, idxB, rowB, hasB, G);
+                if (writer) {
+                    if (lr_real == 0) {
+                        uint4 recv = make_uint4(0, 0, 0, 0);
+                        if (okc) {
+                            recv = lw ? valB : valA;
+                            if (sstar >= p.r) recv = comb16<T, OP>(fold_root16<T, OP, LdShared>(p, 0u, incp, in_lc), recv);
+                        }
+                        reinterpret_cast<uint4*>(reinterpret_cast<char*>(p.out) + s * p.kbytes)[lc] = recv;
+                    }
+                    if (lg == 0) {
+                        uint4 rec;
+                        const uint32_t code = dead ? (uint32_t)FTC_ST_INTERNAL_TIMEOUT : w.code;
+                        rec.x = code | ((okc ? w.sstar : 0xFFu) << 8) | (w.attempts << 16);
+                        rec.y = okc ? p.P - w.npre - w.nexcl : 0u;
+                        rec.z = okc ? w.inop_incl : 0u;
+                        rec.w = (okc && ALLRED) ? w.holders : 0u;
+                        *reinterpret_cast<uint4*>(p.status + s * FTC_STATUS_WORDS) = rec;
+                    }
+                }
+                __syncwarp();
+            };
+            char* buf = bufs + (size_t)b * g.buf_bytes;
+            for (uint32_t i = 0; i < n; i += NS) {
+                const uint32_t si = i + gi;
+                const bool active = si < n;
+                const bool has_word = active && lg < p.W;
+                uint32_t pfw = __shfl_sync(kFullWarp, cur.pfw, has_word ? si * p.W + lg : 0u);
+                if (!has_word) pfw = 0;
+                else if (lg == p.W - 1 && (p.P & 31)) pfw &= (1u << (p.P & 31)) - 1u;
+                uint32_t ev = FTC_INOP_UNUSED, er = 0;
+                if (INOP) {
+                    const uint32_t src = (active && lg < p.max_inop) ? si * p.max_inop + lg : 0u;
+                    ev = __shfl_sync(kFullWarp, cur.vic, src); er = __shfl_sync(kFullWarp, cur.rnd, src);
+                    if (!active) ev = FTC_INOP_UNUSED;
+                }
+                const uint32_t rsrc = __shfl_sync(kFullWarp, cur.root, active ? si : 0u);
+                const uint32_t first_root = p.root >= 0 ? (uint32_t)p.root : rsrc;
+                WarpScen w; bool slow;
+                decode_group<L, (ALLRED ? 1 : 0), (INOP ? 1 : 0)>(p, pfw, ev, er, first_root, w, slow);
+                if (__any_sync(kFullWarp, active && slow)) {
+                    // rare: a scenario for the general routines (a block of one warp may call them). The scenarios of this
+                    // round are played one after the other, every group on the same scenario, the first group writing.
+                    for (uint32_t gg = 0; gg < NS && i + gg < n; ++gg) {
+                        const uint64_t s = grp * g.group + i + gg;
+                        decode_scenario(p, s, cx, pf, inc);
+                        if (cx->code == FTC_ST_OK && ALLRED) count_holders(p, cx, pf, unr);
+                        WarpScen w1;
+                        w1.code = cx->code; w1.sstar = cx->sstar; w1.attempts = cx->attempts; w1.root = cx->root; w1.base = cx->base;
+                        w1.npre = cx->npre; w1.nexcl = cx->nexcl; w1.inop_incl = cx->inop_incl; w1.holders = cx->holders; w1.G = cx->G;
+                        w1.any_victim = 1; w1.incw = 0; w1.iv = 0;
+                        __syncwarp();
+                        evaluate(w1, inc, buf + (size_t)(i + gg) * scen_bytes, gi == 0, s);
+                    }
+                } else {
+                    uint32_t* incp = ginc + gi * (p.W + 1);
+                    if (lg <= p.W) incp[lg] = w.incw;
+                    if (p.W == L && lg == 0) incp[L] = 0;
+                    if (!active) w.code = FTC_ST_BAD_ROOT;              // nothing to play: G = 0, nothing written
+                    __syncwarp();
+                    evaluate(w, incp, buf + (size_t)(active ? si : 0u) * scen_bytes, active, grp * g.group + si);
                 }
             }
-            if (lane == 0) {
-                uint4 rec;
-                const uint32_t code = dead ? (uint32_t)FTC_ST_INTERNAL_TIMEOUT : w.code;
-                rec.x = code | ((okc ? w.sstar : 0xFFu) << 8) | (w.attempts << 16);
-                rec.y = okc ? p.P - w.npre - w.nexcl : 0u;
-                rec.z = okc ? w.inop_incl : 0u;
-                rec.w = (okc && ALLRED) ? w.holders : 0u;
-                *reinterpret_cast<uint4*>(p.status + s * FTC_STATUS_WORDS) = rec;
-            }
-            __syncwarp();
         }
         cur = nx;
     }
@@ -193,6 +287,10 @@ static bool warp_geometry(Params& p, int smem_optin, uint32_t& XL, WarpGeom& g) 
     if (Hmax > lw + 3) return false;
     g.lw = Hmax - 1 < lw ? Hmax - 1 : lw;                      // a shallow heap uses fewer lane rows
     XL = Hmax - g.lw;
+    // Half a warp per scenario where the tile fits 16 lanes: two scenarios then share one instruction stream, and for
+    // scenarios of a KB or so that stream is what bounds them. (Fewer lane rows with deeper lane-local sub-heaps, to make
+    // 2 KB scenarios fit as well, measured slower: 1.4 instead of 2.2 TB/s.)
+    g.lanes = (p.W <= 16 && p.m <= 16 && p.max_inop <= 16 && (C << g.lw) <= 16 && XL <= 2) ? 16 : 32;
     p.C = C; p.cw_log2 = cwl; p.Lt = 0; p.below = 0; p.swz_mask = 0; p.row_shift = 0;
     uint32_t group = (uint32_t)(kWarpBufTarget / scen_bytes);
     if (group < 1) group = 1;
@@ -201,7 +299,7 @@ static bool warp_geometry(Params& p, int smem_optin, uint32_t& XL, WarpGeom& g) 
     g.group = group;
     // behind the last scenario: room for the bytes a full group would have beyond the short last group (read, not used)
     g.buf_bytes = (uint32_t)((group * scen_bytes + (uint64_t)p.m * p.kbytes + 127) & ~(uint64_t)127);
-    size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
+    size_t o = sizeof(Ctx) + (3 + 32 / g.lanes) * (size_t)(p.W + 1) * 4;      // the general routines' masks, then one arrival mask per group
     o = (o + 15) & ~(size_t)15; g.off_bar = (uint32_t)o; o += 16;
     o = (o + 127) & ~(size_t)127; g.off_buf = (uint32_t)o;
     o += 2 * (size_t)g.buf_bytes;
@@ -209,19 +307,27 @@ static bool warp_geometry(Params& p, int smem_optin, uint32_t& XL, WarpGeom& g) 
     return o <= (size_t)smem_optin - 1024;
 }
 
-template <typename T, int OP, int XL, int MODE>
-static cudaError_t launch_warp_m(const Params& p, const WarpGeom& g, int sm_count, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(warp_kernel<T, OP, XL, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
+template <typename T, int OP, int XL, int MODE, int L>
+static cudaError_t launch_warp_l(const Params& p, const WarpGeom& g, int sm_count, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(warp_kernel<T, OP, XL, MODE, L>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, warp_kernel<T, OP, XL, MODE>, 32, g.smem_bytes);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, warp_kernel<T, OP, XL, MODE, L>, 32, g.smem_bytes);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     const uint64_t ngroups = (p.S + g.group - 1) / g.group, cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(ngroups < cap ? ngroups : cap);
     if (p.grid_query) { *p.grid_query = grid; return cudaSuccess; }
-    warp_kernel<T, OP, XL, MODE><<<grid, 32, g.smem_bytes, st>>>(p, g);
+    warp_kernel<T, OP, XL, MODE, L><<<grid, 32, g.smem_bytes, st>>>(p, g);
     return cudaGetLastError();
+}
+
+template <typename T, int OP, int XL, int MODE>
+static cudaError_t launch_warp_m(const Params& p, const WarpGeom& g, int sm_count, cudaStream_t st) {
+    if constexpr (XL <= 2) {
+        if (g.lanes == 16) return launch_warp_l<T, OP, XL, MODE, 16>(p, g, sm_count, st);
+    }
+    return launch_warp_l<T, OP, XL, MODE, 32>(p, g, sm_count, st);
 }
 
 template <typename T, int OP, int XL>
