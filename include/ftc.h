@@ -317,15 +317,17 @@ FTC_API int ftc_read_bandwidth_probe(uint32_t mode, const void* d_buf, uint64_t 
 /* Name of the kernel family the batch calls would use for this descriptor: "staged", "tiled" or "generic". */
 FTC_API const char* ftc_kernel_name(const ftc_desc_t* desc, int is_allreduce);
 
-/* The same, down to the instantiation of the shared-memory kernel: "staged/whole" (scenario staged by one copy),
+/* The same, down to the instantiation of the shared-memory kernel: "staged/warp" (scenarios of a few KB: one warp per
+ * scenario), "staged/warp-pair" (two scenarios per warp, half a warp each), "staged/whole" (scenario staged by one copy),
  * "staged/lean" (blocks of one or two warps), "staged/large" (4-8 warps), "staged/batched-lean" (4-8 warps, groups of at
  * most 128 bytes, exact operations), "staged/lean-swz" and "staged/batched-swz" (float32 vectors of 16 or 32 bytes, tiles
  * by swizzled tensor copies), "staged/whole-large", "tiled", "generic"; assuming the workspace ftc_workspace_bytes() asks for. */
 FTC_API const char* ftc_kernel_variant(const ftc_desc_t* desc, int is_allreduce);
 
 /* Thread blocks the batch calls would launch for S scenarios on the current device (given the workspace
- * ftc_workspace_bytes() asks for). Block b plays scenarios b, b + blocks, b + 2*blocks, ... one after the other; a batch
- * keeps the whole GPU busy when S is a few times this number. Needs a device. Launches nothing. */
+ * ftc_workspace_bytes() asks for). Block b plays scenarios b, b + blocks, b + 2*blocks, ... one after the other (the warp
+ * kernel for scenarios of a few KB hands out short runs of consecutive scenarios the same way); a batch keeps the whole
+ * GPU busy when S is a few times this number. Needs a device. Launches nothing. */
 FTC_API int ftc_launch_blocks(const ftc_desc_t* desc, uint64_t S, int is_allreduce, uint32_t* blocks);
 
 FTC_API const char* ftc_strerror(int code);

@@ -36,6 +36,7 @@ const char* staged_variant(Params p, int tsel, int smem_optin_bytes, int sm_coun
 // Warp kernel (scenarios of a few KB, one warp per scenario): shape check and launch. The staged launcher and the
 // variant query route to it when the shape fits.
 bool warp_supported(Params p, int smem_optin_bytes);
+uint32_t warp_lanes_per_scenario(Params p, int smem_optin_bytes);      // 32, or 16 when two scenarios share a warp; 0: not this kernel
 cudaError_t launch_warp(const Params& p, int tsel, int sm_count, int smem_optin_bytes, cudaStream_t st);
 
 // Every root child's delivery (value, flag, failed-list size): general kernel, workspace slices of candidates_slice_bytes().

@@ -27,7 +27,7 @@ size_t staged_workspace_bytes(Params p, int smem_optin_bytes, int sm_count) {
 
 const char* staged_variant(Params p, int tsel, int smem_optin_bytes, int sm_count, uint32_t* grid_cap_blocks_per_sm) {
     if (grid_cap_blocks_per_sm) *grid_cap_blocks_per_sm = 0;
-    if (warp_supported(p, smem_optin_bytes)) return "staged/warp";
+    if (warp_supported(p, smem_optin_bytes)) return warp_lanes_per_scenario(p, smem_optin_bytes) == 16 ? "staged/warp-pair" : "staged/warp";
     StagedGeom g;
     const StagedVariant v = staged_plan(p, tsel == TS_F32_SUM, true, staged_xl(p), smem_optin_bytes, sm_count, g);
     if (grid_cap_blocks_per_sm) *grid_cap_blocks_per_sm = g.hv_global ? (uint32_t)kHvGlobalBlocksPerSm : 0u;

@@ -11,6 +11,11 @@ bool warp_supported(Params p, int smem_optin_bytes) {
     return warp_geometry(p, smem_optin_bytes, XL, g);
 }
 
+uint32_t warp_lanes_per_scenario(Params p, int smem_optin_bytes) {
+    WarpGeom g; uint32_t XL;
+    return warp_geometry(p, smem_optin_bytes, XL, g) ? g.lanes : 0u;
+}
+
 cudaError_t launch_warp(const Params& p, int tsel, int sm_count, int smem_optin, cudaStream_t st) {
     switch (tsel) {
     case TS_U32_SUM: return launch_warp_t<uint32_t, OP_SUM>(p, sm_count, smem_optin, st);

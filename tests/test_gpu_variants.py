@@ -73,7 +73,10 @@ CASES = [
     ("staged/whole", 700, 6, 4, "i32", "xor", False),                 # 11 KB, a heap too deep for one warp tile
     ("staged/warp", 64, 2, 8, "i64", "sum", False),                   # the P=64 configuration's shape
     ("staged/warp", 150, 3, 4, "f32", "sum", True),                   # short last group, 16-byte vectors
-    ("staged/warp", 64, 3, 4, "i32", "max", True),                    # a heap shallower than the warp tile
+    ("staged/warp-pair", 64, 3, 4, "i32", "max", True),               # a heap shallower than the warp tile: two scenarios per warp
+    ("staged/warp-pair", 30, 1, 4, "f32", "sum", False),              # eight lanes would do
+    ("staged/warp-pair", 120, 7, 4, "u64", "xor", True),              # groups of eight, 32-byte vectors
+    ("staged/warp-pair", 17, 0, 4, "i32", "sum", True),               # no tolerance: every failure goes to the general routines
     ("staged/warp", 500, 1, 4, "i32", "xor", False),                  # 8 KB, lane-local sub-heaps of three levels
     ("staged/warp", 40, 4, 32, "i32", "max", True),                   # 128-byte vectors
     ("staged/warp", 12, 0, 64, "f32", "sum", False),                  # no tolerance: groups of one, 256-byte vectors
@@ -105,7 +108,7 @@ def test_every_variant_with_several_scenarios_per_block(variant, P, f, k, dname,
     assert (codes == 0).sum() > S // 2 and (codes != 0).any()         # most scenarios succeed, some do not
 
 
-DESC_CASES = [c for c in CASES if c[4] == "f32"] + [("staged/large", 4096, 4, 32, "i32", "max", True), ("staged/warp", 64, 2, 8, "i64", "sum", False),
+DESC_CASES = [c for c in CASES if c[4] == "f32"] + [("staged/warp-pair", 64, 3, 4, "f32", "sum", True), ("staged/large", 4096, 4, 32, "i32", "max", True), ("staged/warp", 64, 2, 8, "i64", "sum", False),
                                                     ("tiled", 1024, 3, 16, "f32", "sum", True), ("tiled", 300, 2, 8, "f32", "sum", False)]
 
 
@@ -156,7 +159,8 @@ def test_seeded_random_shapes(P, f, k, dname, op, allreduce):
 # ---------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("P,f,k,dname,op,allreduce", [(1024, 3, 16, "f32", "sum", True), (4096, 4, 32, "i32", "max", True),
                                                       (16384, 3, 8, "f32", "sum", False), (16384, 1, 8, "i32", "sum", True),
-                                                      (64, 2, 8, "i64", "sum", False), (150, 3, 16, "f32", "sum", True)])
+                                                      (64, 2, 8, "i64", "sum", False), (150, 3, 16, "f32", "sum", True),
+                                                      (64, 3, 4, "i32", "max", True)])
 def test_a_wait_that_gives_up_poisons_its_block_and_nothing_else(P, f, k, dname, op, allreduce):
     """With FTC_DEBUG_ONE_POLL the waits for the asynchronous copies look once and give up. Then: a scenario is either
     played correctly (bit-equal to the oracle) or reports FTC_ST_INTERNAL_TIMEOUT with zero bytes; once a block has
@@ -176,9 +180,10 @@ def test_a_wait_that_gives_up_poisons_its_block_and_nothing_else(P, f, k, dname,
     assert not ob[timed_out].any() and not st[timed_out, 1:].any()
     assert ((st[timed_out, 0] >> 8) & 0xFF == 0xFF).all()
     assert np.array_equal(st[~timed_out], want[1][~timed_out]) and np.array_equal(ob[~timed_out], wb[~timed_out])
-    for b in range(blocks):                                           # sticky per block
-        seq = timed_out[b::blocks]
-        assert np.array_equal(seq, np.sort(seq)), (b, seq)
-    if variant not in ("staged/whole", "staged/warp"):               # tile copies are waited for right after their issue
+    if not variant.startswith("staged/warp"):                         # sticky per block (the warp kernel hands its blocks runs of
+        for b in range(blocks):                                       # consecutive scenarios, whose length the test does not know)
+            seq = timed_out[b::blocks]
+            assert np.array_equal(seq, np.sort(seq)), (b, seq)
+    if variant not in ("staged/whole", "staged/warp", "staged/warp-pair"):   # tile copies are waited for right after their issue
         assert timed_out.any()
     assert_same(run_gpu(None, f, op, pf, inop, roots, 0, allreduce, 0, d_x=d_x), want, f"normal call after the give-up run, {variant}")
