@@ -24,144 +24,18 @@ constexpr uint32_t kFullWarp = 0xFFFFFFFFu;
 // reciprocal times x stays below one unit of the quotient's last place)
 __device__ __forceinline__ uint32_t div_m(const Params& p, uint32_t x) { return p.m == 1 ? x : __umulhi(x, p.m_magic); }
 
-// Failure round (global clock) of process `proc`, which may differ from lane to lane. pfw: this lane's word of
-// the pre-operation mask; iv / ir: this lane's in-operation slot (victim or FTC_INOP_UNUSED, merged round).
-__device__ __forceinline__ uint32_t fail_round_lanes(uint32_t pfw, uint32_t iv, uint32_t ir, uint32_t max_inop, uint32_t proc) {
-    const uint32_t word = __shfl_sync(kFullWarp, pfw, proc >> 5);
-    uint32_t fr = ((word >> (proc & 31)) & 1u) ? 0u : kNever;
-    for (uint32_t j = 0; j < max_inop; ++j) {                          // same trip count in every lane
-        const uint32_t vj = __shfl_sync(kFullWarp, iv, j), rj = __shfl_sync(kFullWarp, ir, j);
-        if (fr == kNever && vj == proc) fr = rj;
-    }
-    return fr;
-}
-
-// pfw: word `lane` of the scenario's pre-operation mask, bits >= P cleared, 0 for lanes >= W.
-// ev / er: in-operation slot `lane` as the caller passed it (lanes >= max_inop: anything).
-// Returns false when the scenario is left to the general routines: a root out of range, or more failed processes
-// (before and during the operation) than the f the schedule tolerates. All lanes call; all get the same answer.
-// ALLRED_ / INOP_: 0 or 1 = compile-time copies of p.is_allreduce != 0 and p.max_inop != 0 (code that cannot run is
-// left out); 2 = look at p when running.
-template <int ALLRED_, int INOP_>
-__device__ __forceinline__ bool decode_warp(const Params& p, uint32_t pfw, uint32_t ev, uint32_t er, uint32_t first_root, WarpScen& o) {
-    const bool ALLRED = ALLRED_ == 2 ? p.is_allreduce != 0 : ALLRED_ != 0;
-    const bool INOP = INOP_ == 2 ? p.max_inop != 0 : INOP_ != 0;
-    const uint32_t lane = threadIdx.x & 31;
-    if (first_root >= p.P) return false;
-    const uint32_t npre = __reduce_add_sync(kFullWarp, __popc(pfw));
-
-    // in-operation slots: a victim out of range or failed before the operation does not count; slots naming the
-    // same victim merge into the earliest round; the first of them stands for the victim
-    uint32_t v = (INOP && lane < p.max_inop && ev < p.P) ? ev : FTC_INOP_UNUSED;
-    uint32_t rmin = (INOP && lane < p.max_inop) ? er : 0u;
-    uint32_t ifirst = 0;
-    o.any_victim = 0;
-    if (INOP) {
-        const uint32_t word = __shfl_sync(kFullWarp, pfw, v == FTC_INOP_UNUSED ? 0u : v >> 5);
-        const bool pre = v != FTC_INOP_UNUSED && ((word >> (v & 31)) & 1u);
-        bool first = true;
-        const uint32_t r0 = rmin;
-        for (uint32_t j = 0; j < p.max_inop; ++j) {
-            const uint32_t vj = __shfl_sync(kFullWarp, v, j), rj = __shfl_sync(kFullWarp, r0, j);
-            if (vj == v) { rmin = min(rmin, rj); if (j < lane) first = false; }
-        }
-        if (pre) v = FTC_INOP_UNUSED;
-        o.any_victim = __ballot_sync(kFullWarp, v != FTC_INOP_UNUSED);
-        ifirst = __ballot_sync(kFullWarp, v != FTC_INOP_UNUSED && first);
-    }
-    if (npre + __popc(ifirst) > p.f) return false;
-    const uint32_t iv = v, ir = rmin;
-
-    // the root of the attempt that counts (Algorithm "Allreduce": the first candidate that had not failed beforehand)
-    uint32_t code = FTC_ST_OK, root = first_root, base = 0, attempts = 1;
-    if (!ALLRED) {
-        // the root must be alive when the last tree messages arrive (round f+H-1)
-        if (fail_round_lanes(pfw, iv, ir, INOP ? p.max_inop : 0u, first_root) < p.Rred) code = FTC_ST_ROOT_FAILED;
-    } else {
-        uint32_t c = first_root + (lane < p.m ? lane : 0u);
-        if (c >= p.P) c -= p.P;
-        const uint32_t fr = fail_round_lanes(pfw, iv, ir, INOP ? p.max_inop : 0u, c);
-        const uint32_t inopc = __ballot_sync(kFullWarp, lane < p.m && fr != 0 && fr != kNever);
-        const uint32_t alive = __ballot_sync(kFullWarp, lane < p.m && fr != 0);
-        if (inopc) { code = FTC_ST_PRECONDITION_INOP_ROOT; attempts = 0; }
-        else if (!alive) { code = FTC_ST_NO_LIVE_ROOT_CANDIDATE; attempts = p.m; }
-        else {
-            const uint32_t a = __ffs(alive) - 1;
-            root = first_root + a; if (root >= p.P) root -= p.P;
-            base = a * p.Ratt; attempts = a + 1;
-        }
-    }
-    o.code = code; o.root = root; o.base = base; o.attempts = attempts; o.npre = npre;
-    o.sstar = 0xFF; o.nexcl = 0; o.inop_incl = 0; o.holders = 0; o.G = 0; o.incw = 0; o.iv = iv;
-    if (code != FTC_ST_OK) return true;
-
-    // failed bits of the root's children: a subtree is unclean iff one of its processes does not send up the tree
-    uint32_t F = 0;
-    for (uint32_t word = pfw; word; word &= word - 1) {
-        const uint32_t vr = renumber((lane << 5) + (__ffs(word) - 1), root);
-        if (vr) F |= 1u << ((vr - 1) - div_m(p, vr - 1) * p.m);
-    }
-    const uint32_t vren = (INOP && iv != FTC_INOP_UNUSED) ? renumber(iv, root) : 0u;
-    const uint32_t t = INOP ? local_round(ir, base) : kNever;
-    uint32_t j = 0, sv = 0;
-    if (INOP && vren) {
-        j = div_m(p, vren - 1); sv = (vren - 1) - j * p.m;
-        const uint32_t d = 1 + ilog2u(j + 1);
-        if (!(p.f + p.H - d < t)) F |= 1u << sv;                        // tree send of depth d is round f+H-d
-    }
-    F = __reduce_or_sync(kFullWarp, F);
-    const uint32_t all = p.m >= 32 ? 0xFFFFFFFFu : ((1u << p.m) - 1u);
-    const uint32_t clean = ~F & all;
-    if (!clean) return false;                                          // cannot happen with at most f failures
-    const uint32_t sstar = __ffs(clean) - 1;
-    o.sstar = sstar; o.G = p.q + (sstar < p.r ? 1u : 0u);
-
-    // arrival mask over renumbered ranks: everybody who had not failed before the operation; bit 0 is the root
-    // (alive), bit `root` is process 0
-    const uint32_t W = p.W;
-    uint32_t incw = 0;
-    if (lane < W) {
-        incw = ~pfw;
-        if (lane == W - 1 && (p.P & 31)) incw &= (1u << (p.P & 31)) - 1u;
-    }
-    if (root != 0) {
-        const uint32_t b0 = __shfl_sync(kFullWarp, incw, 0) & 1u;
-        if (lane == 0) incw |= 1u;
-        if (lane == (root >> 5)) incw = b0 ? (incw | (1u << (root & 31))) : (incw & ~(1u << (root & 31)));
-    }
-    // an in-operation victim is included iff its up-correction message to the selected subtree's member of its group
-    // (or to the root, when the group has no member there) was still sent
-    bool included = true;
-    if (INOP && vren) {
-        const bool member_in_subtree = j < p.q || sstar < p.r;
-        if (member_in_subtree) { if (sv != sstar) included = partner_slot(p, j, sv, sstar) < t; }
-        else included = t > root_slot(p);
-    }
-    if (INOP) {
-        o.inop_incl = __ballot_sync(kFullWarp, iv != FTC_INOP_UNUSED && included);
-        const uint32_t excl = __ballot_sync(kFullWarp, iv != FTC_INOP_UNUSED && !included);
-        o.nexcl = __popc(excl & ifirst);
-        for (uint32_t e = excl; e; e &= e - 1) {                        // the same in every lane
-            const uint32_t vj = __shfl_sync(kFullWarp, vren, __ffs(e) - 1);
-            if (lane == (vj >> 5)) incw &= ~(1u << (vj & 31));
-        }
-    }
-    o.incw = incw;
-    // broadcast: with at most f failures a failure-free subtree carries the value to every group, so everybody
-    // alive at the end of the attempt holds it
-    if (ALLRED) {
-        const uint32_t dead_end = INOP ? (__ballot_sync(kFullWarp, iv != FTC_INOP_UNUSED && t < p.Ratt) & ifirst) : 0u;
-        o.holders = p.P - npre - __popc(dead_end);
-    }
-    return true;
-}
-
-// ---- the same decode for several scenarios at once: the warp is cut into groups of L lanes (L = 32, 16 or 8), every
-// group decodes its own scenario (W <= L mask words, max_inop <= L, f+1 <= L). All 32 lanes execute every ballot and
+// The warp is cut into groups of L lanes (L = 32: the whole warp; 16 or 8: several scenarios at once), every group
+// decodes its own scenario (W <= L mask words, max_inop <= L, f+1 <= L). All 32 lanes execute every ballot and
 // shuffle, so nothing here returns early or loops a group-dependent number of times; ballots are cut to the group's
 // lanes, shuffles and reductions stay inside the group. Facts that are "the same in every lane" of WarpScen are the
-// same in every lane of a group. `slow` is set where the scenario is left to the general routines (its other outputs
-// are then meaningless but harmless: G = 0 makes every fold read row 0 only).
+// same in every lane of a group.
+// pfw: word `lane within the group` of the scenario's pre-operation mask, bits >= P cleared, 0 beyond the mask.
+// ev / er: in-operation slot `lane within the group` as the caller passed it (beyond max_inop: anything).
+// `slow` is set where the scenario is left to the general routines: a root out of range, or more failed processes
+// (before and during the operation) than the f the schedule tolerates; the other outputs are then meaningless but
+// harmless (G = 0 makes every fold read row 0 only).
+// ALLRED_ / INOP_: 0 or 1 = compile-time copies of p.is_allreduce != 0 and p.max_inop != 0 (code that cannot run is
+// left out); 2 = look at p when running.
 template <int L> struct LaneGroup {
     static constexpr uint32_t kLanes = L == 32 ? 0xFFFFFFFFu : ((1u << L) - 1u);
     uint32_t lg, base, mask;                                       // lane within the group, the group's first lane and lanes

@@ -487,8 +487,9 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
             if (lane == p.W - 1 && (p.P & 31)) pfw &= (1u << (p.P & 31)) - 1u;
             const uint32_t ev = nx_vic, er = nx_rnd, first_root = p.root >= 0 ? (uint32_t)p.root : nx_root;
             fetch_small(s + gridDim.x);
-            WarpScen w;
-            if (decode_warp<2, 2>(p, pfw, ev, er, first_root, w)) {
+            WarpScen w; bool slow;
+            decode_group<32, 2, 2>(p, pfw, ev, er, first_root, w, slow);
+            if (!slow) {
                 if (lane == 0) {
                     cx->code = w.code; cx->sstar = w.sstar; cx->attempts = w.attempts; cx->root = w.root; cx->base = w.base;
                     cx->npre = w.npre; cx->nexcl = w.nexcl; cx->inop_incl = w.inop_incl; cx->holders = w.holders; cx->G = w.G;

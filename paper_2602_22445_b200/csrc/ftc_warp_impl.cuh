@@ -120,8 +120,9 @@ __global__ void __launch_bounds__(32, WarpMinBlocks<XL, L>::value) warp_kernel(P
                     ev = __shfl_sync(kFullWarp, cur.vic, src); er = __shfl_sync(kFullWarp, cur.rnd, src);
                 }
                 const uint32_t first_root = p.root >= 0 ? (uint32_t)p.root : __shfl_sync(kFullWarp, cur.root, i);
-                WarpScen w;
-                if (decode_warp<(ALLRED ? 1 : 0), (INOP ? 1 : 0)>(p, pfw, ev, er, first_root, w)) {
+                WarpScen w; bool slow;
+                decode_group<32, (ALLRED ? 1 : 0), (INOP ? 1 : 0)>(p, pfw, ev, er, first_root, w, slow);
+                if (!slow) {
                     if (lane <= p.W) inc[lane] = w.incw;
                     if (p.W == 32 && lane == 0) inc[32] = 0;
                     __syncwarp();
