@@ -218,10 +218,11 @@ FTC_API int ftc_reduce_batch_noalloc(const ftc_desc_t* desc, uint64_t S, const v
  *   workspace of at least ftc_candidates_workspace_bytes(desc, S) bytes, 256-byte aligned
  * Other arguments as for ftc_reduce_batch. Scenarios whose root is invalid or violates the allreduce precondition
  * play no attempt: zeros and "nothing delivered".
- * Two kernels (ftc_candidates_kernel_name): "staged" for the exactly associative operations (integer sum, max, xor) on
- * binary heaps with vectors of 16..512 bytes (a power-of-two number of 16-byte chunks) and scenarios above 12 KB -- one pass
- * over the inputs on the tiles of the shared-memory kernel, a group without a failed member being folded once for all
- * children; "generic" (any k, float32, other subtree shapes, FTC_KERNEL_GENERIC) plays child after child.
+ * Two kernels (ftc_candidates_kernel_name): "staged" on binary heaps with vectors of 16..512 bytes (a power-of-two number of
+ * 16-byte chunks) and scenarios above 12 KB -- one pass over the inputs on the tiles of the shared-memory kernel; for the
+ * exactly associative operations (integer sum, max, xor) a group without a failed member is folded once for all children,
+ * for float32 every child's member folds in its own order from the staged copy; "generic" (any k, other subtree shapes,
+ * FTC_KERNEL_GENERIC) plays child after child.
  */
 FTC_API int ftc_candidates_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const void* d_in,
                                  const uint32_t* d_prefail, const ftc_inop_t* d_inop, const uint32_t* d_roots,

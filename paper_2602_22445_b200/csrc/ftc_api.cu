@@ -257,7 +257,7 @@ int ftc_candidates_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, c
     p.in = d_in; p.prefail = d_prefail; p.inop = d_inop; p.roots = d_roots; p.ws = d_workspace;
     if (cand_fast_supported(p, tsel, di.smem_optin, di.sm_count)) {
         const size_t need = cand_fast_workspace_bytes(p, tsel, di.smem_optin, di.sm_count);
-        if (!d_workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return FTC_EWORKSPACE;
+        if (need && (!d_workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(d_workspace) & 255u))) return FTC_EWORKSPACE;
         return launch_cand_fast(p, tsel, d_cand, d_cand_info, di.sm_count, di.smem_optin, static_cast<cudaStream_t>(cuda_stream), nullptr)
                    == cudaSuccess ? FTC_OK : FTC_ECUDA;
     }

@@ -62,13 +62,15 @@ __device__ __noinline__ uint4 cand_fold(const Params& p, CandScen cs, const char
         if (!(partner_slot(p, row, sv, sc) < t)) mask &= ~(1u << sv);
     }
     uint4 acc = member(sc, v);
-    // the root's up-correction send to member sc of its group is its send number sc (descending order: r-1-sc)
+    // the root's up-correction send to member sc of its group is its send number sc (descending order: r-1-sc); in the
+    // fold the root comes first among the partners (descending order: last)
     const bool from_root = row == p.q && (p.pdesc ? p.r - 1 - sc : sc) < cs.troot;
-    if (from_root) acc = comb16<T, OP>(acc, ld_stream(in_lc + (size_t)cs.root * p.kbytes));
-    for (uint32_t sp = 0; sp < mj; ++sp) {
-        const uint32_t vr = vbase + sp;
+    if (from_root && !p.pdesc) acc = comb16<T, OP>(acc, ld_stream(in_lc + (size_t)cs.root * p.kbytes));
+    for (uint32_t i = 0; i < mj; ++i) {
+        const uint32_t sp = p.pdesc ? mj - 1 - i : i, vr = vbase + sp;
         if (sp != sc && ((mask >> sp) & 1u)) acc = comb16<T, OP>(acc, member(sp, vr));
     }
+    if (from_root && p.pdesc) acc = comb16<T, OP>(acc, ld_stream(in_lc + (size_t)cs.root * p.kbytes));
     meta = kMetaExists | kMetaPresent | (mj - __popc(mask) + ((row == p.q && !from_root) ? 1u : 0u));
     return acc;
 }
@@ -242,10 +244,14 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
     uint32_t* trowv = rspec + ((cg.ntop + 31) / 32 + 1);                        // per tile: its one special row, kNoRow or kManyRows
     uint4* hvc = reinterpret_cast<uint4*>(sbase + g.off_hv);                     // common values, heap order
     volatile uint32_t* gaveup = reinterpret_cast<volatile uint32_t*>(sbase + g.off_gaveup);
+    // ORD: the combine order is observable (float32): every member of a group folds in its own order, nothing is common
+    // to the children; every node carries a value and a word per child, all in shared memory.
+    constexpr bool ORD = Ordered<T>::value;
     // per block: values hv[sc][row][chunk], combined words hm[sc][row], own words of the rows above the tiles hmo[sc][row]
-    char* slice = static_cast<char*>(p.ws) + (size_t)blockIdx.x * cg.slice_bytes;
+    // (a slice of the workspace, touched at the dirty nodes only; ORD: shared memory, every node)
+    char* slice = ORD ? sbase + g.off_hv : static_cast<char*>(p.ws) + (size_t)blockIdx.x * cg.slice_bytes;
     uint4* hv = reinterpret_cast<uint4*>(slice);
-    uint32_t* hm = reinterpret_cast<uint32_t*>(slice + (size_t)p.m * cg.nheap * p.C * 16);
+    uint32_t* hm = ORD ? reinterpret_cast<uint32_t*>(sbase + g.off_words) : reinterpret_cast<uint32_t*>(slice + (size_t)p.m * cg.nheap * p.C * 16);
     uint32_t* hmo = hm + (size_t)p.m * cg.nheap;
 
     const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
@@ -410,7 +416,28 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
                 const uint32_t tA = RW - 1 + lr, rowA = ((j0 + 1) << lw) - 1 + lr;
                 const uint32_t tB = ilog2u(lr + 1), idxB = lr + 1 - (1u << tB);
                 const uint32_t rowB = ((j0 + 1) << tB) - 1 + idxB;
-                if (!special) {
+                if (ORD) {
+                    if (!special) {
+                        // every group whole: child sc's member folds its own input first, then the partners in the schedule's order
+                        for (uint32_t sc = 0; sc < p.m; ++sc) {
+                            uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
+                            if (j0 < Gc) {
+                                if (XL > 1 || rowA < Gc) valA = SubHeapPlain<T, OP, XL, 0, false, false>::eval(p, sc, alive, buf_lc, rowbytes, tA, rowA, Gc);
+                                const bool hasB = lr < RW - 1;
+                                if (hasB) valB = fold_plain_staged<T, OP>(p, sc, buf_lc + staged_row_offset<false>(p, rowbytes, lr, rowB));
+                                valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, Gc);
+                            }
+                            if (lr == 0) {
+                                hv[((size_t)sc * cg.nheap + j0) * p.C + lc] = lw ? valB : valA;
+                                if (lc == 0) hm[(size_t)sc * cg.nheap + j0] = j0 < Gc ? (kMetaExists | kMetaPresent) : 0u;
+                            }
+                        }
+                    } else {
+                        const TileJob job{cs, in_s, tile, hv, hm, nullptr, cg.nheap, j0, kManyRows, Lt, D, Gc, rowbytes};
+                        cand_tile_many<T, OP, XL>(p, job);
+                    }
+                    release();
+                } else if (!special) {
                     // every group of the tile is whole: one value per row serves all children (exact operations)
                     if (j0 < Gc) {
                         uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
@@ -428,6 +455,23 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
                     else cand_tile_one<T, OP>(p, job);
                     release();
                 }
+            } else if (ORD) {
+                // ---- rows above the tiles, every child's member in its own order ----
+                for (uint32_t gs = 0; gs < GR; ++gs) {
+                    const uint32_t rloc = gs * RW + lr, row = (it - ntiles) * grows + rloc;
+                    if (row >= ntop) continue;
+                    const bool plain = !special || (row < Gc && !test_bit(rspec, row));
+                    for (uint32_t sc = 0; sc < p.m; ++sc) {
+                        const uint32_t G = p.q + (sc < p.r ? 1u : 0u);
+                        uint32_t mo = 0;
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (plain) { v = fold_plain_staged<T, OP>(p, sc, buf_lc + (size_t)rloc * rowbytes); mo = kMetaExists | kMetaPresent; }
+                        else if (row < G) v = cand_fold<T, OP>(p, cs, in_lc, buf_lc + (size_t)rloc * rowbytes, row, sc, mo);
+                        hv[((size_t)sc * cg.nheap + row) * p.C + lc] = v;
+                        if (lc == 0) hmo[(size_t)sc * cg.ntop + row] = mo;
+                    }
+                }
+                release();
             } else {
                 // ---- rows above the tiles: fold now, combine later ----
                 if (!special) {
@@ -458,7 +502,24 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
         }
         __syncthreads();
         // ---- levels above the tiles, leaves first (Algorithm "reduce_non_root") ----
-        for (int lvl = (int)Lt - 1; lvl >= 0; --lvl) {
+        for (int lvl = ORD ? (int)Lt - 1 : -1; lvl >= 0; --lvl) {              // ORD: every node, per child
+            const uint32_t lo = (1u << lvl) - 1u, n = lo + 1u;
+            for (uint32_t u = tid; u < n * p.m * p.C; u += nt) {
+                const uint32_t c = u & Cmask, x = u >> cwl, sc = x % p.m, row = lo + x / p.m;
+                const size_t me = (size_t)sc * cg.nheap + row;
+                uint32_t meta = hmo[(size_t)sc * cg.ntop + row];
+                uint4 v = hv[me * p.C + c];
+                if (meta & kMetaPresent) {
+                    const size_t c1 = (size_t)sc * cg.nheap + 2 * row + 1;
+                    take_child<T, OP>(v, meta, hv[c1 * p.C + c], hm[c1]);
+                    take_child<T, OP>(v, meta, hv[(c1 + 1) * p.C + c], hm[c1 + 1]);
+                    hv[me * p.C + c] = v;
+                }
+                if (c == 0) hm[me] = meta;
+            }
+            __syncthreads();
+        }
+        for (int lvl = ORD ? -1 : (int)Lt - 1; lvl >= 0; --lvl) {
             const uint32_t lo = (1u << lvl) - 1u, n = lo + 1u;
             // nodes played per child: own value (a special row's per-child fold, else the row's common fold), then each
             // child's delivery (per child if that node is played per child, else its common value)
@@ -496,7 +557,7 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
         }
         // ---- what the root receives from each child ----
         const bool bad = *gaveup != 0;
-        const bool per_child = test_bit(dirty, 0u);                // else: nothing failed anywhere, every child delivers the common value
+        const bool per_child = ORD || test_bit(dirty, 0u);         // else: nothing failed anywhere, every child delivers the common value
         for (uint32_t u = tid; u < p.m * p.C; u += nt) {
             const uint32_t sc = u >> cwl, c = u & Cmask;
             const uint32_t meta = per_child ? hm[(size_t)sc * cg.nheap] : (kMetaExists | kMetaPresent);
@@ -515,14 +576,14 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
 }
 
 // ---- host side ----
-static bool cand_geometry(Params& p, int smem_optin, int sm_count, uint32_t& XL, CandGeom& cg) {
+static bool cand_geometry(Params& p, int smem_optin, int sm_count, uint32_t& XL, CandGeom& cg, bool ordered) {
     if (p.arity != 2) return false;
     XL = staged_xl(p);
     p.ws_bytes = 0; p.swz_mask = 0; p.row_shift = 0;               // its own slices; plain tiles
-    if (!staged_geometry(p, smem_optin, sm_count, XL, cg.st, /*all_children=*/true)) return false;
+    if (!staged_geometry(p, smem_optin, sm_count, XL, cg.st, /*all_children=*/ordered ? 2 : 1)) return false;
     if (cg.st.whole || cg.st.nbuf != 1) return false;
     cg.nheap = (2u << p.Lt) - 1; cg.ntop = (1u << p.Lt) - 1;
-    cg.slice_bytes = (((uint64_t)p.m * cg.nheap * p.C * 16 + (uint64_t)p.m * (cg.nheap + cg.ntop) * 4) + 255) & ~(uint64_t)255;
+    cg.slice_bytes = ordered ? 0 : (((uint64_t)p.m * cg.nheap * p.C * 16 + (uint64_t)p.m * (cg.nheap + cg.ntop) * 4) + 255) & ~(uint64_t)255;
     return true;
 }
 
@@ -534,7 +595,7 @@ static cudaError_t launch_cand_x(const Params& p, const CandGeom& cg, T* cand, u
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, cand_kernel<T, OP, XL>, (int)cg.st.nwarps * 32, cg.st.smem_bytes);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
-    if (per_sm > 4) per_sm = 4;
+    if (cg.slice_bytes && per_sm > 4) per_sm = 4;                 // workspace slices of all blocks stay in L2
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
     if (grid_out) { *grid_out = (uint32_t)cap; return cudaSuccess; }      // one workspace slice per block
@@ -545,7 +606,7 @@ static cudaError_t launch_cand_x(const Params& p, const CandGeom& cg, T* cand, u
 template <typename T, int OP>
 static cudaError_t launch_cand_t(Params p, void* cand, uint32_t* info, int sm_count, int smem_optin, cudaStream_t st, uint32_t* grid_out) {
     CandGeom cg; uint32_t XL;
-    if (!cand_geometry(p, smem_optin, sm_count, XL, cg)) return cudaErrorInvalidConfiguration;
+    if (!cand_geometry(p, smem_optin, sm_count, XL, cg, Ordered<T>::value)) return cudaErrorInvalidConfiguration;
     switch (XL) {
     case 2: return launch_cand_x<T, OP, 2>(p, cg, static_cast<T*>(cand), info, sm_count, st, grid_out);
     case 3: return launch_cand_x<T, OP, 3>(p, cg, static_cast<T*>(cand), info, sm_count, st, grid_out);

@@ -73,6 +73,7 @@ struct StagedGeom {
     uint32_t whole;                        // 1: the whole scenario is staged in one block-wide buffer
     uint32_t off_special, off_rootv, off_hv, off_bar, off_gaveup, off_tiles, smem_bytes;
     uint32_t off_dirty;                    // all-children kernel: bitmaps over the rows of the heap array, then one word per tile
+    uint32_t off_words;                    // all-children kernel, observable order: a word per node and child
     uint32_t hv_global;                    // 1: the heap array of tile roots and upper rows lives in the workspace
     uint64_t hv_bytes;                     // its size per block
 };
@@ -643,7 +644,9 @@ constexpr int kHvGlobalBlocksPerSm = 4;
 
 // all_children: geometry for the kernel that plays every root child (ftc_cand_impl.cuh): every heap level is tiled and
 // the heap arrays live in the workspace, never in shared memory.
-static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL, StagedGeom& g, bool all_children = false) {
+// all_children == 2: its variant for an observable combine order (float32): one heap array per root child, all in
+// shared memory, with their words.
+static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL, StagedGeom& g, int all_children = 0) {
     if (p.kbytes % 16) return false;
     const uint32_t C = p.kbytes / 16;
     if (C == 0 || C > 32 || (C & (C - 1))) return false;
@@ -685,9 +688,12 @@ static bool staged_geometry(Params& p, int smem_optin, int sm_count, uint32_t XL
     g.hv_bytes = (((uint64_t)2 << p.Lt) - 1) * C * 16;
     g.hv_global = (!g.whole && g.hv_bytes >= kHvGlobalMinBytes && g.hv_bytes <= kHvGlobalMaxBytes &&
                    p.ws_bytes / ((uint64_t)sm_count * kHvGlobalBlocksPerSm) >= g.hv_bytes) ? 1u : 0u;
-    g.off_hv = (uint32_t)o; if (!g.hv_global) o += (size_t)g.hv_bytes;
+    if (all_children == 2 && (g.hv_global || g.hv_bytes * p.m > 64 * 1024)) return false;
+    g.off_hv = (uint32_t)o; if (!g.hv_global) o += (size_t)g.hv_bytes * (all_children == 2 ? p.m : 1u);
     g.off_dirty = (uint32_t)o;
     if (all_children) o += ((((((size_t)3 << p.Lt) + 31) / 32 + 4) + ((size_t)1 << p.Lt)) * 4 + 15) & ~(size_t)15;   // keeps the barriers behind it 8-byte aligned
+    g.off_words = (uint32_t)o;
+    if (all_children == 2) o += ((size_t)p.m * (((size_t)3 << p.Lt)) * 4 + 15) & ~(size_t)15;       // words of every node and child
     g.off_bar = (uint32_t)o; o += (size_t)(kStagedMaxThreads / 32) * 4 * 8 + 8;      // room for any warps x nbuf, plus one
     g.off_gaveup = (uint32_t)o; o += 8;
     o = (o + 127) & ~(size_t)127; g.off_tiles = (uint32_t)o;
