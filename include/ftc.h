@@ -299,7 +299,8 @@ FTC_API int ftc_schedule_info(const ftc_desc_t* desc, ftc_sched_t* out);
  * Synthetic scenario inputs on the device (not part of the paper's method): element (s, p, e) of scenario
  * first_scenario+s is a function of (seed, scenario, p, e) only -- the splitmix64 output function applied to
  * seed + 0x9E3779B97F4A7C15 * (counter+1) -- mapped to one of the value kinds
- *   0 int32 in [-2^20, 2^20]   1 int64 in [-2^40, 2^40]   2 float32, sum of twelve 21-bit uniforms scaled to unit variance
+ *   0 int32 in [-2^20, 2^20]   1 int64 in [-2^40, 2^40]   2 float32, sum of twelve 32-bit uniforms (six counters per
+ *   element) centred, rounded to float32 once and scaled to unit variance: close to N(0,1), full mantissas
  *   3 int32 full range         4 uint64 full range
  * d_out is [S][P][k] of the kind's type. Returns FTC_OK, FTC_EINVAL (unknown kind, NULL) or FTC_ECUDA.
  */

@@ -18,14 +18,15 @@ __global__ void fill_kernel(uint64_t seed, uint64_t first_elem, uint64_t n, T* o
     for (uint64_t i = blockIdx.x * (uint64_t)blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
         const uint64_t lin = first_elem + i;
         if (KIND == 2) {
-            // twelve uniforms on [0, 2^21) from four hashes; centred and scaled to unit variance
+            // twelve uniforms on [0, 2^32) from six hashes; twice the centred sum (below 2^37) is rounded to float32 once
+            // (to nearest), the scale to unit variance, 2^-33, is exact
             long long total = 0;
-            for (int t = 0; t < 4; ++t) {
-                uint64_t h = hash_ctr(seed, lin * 4ull + t);
-                total += (long long)(h & 0x1FFFFFull) + (long long)((h >> 21) & 0x1FFFFFull) + (long long)((h >> 42) & 0x1FFFFFull);
+            for (int t = 0; t < 6; ++t) {
+                uint64_t h = hash_ctr(seed, lin * 6ull + t);
+                total += (long long)(h & 0xFFFFFFFFull) + (long long)(h >> 32);
             }
-            long long centred = 2 * total - 12ll * ((1ll << 21) - 1);
-            out[i] = (T)(float)((double)centred / 4194304.0);
+            long long centred = 2 * total - 12ll * ((1ll << 32) - 1);
+            out[i] = (T)(__ll2float_rn(centred) * 1.1641532182693481e-10f);
         } else {
             uint64_t h = hash_ctr(seed, lin);
             if (KIND == 0) out[i] = (T)((long long)(h % ((1ull << 21) + 1ull)) - (1ll << 20));

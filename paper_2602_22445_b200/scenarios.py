@@ -28,7 +28,7 @@ UNUSED = 0xFFFFFFFF
 # value kinds (shared numbering with the device generator)
 KIND_I32_PM20 = 0   # int32 uniform in [-2^20, 2^20]
 KIND_I64_PM40 = 1   # int64 uniform in [-2^40, 2^40]
-KIND_F32_NORMAL = 2  # float32, mean 0 variance 1, sum of twelve 21-bit uniforms (Irwin-Hall)
+KIND_F32_NORMAL = 2  # float32, mean 0 variance 1, sum of twelve 32-bit uniforms (Irwin-Hall), full 24-bit mantissas
 KIND_I32_FULL = 3   # int32 uniform over the full range
 KIND_U64_FULL = 4   # uint64 uniform
 
@@ -65,13 +65,14 @@ def gen_inputs(kind: int, seed: int, scenario_ids, P: int, k: int) -> np.ndarray
     if kind == KIND_F32_NORMAL:
         total = np.zeros(lin.shape, dtype=np.int64)
         with np.errstate(over="ignore"):
-            for t in range(4):
-                h = _hash(seed, lin * np.uint64(4) + np.uint64(t))
-                for part in range(3):
-                    total += ((h >> np.uint64(21 * part)) & np.uint64(0x1FFFFF)).astype(np.int64)
-        # twelve uniforms on [0, 2^21): mean 6*(2^21-1), variance ~ 2^42; scale to unit variance
-        centred = 2 * total - 12 * ((1 << 21) - 1)
-        return (centred.astype(np.float64) / float(1 << 22)).astype(np.float32)
+            for t in range(6):
+                h = _hash(seed, lin * np.uint64(6) + np.uint64(t))
+                total += (h & np.uint64(0xFFFFFFFF)).astype(np.int64) + (h >> np.uint64(32)).astype(np.int64)
+        # twelve uniforms on [0, 2^32): mean 6*(2^32-1), variance ~ 2^64. Twice the centred sum is an integer below 2^37;
+        # its conversion to float32 rounds to nearest (the one rounding), the scale 2^-33 is exact. The values carry full
+        # 24-bit mantissas, so float32 sums of them round at almost every addition (the fold order shows).
+        centred = 2 * total - 12 * ((1 << 32) - 1)
+        return centred.astype(np.float32) * np.float32(2.0 ** -33)
     h = _hash(seed, lin)
     if kind == KIND_I32_PM20:
         return ((h % np.uint64((1 << 21) + 1)).astype(np.int64) - (1 << 20)).astype(np.int32)

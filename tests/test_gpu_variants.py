@@ -26,8 +26,7 @@ def make_batch(P, f, k, dname, allreduce, S, seed):
     import torch
     rng = np.random.Generator(np.random.PCG64(seed))
     if dname == "f32":
-        # the library's float generator yields values whose sums within a group are exact (few mantissa bits), so the
-        # fold order inside a group would not show: take normal deviates, which round at every addition
+        # normal deviates from numpy: full mantissas, so float32 sums round at every addition and every fold order shows
         x = rng.standard_normal((S, P, k), dtype=np.float32)
         d_x = torch.from_numpy(x).cuda()
     else:
