@@ -109,3 +109,21 @@ def test_kernel_choice():
     assert B.ftc_candidates_kernel_name(B.make_desc(64, 2, 8, B.FTC_I64, "sum")) == "generic"             # a few KB per scenario
     assert B.ftc_candidates_kernel_name(B.make_desc(4096, 4, 5, B.FTC_I32, "max")) == "generic"           # odd vector length
     assert B.ftc_candidates_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(4))) == "generic"
+
+
+@pytest.mark.parametrize("P,f,k,dname,op", [(4096, 4, 32, "i32", "max"), (1024, 3, 16, "f32", "sum")])
+def test_a_wait_that_gives_up_is_reported_per_scenario(P, f, k, dname, op):
+    """With FTC_DEBUG_ONE_POLL the kernel's waits for its copies look once and give up: a scenario then either matches the
+    oracle or reports 3 ("a bounded wait ran out") for every child with zero values; the call returns by itself, and a
+    normal call afterwards on the same buffers matches the oracle again."""
+    S = 2 * 4 * 148 + 3
+    d_x, x, pf, inop, roots = make_batch(P, f, k, dname, True, S, seed=5 * P + f)
+    want = oracle_candidates(x, f, op, pf, inop, roots, True)
+    cand, info, _ = gpu_candidates(d_x, f, op, pf, inop, roots, True, B.FTC_DEBUG_ONE_POLL)
+    gave_up = (info[:, :, 0] == 3).all(axis=1)
+    assert ((info[:, :, 0] == 3).any(axis=1) == gave_up).all()          # all children of a scenario or none
+    assert not cand[gave_up].any() and not info[gave_up][:, :, 1].any()
+    assert np.array_equal(info[~gave_up], want[1][~gave_up])
+    assert np.array_equal(cand[~gave_up].view(np.uint8), want[0][~gave_up].view(np.uint8))
+    assert gave_up.any()                                                # tile copies are waited for right after their issue
+    assert_candidates(gpu_candidates(d_x, f, op, pf, inop, roots, True), want, "normal call after the give-up run")
