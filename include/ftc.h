@@ -117,6 +117,8 @@ typedef struct { uint32_t victim; uint32_t round; } ftc_inop_t;
                                             rank, the root last, instead of ascending with the root first: the algorithm leaves the
                                             order open (general kernel) */
 #define FTC_KERNEL_GENERIC 0x100u /* force the general level-by-level kernel (needs the workspace) */
+#define FTC_KERNEL_LEVELS  0x400u /* binary heaps: take the level kernel (shared-memory tiles evaluated level by level), which heaps of
+                                     arity 3 and more use by default, where the shape allows it */
 #define FTC_KERNEL_DIRECT  0x200u /* force the register-tiled kernel (direct global loads) where the shape allows it */
 #define FTC_DEBUG_ONE_POLL 0x4000000u /* testing aid: the kernel's bounded waits for its asynchronous copies look once instead of
                                          polling, so most of them give up and the give-up path runs: affected scenarios report

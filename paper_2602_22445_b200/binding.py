@@ -35,6 +35,7 @@ def FTC_TREE_ARITY(a: int) -> int:
     return (a & 0xFF) << 16
 
 FTC_KERNEL_DIRECT = 0x200
+FTC_KERNEL_LEVELS = 0x400
 FTC_DEBUG_ONE_POLL = 0x4000000
 OPS = {"sum": FTC_SUM, "max": FTC_MAX, "xor": FTC_XOR}
 

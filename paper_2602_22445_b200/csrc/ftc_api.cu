@@ -77,9 +77,12 @@ static int device_info(DeviceInfo& di) {
 // B200 figures, used where no device can be asked (sizing queries on a machine without a GPU).
 static const DeviceInfo kB200 = {148, 232448};
 
-enum KernelKind { K_GENERIC = 0, K_TILED = 1, K_STAGED = 2 };
+enum KernelKind { K_GENERIC = 0, K_TILED = 1, K_STAGED = 2, K_LEVELS = 3 };
 static KernelKind pick_kernel(Params& p, const DeviceInfo& di) {
-    if ((p.flags & FTC_KERNEL_GENERIC) || p.arity != 2) return K_GENERIC;   // the tiled kernels are built on the binary heap
+    if (p.flags & FTC_KERNEL_GENERIC) return K_GENERIC;
+    if (p.arity > 2 || (p.arity == 2 && (p.flags & FTC_KERNEL_LEVELS)))      // heaps of any arity: tiles evaluated level by level
+        if (aheap_supported(p, di.smem_optin)) return K_LEVELS;
+    if (p.arity != 2) return K_GENERIC;                                      // the register-tiled kernels are built on the binary heap
     if (!(p.flags & FTC_KERNEL_DIRECT) && staged_supported(p, di.smem_optin, di.sm_count)) return K_STAGED;
     return tiled_supported(p, di.smem_optin) ? K_TILED : K_GENERIC;
 }
@@ -134,6 +137,8 @@ static int run_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const
         e = launch_staged(p, tsel, di.sm_count, di.smem_optin, st);
     } else if (kind == K_TILED) {
         e = launch_tiled(p, tsel, di.sm_count, st);
+    } else if (kind == K_LEVELS) {
+        e = launch_aheap(p, tsel, di.sm_count, di.smem_optin, st);
     } else {
         const size_t need = (size_t)generic_grid(p, di.sm_count) * p.Gmax * p.kbytes;
         if (!d_ws || ws_bytes < need || !aligned16(d_ws)) return FTC_EWORKSPACE;
@@ -392,7 +397,7 @@ const char* ftc_kernel_name(const ftc_desc_t* desc, int is_allreduce) {
     if (device_info(di) != FTC_OK) di = kB200;
     p.ws_bytes = ~0ull;                                   // given the workspace ftc_workspace_bytes() asks for
     const KernelKind kind = pick_kernel(p, di);
-    return kind == K_STAGED ? "staged" : kind == K_TILED ? "tiled" : "generic";
+    return kind == K_STAGED ? "staged" : kind == K_TILED ? "tiled" : kind == K_LEVELS ? "levels" : "generic";
 }
 
 const char* ftc_kernel_variant(const ftc_desc_t* desc, int is_allreduce) {
@@ -403,7 +408,7 @@ const char* ftc_kernel_variant(const ftc_desc_t* desc, int is_allreduce) {
     p.ws_bytes = ~0ull;
     const KernelKind kind = pick_kernel(p, di);
     if (kind == K_STAGED) return staged_variant(p, type_select(desc->dtype, desc->op), di.smem_optin, di.sm_count, nullptr);
-    return kind == K_TILED ? "tiled" : "generic";
+    return kind == K_TILED ? "tiled" : kind == K_LEVELS ? "levels" : "generic";
 }
 
 int ftc_launch_blocks(const ftc_desc_t* desc, uint64_t S, int is_allreduce, uint32_t* blocks) {
@@ -420,7 +425,8 @@ int ftc_launch_blocks(const ftc_desc_t* desc, uint64_t S, int is_allreduce, uint
     const int tsel = type_select(desc->dtype, desc->op);
     const KernelKind kind = pick_kernel(p, di);
     cudaError_t e = kind == K_STAGED ? launch_staged(p, tsel, di.sm_count, di.smem_optin, nullptr)
-                  : kind == K_TILED ? launch_tiled(p, tsel, di.sm_count, nullptr) : launch_generic(p, tsel, di.sm_count, nullptr);
+                  : kind == K_TILED ? launch_tiled(p, tsel, di.sm_count, nullptr)
+                  : kind == K_LEVELS ? launch_aheap(p, tsel, di.sm_count, di.smem_optin, nullptr) : launch_generic(p, tsel, di.sm_count, nullptr);
     return e == cudaSuccess ? FTC_OK : FTC_ECUDA;
 }
 

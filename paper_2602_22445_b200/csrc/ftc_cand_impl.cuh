@@ -313,7 +313,8 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
             else { stop = true; if (lane == 0) atomicOr(const_cast<uint32_t*>(gaveup), 1u); }
         }
     };
-    auto release = [&]() { __syncwarp(); issue_next(); };
+    // values were written into the tile in place: order those writes before the next copy into the same bytes
+    auto release = [&]() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); __syncwarp(); issue_next(); };
     issue_next();
 
     for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {

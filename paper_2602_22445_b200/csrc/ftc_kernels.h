@@ -39,6 +39,11 @@ bool warp_supported(Params p, int smem_optin_bytes);
 uint32_t warp_lanes_per_scenario(Params p, int smem_optin_bytes);      // 32, or 16 when two scenarios share a warp; 0: not this kernel
 cudaError_t launch_warp(const Params& p, int tsel, int sm_count, int smem_optin_bytes, cudaStream_t st);
 
+// Level kernel: staged tiles evaluated level by level in shared memory, for subtrees that are a-ary heaps of any
+// arity >= 2 (the binary heap takes it only on request).
+bool aheap_supported(Params p, int smem_optin_bytes);
+cudaError_t launch_aheap(const Params& p, int tsel, int sm_count, int smem_optin_bytes, cudaStream_t st);
+
 // Every root child's delivery (value, flag, failed-list size): general kernel, workspace slices of candidates_slice_bytes().
 size_t candidates_slice_bytes(const Params& p);
 cudaError_t launch_candidates(const Params& p, int tsel, void* cand, uint32_t* info, int sm_count, cudaStream_t st);

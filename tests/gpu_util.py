@@ -59,7 +59,7 @@ def run_oracle(x, f, op, prefail, inop=None, roots=None, root=0, allreduce=False
                    partners_descending=partners_descending)
 
 
-def run_oracle_mt(x, f, op, prefail, inop=None, roots=None, root=0, allreduce=False, chunk=None, partners_descending=False):
+def run_oracle_mt(x, f, op, prefail, inop=None, roots=None, root=0, allreduce=False, chunk=None, partners_descending=False, arity=2):
     """run_oracle over chunks of scenarios on all host cores (threads: the C call releases the interpreter lock)."""
     import os
     from concurrent.futures import ThreadPoolExecutor
@@ -73,7 +73,7 @@ def run_oracle_mt(x, f, op, prefail, inop=None, roots=None, root=0, allreduce=Fa
         a, b = ab
         return O.batch(x[a:b], f, op, prefail[a:b], inop=None if inop is None else inop[a:b],
                        roots=None if roots is None else roots[a:b], root=root, allreduce=allreduce,
-                       partners_descending=partners_descending)
+                       arity=arity, partners_descending=partners_descending)
 
     with ThreadPoolExecutor(max_workers=cores) as ex:
         parts = list(ex.map(work, cuts))

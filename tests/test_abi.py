@@ -35,10 +35,15 @@ def test_host_only_calls():
     assert B.ftc_workspace_bytes(B.make_desc(8, 1, 1, B.FTC_I32, "sum"), 9) == 9 * 4 * 4
     assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_KERNEL_DIRECT)) == "tiled"
     assert B.ftc_kernel_name(B.make_desc(2, 1, 1, B.FTC_I32, "sum")) == "invalid"
-    # other subtree shapes: depth of the deepest node of an a-ary heap; they run on the general kernel
+    # other subtree shapes: depth of the deepest node of an a-ary heap; heaps run on the level kernel where the vector is a
+    # power-of-two number of 16-byte chunks, binomial trees and the rest on the general kernel
     t = B.ftc_schedule_info(B.make_desc(1024, 3, 16, B.FTC_F32, "sum", flags=B.FTC_TREE_ARITY(4)))
     assert (t["H"], t["rounds_reduce"], t["rounds_attempt"]) == (5, 8, 16)       # 256 rows: levels of 1, 4, 16, 64, 171
-    assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(3))) == "generic"
+    assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(3))) == "levels"
+    assert B.ftc_kernel_name(B.make_desc(4096, 4, 3, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(3))) == "generic"
+    assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_BINOMIAL)) == "generic"
+    assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_KERNEL_LEVELS)) == "levels"
+    assert B.ftc_workspace_bytes(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(3)), 1000, True) == 0
     assert B.ftc_kernel_name(B.make_desc(8, 1, 1, B.FTC_I32, "sum", flags=B.FTC_TREE_ARITY(1))) == "invalid"
     # many processes with wide vectors: the shared-memory kernel asks for a workspace for its array of tile results
     wide = B.make_desc(16384, 5, 16, B.FTC_U64, "sum")

@@ -1,0 +1,76 @@
+"""GPU parity for the level kernel (shared-memory tiles evaluated level by level), which plays subtrees that are a-ary heaps
+of arity 3 and more, and binary heaps on request: against the CPU oracle playing the same shape, bit for bit."""
+import numpy as np
+import pytest
+
+from paper_2602_22445_b200 import binding as B
+from tests.gpu_util import assert_same, run_gpu, run_oracle_mt
+from tests.test_gpu_variants import DT, make_batch
+
+pytestmark = pytest.mark.gpu
+
+
+def flags_for(arity):
+    return B.FTC_KERNEL_LEVELS if arity == 2 else B.FTC_TREE_ARITY(arity)
+
+
+SHAPES = [
+    # P, f, k, dtype, op: one tile, several tiles, several levels above the tiles, ragged last levels, a short last group
+    (7, 1, 4, "i32", "sum"), (40, 3, 2, "u64", "xor"), (150, 3, 16, "f32", "sum"), (1024, 3, 16, "f32", "sum"),
+    (1000, 0, 4, "f32", "sum"), (2003, 2, 8, "i64", "max"), (4096, 4, 32, "i32", "max"), (5000, 15, 4, "i32", "xor"),
+    (16384, 1, 8, "i32", "sum"), (65536, 8, 4, "u64", "sum"), (30011, 7, 64, "f32", "sum"), (9000, 31, 2, "i64", "sum"),
+]
+
+
+@pytest.mark.parametrize("arity", [2, 3, 4, 5, 8, 32])
+@pytest.mark.parametrize("P,f,k,dname,op", SHAPES)
+def test_level_kernel_matches_the_oracle(arity, P, f, k, dname, op):
+    S = max(3, min(40, int(4e6 // (P * k))))
+    for allreduce in (False, True):
+        d_x, x, pf, inop, roots = make_batch(P, f, k, dname, allreduce, S, seed=arity * 1000 + P + k)
+        got = run_gpu(None, f, op, pf, inop, roots, 0, allreduce, flags_for(arity), d_x=d_x)
+        # the widest shape's heap array does not fit into shared memory: the general kernel (binary heap: the staged one) plays it
+        assert B.ftc_kernel_name(got[2], allreduce) == (("staged" if arity == 2 else "generic") if (P, k) == (30011, 64) else "levels")
+        assert_same(got, run_oracle_mt(x, f, op, pf, inop, roots, 0, allreduce, arity=arity), f"P={P} f={f} k={k} {dname} {op} arity={arity} allreduce={allreduce}")
+
+
+@pytest.mark.parametrize("arity", [3, 4])
+def test_level_kernel_with_descending_partners(arity):
+    for P, f, k in ((150, 3, 16), (4099, 4, 8)):
+        d_x, x, pf, inop, roots = make_batch(P, f, k, "f32", True, 30, seed=P)
+        got = run_gpu(None, f, "sum", pf, inop, roots, 0, True, flags_for(arity) | B.FTC_PARTNERS_DESCENDING, d_x=d_x)
+        assert B.ftc_kernel_name(got[2], True) == "levels"
+        assert_same(got, run_oracle_mt(x, f, "sum", pf, inop, roots, 0, True, arity=arity, partners_descending=True), f"P={P} arity={arity}")
+
+
+def test_shapes_the_level_kernel_leaves_to_the_general_one():
+    for k, dt in ((3, B.FTC_F32), (6, B.FTC_I32), (1, B.FTC_U64)):            # not a power-of-two number of 16-byte chunks
+        assert B.ftc_kernel_name(B.make_desc(100, 2, k, dt, "sum", flags=B.FTC_TREE_ARITY(4)), True) == "generic"
+    assert B.ftc_kernel_name(B.make_desc(100, 2, 4, B.FTC_I32, "sum", flags=B.FTC_TREE_ARITY(4) | B.FTC_KERNEL_GENERIC), True) == "generic"
+    assert B.ftc_kernel_name(B.make_desc(100, 2, 4, B.FTC_I32, "sum", flags=B.FTC_TREE_BINOMIAL), True) == "generic"
+    assert B.ftc_kernel_name(B.make_desc(100, 2, 4, B.FTC_I32, "sum"), True) == "staged"
+
+
+@pytest.mark.parametrize("arity,P,f,k,dname,op,allreduce", [(4, 4096, 4, 32, "i32", "max", True), (3, 1024, 3, 16, "f32", "sum", True),
+                                                            (8, 65536, 8, 4, "u64", "sum", False), (2, 150, 3, 16, "f32", "sum", True)])
+def test_level_kernel_gives_up_cleanly(arity, P, f, k, dname, op, allreduce):
+    """With FTC_DEBUG_ONE_POLL the waits for the asynchronous copies look once and give up: a scenario is then either
+    played correctly or reports FTC_ST_INTERNAL_TIMEOUT with zero bytes, a block that reported it does so for all its
+    later scenarios, the call returns by itself, and the next normal call on the same buffers matches the oracle."""
+    flags = flags_for(arity)
+    desc = B.make_desc(P, f, k, B.dtype_code(np.dtype(DT[dname])), op, root=-1, max_inop=2, flags=flags)
+    assert B.ftc_kernel_name(desc, allreduce) == "levels"
+    blocks = B.ftc_launch_blocks(desc, 1 << 30, allreduce)
+    S = 2 * blocks + 3
+    d_x, x, pf, inop, roots = make_batch(P, f, k, dname, allreduce, S, seed=5 + P)
+    want = run_oracle_mt(x, f, op, pf, inop, roots, 0, allreduce, arity=arity)
+    out, st, _ = run_gpu(None, f, op, pf, inop, roots, 0, allreduce, flags | B.FTC_DEBUG_ONE_POLL, d_x=d_x)
+    timed_out = (st[:, 0] & 0xFF) == B.FTC_ST_INTERNAL_TIMEOUT
+    ob, wb = out.view(np.uint8).reshape(S, -1), want[0].view(np.uint8).reshape(S, -1)
+    assert not ob[timed_out].any() and not st[timed_out, 1:].any()
+    assert np.array_equal(st[~timed_out], want[1][~timed_out]) and np.array_equal(ob[~timed_out], wb[~timed_out])
+    for b in range(blocks):
+        seq = timed_out[b::blocks]
+        assert np.array_equal(seq, np.sort(seq)), (b, seq)
+    assert timed_out.any()
+    assert_same(run_gpu(None, f, op, pf, inop, roots, 0, allreduce, flags, d_x=d_x), want, "normal call after the give-up run")
