@@ -1,8 +1,9 @@
 // Level kernel: the shared-memory path for subtrees that are a-ary heaps (FTC_TREE_ARITY(a), a = 2..32; the paper's
 // I(f)-tree fixes only the root's f+1 children and their subtree sizes, so any such shape is one). The heap of the
-// selected subtree's rows is cut into tiles as in the staged kernel -- a tile is a sub-heap of D levels, each level one
-// contiguous run of rows, brought into shared memory by one bulk copy per level -- but a tile is evaluated level by
-// level in shared memory instead of in registers and shuffles, which works for any number of children per node:
+// selected subtree's rows is cut into tiles as in the staged kernel -- a tile is a forest of neighbouring sub-heaps of D
+// levels, each level one contiguous run of rows, brought into shared memory by one bulk copy per level -- but a tile is
+// evaluated level by level in shared memory instead of in registers and shuffles, which works for any number of children
+// per node:
 //   1. every (row, 16-byte chunk) of the tile folds its group (Algorithm "Up-correction": own input, then the partners
 //      whose message arrived, in the schedule's order) and leaves the result in place of the row's first member;
 //   2. the tile's levels are combined from the leaves up (Algorithm "reduce_non_root": data, then child 1, child 2, ...),
@@ -17,14 +18,20 @@ namespace ftc {
 
 constexpr uint32_t kAheapMaxLevels = 24;
 
+// A work item of the tile kind is a forest: n neighbouring nodes of heap level Lt with everything below them, d levels in
+// all. Neighbouring nodes have neighbouring children, so every level of the forest is one contiguous run of rows. The
+// heap's last level is filled from the left only: the first nA nodes of level Lt have rows on it (forests of D levels, n1
+// nodes each), the others end one level higher (forests of D - 1 levels, n2 nodes each, n2 > n1), so that both kinds fill
+// a warp's buffer about equally.
 struct AheapGeom {
     uint32_t nwarps, tile_cap;             // warps per block, bytes of a warp's buffer
-    uint32_t D, Lt;                        // levels of a tile; heap level at which the tiles are rooted
-    uint32_t R;                            // rows of a tile: (a^D - 1) / (a - 1)
-    uint32_t ntop, ntiles, nheap;          // rows above the tiles, tiles, rows of the heap array (ntop + ntiles)
-    uint32_t ngroups;                      // work items over the rows above the tiles (R rows each)
+    uint32_t D, Lt;                        // levels of a deep forest; heap level of the forests' roots
+    uint32_t n1, n2, nA, nroots;           // roots per deep / shallow forest; roots with rows on the last level; all roots
+    uint32_t itemsA, itemsB, ngroups;      // deep forests, shallow forests, work items over the rows above level Lt
+    uint32_t cap_rows;                     // rows a warp's buffer holds
+    uint32_t ntop, nheap;                  // rows above level Lt; rows of the block's heap array (levels 0 .. Lt)
     uint32_t lstart[kAheapMaxLevels + 1];  // first row of heap level l: (a^l - 1) / (a - 1)
-    uint32_t tstart[4], apow[4];           // tile level u: its first node, and a^u (0xFFFFFFFF / 0 beyond the tile's levels)
+    uint32_t tstart[5], apow[5];           // a forest's level u per root: nodes above it, (a^u - 1) / (a - 1), and nodes on it, a^u
     uint32_t off_rootv, off_hv, off_bar, off_gaveup, off_tiles, smem_bytes;
 };
 
@@ -42,14 +49,16 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) aheap_kernel(Params p, c
 
     const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
     const uint32_t a = p.arity, C = p.C, cwl = p.cw_log2, Cmask = C - 1;
-    const uint32_t D = g.D, R = g.R, ntop = g.ntop, ntiles = g.ntiles;
-    const uint32_t nitems = ntiles + g.ngroups + 1;
+    const uint32_t D = g.D, Lt = g.Lt, ntop = g.ntop;
+    const uint32_t itemsAB = g.itemsA + g.itemsB, nitems = itemsAB + g.ngroups + 1;
     const uint32_t rowbytes = p.m * p.kbytes;
     const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
     const uint32_t tries = (p.flags & FTC_DEBUG_ONE_POLL) ? 1u : kWaitTries;
-    // a^u for the tile level u that holds tile node t
-    const uint32_t ts1 = g.tstart[1], ts2 = g.tstart[2], ts3 = g.tstart[3], a2 = a * a, a3 = a2 * a;
-    auto level_width = [&](uint32_t t) { return t >= ts3 ? a3 : t >= ts2 ? a2 : t >= ts1 ? a : 1u; };
+    // forest `it`: first root (position on level Lt), roots, levels
+    auto forest = [&](uint32_t it, uint32_t& x0, uint32_t& n, uint32_t& d) {
+        if (it < g.itemsA) { x0 = it * g.n1; n = min(g.n1, g.nA - x0); d = D; }
+        else { x0 = g.nA + (it - g.itemsA) * g.n2; n = min(g.n2, g.nroots - x0); d = D - 1; }
+    };
 
     const uint32_t bar0 = smem_addr(sbase + g.off_bar) + wid * 8;
     char* tile = sbase + g.off_tiles + (size_t)wid * g.tile_cap;
@@ -60,21 +69,22 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) aheap_kernel(Params p, c
     uint32_t phase = 0;
     bool pending = false, stop = false;
 
-    // ---- this warp's copy pipeline over the flat sequence (scenario, work item), one buffer, one item ahead ----
+    // ---- this warp's copy pipeline over the flat sequence (scenario, work item): one buffer, refilled as soon as it is free ----
     const uint32_t n_my = wid < nitems ? (nitems - wid + nw - 1) / nw : 0;
     uint64_t is_s = blockIdx.x;
     const char* is_src = reinterpret_cast<const char*>(p.in) + is_s * scen_bytes;
     uint32_t is_i = 0;
-    uint32_t my_rows = 0, my_start = 0;                               // lane u < D copies level u of a tile
-    if (lane < D) { my_rows = g.apow[lane]; my_start = g.tstart[lane]; }
+    uint32_t my_pw = 0, my_ts = 0, my_ls = 0;                         // lane u < D copies level u of a forest
+    if (lane < D) { my_pw = g.apow[lane]; my_ts = g.tstart[lane]; my_ls = g.lstart[Lt + lane]; }
     auto issue_next = [&]() {
         if (n_my == 0 || is_s >= p.S || stop) return;
         const uint32_t it = wid + is_i * nw;
         uint64_t first_row = 0; uint32_t nrows = 0, dst_off = 0;
-        if (it < ntiles) {
-            if (lane < D) { first_row = (uint64_t)my_rows * (ntop + it) + my_start; nrows = my_rows; dst_off = my_start * rowbytes; }
-        } else if (it < ntiles + g.ngroups) {
-            if (lane == 0) { first_row = (uint64_t)(it - ntiles) * R; nrows = min(R, ntop - (uint32_t)first_row); }
+        if (it < itemsAB) {
+            uint32_t x0, n, d; forest(it, x0, n, d);
+            if (lane < d) { first_row = (uint64_t)my_ls + (uint64_t)x0 * my_pw; nrows = n * my_pw; dst_off = n * my_ts * rowbytes; }
+        } else if (it < itemsAB + g.ngroups) {
+            if (lane == 0) { first_row = (uint64_t)(it - itemsAB) * g.cap_rows; nrows = min(g.cap_rows, ntop - (uint32_t)first_row); }
         }
         const uint64_t b0 = first_row * rowbytes + p.kbytes;
         uint32_t bytes = 0;
@@ -122,44 +132,60 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) aheap_kernel(Params p, c
         }
         if (p.is_allreduce) count_holders(p, cx, pf, unr);
         const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
+        // a row's value after up-correction (Algorithm "Up-correction") from its staged copy
+        auto fold_row = [&](const char* srow_lc, const char* in_lc, uint32_t row) -> uint4 {
+            if (group_is_plain(p, root, inc, row)) return fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdShared(), p.pdesc != 0);
+            return fold_staged_call<T, OP, false>(fold_shape(p), root, sstar, inc, in_lc, srow_lc, row);
+        };
 
         for (uint32_t i = 0; i < n_my; ++i) {
             const uint32_t it = wid + i * nw;
             acquire();
-            if (it < ntiles) {
-                const uint32_t j0 = ntop + it;
-                if (j0 < G) {
+            if (it < itemsAB) {
+                uint32_t x0, n, d; forest(it, x0, n, d);
+                // local node t of forest level l is row rb_l + t; level l starts at local node th_l
+                const uint32_t th1 = d > 1 ? n * g.tstart[1] : 0xFFFFFFFFu, th2 = d > 2 ? n * g.tstart[2] : 0xFFFFFFFFu,
+                               th3 = d > 3 ? n * g.tstart[3] : 0xFFFFFFFFu;
+                const uint32_t rb0 = g.lstart[Lt] + x0, rb1 = g.lstart[Lt + 1] + x0 * g.apow[1] - th1,
+                               rb2 = g.lstart[Lt + 2] + x0 * g.apow[2] - th2, rb3 = g.lstart[Lt + 3] + x0 * g.apow[3] - th3;
+                if (rb0 < G) {
                     // 1. every (row, chunk) folds its group; the result takes the place of the row's first member
-                    for (uint32_t u = lane; u < R * C; u += 32) {
-                        const uint32_t t = u >> cwl, c = u & Cmask, row = level_width(t) * j0 + t;
+                    const uint32_t units = (n * g.tstart[d]) << cwl;
+                    for (uint32_t u = lane; u < units; u += 32) {
+                        const uint32_t t = u >> cwl, c = u & Cmask;
+                        const uint32_t row = t + (t >= th3 ? rb3 : t >= th2 ? rb2 : t >= th1 ? rb1 : rb0);
                         if (row >= G) continue;
                         char* srow = tile + (size_t)t * rowbytes + c * 16;
-                        *reinterpret_cast<uint4*>(srow) = fold_staged<T, OP, false>(p, root, sstar, inc, in_s + c * 16, srow, row);
+                        *reinterpret_cast<uint4*>(srow) = fold_row(srow, in_s + c * 16, row);
                     }
                     __syncwarp();
-                    // 2. the levels of the tile, leaves first: data, then the children in ascending order
-                    for (int lv = (int)D - 2; lv >= 0; --lv) {
-                        const uint32_t t0 = g.tstart[lv], nn = g.apow[lv];
-                        for (uint32_t u = lane; u < nn * C; u += 32) {
-                            const uint32_t t = t0 + (u >> cwl), c = u & Cmask, row = nn * j0 + t;
-                            if (row >= G) continue;
-                            uint4 v = *reinterpret_cast<const uint4*>(tile + (size_t)t * rowbytes + c * 16);
-                            for (uint32_t ch = 1; ch <= a; ++ch)
-                                if ((uint64_t)a * row + ch < G) v = comb16<T, OP>(v, *reinterpret_cast<const uint4*>(tile + (size_t)(a * t + ch) * rowbytes + c * 16));
-                            *reinterpret_cast<uint4*>(tile + (size_t)t * rowbytes + c * 16) = v;
+                    // 2. the levels of the forest, leaves first: data, then the children in ascending order
+                    for (int lv = (int)d - 2; lv >= 0; --lv) {
+                        const uint32_t t0 = n * g.tstart[lv], t1 = n * g.tstart[lv + 1], nn = n * g.apow[lv];
+                        const uint32_t rbl = g.lstart[Lt + lv] + x0 * g.apow[lv];
+                        for (uint32_t u = lane; u < (nn << cwl); u += 32) {
+                            const uint32_t pos = u >> cwl, c = u & Cmask, row = rbl + pos, first = a * row + 1;
+                            if (row >= G || first >= G) continue;
+                            const uint32_t cnt = min(a, G - first);
+                            char* mine = tile + (size_t)(t0 + pos) * rowbytes + c * 16;
+                            const char* child = tile + (size_t)(t1 + a * pos) * rowbytes + c * 16;
+                            uint4 v = *reinterpret_cast<const uint4*>(mine);
+                            for (uint32_t ch = 0; ch < cnt; ++ch) v = comb16<T, OP>(v, *reinterpret_cast<const uint4*>(child + (size_t)ch * rowbytes));
+                            *reinterpret_cast<uint4*>(mine) = v;
                         }
                         __syncwarp();
                     }
-                    // 3. the tile's root
-                    if (lane < C) hv[(size_t)j0 * C + lane] = *reinterpret_cast<const uint4*>(tile + lane * 16);
+                    // 3. the forest's roots
+                    for (uint32_t u = lane; u < (n << cwl); u += 32)
+                        hv[(size_t)(rb0 + (u >> cwl)) * C + (u & Cmask)] = *reinterpret_cast<const uint4*>(tile + (size_t)(u >> cwl) * rowbytes + (u & Cmask) * 16);
                 }
-            } else if (it < ntiles + g.ngroups) {
-                // rows above the tiles: fold now, combine later
-                const uint32_t r0 = (it - ntiles) * R;
-                for (uint32_t u = lane; u < R * C; u += 32) {
+            } else if (it < itemsAB + g.ngroups) {
+                // rows above the forests: fold now, combine later
+                const uint32_t r0 = (it - itemsAB) * g.cap_rows;
+                for (uint32_t u = lane; u < (g.cap_rows << cwl); u += 32) {
                     const uint32_t t = u >> cwl, c = u & Cmask, row = r0 + t;
-                    if (row >= ntop || row >= G) continue;
-                    hv[(size_t)row * C + c] = fold_staged<T, OP, false>(p, root, sstar, inc, in_s + c * 16, tile + (size_t)t * rowbytes + c * 16, row);
+                    if (row >= ntop || row >= G) break;
+                    hv[(size_t)row * C + c] = fold_row(tile + (size_t)t * rowbytes + c * 16, in_s + c * 16, row);
                 }
             } else if (sstar >= p.r) {
                 if (lane < C) rootv[lane] = fold_root16<T, OP, LdGlobal>(p, root, inc, in_s + lane * 16);
@@ -167,15 +193,15 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) aheap_kernel(Params p, c
             release();
         }
         __syncthreads();
-        // ---- levels above the tiles, leaves first ----
-        for (int lvl = (int)g.Lt - 1; lvl >= 0; --lvl) {
+        // ---- levels above the forests, leaves first ----
+        for (int lvl = (int)Lt - 1; lvl >= 0; --lvl) {
             const uint32_t lo = g.lstart[lvl], n = g.lstart[lvl + 1] - lo;
-            for (uint32_t u = tid; u < n * C; u += nt) {
-                const uint32_t row = lo + (u >> cwl), c = u & Cmask;
-                if (row >= G) continue;
+            for (uint32_t u = tid; u < (n << cwl); u += nt) {
+                const uint32_t row = lo + (u >> cwl), c = u & Cmask, first = a * row + 1;
+                if (row >= G || first >= G) continue;
+                const uint32_t cnt = min(a, G - first);
                 uint4 v = hv[(size_t)row * C + c];
-                for (uint32_t ch = 1; ch <= a; ++ch)
-                    if ((uint64_t)a * row + ch < G) v = comb16<T, OP>(v, hv[(size_t)(a * row + ch) * C + c]);
+                for (uint32_t ch = 0; ch < cnt; ++ch) v = comb16<T, OP>(v, hv[(size_t)(first + ch) * C + c]);
                 hv[(size_t)row * C + c] = v;
             }
             __syncthreads();
@@ -198,10 +224,10 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) aheap_kernel(Params p, c
 
 // ---- host side ----
 #ifndef FTC_AHEAP_TILE_KB
-#define FTC_AHEAP_TILE_KB 24
+#define FTC_AHEAP_TILE_KB 14
 #endif
-constexpr uint64_t kAheapTileBytes = FTC_AHEAP_TILE_KB * 1024;   // a tile takes as many whole levels as fit into this
-constexpr size_t kAheapMaxHeapBytes = 96 * 1024;                 // the block's heap array (tile roots and the rows above them)
+constexpr uint64_t kAheapTileBytes = FTC_AHEAP_TILE_KB * 1024;   // a warp's buffer: forests are sized to fill it
+constexpr size_t kAheapMaxHeapBytes = 96 * 1024;                 // the block's heap array (levels 0 .. Lt)
 
 static bool aheap_geometry(Params& p, int smem_optin, AheapGeom& g) {
     if (p.kbytes % 16 || p.arity < 2) return false;
@@ -210,33 +236,42 @@ static bool aheap_geometry(Params& p, int smem_optin, AheapGeom& g) {
     uint32_t cwl = 0; while ((1u << cwl) < C) ++cwl;
     p.C = C; p.cw_log2 = cwl;
     const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
+    const uint64_t budget = kAheapTileBytes > rowbytes ? kAheapTileBytes : rowbytes;
     // levels of the heap: first row of each level
     uint32_t Hmax = 0; uint64_t start = 0, width = 1;
     g.lstart[0] = 0;
     while (start < p.Gmax) {
         start += width; width *= a; ++Hmax;
-        if (Hmax > kAheapMaxLevels) return false;
+        if (Hmax + 4 > kAheapMaxLevels) return false;
         g.lstart[Hmax] = (uint32_t)(start < 0xFFFFFFFFull ? start : 0xFFFFFFFFull);
     }
     for (uint32_t l = Hmax + 1; l <= kAheapMaxLevels; ++l) g.lstart[l] = 0xFFFFFFFFu;
-    // the deepest tile within the byte budget (at most four levels)
+    // the deepest forest of one root within the budget (at most four levels)
     uint32_t D = 1; uint64_t R = 1, w = a;
-    while (D < 4 && D < Hmax && (R + w) * rowbytes <= kAheapTileBytes) { R += w; w *= a; ++D; }
-    if (R * rowbytes > 64 * 1024) return false;
-    g.D = D; g.R = (uint32_t)R;
-    { uint32_t s0 = 0, pw = 1; for (uint32_t u = 0; u < 4; ++u) { g.tstart[u] = u < D ? s0 : 0xFFFFFFFFu; g.apow[u] = u < D ? pw : 0; s0 += pw; pw *= a; } }
-    g.Lt = Hmax > D ? Hmax - D : 0;
-    g.ntop = g.lstart[g.Lt];
-    uint64_t nt = 1; for (uint32_t l = 0; l < g.Lt; ++l) nt *= a;
-    if (nt > (1u << 20)) return false;
-    g.ntiles = (uint32_t)nt; g.nheap = g.ntop + g.ntiles;
-    g.ngroups = (g.ntop + g.R - 1) / g.R;
+    while (D < 4 && D < Hmax && (R + w) * rowbytes <= budget) { R += w; w *= a; ++D; }
+    { uint64_t s0 = 0, pw = 1; for (uint32_t u = 0; u < 5; ++u) { g.tstart[u] = (uint32_t)s0; g.apow[u] = (uint32_t)pw; s0 += pw; pw *= a; } }
+    g.D = D; g.Lt = Hmax - D;
+    const uint64_t Rshallow = g.tstart[D - 1];                                   // rows of a root with D - 1 levels (0: D = 1)
+    uint64_t nroots = 1; for (uint32_t l = 0; l < g.Lt; ++l) nroots *= a;
+    if (nroots > (1u << 20)) return false;
+    const uint64_t nlast = p.Gmax - g.lstart[Hmax - 1];                          // rows on the heap's last level
+    const uint64_t per_root_last = g.apow[D - 1];
+    g.nA = (uint32_t)((nlast + per_root_last - 1) / per_root_last);
+    g.nroots = D == 1 ? g.nA : (uint32_t)nroots;
+    g.n1 = (uint32_t)(budget / (R * rowbytes)); if (g.n1 < 1) g.n1 = 1;
+    g.n2 = Rshallow ? (uint32_t)(budget / (Rshallow * rowbytes)) : 1; if (g.n2 < 1) g.n2 = 1;
+    g.itemsA = (g.nA + g.n1 - 1) / g.n1;
+    g.itemsB = (g.nroots - g.nA + g.n2 - 1) / g.n2;
+    uint64_t cap_rows = g.n1 * R; if (g.n2 * Rshallow > cap_rows) cap_rows = g.n2 * Rshallow;
+    g.cap_rows = (uint32_t)cap_rows;
+    g.ntop = g.lstart[g.Lt]; g.nheap = g.ntop + (uint32_t)nroots;
+    g.ngroups = (g.ntop + g.cap_rows - 1) / g.cap_rows;
     const size_t hv_bytes = (size_t)g.nheap * C * 16;
     if (hv_bytes > kAheapMaxHeapBytes) return false;
-    g.tile_cap = (uint32_t)((R * rowbytes + 127) & ~(uint64_t)127);
-    const uint32_t nitems = g.ntiles + g.ngroups + 1;
+    g.tile_cap = (uint32_t)((cap_rows * rowbytes + 127) & ~(uint64_t)127);
+    const uint32_t nitems = g.itemsA + g.itemsB + g.ngroups + 1;
     uint32_t warps = 1;
-    while (warps < 8 && warps * 2 * 8 <= nitems) warps *= 2;
+    while (warps < 8 && warps * 2 * 4 <= nitems) warps *= 2;
     size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
     o = (o + 15) & ~(size_t)15; g.off_rootv = (uint32_t)o; o += (size_t)C * 16;
     g.off_hv = (uint32_t)o; o += hv_bytes;

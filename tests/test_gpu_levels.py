@@ -22,6 +22,11 @@ SHAPES = [
 ]
 
 
+# (arity, P) of SHAPES whose heap array (the rows of all levels down to the tiles' roots) exceeds the kernel's shared-memory
+# budget, as the shape with P = 30011 and 256-byte vectors does at every arity: the general kernel plays those
+TOO_WIDE = {(5, 4096), (32, 4096), (8, 65536)}
+
+
 @pytest.mark.parametrize("arity", [2, 3, 4, 5, 8, 32])
 @pytest.mark.parametrize("P,f,k,dname,op", SHAPES)
 def test_level_kernel_matches_the_oracle(arity, P, f, k, dname, op):
@@ -29,8 +34,8 @@ def test_level_kernel_matches_the_oracle(arity, P, f, k, dname, op):
     for allreduce in (False, True):
         d_x, x, pf, inop, roots = make_batch(P, f, k, dname, allreduce, S, seed=arity * 1000 + P + k)
         got = run_gpu(None, f, op, pf, inop, roots, 0, allreduce, flags_for(arity), d_x=d_x)
-        # the widest shape's heap array does not fit into shared memory: the general kernel (binary heap: the staged one) plays it
-        assert B.ftc_kernel_name(got[2], allreduce) == (("staged" if arity == 2 else "generic") if (P, k) == (30011, 64) else "levels")
+        fits = (P, k) != (30011, 64) and (arity, P) not in TOO_WIDE
+        assert B.ftc_kernel_name(got[2], allreduce) == ("levels" if fits else "staged" if arity == 2 else "generic")
         assert_same(got, run_oracle_mt(x, f, op, pf, inop, roots, 0, allreduce, arity=arity), f"P={P} f={f} k={k} {dname} {op} arity={arity} allreduce={allreduce}")
 
 
@@ -52,7 +57,7 @@ def test_shapes_the_level_kernel_leaves_to_the_general_one():
 
 
 @pytest.mark.parametrize("arity,P,f,k,dname,op,allreduce", [(4, 4096, 4, 32, "i32", "max", True), (3, 1024, 3, 16, "f32", "sum", True),
-                                                            (8, 65536, 8, 4, "u64", "sum", False), (2, 150, 3, 16, "f32", "sum", True)])
+                                                            (8, 16384, 1, 8, "i32", "sum", False), (2, 150, 3, 16, "f32", "sum", True)])
 def test_level_kernel_gives_up_cleanly(arity, P, f, k, dname, op, allreduce):
     """With FTC_DEBUG_ONE_POLL the waits for the asynchronous copies look once and give up: a scenario is then either
     played correctly or reports FTC_ST_INTERNAL_TIMEOUT with zero bytes, a block that reported it does so for all its
