@@ -13,10 +13,15 @@
 // or the general fold is needed (a renumbered slot, the short last group): no marking pass.
 #pragma once
 #include "ftc_staged_impl.cuh"
+#include "ftc_decode_warp.cuh"
 
 namespace ftc {
 
 constexpr uint32_t kAheapMaxLevels = 24;
+#ifndef FTC_AHEAP_MINB
+#define FTC_AHEAP_MINB 2
+#endif
+constexpr uint32_t kAheapWarpsPerSM = 8 * FTC_AHEAP_MINB;   // what the register bound of the kernel lets an SM hold
 
 // A work item of the tile kind is a forest: n neighbouring nodes of heap level Lt with everything below them, d levels in
 // all. Neighbouring nodes have neighbouring children, so every level of the forest is one contiguous run of rows. The
@@ -36,7 +41,7 @@ struct AheapGeom {
 };
 
 template <typename T, int OP>
-__global__ void __launch_bounds__(kStagedMaxThreads, 2) aheap_kernel(Params p, const __grid_constant__ AheapGeom g) {
+__global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kernel(Params p, const __grid_constant__ AheapGeom g) {
     extern __shared__ __align__(128) uint32_t smem[];
     char* sbase = reinterpret_cast<char*>(smem);
     Ctx* cx = reinterpret_cast<Ctx*>(smem);
@@ -113,11 +118,45 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) aheap_kernel(Params p, c
     auto release = [&]() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); __syncwarp(); issue_next(); };
     issue_next();
 
+    // A block of one warp whose masks are one word per lane decodes in registers (ftc_decode_warp.cuh) and fetches the
+    // next scenario's mask word, in-operation entry and root while the current scenario is played.
+    const bool warp_decode = nw == 1 && p.W <= 32 && p.max_inop <= 32;
+    uint32_t nx_pf = 0, nx_vic = FTC_INOP_UNUSED, nx_rnd = 0, nx_root = 0;
+    auto fetch_small = [&](uint64_t s) {
+        nx_pf = 0; nx_vic = FTC_INOP_UNUSED; nx_rnd = 0; nx_root = 0;
+        if (s >= p.S) return;
+        if (lane < p.W) nx_pf = __ldg(p.prefail + s * p.W + lane);
+        if (lane < p.max_inop) { const ftc_inop_t* e = p.inop + s * p.max_inop + lane; nx_vic = __ldg(&e->victim); nx_rnd = __ldg(&e->round); }
+        if (p.root < 0) nx_root = __ldg(p.roots + s);
+    };
+    if (warp_decode) fetch_small(blockIdx.x);
+
     for (uint64_t s = blockIdx.x; s < p.S; s += gridDim.x) {
         const char* in_s = reinterpret_cast<const char*>(p.in) + s * scen_bytes;
         const bool dead = *gaveup != 0;
         if (dead) stop = true;
-        decode_scenario(p, s, cx, pf, inc);
+        bool decoded = false;
+        if (warp_decode) {
+            uint32_t pfw = nx_pf;
+            if (lane == p.W - 1 && (p.P & 31)) pfw &= (1u << (p.P & 31)) - 1u;
+            const uint32_t ev = nx_vic, er = nx_rnd, first_root = p.root >= 0 ? (uint32_t)p.root : nx_root;
+            fetch_small(s + gridDim.x);
+            WarpScen w; bool slow;
+            decode_group<32, 2, 2>(p, pfw, ev, er, first_root, w, slow);
+            if (!slow) {
+                if (lane == 0) {
+                    cx->code = w.code; cx->sstar = w.sstar; cx->attempts = w.attempts; cx->root = w.root; cx->base = w.base;
+                    cx->npre = w.npre; cx->nexcl = w.nexcl; cx->inop_incl = w.inop_incl; cx->holders = w.holders; cx->G = w.G;
+                    pf[p.W] = 0;
+                }
+                if (lane < p.W) pf[lane] = pfw;
+                if (lane <= p.W) inc[lane] = w.incw;
+                if (p.W == 32 && lane == 0) inc[32] = 0;
+                decoded = true;
+                __syncwarp();
+            }
+        }
+        if (!decoded) decode_scenario(p, s, cx, pf, inc);
         char* out_s = reinterpret_cast<char*>(p.out) + s * p.kbytes;
         if (cx->code != FTC_ST_OK || dead) {
             if (tid < C) reinterpret_cast<uint4*>(out_s)[tid] = make_uint4(0, 0, 0, 0);
@@ -130,11 +169,13 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) aheap_kernel(Params p, c
             __syncthreads();
             continue;
         }
-        if (p.is_allreduce) count_holders(p, cx, pf, unr);
+        if (p.is_allreduce && !decoded) count_holders(p, cx, pf, unr);
         const uint32_t root = cx->root, sstar = cx->sstar, G = cx->G;
-        // a row's value after up-correction (Algorithm "Up-correction") from its staged copy
+        // a row's value after up-correction (Algorithm "Up-correction") from its staged copy: folded as a plain group at once
+        // (the loads do not wait for the row's mask), and once more by the general rules where the group is not plain
         auto fold_row = [&](const char* srow_lc, const char* in_lc, uint32_t row) -> uint4 {
-            if (group_is_plain(p, root, inc, row)) return fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdShared(), p.pdesc != 0);
+            const uint4 v = fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdShared(), p.pdesc != 0);
+            if (group_is_plain(p, root, inc, row)) return v;
             return fold_staged_call<T, OP, false>(fold_shape(p), root, sstar, inc, in_lc, srow_lc, row);
         };
 
@@ -228,15 +269,25 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) aheap_kernel(Params p, c
 #endif
 constexpr uint64_t kAheapTileBytes = FTC_AHEAP_TILE_KB * 1024;   // a warp's buffer: forests are sized to fill it
 constexpr size_t kAheapMaxHeapBytes = 96 * 1024;                 // the block's heap array (levels 0 .. Lt)
+constexpr size_t kAheapSmallHeapBytes = 32 * 1024;               // a heap array that leaves the buffers room
+#ifndef FTC_AHEAP_MAX_WARPS
+#define FTC_AHEAP_MAX_WARPS 8
+#endif
+#ifndef FTC_AHEAP_ITEMS_PER_WARP
+#define FTC_AHEAP_ITEMS_PER_WARP 4
+#endif
+constexpr uint32_t kAheapMaxWarps = FTC_AHEAP_MAX_WARPS;
+constexpr uint32_t kAheapItemsPerWarp = FTC_AHEAP_ITEMS_PER_WARP; // a block gets a further warp only if each then has this many items a scenario
 
-static bool aheap_geometry(Params& p, int smem_optin, AheapGeom& g) {
+// The geometry for one buffer size; `inflight` = bytes of buffers the blocks of an SM hold together.
+static bool aheap_geometry_at(Params& p, int smem_optin, AheapGeom& g, uint64_t tile_bytes, uint64_t& inflight) {
     if (p.kbytes % 16 || p.arity < 2) return false;
     const uint32_t C = p.kbytes / 16, a = p.arity;
     if (C == 0 || C > 32 || (C & (C - 1))) return false;
     uint32_t cwl = 0; while ((1u << cwl) < C) ++cwl;
     p.C = C; p.cw_log2 = cwl;
     const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
-    const uint64_t budget = kAheapTileBytes > rowbytes ? kAheapTileBytes : rowbytes;
+    const uint64_t budget = tile_bytes > rowbytes ? tile_bytes : rowbytes;
     // levels of the heap: first row of each level
     uint32_t Hmax = 0; uint64_t start = 0, width = 1;
     g.lstart[0] = 0;
@@ -259,7 +310,10 @@ static bool aheap_geometry(Params& p, int smem_optin, AheapGeom& g) {
     g.nA = (uint32_t)((nlast + per_root_last - 1) / per_root_last);
     g.nroots = D == 1 ? g.nA : (uint32_t)nroots;
     g.n1 = (uint32_t)(budget / (R * rowbytes)); if (g.n1 < 1) g.n1 = 1;
-    g.n2 = Rshallow ? (uint32_t)(budget / (Rshallow * rowbytes)) : 1; if (g.n2 < 1) g.n2 = 1;
+    g.n2 = Rshallow ? (uint32_t)(budget / (Rshallow * rowbytes)) : 1;
+    // where the deep forests hold most of the rows the buffer is sized for them: no larger shallow forests
+    if (Rshallow && (uint64_t)g.nA * R >= (g.nroots - g.nA) * Rshallow && g.n2 * Rshallow > g.n1 * R) g.n2 = (uint32_t)(g.n1 * R / Rshallow);
+    if (g.n2 < 1) g.n2 = 1;
     g.itemsA = (g.nA + g.n1 - 1) / g.n1;
     g.itemsB = (g.nroots - g.nA + g.n2 - 1) / g.n2;
     uint64_t cap_rows = g.n1 * R; if (g.n2 * Rshallow > cap_rows) cap_rows = g.n2 * Rshallow;
@@ -270,19 +324,47 @@ static bool aheap_geometry(Params& p, int smem_optin, AheapGeom& g) {
     if (hv_bytes > kAheapMaxHeapBytes) return false;
     g.tile_cap = (uint32_t)((cap_rows * rowbytes + 127) & ~(uint64_t)127);
     const uint32_t nitems = g.itemsA + g.itemsB + g.ngroups + 1;
-    uint32_t warps = 1;
-    while (warps < 8 && warps * 2 * 4 <= nitems) warps *= 2;
     size_t o = sizeof(Ctx) + 3 * (size_t)(p.W + 1) * 4;
     o = (o + 15) & ~(size_t)15; g.off_rootv = (uint32_t)o; o += (size_t)C * 16;
     g.off_hv = (uint32_t)o; o += hv_bytes;
     g.off_bar = (uint32_t)o; o += 8 * 8;
     g.off_gaveup = (uint32_t)o; o += 8;
     o = (o + 127) & ~(size_t)127; g.off_tiles = (uint32_t)o;
-    while (warps > 1 && o + (size_t)warps * g.tile_cap > (size_t)smem_optin - 1024) warps /= 2;
+    // Warps per block: what counts is how many buffers the blocks of an SM keep in flight together (each warp waits for
+    // its one buffer, folds it and asks for the next), so take the count that fits the most, among those that leave every
+    // warp a few items per scenario; on a tie the smaller blocks, whose decodes overlap the others' streaming.
+    const size_t per_sm = (size_t)smem_optin + 1024, limit = (size_t)smem_optin - 1024;
+    uint32_t warps = 0, best = 0;
+    for (uint32_t w = 1; w <= kAheapMaxWarps; ++w) {
+        const size_t block = o + (size_t)w * g.tile_cap;
+        if (block > limit) break;
+        if (w > 1 && w * kAheapItemsPerWarp > nitems) break;
+        size_t blocks = per_sm / (block + 1024);
+        const size_t by_regs = kAheapWarpsPerSM / w, by_slots = 32;
+        if (blocks > by_regs) blocks = by_regs;
+        if (blocks > by_slots) blocks = by_slots;
+        if (blocks * w > best) { best = (uint32_t)(blocks * w); warps = w; }
+    }
+    if (!warps) return false;
     o += (size_t)warps * g.tile_cap;
-    if (o > (size_t)smem_optin - 1024) return false;
     g.nwarps = warps; g.smem_bytes = (uint32_t)o;
+    inflight = (uint64_t)best * g.tile_cap;
     return true;
+}
+
+// Buffer size: a larger buffer can take forests one level deeper, which divides the forests' roots -- and with them the
+// block's heap array -- by the arity. The smallest size whose heap array leaves most of the shared memory to the buffers
+// is taken; where none does, the size that keeps the most bytes in flight.
+static bool aheap_geometry(Params& p, int smem_optin, AheapGeom& g) {
+    bool found = false; uint64_t best = 0;
+    for (uint64_t tile = kAheapTileBytes; tile <= kAheapTileBytes + 12 * 1024; tile += 4 * 1024) {
+        AheapGeom t; Params q = p; uint64_t inflight = 0;
+        if (!aheap_geometry_at(q, smem_optin, t, tile, inflight)) continue;
+        const size_t hv_bytes = (size_t)t.nheap * q.C * 16;
+        if (hv_bytes <= kAheapSmallHeapBytes) { p = q; g = t; return true; }
+        if (!found || inflight > best) { found = true; best = inflight; p = q; g = t; }
+    }
+    return found;
 }
 
 template <typename T, int OP>

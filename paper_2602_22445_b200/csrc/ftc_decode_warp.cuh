@@ -115,7 +115,7 @@ __device__ __forceinline__ void decode_group(const Params& p, uint32_t pfw, uint
     uint32_t j = 0, sv = 0;
     if (INOP && vren) {
         j = div_m(p, vren - 1); sv = (vren - 1) - j * p.m;
-        const uint32_t d = 1 + ilog2u(j + 1);
+        const uint32_t d = 1 + heap_level(p.arity, j);
         if (!(p.f + p.H - d < t)) F |= 1u << sv;
     }
     F = g.any_or(F);

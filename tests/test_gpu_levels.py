@@ -22,9 +22,10 @@ SHAPES = [
 ]
 
 
-# (arity, P) of SHAPES whose heap array (the rows of all levels down to the tiles' roots) exceeds the kernel's shared-memory
-# budget, as the shape with P = 30011 and 256-byte vectors does at every arity: the general kernel plays those
-TOO_WIDE = {(5, 4096), (32, 4096), (8, 65536)}
+# The shape with P = 30011 and 256-byte vectors has a heap array (the rows of all levels down to the tiles' roots) beyond the
+# kernel's shared-memory budget at every arity: the general kernel plays it. (4096 processes at arity 5 or 32 and 65536 at
+# arity 8 fit only because the kernel may take a larger buffer to make its forests one level deeper.)
+TOO_WIDE = set()
 
 
 @pytest.mark.parametrize("arity", [2, 3, 4, 5, 8, 32])
