@@ -306,7 +306,7 @@ class Leg:
         self.tdt = getattr(torch, np.dtype(w.dtype).name)
         kflags = {"auto": 0, "direct": B.FTC_KERNEL_DIRECT, "generic": B.FTC_KERNEL_GENERIC, "levels": B.FTC_KERNEL_LEVELS}[args.kernel]
         if args.arity:
-            kflags |= B.FTC_TREE_ARITY(args.arity)
+            kflags |= B.FTC_TREE_BINOMIAL if args.arity == 1 else B.FTC_TREE_ARITY(args.arity)
         self.desc = B.make_desc(w.P, w.f, w.k, B.dtype_code(self.tdt), w.op, root=-1 if w.roots is not None else 0,
                                 max_inop=0 if w.inop is None else w.inop.shape[1], flags=kflags)
         self.fn = B.ftc_allreduce_batch if self.allred else B.ftc_reduce_batch
@@ -671,7 +671,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="scenarios per step per GPU")
     ap.add_argument("--e2e-scenarios", type=int, default=0)
     ap.add_argument("--kernel", default="auto", choices=["auto", "direct", "generic", "levels"], help="force a kernel family")
-    ap.add_argument("--arity", type=int, default=0, help="subtrees below the root's children as a-ary heaps (diagnostic: 0 = the binary heap of the configurations)")
+    ap.add_argument("--arity", type=int, default=0, help="subtrees below the root's children as a-ary heaps, 1 = binomial trees (diagnostic: 0 = the binary heap of the configurations)")
     ap.add_argument("--collective", default="", choices=["", "reduce", "allreduce"], help="override the workload's collective")
     ap.add_argument("--failure-free", action="store_true", help="clear every failure of the workload (diagnostic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -55,6 +55,7 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
     const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
     const uint32_t a = p.arity, C = p.C, cwl = p.cw_log2, Cmask = C - 1;
     const uint32_t D = g.D, Lt = g.Lt, ntop = g.ntop;
+    const bool binom = a == 1;                                         // binomial subtrees: D = log2 of a tile's rows
     const uint32_t itemsAB = g.itemsA + g.itemsB, nitems = itemsAB + g.ngroups + 1;
     const uint32_t rowbytes = p.m * p.kbytes;
     const uint64_t scen_bytes = (uint64_t)p.P * p.kbytes;
@@ -80,12 +81,14 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
     const char* is_src = reinterpret_cast<const char*>(p.in) + is_s * scen_bytes;
     uint32_t is_i = 0;
     uint32_t my_pw = 0, my_ts = 0, my_ls = 0;                         // lane u < D copies level u of a forest
-    if (lane < D) { my_pw = g.apow[lane]; my_ts = g.tstart[lane]; my_ls = g.lstart[Lt + lane]; }
+    if (!binom && lane < D) { my_pw = g.apow[lane]; my_ts = g.tstart[lane]; my_ls = g.lstart[Lt + lane]; }
     auto issue_next = [&]() {
         if (n_my == 0 || is_s >= p.S || stop) return;
         const uint32_t it = wid + is_i * nw;
         uint64_t first_row = 0; uint32_t nrows = 0, dst_off = 0;
-        if (it < itemsAB) {
+        if (binom) {
+            if (it < itemsAB && lane == 0) { first_row = (uint64_t)it << D; nrows = 1u << D; }
+        } else if (it < itemsAB) {
             uint32_t x0, n, d; forest(it, x0, n, d);
             if (lane < d) { first_row = (uint64_t)my_ls + (uint64_t)x0 * my_pw; nrows = n * my_pw; dst_off = n * my_ts * rowbytes; }
         } else if (it < itemsAB + g.ngroups) {
@@ -182,7 +185,31 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
         for (uint32_t i = 0; i < n_my; ++i) {
             const uint32_t it = wid + i * nw;
             acquire();
-            if (it < itemsAB) {
+            if (binom && it < itemsAB) {
+                // rows [it * 2^D, (it + 1) * 2^D) are the binomial subtree of the tile's first row: node x takes its children
+                // x + 1, x + 2, x + 4, ... in that order, each complete before it is taken (it ends on fewer zero bits)
+                const uint32_t r0 = it << D, nr = 1u << D;
+                if (r0 < G) {
+                    for (uint32_t u = lane; u < (nr << cwl); u += 32) {
+                        const uint32_t t = u >> cwl, c = u & Cmask;
+                        if (r0 + t >= G) continue;
+                        char* srow = tile + (size_t)t * rowbytes + c * 16;
+                        *reinterpret_cast<uint4*>(srow) = fold_row(srow, in_s + c * 16, r0 + t);
+                    }
+                    __syncwarp();
+                    for (uint32_t i = 0; i < D; ++i) {
+                        for (uint32_t u = lane; u < ((nr >> (i + 1)) << cwl); u += 32) {
+                            const uint32_t x = (u >> cwl) << (i + 1), c = u & Cmask;
+                            if (r0 + x + (1u << i) >= G) continue;
+                            char* mine = tile + (size_t)x * rowbytes + c * 16;
+                            const uint4 child = *reinterpret_cast<const uint4*>(mine + ((size_t)rowbytes << i));
+                            *reinterpret_cast<uint4*>(mine) = comb16<T, OP>(*reinterpret_cast<const uint4*>(mine), child);
+                        }
+                        __syncwarp();
+                    }
+                    if (lane < C) hv[(size_t)it * C + lane] = *reinterpret_cast<const uint4*>(tile + lane * 16);
+                }
+            } else if (it < itemsAB) {
                 uint32_t x0, n, d; forest(it, x0, n, d);
                 // local node t of forest level l is row rb_l + t; level l starts at local node th_l
                 const uint32_t th1 = d > 1 ? n * g.tstart[1] : 0xFFFFFFFFu, th2 = d > 2 ? n * g.tstart[2] : 0xFFFFFFFFu,
@@ -234,6 +261,17 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
             release();
         }
         __syncthreads();
+        // ---- binomial subtrees: the tiles' first rows form a binomial tree on the tile index ----
+        if (binom) {
+            const uint32_t used = (G + (1u << D) - 1) >> D;
+            for (uint32_t i = 0; (1u << i) < used; ++i) {
+                for (uint32_t u = tid; u < (((used >> (i + 1)) + 1) << cwl); u += nt) {
+                    const uint32_t X = (u >> cwl) << (i + 1), Y = X + (1u << i), c = u & Cmask;
+                    if (Y < used) hv[(size_t)X * C + c] = comb16<T, OP>(hv[(size_t)X * C + c], hv[(size_t)Y * C + c]);
+                }
+                __syncthreads();
+            }
+        }
         // ---- levels above the forests, leaves first ----
         for (int lvl = (int)Lt - 1; lvl >= 0; --lvl) {
             const uint32_t lo = g.lstart[lvl], n = g.lstart[lvl + 1] - lo;
@@ -281,45 +319,60 @@ constexpr uint32_t kAheapItemsPerWarp = FTC_AHEAP_ITEMS_PER_WARP; // a block get
 
 // The geometry for one buffer size; `inflight` = bytes of buffers the blocks of an SM hold together.
 static bool aheap_geometry_at(Params& p, int smem_optin, AheapGeom& g, uint64_t tile_bytes, uint64_t& inflight) {
-    if (p.kbytes % 16 || p.arity < 2) return false;
+    if (p.kbytes % 16 || p.arity < 1) return false;
     const uint32_t C = p.kbytes / 16, a = p.arity;
     if (C == 0 || C > 32 || (C & (C - 1))) return false;
     uint32_t cwl = 0; while ((1u << cwl) < C) ++cwl;
     p.C = C; p.cw_log2 = cwl;
     const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
     const uint64_t budget = tile_bytes > rowbytes ? tile_bytes : rowbytes;
-    // levels of the heap: first row of each level
-    uint32_t Hmax = 0; uint64_t start = 0, width = 1;
-    g.lstart[0] = 0;
-    while (start < p.Gmax) {
-        start += width; width *= a; ++Hmax;
-        if (Hmax + 4 > kAheapMaxLevels) return false;
-        g.lstart[Hmax] = (uint32_t)(start < 0xFFFFFFFFull ? start : 0xFFFFFFFFull);
+    uint64_t cap_rows = 0;
+    if (a == 1) {
+        // binomial subtrees: a tile is 2^D rows starting at a multiple of 2^D (the binomial subtree of its first row), one
+        // contiguous run; the tiles' first rows form a binomial tree again, on the tile index
+        uint32_t t = 0;
+        while (t < 12 && ((uint64_t)2 << t) * rowbytes <= budget && ((uint64_t)1 << t) < p.Gmax) ++t;
+        const uint64_t ntiles = ((uint64_t)p.Gmax + ((uint64_t)1 << t) - 1) >> t;
+        if (ntiles > (1u << 20)) return false;
+        for (uint32_t l = 0; l <= kAheapMaxLevels; ++l) g.lstart[l] = 0;
+        for (uint32_t u = 0; u < 5; ++u) { g.tstart[u] = 0; g.apow[u] = 0; }
+        g.D = t; g.Lt = 0; g.n1 = 1u << t; g.n2 = 1; g.nA = g.nroots = (uint32_t)ntiles;
+        g.itemsA = (uint32_t)ntiles; g.itemsB = 0; g.ngroups = 0; g.ntop = 0; g.nheap = (uint32_t)ntiles;
+        cap_rows = (uint64_t)1 << t; g.cap_rows = (uint32_t)cap_rows;
+    } else {
+        // levels of the heap: first row of each level
+        uint32_t Hmax = 0; uint64_t start = 0, width = 1;
+        g.lstart[0] = 0;
+        while (start < p.Gmax) {
+            start += width; width *= a; ++Hmax;
+            if (Hmax + 4 > kAheapMaxLevels) return false;
+            g.lstart[Hmax] = (uint32_t)(start < 0xFFFFFFFFull ? start : 0xFFFFFFFFull);
+        }
+        for (uint32_t l = Hmax + 1; l <= kAheapMaxLevels; ++l) g.lstart[l] = 0xFFFFFFFFu;
+        // the deepest forest of one root within the budget (at most four levels)
+        uint32_t D = 1; uint64_t R = 1, w = a;
+        while (D < 4 && D < Hmax && (R + w) * rowbytes <= budget) { R += w; w *= a; ++D; }
+        { uint64_t s0 = 0, pw = 1; for (uint32_t u = 0; u < 5; ++u) { g.tstart[u] = (uint32_t)s0; g.apow[u] = (uint32_t)pw; s0 += pw; pw *= a; } }
+        g.D = D; g.Lt = Hmax - D;
+        const uint64_t Rshallow = g.tstart[D - 1];                                   // rows of a root with D - 1 levels (0: D = 1)
+        uint64_t nroots = 1; for (uint32_t l = 0; l < g.Lt; ++l) nroots *= a;
+        if (nroots > (1u << 20)) return false;
+        const uint64_t nlast = p.Gmax - g.lstart[Hmax - 1];                          // rows on the heap's last level
+        const uint64_t per_root_last = g.apow[D - 1];
+        g.nA = (uint32_t)((nlast + per_root_last - 1) / per_root_last);
+        g.nroots = D == 1 ? g.nA : (uint32_t)nroots;
+        g.n1 = (uint32_t)(budget / (R * rowbytes)); if (g.n1 < 1) g.n1 = 1;
+        g.n2 = Rshallow ? (uint32_t)(budget / (Rshallow * rowbytes)) : 1;
+        // where the deep forests hold most of the rows the buffer is sized for them: no larger shallow forests
+        if (Rshallow && (uint64_t)g.nA * R >= (g.nroots - g.nA) * Rshallow && g.n2 * Rshallow > g.n1 * R) g.n2 = (uint32_t)(g.n1 * R / Rshallow);
+        if (g.n2 < 1) g.n2 = 1;
+        g.itemsA = (g.nA + g.n1 - 1) / g.n1;
+        g.itemsB = (g.nroots - g.nA + g.n2 - 1) / g.n2;
+        cap_rows = g.n1 * R; if (g.n2 * Rshallow > cap_rows) cap_rows = g.n2 * Rshallow;
+        g.cap_rows = (uint32_t)cap_rows;
+        g.ntop = g.lstart[g.Lt]; g.nheap = g.ntop + (uint32_t)nroots;
+        g.ngroups = (g.ntop + g.cap_rows - 1) / g.cap_rows;
     }
-    for (uint32_t l = Hmax + 1; l <= kAheapMaxLevels; ++l) g.lstart[l] = 0xFFFFFFFFu;
-    // the deepest forest of one root within the budget (at most four levels)
-    uint32_t D = 1; uint64_t R = 1, w = a;
-    while (D < 4 && D < Hmax && (R + w) * rowbytes <= budget) { R += w; w *= a; ++D; }
-    { uint64_t s0 = 0, pw = 1; for (uint32_t u = 0; u < 5; ++u) { g.tstart[u] = (uint32_t)s0; g.apow[u] = (uint32_t)pw; s0 += pw; pw *= a; } }
-    g.D = D; g.Lt = Hmax - D;
-    const uint64_t Rshallow = g.tstart[D - 1];                                   // rows of a root with D - 1 levels (0: D = 1)
-    uint64_t nroots = 1; for (uint32_t l = 0; l < g.Lt; ++l) nroots *= a;
-    if (nroots > (1u << 20)) return false;
-    const uint64_t nlast = p.Gmax - g.lstart[Hmax - 1];                          // rows on the heap's last level
-    const uint64_t per_root_last = g.apow[D - 1];
-    g.nA = (uint32_t)((nlast + per_root_last - 1) / per_root_last);
-    g.nroots = D == 1 ? g.nA : (uint32_t)nroots;
-    g.n1 = (uint32_t)(budget / (R * rowbytes)); if (g.n1 < 1) g.n1 = 1;
-    g.n2 = Rshallow ? (uint32_t)(budget / (Rshallow * rowbytes)) : 1;
-    // where the deep forests hold most of the rows the buffer is sized for them: no larger shallow forests
-    if (Rshallow && (uint64_t)g.nA * R >= (g.nroots - g.nA) * Rshallow && g.n2 * Rshallow > g.n1 * R) g.n2 = (uint32_t)(g.n1 * R / Rshallow);
-    if (g.n2 < 1) g.n2 = 1;
-    g.itemsA = (g.nA + g.n1 - 1) / g.n1;
-    g.itemsB = (g.nroots - g.nA + g.n2 - 1) / g.n2;
-    uint64_t cap_rows = g.n1 * R; if (g.n2 * Rshallow > cap_rows) cap_rows = g.n2 * Rshallow;
-    g.cap_rows = (uint32_t)cap_rows;
-    g.ntop = g.lstart[g.Lt]; g.nheap = g.ntop + (uint32_t)nroots;
-    g.ngroups = (g.ntop + g.cap_rows - 1) / g.cap_rows;
     const size_t hv_bytes = (size_t)g.nheap * C * 16;
     if (hv_bytes > kAheapMaxHeapBytes) return false;
     g.tile_cap = (uint32_t)((cap_rows * rowbytes + 127) & ~(uint64_t)127);

@@ -80,7 +80,7 @@ static const DeviceInfo kB200 = {148, 232448};
 enum KernelKind { K_GENERIC = 0, K_TILED = 1, K_STAGED = 2, K_LEVELS = 3 };
 static KernelKind pick_kernel(Params& p, const DeviceInfo& di) {
     if (p.flags & FTC_KERNEL_GENERIC) return K_GENERIC;
-    if (p.arity > 2 || (p.arity == 2 && (p.flags & FTC_KERNEL_LEVELS)))      // heaps of any arity: tiles evaluated level by level
+    if (p.arity != 2 || (p.flags & FTC_KERNEL_LEVELS))                       // heaps of any arity, binomial trees: tiles evaluated level by level
         if (aheap_supported(p, di.smem_optin)) return K_LEVELS;
     if (p.arity != 2) return K_GENERIC;                                      // the register-tiled kernels are built on the binary heap
     if (!(p.flags & FTC_KERNEL_DIRECT) && staged_supported(p, di.smem_optin, di.sm_count)) return K_STAGED;

@@ -41,7 +41,7 @@ def test_host_only_calls():
     assert (t["H"], t["rounds_reduce"], t["rounds_attempt"]) == (5, 8, 16)       # 256 rows: levels of 1, 4, 16, 64, 171
     assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(3))) == "levels"
     assert B.ftc_kernel_name(B.make_desc(4096, 4, 3, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(3))) == "generic"
-    assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_BINOMIAL)) == "generic"
+    assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_BINOMIAL)) == "levels"
     assert B.ftc_kernel_name(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_KERNEL_LEVELS)) == "levels"
     assert B.ftc_workspace_bytes(B.make_desc(4096, 4, 32, B.FTC_I32, "max", flags=B.FTC_TREE_ARITY(3)), 1000, True) == 0
     assert B.ftc_kernel_name(B.make_desc(8, 1, 1, B.FTC_I32, "sum", flags=B.FTC_TREE_ARITY(1))) == "invalid"

@@ -1,5 +1,6 @@
 """GPU parity for the level kernel (shared-memory tiles evaluated level by level), which plays subtrees that are a-ary heaps
-of arity 3 and more, and binary heaps on request: against the CPU oracle playing the same shape, bit for bit."""
+of arity 3 and more, binomial trees (arity 1 here, the oracle's code for them), and binary heaps on request: against the CPU
+oracle playing the same shape, bit for bit."""
 import numpy as np
 import pytest
 
@@ -11,7 +12,7 @@ pytestmark = pytest.mark.gpu
 
 
 def flags_for(arity):
-    return B.FTC_KERNEL_LEVELS if arity == 2 else B.FTC_TREE_ARITY(arity)
+    return B.FTC_KERNEL_LEVELS if arity == 2 else B.FTC_TREE_BINOMIAL if arity == 1 else B.FTC_TREE_ARITY(arity)
 
 
 SHAPES = [
@@ -28,7 +29,7 @@ SHAPES = [
 TOO_WIDE = set()
 
 
-@pytest.mark.parametrize("arity", [2, 3, 4, 5, 8, 32])
+@pytest.mark.parametrize("arity", [1, 2, 3, 4, 5, 8, 32])
 @pytest.mark.parametrize("P,f,k,dname,op", SHAPES)
 def test_level_kernel_matches_the_oracle(arity, P, f, k, dname, op):
     S = max(3, min(40, int(4e6 // (P * k))))
@@ -40,7 +41,7 @@ def test_level_kernel_matches_the_oracle(arity, P, f, k, dname, op):
         assert_same(got, run_oracle_mt(x, f, op, pf, inop, roots, 0, allreduce, arity=arity), f"P={P} f={f} k={k} {dname} {op} arity={arity} allreduce={allreduce}")
 
 
-@pytest.mark.parametrize("arity", [3, 4])
+@pytest.mark.parametrize("arity", [1, 3, 4])
 def test_level_kernel_with_descending_partners(arity):
     for P, f, k in ((150, 3, 16), (4099, 4, 8)):
         d_x, x, pf, inop, roots = make_batch(P, f, k, "f32", True, 30, seed=P)
@@ -53,12 +54,14 @@ def test_shapes_the_level_kernel_leaves_to_the_general_one():
     for k, dt in ((3, B.FTC_F32), (6, B.FTC_I32), (1, B.FTC_U64)):            # not a power-of-two number of 16-byte chunks
         assert B.ftc_kernel_name(B.make_desc(100, 2, k, dt, "sum", flags=B.FTC_TREE_ARITY(4)), True) == "generic"
     assert B.ftc_kernel_name(B.make_desc(100, 2, 4, B.FTC_I32, "sum", flags=B.FTC_TREE_ARITY(4) | B.FTC_KERNEL_GENERIC), True) == "generic"
-    assert B.ftc_kernel_name(B.make_desc(100, 2, 4, B.FTC_I32, "sum", flags=B.FTC_TREE_BINOMIAL), True) == "generic"
+    assert B.ftc_kernel_name(B.make_desc(100, 2, 6, B.FTC_I32, "sum", flags=B.FTC_TREE_BINOMIAL), True) == "generic"
+    assert B.ftc_kernel_name(B.make_desc(100, 2, 4, B.FTC_I32, "sum", flags=B.FTC_TREE_BINOMIAL), True) == "levels"
     assert B.ftc_kernel_name(B.make_desc(100, 2, 4, B.FTC_I32, "sum"), True) == "staged"
 
 
 @pytest.mark.parametrize("arity,P,f,k,dname,op,allreduce", [(4, 4096, 4, 32, "i32", "max", True), (3, 1024, 3, 16, "f32", "sum", True),
-                                                            (8, 16384, 1, 8, "i32", "sum", False), (2, 150, 3, 16, "f32", "sum", True)])
+                                                            (8, 16384, 1, 8, "i32", "sum", False), (2, 150, 3, 16, "f32", "sum", True),
+                                                            (1, 5000, 2, 8, "i64", "max", True)])
 def test_level_kernel_gives_up_cleanly(arity, P, f, k, dname, op, allreduce):
     """With FTC_DEBUG_ONE_POLL the waits for the asynchronous copies look once and give up: a scenario is then either
     played correctly or reports FTC_ST_INTERNAL_TIMEOUT with zero bytes, a block that reported it does so for all its

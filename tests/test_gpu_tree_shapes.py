@@ -43,7 +43,7 @@ def test_exhaustive_failure_sets_small_P(arity, allreduce):
             x = rng.integers(0, 2**64, size=(len(sets), P, 2), dtype=np.uint64)
             pf = sc.sets_to_masks(sets, P)
             got = run_gpu(x, f, "sum", pf, None, roots, 0, allreduce, shape_flags(arity))
-            assert B.ftc_kernel_name(got[2], allreduce) == ("generic" if arity == 1 else "levels")
+            assert B.ftc_kernel_name(got[2], allreduce) == "levels"
             want = run_oracle(x, f, "sum", pf, None, roots, 0, allreduce, arity)
             assert_same(got, want, f"P={P} f={f} arity={arity}")
 
@@ -169,7 +169,7 @@ def test_descending_partners(arity, allreduce):
         inop[:, 0, 0] = [c[1] for c in cases]
         inop[:, 0, 1] = [c[2] for c in cases]
         got = run_gpu(x, f, "sum", pf, inop, None, 0, allreduce, flags)
-        assert B.ftc_kernel_name(got[2], allreduce) == {2: "staged", 3: "levels", 1: "generic"}[arity]    # heaps: the order is known to the shared-memory kernels
+        assert B.ftc_kernel_name(got[2], allreduce) == {2: "staged", 3: "levels", 1: "levels"}[arity]    # the order is known to the shared-memory kernels
         assert_same(got, run_oracle(x, f, "sum", pf, inop, None, 0, allreduce, arity, True), f"P={P} f={f} arity={arity}")
     # float32 bit for bit, random failures and roots, expanded output and message counts
     import torch
