@@ -400,9 +400,12 @@ def add_sustained(roof, leg, torch, sampler, seconds):
                          "sm_mhz_median": mhz, "ms_x_mhz": (ms * mhz) if mhz else None, "clocks": clocks}
 
 
-def run_side_leg(name, args, B, torch, sampler, peak, peak_kind, candidates=False):
+def run_side_leg(name, args, B, torch, sampler, peak, peak_kind, candidates=False, arity=0):
     """One more workload, timed like the headline one: K steps, then a sustained run; its own roofline record.
-    candidates: what every root child delivers (ftc_candidates_batch) instead of the batch call."""
+    candidates: what every root child delivers (ftc_candidates_batch) instead of the batch call.
+    arity: another subtree shape below the root's children (a-ary heaps; 1 = binomial trees) on the same inputs."""
+    if arity:
+        args = argparse.Namespace(**{**vars(args), "arity": arity})
     S = (args.batch if args.candidates and args.batch else 0) or DEFAULT_BATCH[name]
     leg = Leg(name, S, 0, args, B, torch, 28, candidates=candidates)
     for _ in range(max(args.warmup, 3)):
@@ -415,7 +418,8 @@ def run_side_leg(name, args, B, torch, sampler, peak, peak_kind, candidates=Fals
         roof["traffic"] = None
     add_sustained(roof, leg, torch, sampler, args.sustain_seconds / 2)
     ms = total_ms / args.steps
-    rec = {"workload": f"{name}: {DESCRIPTION[name]}" + (" [what every root child delivers: all f+1 subtrees played]" if candidates else ""),
+    shape = "" if not arity else " [subtrees: binomial trees]" if arity == 1 else f" [subtrees: {arity}-ary heaps]"
+    rec = {"workload": f"{name}: {DESCRIPTION[name]}" + (" [what every root child delivers: all f+1 subtrees played]" if candidates else "") + shape,
            "value": S / (ms / 1e3), "unit": "scenarios/s", "ms_per_step": ms,
            "steps": args.steps, "scenarios_per_step": S, "process_rounds_per_sec": S / (ms / 1e3) * leg.w.P * leg.rounds(),
            "dtype": np.dtype(leg.w.dtype).name, "roofline": roof, "clocks": clocks}
@@ -447,24 +451,23 @@ def read_only_ceiling(B, torch, d_x, steps):
     return out
 
 
-def run_full_config(args, B, torch, sampler, peak, peak_kind):
-    """Every batch of the configuration at its stated scenario count: per batch the inputs are regenerated on the device,
-    K steps are timed, and the batch is checked against the any-size properties; times are summed over the batches."""
+def full_config_pass(name, args, B, torch, peak, peak_kind, steps, batch=0):
+    """Every batch of configuration `name` at its stated scenario count: per batch the inputs are regenerated on the device,
+    `steps` steps are timed, and the batch is checked against the any-size properties; times are summed over the batches.
+    Returns (leg facts, sum of the batches' mean step times in ms, all step times, checks)."""
     from paper_2602_22445_b200 import verify
-    name = args.workload
     total = CONFIG_SCENARIOS[name]
-    S = args.batch or min(DEFAULT_BATCH[name], total)
+    S = batch or min(DEFAULT_BATCH[name], total)
     nb = (total + S - 1) // S
     leg = Leg(name, S, 0, args, B, torch, 28)
     sum_ms, all_ms, checks = 0.0, [], {"ok_scenarios": 0, "noop_scenarios": 0, "retried": 0, "excluded_pairs": 0}
-    m0 = sampler.lines() if sampler else 0
     for b in range(nb):
         if b:
             leg.regenerate(b * S, 28)
-        for _ in range(max(args.warmup, 3)):
+        for _ in range(3):
             leg.step()
-        per_ms, total_ms = time_steps(torch, leg.step, args.steps)
-        sum_ms += total_ms / args.steps
+        per_ms, total_ms = time_steps(torch, leg.step, steps)
+        sum_ms += total_ms / steps
         all_ms += per_ms
         st = leg.status()
         for k, v in verify.check_status_fields(leg.w, st).items():
@@ -473,18 +476,30 @@ def run_full_config(args, B, torch, sampler, peak, peak_kind):
         checks["excluded_pairs"] += rep["excluded_pairs"]
         if "worst_relative_error" in rep:
             checks["worst_relative_error"] = max(checks.get("worst_relative_error", 0.0), rep["worst_relative_error"])
+    facts = {"scenarios_total": nb * S, "batches": nb, "scenarios_per_batch": S, "bytes_per_launch": leg.bytes_per_launch,
+             "kernel": B.ftc_kernel_variant(leg.desc, leg.allred), "rounds": leg.rounds(), "P": leg.w.P, "f": leg.w.f,
+             "dtype": np.dtype(leg.w.dtype).name}
+    leg.free()
+    return facts, sum_ms, all_ms, checks
+
+
+def run_full_config(args, B, torch, sampler, peak, peak_kind):
+    """`--full-config`: one line for the whole configuration (see full_config_pass)."""
+    name = args.workload
+    facts, sum_ms, all_ms, checks = full_config_pass(name, args, B, torch, peak, peak_kind, args.steps, args.batch)
     clocks = sampler.stop() if sampler else None
-    roof = roofline_record(name, leg.bytes_per_launch, all_ms, S, peak, peak_kind)
+    nb, S = facts["batches"], facts["scenarios_per_batch"]
+    roof = roofline_record(name, facts["bytes_per_launch"], all_ms, S, peak, peak_kind)
     value = nb * S / (sum_ms / 1e3)
     line = {
         "metric": "scenarios_per_sec", "value": value, "unit": "scenarios/s", "n_gpus": 1, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": sum_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": {"int32": "i32", "int64": "i64", "uint64": "u64", "float32": "f32"}[np.dtype(leg.w.dtype).name], "data": "synthetic",
-        "process_rounds_per_sec": value * leg.w.P * leg.rounds(),
+        "dtype": {"int32": "i32", "int64": "i64", "uint64": "u64", "float32": "f32"}[facts["dtype"]], "data": "synthetic",
+        "process_rounds_per_sec": value * facts["P"] * facts["rounds"],
         "config": {"workload": f"{name}: {DESCRIPTION[name]} [whole configuration]", "scenarios_total": nb * S, "batches": nb,
                    "scenarios_per_batch": S, "step": "one pass over all batches (times of the batches summed)",
-                   "cache": "inputs larger than L2, no flush", "kernel": B.ftc_kernel_variant(leg.desc, leg.allred),
-                   "rounds_per_scenario": leg.rounds(), "subtrees_played": f"1 of {leg.w.f + 1}",
+                   "cache": "inputs larger than L2, no flush", "kernel": facts["kernel"],
+                   "rounds_per_scenario": facts["rounds"], "subtrees_played": f"1 of {facts['f'] + 1}",
                    "checked": "every scenario: outcome and counts from the masks, result by the plain definition (torch)", **checks},
         "roofline": roof, "cpu_baseline": None, "e2e": None, "gpu_launches": args.steps * nb, "clocks": clocks,
     }
@@ -593,7 +608,7 @@ def run_gpu(args):
         return
 
     launches = args.steps
-    workloads = {}
+    workloads, whole = {}, {}
     cpu = None
     if not args.kernel_only:
         # ---- the same step for seconds, with the clocks it ran at; and what a kernel that only reads can reach ----
@@ -626,10 +641,24 @@ def run_gpu(args):
             for other in [x for x in ("c5", "c5r", "c3", "c4", "c2") if x != name]:
                 workloads[other] = run_side_leg(other, args, B, torch, sampler, peak, peak_kind)
                 launches += args.steps + workloads[other]["roofline"]["sustained"]["steps"]
+            for other, ar, tag in (("c4", 4, "c4_4ary"), ("c4", 1, "c4_binomial")):     # other I(f)-tree shapes on the same inputs
+                workloads[tag] = run_side_leg(other, args, B, torch, sampler, peak, peak_kind, arity=ar)
+                workloads[tag]["roofline"]["traffic"] = None
+                launches += args.steps + workloads[tag]["roofline"]["sustained"]["steps"]
             for other in ("c4", "c5"):                      # all f+1 root children played (integer configurations)
                 key = other + "_all_children"
                 workloads[key] = run_side_leg(other, args, B, torch, sampler, peak, peak_kind, candidates=True)
                 launches += args.steps + workloads[key]["roofline"]["sustained"]["steps"]
+        # ---- the configurations at their stated scenario counts: every batch played and checked, times summed ----
+        if world == 1 and not args.no_legs and not args.no_whole:
+            for cfg in ("c4", "c5", "c3"):
+                facts, sum_ms, all_ms, checks = full_config_pass(cfg, args, B, torch, peak, peak_kind, 3)
+                gbs = facts["bytes_per_launch"] * facts["batches"] / (sum_ms / 1e3) / 1e9
+                whole[cfg] = {"scenarios_total": facts["scenarios_total"], "batches": facts["batches"], "steps_per_batch": 3,
+                              "ms_all_batches": sum_ms, "scenarios_per_sec": facts["scenarios_total"] / (sum_ms / 1e3),
+                              "achieved_gbs": gbs, "frac": gbs / peak, "kernel": facts["kernel"],
+                              "checked": "every scenario: outcome and counts from the masks, result by the plain definition (torch)", **checks}
+                launches += 6 * facts["batches"]
     if sampler:
         sampler.stop()
 
@@ -653,7 +682,7 @@ def run_gpu(args):
         "cpu_baseline": cpu,
         "e2e": e2e,
         "gpu_launches": args.steps,
-        "launches_all_legs": launches,
+        "whole_configurations": whole, "launches_all_legs": launches,
         "clocks": clocks,
     }
     print(json.dumps(line))
@@ -677,6 +706,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--kernel-only", action="store_true", help="skip the end-to-end, sustained, CPU and other-workload legs (for profiler runs)")
     ap.add_argument("--no-legs", action="store_true", help="skip the legs over the other configurations")
+    ap.add_argument("--no-whole", action="store_true", help="skip the pass over every batch of C3, C4 and C5 at their stated scenario counts")
     ap.add_argument("--sustain-seconds", type=float, default=2.0, help="GPU time of the sustained run of the headline workload")
     ap.add_argument("--candidates", action="store_true",
                     help="time ftc_candidates_batch (what every root child delivers: all f+1 subtrees) on the workload")

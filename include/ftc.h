@@ -29,7 +29,8 @@
  *     section "Properties"); within a subtree the nodes j = floor((v-1)/(f+1)) form a
  *     heap, binary unless FTC_TREE_ARITY(a) in the flags asks for a children per node: children a*j+1 .. a*j+a,
  *     received in that order, accumulator on the left (the paper's I(f)-tree fixes only the root's f+1 children
- *     and their subtree sizes; shapes other than binary run on the general kernel and need its workspace);
+ *     and their subtree sizes; heaps of other arities and binomial trees run on the level kernel in shared memory
+ *     where their shape fits it, else on the general kernel, which needs its workspace);
  *   - failure information is the single failed bit (third scheme of section "Failure
  *     information"); the root takes the lowest-numbered child that delivered with the
  *     bit clear (Algorithm "reduce_root");
@@ -112,13 +113,13 @@ typedef struct { uint32_t victim; uint32_t round; } ftc_inop_t;
 #define FTC_MAX_ARITY 32u
 #define FTC_TREE_BINOMIAL   0x1000000u /* subtrees below the root's children are binomial trees on the local index j: parent of j =
                                          j without its lowest set bit, children in ascending order, depth = 1 + set bits of j
-                                         (not together with FTC_TREE_ARITY; general kernel) */
+                                         (not together with FTC_TREE_ARITY) */
 #define FTC_PARTNERS_DESCENDING 0x2000000u /* up-correction (and the broadcast's correction) visits the group partners in descending
                                             rank, the root last, instead of ascending with the root first: the algorithm leaves the
-                                            order open (general kernel) */
+                                            order open (every kernel plays it) */
 #define FTC_KERNEL_GENERIC 0x100u /* force the general level-by-level kernel (needs the workspace) */
 #define FTC_KERNEL_LEVELS  0x400u /* binary heaps: take the level kernel (shared-memory tiles evaluated level by level), which heaps of
-                                     arity 3 and more use by default, where the shape allows it */
+                                     arity 3 and more and binomial trees use by default, where the shape allows it */
 #define FTC_KERNEL_DIRECT  0x200u /* force the register-tiled kernel (direct global loads) where the shape allows it */
 #define FTC_DEBUG_ONE_POLL 0x4000000u /* testing aid: the kernel's bounded waits for its asynchronous copies look once instead of
                                          polling, so most of them give up and the give-up path runs: affected scenarios report

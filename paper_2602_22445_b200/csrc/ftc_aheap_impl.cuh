@@ -11,6 +11,9 @@
 //   3. the tile's root goes to the block's heap array, which is combined level by level as in the staged kernel.
 // Each row decides by itself whether the plain fold from its staged copy serves it (a full group under its arrival mask)
 // or the general fold is needed (a renumbered slot, the short last group): no marking pass.
+// Binomial subtrees (FTC_TREE_BINOMIAL, arity 1 internally) run here too: a tile is 2^D rows from a multiple of 2^D, which
+// is the binomial subtree of its first row and one contiguous run; step 2 becomes D doubling steps, and step 3 the same
+// doubling steps on the tile index.
 #pragma once
 #include "ftc_staged_impl.cuh"
 #include "ftc_decode_warp.cuh"
