@@ -41,6 +41,7 @@ struct AheapGeom {
     uint32_t lstart[kAheapMaxLevels + 1];  // first row of heap level l: (a^l - 1) / (a - 1)
     uint32_t tstart[5], apow[5];           // a forest's level u per root: nodes above it, (a^u - 1) / (a - 1), and nodes on it, a^u
     uint32_t off_rootv, off_hv, off_bar, off_gaveup, off_tiles, smem_bytes;
+    uint32_t c_magic;                      // 0: the vector is a power-of-two number of 16-byte chunks; else ceil(2^32 / chunks)
 };
 
 template <typename T, int OP>
@@ -56,7 +57,12 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
     volatile uint32_t* gaveup = reinterpret_cast<volatile uint32_t*>(sbase + g.off_gaveup);
 
     const uint32_t tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, wid = tid >> 5, nw = nt >> 5;
-    const uint32_t a = p.arity, C = p.C, cwl = p.cw_log2, Cmask = C - 1;
+    const uint32_t a = p.arity, C = p.C;
+    // unit u of a run of rows = (row u / C, chunk u % C); C is a power of two (shift and mask) or not (multiply by the
+    // reciprocal g.c_magic = ceil(2^32 / C): exact for u below 2^26)
+    const uint32_t cwl = p.cw_log2, cmagic = g.c_magic;
+    auto urow = [&](uint32_t u) -> uint32_t { return cmagic ? __umulhi(u, cmagic) : u >> cwl; };
+    auto uchunk = [&](uint32_t u, uint32_t t) -> uint32_t { return u - t * C; };
     const uint32_t D = g.D, Lt = g.Lt, ntop = g.ntop;
     const bool binom = a == 1;                                         // binomial subtrees: D = log2 of a tile's rows
     const uint32_t itemsAB = g.itemsA + g.itemsB, nitems = itemsAB + g.ngroups + 1;
@@ -193,16 +199,16 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
                 // x + 1, x + 2, x + 4, ... in that order, each complete before it is taken (it ends on fewer zero bits)
                 const uint32_t r0 = it << D, nr = 1u << D;
                 if (r0 < G) {
-                    for (uint32_t u = lane; u < (nr << cwl); u += 32) {
-                        const uint32_t t = u >> cwl, c = u & Cmask;
+                    for (uint32_t u = lane; u < nr * C; u += 32) {
+                        const uint32_t t = urow(u), c = uchunk(u, t);
                         if (r0 + t >= G) continue;
                         char* srow = tile + (size_t)t * rowbytes + c * 16;
                         *reinterpret_cast<uint4*>(srow) = fold_row(srow, in_s + c * 16, r0 + t);
                     }
                     __syncwarp();
                     for (uint32_t i = 0; i < D; ++i) {
-                        for (uint32_t u = lane; u < ((nr >> (i + 1)) << cwl); u += 32) {
-                            const uint32_t x = (u >> cwl) << (i + 1), c = u & Cmask;
+                        for (uint32_t u = lane; u < (nr >> (i + 1)) * C; u += 32) {
+                            const uint32_t ur = urow(u), x = ur << (i + 1), c = uchunk(u, ur);
                             if (r0 + x + (1u << i) >= G) continue;
                             char* mine = tile + (size_t)x * rowbytes + c * 16;
                             const uint4 child = *reinterpret_cast<const uint4*>(mine + ((size_t)rowbytes << i));
@@ -221,9 +227,9 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
                                rb2 = g.lstart[Lt + 2] + x0 * g.apow[2] - th2, rb3 = g.lstart[Lt + 3] + x0 * g.apow[3] - th3;
                 if (rb0 < G) {
                     // 1. every (row, chunk) folds its group; the result takes the place of the row's first member
-                    const uint32_t units = (n * g.tstart[d]) << cwl;
+                    const uint32_t units = n * g.tstart[d] * C;
                     for (uint32_t u = lane; u < units; u += 32) {
-                        const uint32_t t = u >> cwl, c = u & Cmask;
+                        const uint32_t t = urow(u), c = uchunk(u, t);
                         const uint32_t row = t + (t >= th3 ? rb3 : t >= th2 ? rb2 : t >= th1 ? rb1 : rb0);
                         if (row >= G) continue;
                         char* srow = tile + (size_t)t * rowbytes + c * 16;
@@ -234,8 +240,8 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
                     for (int lv = (int)d - 2; lv >= 0; --lv) {
                         const uint32_t t0 = n * g.tstart[lv], t1 = n * g.tstart[lv + 1], nn = n * g.apow[lv];
                         const uint32_t rbl = g.lstart[Lt + lv] + x0 * g.apow[lv];
-                        for (uint32_t u = lane; u < (nn << cwl); u += 32) {
-                            const uint32_t pos = u >> cwl, c = u & Cmask, row = rbl + pos, first = a * row + 1;
+                        for (uint32_t u = lane; u < nn * C; u += 32) {
+                            const uint32_t pos = urow(u), c = uchunk(u, pos), row = rbl + pos, first = a * row + 1;
                             if (row >= G || first >= G) continue;
                             const uint32_t cnt = min(a, G - first);
                             char* mine = tile + (size_t)(t0 + pos) * rowbytes + c * 16;
@@ -247,14 +253,16 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
                         __syncwarp();
                     }
                     // 3. the forest's roots
-                    for (uint32_t u = lane; u < (n << cwl); u += 32)
-                        hv[(size_t)(rb0 + (u >> cwl)) * C + (u & Cmask)] = *reinterpret_cast<const uint4*>(tile + (size_t)(u >> cwl) * rowbytes + (u & Cmask) * 16);
+                    for (uint32_t u = lane; u < n * C; u += 32) {
+                        const uint32_t t = urow(u), c = uchunk(u, t);
+                        hv[(size_t)(rb0 + t) * C + c] = *reinterpret_cast<const uint4*>(tile + (size_t)t * rowbytes + c * 16);
+                    }
                 }
             } else if (it < itemsAB + g.ngroups) {
                 // rows above the forests: fold now, combine later
                 const uint32_t r0 = (it - itemsAB) * g.cap_rows;
-                for (uint32_t u = lane; u < (g.cap_rows << cwl); u += 32) {
-                    const uint32_t t = u >> cwl, c = u & Cmask, row = r0 + t;
+                for (uint32_t u = lane; u < g.cap_rows * C; u += 32) {
+                    const uint32_t t = urow(u), c = uchunk(u, t), row = r0 + t;
                     if (row >= ntop || row >= G) break;
                     hv[(size_t)row * C + c] = fold_row(tile + (size_t)t * rowbytes + c * 16, in_s + c * 16, row);
                 }
@@ -268,8 +276,8 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
         if (binom) {
             const uint32_t used = (G + (1u << D) - 1) >> D;
             for (uint32_t i = 0; (1u << i) < used; ++i) {
-                for (uint32_t u = tid; u < (((used >> (i + 1)) + 1) << cwl); u += nt) {
-                    const uint32_t X = (u >> cwl) << (i + 1), Y = X + (1u << i), c = u & Cmask;
+                for (uint32_t u = tid; u < ((used >> (i + 1)) + 1) * C; u += nt) {
+                    const uint32_t ur = urow(u), X = ur << (i + 1), Y = X + (1u << i), c = uchunk(u, ur);
                     if (Y < used) hv[(size_t)X * C + c] = comb16<T, OP>(hv[(size_t)X * C + c], hv[(size_t)Y * C + c]);
                 }
                 __syncthreads();
@@ -278,8 +286,8 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
         // ---- levels above the forests, leaves first ----
         for (int lvl = (int)Lt - 1; lvl >= 0; --lvl) {
             const uint32_t lo = g.lstart[lvl], n = g.lstart[lvl + 1] - lo;
-            for (uint32_t u = tid; u < (n << cwl); u += nt) {
-                const uint32_t row = lo + (u >> cwl), c = u & Cmask, first = a * row + 1;
+            for (uint32_t u = tid; u < n * C; u += nt) {
+                const uint32_t ur = urow(u), row = lo + ur, c = uchunk(u, ur), first = a * row + 1;
                 if (row >= G || first >= G) continue;
                 const uint32_t cnt = min(a, G - first);
                 uint4 v = hv[(size_t)row * C + c];
@@ -324,9 +332,10 @@ constexpr uint32_t kAheapItemsPerWarp = FTC_AHEAP_ITEMS_PER_WARP; // a block get
 static bool aheap_geometry_at(Params& p, int smem_optin, AheapGeom& g, uint64_t tile_bytes, uint64_t& inflight) {
     if (p.kbytes % 16 || p.arity < 1) return false;
     const uint32_t C = p.kbytes / 16, a = p.arity;
-    if (C == 0 || C > 32 || (C & (C - 1))) return false;
+    if (C == 0 || C > 32) return false;
     uint32_t cwl = 0; while ((1u << cwl) < C) ++cwl;
-    p.C = C; p.cw_log2 = cwl;
+    p.C = C; p.cw_log2 = cwl; p.swz_mask = 0; p.row_shift = 0;       // plain tiles
+    g.c_magic = (C & (C - 1)) ? (uint32_t)((((uint64_t)1 << 32) + C - 1) / C) : 0u;
     const uint64_t rowbytes = (uint64_t)p.m * p.kbytes;
     const uint64_t budget = tile_bytes > rowbytes ? tile_bytes : rowbytes;
     uint64_t cap_rows = 0;

@@ -84,7 +84,11 @@ static KernelKind pick_kernel(Params& p, const DeviceInfo& di) {
         if (aheap_supported(p, di.smem_optin)) return K_LEVELS;
     if (p.arity != 2) return K_GENERIC;                                      // the register-tiled kernels are built on the binary heap
     if (!(p.flags & FTC_KERNEL_DIRECT) && staged_supported(p, di.smem_optin, di.sm_count)) return K_STAGED;
-    return tiled_supported(p, di.smem_optin) ? K_TILED : K_GENERIC;
+    if (tiled_supported(p, di.smem_optin)) return K_TILED;
+    // vectors that are not a power-of-two number of 16-byte chunks: the register tiles cannot hold them, the level kernel can
+    const uint32_t chunks = p.kbytes / 16;
+    if (p.kbytes % 16 == 0 && (chunks & (chunks - 1)) && !(p.flags & FTC_KERNEL_DIRECT) && aheap_supported(p, di.smem_optin)) return K_LEVELS;
+    return K_GENERIC;
 }
 
 static size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }

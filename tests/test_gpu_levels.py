@@ -50,8 +50,28 @@ def test_level_kernel_with_descending_partners(arity):
         assert_same(got, run_oracle_mt(x, f, "sum", pf, inop, roots, 0, True, arity=arity, partners_descending=True), f"P={P} arity={arity}")
 
 
+WIDE_SHAPES = [
+    # vectors of 3, 5, 6 and 12 chunks of 16 bytes (not a power of two: the register tiles cannot hold them)
+    (300, 2, 12, "f32", "sum"), (4099, 4, 20, "i32", "max"), (1024, 3, 12, "u64", "xor"), (20011, 7, 6, "i64", "sum"), (700, 1, 48, "f32", "sum"),
+]
+
+
+@pytest.mark.parametrize("arity", [1, 2, 4])
+@pytest.mark.parametrize("P,f,k,dname,op", WIDE_SHAPES)
+def test_vectors_of_any_number_of_chunks(arity, P, f, k, dname, op):
+    """Vectors that are a multiple of 16 bytes but not a power-of-two number of chunks: binary heaps take the level kernel by
+    themselves here (no flag), the other shapes as always."""
+    S = max(3, min(40, int(4e6 // (P * k))))
+    flags = 0 if arity == 2 else flags_for(arity)
+    for allreduce in (False, True):
+        d_x, x, pf, inop, roots = make_batch(P, f, k, dname, allreduce, S, seed=arity * 77 + P + k)
+        got = run_gpu(None, f, op, pf, inop, roots, 0, allreduce, flags, d_x=d_x)
+        assert B.ftc_kernel_name(got[2], allreduce) == "levels"
+        assert_same(got, run_oracle_mt(x, f, op, pf, inop, roots, 0, allreduce, arity=arity), f"P={P} f={f} k={k} {dname} {op} arity={arity} allreduce={allreduce}")
+
+
 def test_shapes_the_level_kernel_leaves_to_the_general_one():
-    for k, dt in ((3, B.FTC_F32), (6, B.FTC_I32), (1, B.FTC_U64)):            # not a power-of-two number of 16-byte chunks
+    for k, dt in ((3, B.FTC_F32), (6, B.FTC_I32), (1, B.FTC_U64)):            # not a multiple of 16 bytes
         assert B.ftc_kernel_name(B.make_desc(100, 2, k, dt, "sum", flags=B.FTC_TREE_ARITY(4)), True) == "generic"
     assert B.ftc_kernel_name(B.make_desc(100, 2, 4, B.FTC_I32, "sum", flags=B.FTC_TREE_ARITY(4) | B.FTC_KERNEL_GENERIC), True) == "generic"
     assert B.ftc_kernel_name(B.make_desc(100, 2, 6, B.FTC_I32, "sum", flags=B.FTC_TREE_BINOMIAL), True) == "generic"

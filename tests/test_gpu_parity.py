@@ -162,12 +162,13 @@ def test_random_shapes_ops_and_failure_patterns(seed):
 
 
 def test_chunk_counts_up_to_32_and_beyond():
-    """k*elem = 16 B .. 512 B run on the tiled kernel, larger or odd sizes on the general one."""
+    """k*elem = 16 B .. 512 B in a power-of-two number of 16-byte chunks run on the staged tiles, other multiples of 16 bytes
+    (80 B here) on the level kernel, larger vectors and sizes that are no multiple of 16 bytes on the general one."""
     rng = np.random.Generator(np.random.PCG64(3))
     P, f, S = 300, 2, 16
     pf = sc.picks_to_masks(sc.random_subsets(rng, S, P, rng.integers(0, 3, size=S)), P)
     for k, kernel in ((4, "staged"), (8, "staged"), (16, "staged"), (32, "staged"), (64, "staged"), (128, "staged"),
-                      (256, "generic"), (20, "generic"), (5, "generic")):
+                      (256, "generic"), (20, "levels"), (5, "generic")):
         x = rng.integers(-2**31, 2**31 - 1, size=(S, P, k), dtype=np.int32)
         got = run_gpu(x, f, "max", pf)
         assert B.ftc_kernel_name(got[2]) == kernel
