@@ -44,7 +44,8 @@ struct AheapGeom {
     uint32_t c_magic;                      // 0: the vector is a power-of-two number of 16-byte chunks; else ceil(2^32 / chunks)
 };
 
-template <typename T, int OP>
+// NP2: the vector is not a power-of-two number of 16-byte chunks
+template <typename T, int OP, bool NP2>
 __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kernel(Params p, const __grid_constant__ AheapGeom g) {
     extern __shared__ __align__(128) uint32_t smem[];
     char* sbase = reinterpret_cast<char*>(smem);
@@ -61,8 +62,8 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
     // unit u of a run of rows = (row u / C, chunk u % C); C is a power of two (shift and mask) or not (multiply by the
     // reciprocal g.c_magic = ceil(2^32 / C): exact for u below 2^26)
     const uint32_t cwl = p.cw_log2, cmagic = g.c_magic;
-    auto urow = [&](uint32_t u) -> uint32_t { return cmagic ? __umulhi(u, cmagic) : u >> cwl; };
-    auto uchunk = [&](uint32_t u, uint32_t t) -> uint32_t { return u - t * C; };
+    auto urow = [&](uint32_t u) -> uint32_t { return NP2 ? __umulhi(u, cmagic) : u >> cwl; };
+    auto uchunk = [&](uint32_t u, uint32_t t) -> uint32_t { return NP2 ? u - t * C : u & (C - 1); };
     const uint32_t D = g.D, Lt = g.Lt, ntop = g.ntop;
     const bool binom = a == 1;                                         // binomial subtrees: D = log2 of a tile's rows
     const uint32_t itemsAB = g.itemsA + g.itemsB, nitems = itemsAB + g.ngroups + 1;
@@ -432,21 +433,26 @@ static bool aheap_geometry(Params& p, int smem_optin, AheapGeom& g) {
     return found;
 }
 
-template <typename T, int OP>
-static cudaError_t launch_aheap_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
-    AheapGeom g;
-    if (!aheap_geometry(p, smem_optin, g)) return cudaErrorInvalidConfiguration;
-    cudaError_t e = cudaFuncSetAttribute(aheap_kernel<T, OP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
+template <typename T, int OP, bool NP2>
+static cudaError_t launch_aheap_k(const Params& p, const AheapGeom& g, int sm_count, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(aheap_kernel<T, OP, NP2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, aheap_kernel<T, OP>, (int)g.nwarps * 32, g.smem_bytes);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, aheap_kernel<T, OP, NP2>, (int)g.nwarps * 32, g.smem_bytes);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
     if (p.grid_query) { *p.grid_query = grid; return cudaSuccess; }
-    aheap_kernel<T, OP><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
+    aheap_kernel<T, OP, NP2><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
     return cudaGetLastError();
+}
+
+template <typename T, int OP>
+static cudaError_t launch_aheap_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
+    AheapGeom g;
+    if (!aheap_geometry(p, smem_optin, g)) return cudaErrorInvalidConfiguration;
+    return g.c_magic ? launch_aheap_k<T, OP, true>(p, g, sm_count, st) : launch_aheap_k<T, OP, false>(p, g, sm_count, st);
 }
 
 cudaError_t launch_aheap_u64(const Params& p, int tsel, int sm_count, int smem_optin, cudaStream_t st);
