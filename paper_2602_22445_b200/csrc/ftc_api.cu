@@ -104,7 +104,7 @@ static size_t workspace_for(Params& p, const DeviceInfo& di) {
     size_t need = compact_area(p);
     p.ws_bytes = ~0ull;
     const KernelKind kind = pick_kernel(p, di);
-    if (kind == K_GENERIC) need += (size_t)generic_grid(p, di.sm_count) * p.Gmax * p.kbytes;
+    if (kind == K_GENERIC) need += (size_t)generic_reduce_grid(p, di.sm_count) * p.Gmax * p.kbytes;
     else if (kind == K_STAGED) need += staged_workspace_bytes(p, di.smem_optin, di.sm_count);
     return need;
 }
@@ -144,7 +144,7 @@ static int run_batch(const ftc_desc_t* desc, uint64_t S, int is_allreduce, const
     } else if (kind == K_LEVELS) {
         e = launch_aheap(p, tsel, di.sm_count, di.smem_optin, st);
     } else {
-        const size_t need = (size_t)generic_grid(p, di.sm_count) * p.Gmax * p.kbytes;
+        const size_t need = (size_t)generic_reduce_grid(p, di.sm_count) * p.Gmax * p.kbytes;
         if (!d_ws || ws_bytes < need || !aligned16(d_ws)) return FTC_EWORKSPACE;
         if (generic_smem_bytes(p) > (size_t)di.smem_optin) return FTC_EUNSUPPORTED;
         p.ws = d_ws;

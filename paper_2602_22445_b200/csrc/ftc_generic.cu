@@ -160,6 +160,23 @@ uint32_t generic_grid(const Params& p, int sm_count) {
     return (uint32_t)(p.S < g ? p.S : g);
 }
 
+// Threads of a block of the general reduce kernel: a level of the widest subtree keeps at most Gmax rows x the lanes
+// that walk a row busy, so scenarios of a few dozen processes get one warp (cheap barriers, 32 blocks per SM) and
+// large ones the full 256 threads.
+uint32_t generic_reduce_threads(const Params& p) {
+    const uint32_t nu = p.kbytes % 16 == 0 ? p.kbytes / 16 : p.k;
+    uint32_t upw = 1; while (upw < nu && upw < 32) upw <<= 1;
+    const uint64_t busy = (uint64_t)p.Gmax * upw;
+    uint32_t t = 32; while (t < 256 && t < busy) t <<= 1;
+    return t;
+}
+
+uint32_t generic_reduce_grid(const Params& p, int sm_count) {
+    const uint32_t per_sm = 2048 / generic_reduce_threads(p) > 32 ? 32 : 2048 / generic_reduce_threads(p);
+    uint64_t g = (uint64_t)sm_count * per_sm;
+    return (uint32_t)(p.S < g ? p.S : g);
+}
+
 template <typename T, int OP, bool VEC>
 static cudaError_t launch_generic_v(const Params& p, uint32_t grid, cudaStream_t st) {
     size_t smem = generic_smem_bytes(p);
@@ -168,15 +185,15 @@ static cudaError_t launch_generic_v(const Params& p, uint32_t grid, cudaStream_t
         cudaError_t e = cudaFuncSetAttribute(generic_kernel<T, OP, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    generic_kernel<T, OP, VEC><<<grid, 256, smem, st>>>(p);
+    generic_kernel<T, OP, VEC><<<grid, generic_reduce_threads(p), smem, st>>>(p);
     return cudaGetLastError();
 }
 
 // 16-byte units when the process vectors are a whole number of them (inputs, results and workspace are 16-byte aligned)
 template <typename T, int OP>
 static cudaError_t launch_generic_t(const Params& p, int sm_count, cudaStream_t st) {
-    return p.kbytes % 16 == 0 ? launch_generic_v<T, OP, true>(p, generic_grid(p, sm_count), st)
-                              : launch_generic_v<T, OP, false>(p, generic_grid(p, sm_count), st);
+    return p.kbytes % 16 == 0 ? launch_generic_v<T, OP, true>(p, generic_reduce_grid(p, sm_count), st)
+                              : launch_generic_v<T, OP, false>(p, generic_reduce_grid(p, sm_count), st);
 }
 
 cudaError_t launch_generic(const Params& p, int tsel, int sm_count, cudaStream_t st) {
@@ -237,7 +254,7 @@ cudaError_t launch_generic_static(Params p, int tsel, int sm_count, cudaStream_t
     void* ptr = nullptr;
     cudaError_t e = static_scratch_address(&ptr);
     if (e != cudaSuccess) return e;
-    uint32_t grid = generic_grid(p, sm_count);
+    uint32_t grid = generic_reduce_grid(p, sm_count);
     const size_t fit = (size_t)FTC_NOALLOC_SCRATCH_BYTES / slice;
     if (grid > fit) grid = (uint32_t)fit;
     p.ws = ptr;

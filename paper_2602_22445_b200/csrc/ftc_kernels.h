@@ -14,6 +14,8 @@ enum TypeSel { TS_U32_SUM = 0, TS_I32_MAX, TS_U32_XOR, TS_U64_SUM, TS_I64_MAX, T
 
 size_t generic_smem_bytes(const Params& p);
 uint32_t generic_grid(const Params& p, int sm_count);
+uint32_t generic_reduce_threads(const Params& p);            // block size of the general reduce kernel for this shape
+uint32_t generic_reduce_grid(const Params& p, int sm_count);  // its blocks (each needs a workspace slice of Gmax * kbytes)
 cudaError_t launch_generic(const Params& p, int tsel, int sm_count, cudaStream_t st);
 
 // General kernel on the library's built-in scratch array (no workspace from the caller).
