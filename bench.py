@@ -291,7 +291,7 @@ def measured_peak():
 class Leg:
     """One workload resident on the device: inputs generated there, failure patterns uploaded, outputs and workspace."""
 
-    def __init__(self, name, S, first, args, B, torch, sched_rounds, candidates=False):
+    def __init__(self, name, S, first, args, B, torch, sched_rounds, candidates=False, expanded=False):
         self.name, self.S, self.B, self.torch = name, S, B, torch
         self.candidates = candidates
         w = make_workload(name, S, first, sched_rounds)
@@ -307,6 +307,8 @@ class Leg:
         kflags = {"auto": 0, "direct": B.FTC_KERNEL_DIRECT, "generic": B.FTC_KERNEL_GENERIC, "levels": B.FTC_KERNEL_LEVELS}[args.kernel]
         if args.arity:
             kflags |= B.FTC_TREE_BINOMIAL if args.arity == 1 else B.FTC_TREE_ARITY(args.arity)
+        if expanded:
+            kflags |= B.FTC_OUT_EXPANDED            # allreduce: the value in the slot of every process that holds it, [S][P][k]
         self.desc = B.make_desc(w.P, w.f, w.k, B.dtype_code(self.tdt), w.op, root=-1 if w.roots is not None else 0,
                                 max_inop=0 if w.inop is None else w.inop.shape[1], flags=kflags)
         self.fn = B.ftc_allreduce_batch if self.allred else B.ftc_reduce_batch
@@ -325,6 +327,9 @@ class Leg:
             self.d_ws = torch.empty(max(B.ftc_candidates_workspace_bytes(self.desc, S), 256), dtype=torch.uint8, device="cuda")
             self.bytes_per_launch += S * w.f * (w.k * self.esz + 8) - S * 8
         else:
+            if expanded:
+                self.d_out = torch.empty((S, w.P, w.k), dtype=self.tdt, device="cuda")
+                self.bytes_per_launch += S * (w.P - 1) * w.k * self.esz
             self.d_ws = torch.empty(max(B.ftc_workspace_bytes(self.desc, S, self.allred), 16), dtype=torch.uint8, device="cuda")
         torch.cuda.synchronize()
 
@@ -400,14 +405,14 @@ def add_sustained(roof, leg, torch, sampler, seconds):
                          "sm_mhz_median": mhz, "ms_x_mhz": (ms * mhz) if mhz else None, "clocks": clocks}
 
 
-def run_side_leg(name, args, B, torch, sampler, peak, peak_kind, candidates=False, arity=0):
+def run_side_leg(name, args, B, torch, sampler, peak, peak_kind, candidates=False, arity=0, expanded=False):
     """One more workload, timed like the headline one: K steps, then a sustained run; its own roofline record.
     candidates: what every root child delivers (ftc_candidates_batch) instead of the batch call.
     arity: another subtree shape below the root's children (a-ary heaps; 1 = binomial trees) on the same inputs."""
     if arity:
         args = argparse.Namespace(**{**vars(args), "arity": arity})
     S = (args.batch if args.candidates and args.batch else 0) or DEFAULT_BATCH[name]
-    leg = Leg(name, S, 0, args, B, torch, 28, candidates=candidates)
+    leg = Leg(name, S, 0, args, B, torch, 28, candidates=candidates, expanded=expanded)
     for _ in range(max(args.warmup, 3)):
         leg.step()
     m0 = sampler.lines() if sampler else 0
@@ -419,6 +424,8 @@ def run_side_leg(name, args, B, torch, sampler, peak, peak_kind, candidates=Fals
     add_sustained(roof, leg, torch, sampler, args.sustain_seconds / 2)
     ms = total_ms / args.steps
     shape = "" if not arity else " [subtrees: binomial trees]" if arity == 1 else f" [subtrees: {arity}-ary heaps]"
+    if expanded:
+        shape += " [expanded output: the value written into the slot of every process that holds it, zeros elsewhere]"
     rec = {"workload": f"{name}: {DESCRIPTION[name]}" + (" [what every root child delivers: all f+1 subtrees played]" if candidates else "") + shape,
            "value": S / (ms / 1e3), "unit": "scenarios/s", "ms_per_step": ms,
            "steps": args.steps, "scenarios_per_step": S, "process_rounds_per_sec": S / (ms / 1e3) * leg.w.P * leg.rounds(),
@@ -645,6 +652,9 @@ def run_gpu(args):
                 workloads[tag] = run_side_leg(other, args, B, torch, sampler, peak, peak_kind, arity=ar)
                 workloads[tag]["roofline"]["traffic"] = None
                 launches += args.steps + workloads[tag]["roofline"]["sustained"]["steps"]
+            workloads["c4_expanded"] = run_side_leg("c4", args, B, torch, sampler, peak, peak_kind, expanded=True)
+            workloads["c4_expanded"]["roofline"]["traffic"] = None
+            launches += 2 * (args.steps + workloads["c4_expanded"]["roofline"]["sustained"]["steps"])     # two kernels a step
             for other in ("c4", "c5"):                      # all f+1 root children played (integer configurations)
                 key = other + "_all_children"
                 workloads[key] = run_side_leg(other, args, B, torch, sampler, peak, peak_kind, candidates=True)
