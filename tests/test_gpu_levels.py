@@ -70,6 +70,26 @@ def test_vectors_of_any_number_of_chunks(arity, P, f, k, dname, op):
         assert_same(got, run_oracle_mt(x, f, op, pf, inop, roots, 0, allreduce, arity=arity), f"P={P} f={f} k={k} {dname} {op} arity={arity} allreduce={allreduce}")
 
 
+EDGE_SHAPES = [
+    # the smallest process counts (P = f + 2: one group, one row), a single full group plus the root, one row more than a tile,
+    # the widest group (f = 31), the widest vectors (31 and 32 chunks), two processes
+    (3, 1, 4, "i32", "sum"), (2, 0, 4, "f32", "sum"), (33, 31, 4, "i32", "xor"), (34, 31, 2, "u64", "sum"), (65, 31, 4, "f32", "sum"),
+    (5, 3, 8, "f32", "sum"), (6, 3, 8, "i64", "max"), (1000, 0, 124, "f32", "sum"), (300, 2, 128, "i32", "max"), (130, 1, 64, "u64", "xor"),
+]
+
+
+@pytest.mark.parametrize("arity", [1, 2, 3, 32])
+@pytest.mark.parametrize("P,f,k,dname,op", EDGE_SHAPES)
+def test_level_kernel_edge_shapes(arity, P, f, k, dname, op):
+    """Degenerate shapes, and batches of one and two scenarios: whichever kernel the shape gets, the oracle decides."""
+    for allreduce in (False, True):
+        for S in (1, 2, 37):
+            d_x, x, pf, inop, roots = make_batch(P, f, k, dname, allreduce, S, seed=arity + 13 * P + k + S)
+            got = run_gpu(None, f, op, pf, inop, roots, 0, allreduce, flags_for(arity), d_x=d_x)
+            assert B.ftc_kernel_name(got[2], allreduce) in ("levels", "generic", "staged")
+            assert_same(got, run_oracle_mt(x, f, op, pf, inop, roots, 0, allreduce, arity=arity), f"P={P} f={f} k={k} {dname} {op} arity={arity} allreduce={allreduce} S={S}")
+
+
 def test_shapes_the_level_kernel_leaves_to_the_general_one():
     for k, dt in ((3, B.FTC_F32), (6, B.FTC_I32), (1, B.FTC_U64)):            # not a multiple of 16 bytes
         assert B.ftc_kernel_name(B.make_desc(100, 2, k, dt, "sum", flags=B.FTC_TREE_ARITY(4)), True) == "generic"
