@@ -4,6 +4,9 @@ oracle playing the same shape, bit for bit."""
 import numpy as np
 import pytest
 
+from oracle import oracle as O
+from paper_2602_22445_b200 import scenarios as sc
+
 from paper_2602_22445_b200 import binding as B
 from tests.gpu_util import assert_same, run_gpu, run_oracle_mt
 from tests.test_gpu_variants import DT, make_batch
@@ -123,3 +126,43 @@ def test_level_kernel_gives_up_cleanly(arity, P, f, k, dname, op, allreduce):
         assert np.array_equal(seq, np.sort(seq)), (b, seq)
     assert timed_out.any()
     assert_same(run_gpu(None, f, op, pf, inop, roots, 0, allreduce, flags, d_x=d_x), want, "normal call after the give-up run")
+
+
+def seeded_shapes():
+    rng = np.random.Generator(np.random.PCG64(20260223))
+    out = []
+    for _ in range(40):
+        f = int(rng.choice([0, 1, 1, 2, 3, 3, 4, 7, 15]))
+        P = int(rng.choice([rng.integers(f + 2, 300), rng.integers(300, 3000), rng.integers(3000, 30000)]))
+        dname = ["i32", "i64", "u64", "f32", "f32"][int(rng.integers(0, 5))]
+        op = "sum" if dname == "f32" else ["sum", "max", "xor"][int(rng.integers(0, 3))]
+        k = int(rng.choice([4, 8, 12, 16, 20, 24, 32, 44, 64, 128] if np.dtype(DT[dname]).itemsize == 4 else [2, 4, 6, 8, 10, 16, 22, 64]))
+        out.append((P, f, k, dname, op, bool(rng.integers(0, 2)), int(rng.choice([1, 2, 3, 4, 5, 7, 8, 16, 32])), bool(rng.integers(0, 3) == 0)))
+    return out
+
+
+@pytest.mark.parametrize("P,f,k,dname,op,allreduce,arity,descending", seeded_shapes())
+def test_seeded_random_shapes_and_patterns(P, f, k, dname, op, allreduce, arity, descending):
+    """Random shapes, subtree shapes and partner orders with failure patterns beyond what the schedule tolerates (up to f + 2
+    processes failed beforehand, two in-operation victims at any round up to twice an attempt, any root): whatever kernel the
+    shape gets, results and status records equal the oracle's."""
+    rng = np.random.Generator(np.random.PCG64(P * 31 + k + arity))
+    S = max(2, min(24, int(3e6 // (P * k))))
+    dt = DT[dname]
+    x = rng.standard_normal((S, P, k)).astype(np.float32) if dname == "f32" else \
+        rng.integers(np.iinfo(dt).min, np.iinfo(dt).max, size=(S, P, k), dtype=dt, endpoint=True)
+    pf = sc.picks_to_masks(sc.random_subsets(rng, S, P, np.minimum(rng.integers(0, f + 3, size=S), P - 1)), P)
+    R = O.schedule(P, f, arity)["rounds_attempt"]
+    inop = np.zeros((S, 2, 2), dtype=np.uint32)
+    lo = f + 1 if allreduce and P > 2 * f + 4 else 0                 # keeps the victims clear of the root candidates 0..f
+    inop[:, :, 0] = rng.integers(lo, P, size=(S, 2))
+    inop[:, :, 1] = rng.integers(0, 2 * R + 2, size=(S, 2))
+    inop[rng.random((S, 2)) < 0.4, 0] = sc.UNUSED
+    roots = rng.integers(0, P, size=S).astype(np.uint32)
+    if allreduce and lo:
+        roots[:] = 0
+    flags = flags_for(arity) | (B.FTC_PARTNERS_DESCENDING if descending else 0)
+    got = run_gpu(x, f, op, pf, inop, roots, 0, allreduce, flags)
+    assert B.ftc_kernel_name(got[2], allreduce) in ("levels", "generic", "staged")
+    assert_same(got, run_oracle_mt(x, f, op, pf, inop, roots, 0, allreduce, arity=arity, partners_descending=descending),
+                f"P={P} f={f} k={k} {dname} {op} allreduce={allreduce} arity={arity} descending={descending}")
