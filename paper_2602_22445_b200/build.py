@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libftc.so")
-SOURCES = ["ftc_api.cu", "ftc_generic.cu", "ftc_tiled.cu", "ftc_staged.cu", "ftc_staged_inst0.cu", "ftc_staged_inst1.cu", "ftc_staged_inst2.cu", "ftc_staged_inst3.cu", "ftc_expand.cu", "ftc_candidates.cu", "ftc_messages.cu", "ftc_fill.cu", "ftc_probe.cu", "ftc_warp_inst0.cu", "ftc_warp_inst1.cu", "ftc_cand_inst0.cu", "ftc_cand_inst1.cu", "ftc_aheap_inst0.cu", "ftc_aheap_inst1.cu"]
+SOURCES = ["ftc_api.cu", "ftc_generic.cu", "ftc_tiled.cu", "ftc_staged.cu", "ftc_staged_inst0.cu", "ftc_staged_inst1.cu", "ftc_staged_inst2.cu", "ftc_staged_inst3.cu", "ftc_expand.cu", "ftc_candidates.cu", "ftc_messages.cu", "ftc_fill.cu", "ftc_probe.cu", "ftc_warp_inst0.cu", "ftc_warp_inst1.cu", "ftc_cand_inst0.cu", "ftc_cand_inst1.cu", "ftc_aheap_inst0.cu", "ftc_aheap_inst1.cu", "ftc_aheap_inst2.cu", "ftc_aheap_inst3.cu"]
 HEADERS = ["ftc_device.cuh", "ftc_tile_common.cuh", "ftc_staged_impl.cuh", "ftc_warp_impl.cuh", "ftc_cand_impl.cuh", "ftc_aheap_impl.cuh", "ftc_decode_warp.cuh", "ftc_kernels.h", os.path.join("..", "..", "include", "ftc.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--fmad=false"]

@@ -44,8 +44,9 @@ struct AheapGeom {
     uint32_t c_magic;                      // 0: the vector is a power-of-two number of 16-byte chunks; else ceil(2^32 / chunks)
 };
 
-// NP2: the vector is not a power-of-two number of 16-byte chunks
-template <typename T, int OP, bool NP2>
+// NP2: the vector is not a power-of-two number of 16-byte chunks. M: the group size f + 1 when it is one of the usual ones (its
+// fold is then straight-line code with all loads issued together: the fold is most of the instruction stream), 0: any.
+template <typename T, int OP, bool NP2, int M>
 __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kernel(Params p, const __grid_constant__ AheapGeom g) {
     extern __shared__ __align__(128) uint32_t smem[];
     char* sbase = reinterpret_cast<char*>(smem);
@@ -187,7 +188,7 @@ __global__ void __launch_bounds__(kStagedMaxThreads, FTC_AHEAP_MINB) aheap_kerne
         // a row's value after up-correction (Algorithm "Up-correction") from its staged copy: folded as a plain group at once
         // (the loads do not wait for the row's mask), and once more by the general rules where the group is not plain
         auto fold_row = [&](const char* srow_lc, const char* in_lc, uint32_t row) -> uint4 {
-            const uint4 v = fold16_full<T, OP, 0>(srow_lc, p.kbytes, p.m, sstar, LdShared(), p.pdesc != 0);
+            const uint4 v = fold16_full<T, OP, M>(srow_lc, p.kbytes, M ? (uint32_t)M : p.m, sstar, LdShared(), p.pdesc != 0);
             if (group_is_plain(p, root, inc, row)) return v;
             return fold_staged_call<T, OP, false>(fold_shape(p), root, sstar, inc, in_lc, srow_lc, row);
         };
@@ -433,18 +434,18 @@ static bool aheap_geometry(Params& p, int smem_optin, AheapGeom& g) {
     return found;
 }
 
-template <typename T, int OP, bool NP2>
+template <typename T, int OP, bool NP2, int M>
 static cudaError_t launch_aheap_k(const Params& p, const AheapGeom& g, int sm_count, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(aheap_kernel<T, OP, NP2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
+    cudaError_t e = cudaFuncSetAttribute(aheap_kernel<T, OP, NP2, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, aheap_kernel<T, OP, NP2>, (int)g.nwarps * 32, g.smem_bytes);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, aheap_kernel<T, OP, NP2, M>, (int)g.nwarps * 32, g.smem_bytes);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
     if (p.grid_query) { *p.grid_query = grid; return cudaSuccess; }
-    aheap_kernel<T, OP, NP2><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
+    aheap_kernel<T, OP, NP2, M><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g);
     return cudaGetLastError();
 }
 
@@ -452,9 +453,18 @@ template <typename T, int OP>
 static cudaError_t launch_aheap_t(Params p, int sm_count, int smem_optin, cudaStream_t st) {
     AheapGeom g;
     if (!aheap_geometry(p, smem_optin, g)) return cudaErrorInvalidConfiguration;
-    return g.c_magic ? launch_aheap_k<T, OP, true>(p, g, sm_count, st) : launch_aheap_k<T, OP, false>(p, g, sm_count, st);
+    if (g.c_magic) return launch_aheap_k<T, OP, true, 0>(p, g, sm_count, st);
+    switch (p.m) {                                                  // the group sizes of f = 2, 3, 4 and 8
+    case 3: return launch_aheap_k<T, OP, false, 3>(p, g, sm_count, st);
+    case 4: return launch_aheap_k<T, OP, false, 4>(p, g, sm_count, st);
+    case 5: return launch_aheap_k<T, OP, false, 5>(p, g, sm_count, st);
+    case 9: return launch_aheap_k<T, OP, false, 9>(p, g, sm_count, st);
+    default: return launch_aheap_k<T, OP, false, 0>(p, g, sm_count, st);
+    }
 }
 
 cudaError_t launch_aheap_u64(const Params& p, int tsel, int sm_count, int smem_optin, cudaStream_t st);
+cudaError_t launch_aheap_b32(const Params& p, int tsel, int sm_count, int smem_optin, cudaStream_t st);
+cudaError_t launch_aheap_b64(const Params& p, int tsel, int sm_count, int smem_optin, cudaStream_t st);
 
 }  // namespace ftc
