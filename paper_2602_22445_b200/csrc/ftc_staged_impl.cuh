@@ -20,6 +20,7 @@
 //   - scenarios staged whole by one copy (up to 12-16 KB): 64 registers.
 #pragma once
 #include <cuda.h>
+#include <type_traits>
 #include "ftc_tile_common.cuh"
 #include "ftc_decode_warp.cuh"
 #include "ftc_kernels.h"
@@ -133,17 +134,26 @@ __device__ __forceinline__ uint4 fold_fast_staged(const Params& p, uint32_t ssta
     return fold_plain_staged<T, OP>(p, sstar, srow_lc);
 }
 
-template <typename T, int OP, int XL, int U, bool WHOLE, bool MASKED>
+// Fold of a plain group from its staged copy with the group size as a constant (M = f + 1: straight-line code, all loads
+// issued together); M = 0: the size is read from p.
+template <typename T, int OP, int M>
+__device__ __forceinline__ uint4 fold_plain_m(const Params& p, uint32_t sstar, const char* srow_lc) {
+    return fold16_full<T, OP, M>(srow_lc, p.kbytes, M ? (uint32_t)M : p.m, sstar, LdShared(), p.pdesc != 0);
+}
+
+// M: the group size as a constant for the plain folds (the large-block kernel picks it once per tile), 0: from p
+template <typename T, int OP, int XL, int U, bool WHOLE, bool MASKED, int M = 0>
 struct SubHeapPlain {
     static __device__ __forceinline__ uint4 eval(const Params& p, uint32_t sstar, const uint32_t* inc, const char* buf_lc, uint32_t rowbytes,
                                                  uint32_t trow, uint32_t grow, uint32_t G) {
-        uint4 v = fold_fast_staged<T, OP, MASKED>(p, sstar, inc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, trow, grow), grow);
+        const char* srow = buf_lc + staged_row_offset<WHOLE>(p, rowbytes, trow, grow);
+        uint4 v = (M && !MASKED) ? fold_plain_m<T, OP, M>(p, sstar, srow) : fold_fast_staged<T, OP, MASKED>(p, sstar, inc, srow, grow);
         if (U + 1 < XL) {
             constexpr int UN = (U + 1 < XL ? U + 1 : U);
             if (U + 2 < XL || 2 * grow + 1 < G)
-                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE, MASKED>::eval(p, sstar, inc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
+                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE, MASKED, M>::eval(p, sstar, inc, buf_lc, rowbytes, 2 * trow + 1, 2 * grow + 1, G));
             if (U + 2 < XL || 2 * grow + 2 < G)
-                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE, MASKED>::eval(p, sstar, inc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
+                v = comb16<T, OP>(v, SubHeapPlain<T, OP, XL, UN, WHOLE, MASKED, M>::eval(p, sstar, inc, buf_lc, rowbytes, 2 * trow + 2, 2 * grow + 2, G));
         }
         return v;
     }
@@ -560,9 +570,17 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
                 } else if (!careful && !masked) {
                     // XL == 1: the bottom rows are the tile's last level and may be missing; XL > 1: they exist
                     uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
-                    if (XL > 1 || rowA < G) valA = SubHeapPlain<T, OP, XL, 0, WHOLE, false>::eval(p, sstar, inc, buf_lc, rowbytes, tA, rowA, G);
                     const bool hasB = lr < RW - 1;
-                    if (hasB) valB = fold_fast_staged<T, OP, false>(p, sstar, inc, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB), rowB);
+                    // the tile's folds with the group size as a constant where it is one of f = 4, f = 8 (the configurations
+                    // with many processes): one uniform branch per tile
+                    auto folds = [&](auto mtag) {
+                        constexpr int M = decltype(mtag)::value;
+                        if (XL > 1 || rowA < G) valA = SubHeapPlain<T, OP, XL, 0, WHOLE, false, M>::eval(p, sstar, inc, buf_lc, rowbytes, tA, rowA, G);
+                        if (hasB) valB = fold_plain_m<T, OP, M>(p, sstar, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB));
+                    };
+                    if (!WHOLE && p.m == 5) folds(std::integral_constant<int, 5>());
+                    else if (!WHOLE && p.m == 9) folds(std::integral_constant<int, 9>());
+                    else folds(std::integral_constant<int, 0>());
                     valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                     if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                 } else if (!careful) {
