@@ -442,9 +442,16 @@ __global__ void __launch_bounds__(kStagedMaxThreads, 2) cand_kernel(Params p, Ca
                     // every group of the tile is whole: one value per row serves all children (exact operations)
                     if (j0 < Gc) {
                         uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
-                        if (XL > 1 || rowA < Gc) valA = SubHeapPlain<T, OP, XL, 0, false, false>::eval(p, 0u, alive, buf_lc, rowbytes, tA, rowA, Gc);
                         const bool hasB = lr < RW - 1;
-                        if (hasB) valB = fold_plain_staged<T, OP>(p, 0u, buf_lc + staged_row_offset<false>(p, rowbytes, lr, rowB));
+                        // the group size as a constant where it is that of f = 4 or f = 8: one uniform branch per tile
+                        auto folds = [&](auto mtag) {
+                            constexpr int M = decltype(mtag)::value;
+                            if (XL > 1 || rowA < Gc) valA = SubHeapPlain<T, OP, XL, 0, false, false, M>::eval(p, 0u, alive, buf_lc, rowbytes, tA, rowA, Gc);
+                            if (hasB) valB = fold_plain_m<T, OP, M>(p, 0u, buf_lc + staged_row_offset<false>(p, rowbytes, lr, rowB));
+                        };
+                        if (p.m == 5) folds(std::integral_constant<int, 5>());
+                        else if (p.m == 9) folds(std::integral_constant<int, 9>());
+                        else folds(std::integral_constant<int, 0>());
                         valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, Gc);
                         if (lr == 0) hvc[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                     }
