@@ -333,7 +333,9 @@ constexpr int kStagedBatchedSwzTag = 5;      // the same in large blocks
 // Tensor maps of the swizzled variant: one per tile level (its box is that level's rows); unused otherwise.
 struct alignas(64) TmaMaps { CUtensorMap lvl[8]; };
 
-template <typename T, int OP, int XL, bool WHOLE, int MINB>
+// GM: the group size f + 1 as a constant for the plain folds of the large-block kernel (5, 9: the configurations with many
+// processes), 0: read from p
+template <typename T, int OP, int XL, bool WHOLE, int MINB, int GM = 0>
 __global__ void __launch_bounds__((MINB == kStagedLeanMinBlocks || MINB == kStagedLeanSwzTag) ? kStagedLeanThreads : kStagedMaxThreads,
                                   (MINB == kStagedBatchedTag || MINB == kStagedBatchedSwzTag) ? 2 : (MINB == kStagedLeanSwzTag ? kStagedLeanMinBlocks : MINB))
 staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
@@ -571,16 +573,13 @@ staged_kernel(Params p, StagedGeom g, const __grid_constant__ TmaMaps maps) {
                     // XL == 1: the bottom rows are the tile's last level and may be missing; XL > 1: they exist
                     uint4 valA = make_uint4(0, 0, 0, 0), valB = make_uint4(0, 0, 0, 0);
                     const bool hasB = lr < RW - 1;
-                    // the tile's folds with the group size as a constant where it is one of f = 4, f = 8 (the configurations
-                    // with many processes): one uniform branch per tile
+                    // the tile's folds, with the group size as a constant in the instantiations that have one
                     auto folds = [&](auto mtag) {
                         constexpr int M = decltype(mtag)::value;
                         if (XL > 1 || rowA < G) valA = SubHeapPlain<T, OP, XL, 0, WHOLE, false, M>::eval(p, sstar, inc, buf_lc, rowbytes, tA, rowA, G);
                         if (hasB) valB = fold_plain_m<T, OP, M>(p, sstar, buf_lc + staged_row_offset<WHOLE>(p, rowbytes, lr, rowB));
                     };
-                    if (!WHOLE && p.m == 5) folds(std::integral_constant<int, 5>());
-                    else if (!WHOLE && p.m == 9) folds(std::integral_constant<int, 9>());
-                    else folds(std::integral_constant<int, 0>());
+                    folds(std::integral_constant<int, GM>());
                     valB = tile_tree_phase<T, OP, (XL > 1), true>(valA, valB, lw, cwl, p.C, lane, lc, tB, idxB, rowB, hasB, G);
                     if (lr == 0) hv[(size_t)j0 * p.C + lc] = lw ? valB : valA;
                 } else if (!careful) {
@@ -744,19 +743,19 @@ static const TmaMaps kNoMaps = {};
 // Tensor maps for the swizzled variant (host side, below).
 static bool staged_tensor_maps(const Params& p, uint32_t D, TmaMaps& maps);
 
-template <typename T, int OP, int XL, bool WHOLE, int MINB>
+template <typename T, int OP, int XL, bool WHOLE, int MINB, int GM = 0>
 static cudaError_t launch_staged_w(const Params& p, const StagedGeom& g, int sm_count, cudaStream_t st, const TmaMaps& maps = kNoMaps) {
-    cudaError_t e = cudaFuncSetAttribute(staged_kernel<T, OP, XL, WHOLE, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
+    cudaError_t e = cudaFuncSetAttribute(staged_kernel<T, OP, XL, WHOLE, MINB, GM>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g.smem_bytes);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, staged_kernel<T, OP, XL, WHOLE, MINB>, (int)g.nwarps * 32, g.smem_bytes);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, staged_kernel<T, OP, XL, WHOLE, MINB, GM>, (int)g.nwarps * 32, g.smem_bytes);
     if (e != cudaSuccess) return e;
     if (per_sm < 1) per_sm = 1;
     if (g.hv_global && per_sm > kHvGlobalBlocksPerSm) per_sm = kHvGlobalBlocksPerSm;      // one workspace slice per block
     const uint64_t cap = (uint64_t)sm_count * per_sm;
     const uint32_t grid = (uint32_t)(p.S < cap ? p.S : cap);
     if (p.grid_query) { *p.grid_query = grid; return cudaSuccess; }
-    staged_kernel<T, OP, XL, WHOLE, MINB><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g, maps);
+    staged_kernel<T, OP, XL, WHOLE, MINB, GM><<<grid, g.nwarps * 32, g.smem_bytes, st>>>(p, g, maps);
     return cudaGetLastError();
 }
 
@@ -832,7 +831,10 @@ static cudaError_t launch_staged_t(Params p, int sm_count, int smem_optin, cudaS
     case SV_BATCHED_LEAN:
         if constexpr (!Ordered<T>::value) return launch_staged_w<T, OP, XL, false, kStagedBatchedTag>(p, g, sm_count, st);
         return cudaErrorInvalidConfiguration;
-    case SV_LARGE: return launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
+    case SV_LARGE:
+        if (p.m == 5) return launch_staged_w<T, OP, XL, false, 2, 5>(p, g, sm_count, st);
+        if (p.m == 9) return launch_staged_w<T, OP, XL, false, 2, 9>(p, g, sm_count, st);
+        return launch_staged_w<T, OP, XL, false, 2>(p, g, sm_count, st);
     default: return cudaErrorInvalidConfiguration;
     }
 }
